@@ -1,0 +1,191 @@
+/*
+ * fasttps.h -- C ABI of the FastTPS decode (token-phase) library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements one decode step of a decoder-only transformer layer as
+ * described by the FastTPS paper: joint RoPE on the new q/k, in-place append of
+ * k/v into a preallocated ("static") KV cache, single-query attention over that
+ * cache (Algorithm 3 "GKVC & TPSFLAT", Eq. 2), and the fused SwiGLU MLP
+ * (Algorithm 4 "MLP Implementation", Eq. 1, Eq. 31), plus the projections and
+ * norms that chain them into a layer and a model (Figure 1, Section 2.2, 2.3).
+ *
+ * Conventions that hold for every entry point
+ *   - "device" pointers are CUDA device memory on the context's GPU, owned by the
+ *     caller, contiguous, 16-byte aligned.  bf16 unless stated.  Nothing is
+ *     retained after the call returns except where stated (packed weights are
+ *     read on every call and must stay alive).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *     only enqueue work and return without synchronising.  One context must not be
+ *     used from two streams at the same time (its workspace is shared).
+ *   - Return value: FASTTPS_OK or a negative fasttps_status code.  Nothing is
+ *     thrown across the boundary.  Conditions that only the device can see (a
+ *     sequence whose cache is full, a negative position, a bounded wait that ran
+ *     out) never trap: the affected sequence is skipped and a bit is set in the
+ *     context's device status word, read with fasttps_get_status().
+ *   - There is no CPU fallback: every step runs in the library's CUDA kernels.
+ */
+#ifndef FASTTPS_H
+#define FASTTPS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fasttps_ctx fasttps_ctx;
+
+typedef enum {
+    FASTTPS_OK = 0,
+    FASTTPS_INVALID_ARG = -1,   /* null/misaligned pointer, batch out of range, unsupported dims */
+    FASTTPS_CUDA_ERROR = -2,    /* a CUDA runtime call or launch failed; see fasttps_last_error() */
+    FASTTPS_OUT_OF_MEMORY = -3  /* workspace allocation failed in fasttps_create() */
+} fasttps_status;
+
+/* bits of the device status word */
+#define FASTTPS_DEV_CACHE_FULL   1u   /* some seq_lens[b] >= max_seq (or < 0): sequence skipped */
+#define FASTTPS_DEV_BAD_POSITION 2u   /* some pos[b] < 0 or >= max_seq: sequence skipped        */
+#define FASTTPS_DEV_WAIT_TIMEOUT 4u   /* a bounded wait on an asynchronous copy ran out         */
+#define FASTTPS_DEV_BAD_TOKEN    8u   /* a token id outside [0, vocab): row 0 used instead      */
+
+/* Model shape and limits.  Supported: hidden % 8 == 0, hidden <= 8192;
+ * head_dim in {32, 64, 96, 128}; n_q_heads % n_kv_heads == 0; inter % 8 == 0;
+ * (n_q_heads * head_dim) % 8 == 0 and <= 8192; max_batch >= 1; max_seq >= 1.
+ * vocab and n_layers may be 0 when only the block-level calls are used. */
+typedef struct {
+    int hidden;        /* D                                   */
+    int n_q_heads;     /* H_q                                 */
+    int n_kv_heads;    /* H_kv (H_q for multi-head attention) */
+    int head_dim;      /* d                                   */
+    int inter;         /* K, MLP intermediate size            */
+    int vocab;         /* V                                   */
+    int n_layers;
+    int max_batch;     /* largest batch any call will use     */
+    int max_seq;       /* N_p + N_r: rows per head in a cache; also the largest position + 1 */
+    float rms_eps;
+    float rope_theta;
+    int device;        /* CUDA device ordinal                 */
+} fasttps_config;
+
+/* Packed weights of one layer (device pointers; see the packing calls). */
+typedef struct {
+    const void *g_attn_norm;  /* [D] bf16 gain of the norm before attention */
+    const void *w_qkv;        /* packed FASTTPS_W_QKV     */
+    const void *w_o;          /* packed FASTTPS_W_O       */
+    const void *g_mlp_norm;   /* [D] bf16 gain of the norm before the MLP   */
+    const void *w_gate_up;    /* packed FASTTPS_W_GATE_UP */
+    const void *w_down;       /* packed FASTTPS_W_DOWN    */
+} fasttps_layer_weights;
+
+typedef enum {
+    FASTTPS_W_QKV = 0,      /* logical [D, (H_q + 2 H_kv) d], columns q | k | v, head-major */
+    FASTTPS_W_O = 1,        /* logical [H_q d, D]                                           */
+    FASTTPS_W_GATE_UP = 2,  /* logical [D, 2K], columns [0,K) gate and [K,2K) up            */
+    FASTTPS_W_DOWN = 3,     /* logical [K, D]                                               */
+    FASTTPS_W_LM_HEAD = 4   /* logical [V, D]                                               */
+} fasttps_weight_kind;
+
+/* Create a context: validates cfg, selects cfg->device, allocates the workspace
+ * (split-KV partials, FP32 accumulators, tickets, activation scratch for the
+ * layer/model chains, the RoPE cos/sin table, the status word) and builds the
+ * cos/sin table on the host in double precision.  The only call that allocates
+ * or synchronises besides fasttps_destroy/get_status/model_decode_host. */
+int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg);
+int fasttps_destroy(fasttps_ctx *ctx);
+
+/* One-time weight packing, outside the decode path: the offline re-layout of
+ * Section 3.2 item 1 ("interlaced layout of gate-up weights").  `src` is the
+ * logical row-major bf16 matrix described at fasttps_weight_kind, `dst` a
+ * device buffer of fasttps_packed_bytes(kind) bytes.  Packed layouts:
+ *   QKV, O, LM_HEAD: [out, in] (each output's weights contiguous);
+ *   GATE_UP: [2K, D] rows interlaced in blocks of 8: for j-octet J the rows
+ *            16J..16J+7 are gate columns 8J..8J+7 and 16J+8..16J+15 the matching
+ *            up columns, so a gate value and its up value meet in one CTA;
+ *   DOWN: [K, D] unchanged. */
+size_t fasttps_packed_bytes(const fasttps_ctx *ctx, int kind);
+int fasttps_pack_weight(fasttps_ctx *ctx, int kind, const void *src, void *dst, void *stream);
+/* Inverse of fasttps_pack_weight (for round-trip checks). */
+int fasttps_unpack_weight(fasttps_ctx *ctx, int kind, const void *src_packed, void *dst_logical, void *stream);
+
+/* Algorithm 3 (GKVC & TPSFLAT), one decode step for `batch` sequences.
+ *   q [B,H_q,d], k_new [B,H_kv,d], v_new [B,H_kv,d]   (before RoPE)
+ *   k_cache, v_cache [B,H_kv,max_seq,d]   in/out: row seq_lens[b] of every head
+ *       receives bf16(rope(k_new)) resp. v_new -- exactly B*H_kv runs of d
+ *       elements at element offset (b*H_kv+h)*max_seq*d + seq_lens[b]*d (Eq. 2);
+ *       no other element is written and none is re-loaded to be moved.
+ *   pos [B] int32 device: rotary position of the new token.
+ *   seq_lens [B] int32 device: rows already cached (N_p) = the row written now.
+ *   out [B,H_q,d]: softmax(q' K^T / sqrt(d)) V over rows 0..seq_lens[b] inclusive.
+ * Query head h uses kv head h / (H_q/H_kv).  Neither pos nor seq_lens is advanced. */
+int fasttps_attn_decode(fasttps_ctx *ctx, const void *q, const void *k_new, const void *v_new,
+                        void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
+                        void *out, int batch, void *stream);
+
+/* Algorithm 4 steps 2-15 / Eq. 1: out = (silu(x W_gate) * (x W_up)) W_down.
+ *   x [B,D]; w_gate_up, w_down packed; out [B,D].  The gate_up products, the
+ *   SiLU*mul result and the down-projection partial sums stay on chip; partial
+ *   sums of the CTAs meet in an FP32 accumulator of the workspace. */
+int fasttps_mlp_decode(fasttps_ctx *ctx, const void *x, const void *w_gate_up, const void *w_down,
+                       void *out, int batch, void *stream);
+
+/* Building block of the chain (QKV, output projection, lm_head; Figure 1):
+ *   out[b,n] = (g_norm ? rmsnorm(x[b], g_norm) : x[b]) . W[n,:] (+ residual[b,n])
+ *   x [B,in]; w packed [out,in]; residual [B,out] or NULL; out_bf16 [B,out] or NULL;
+ *   out_f32 [B,out] float or NULL (at least one output).  in = D for QKV/LM_HEAD,
+ *   H_q d for O.  The normalised input is rounded to bf16 before the product. */
+int fasttps_linear_decode(fasttps_ctx *ctx, int kind, const void *x, const void *g_norm, const void *w,
+                          const void *residual, void *out_bf16, float *out_f32, int batch, void *stream);
+
+/* One decoder layer: RMSNorm -> QKV -> attn_decode -> o_proj (+x) -> RMSNorm -> MLP (+h).
+ *   x_in [B,D], x_out [B,D] (may alias x_in); caches, pos, seq_lens as in
+ *   fasttps_attn_decode (caches of THIS layer). */
+int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const void *x_in, void *x_out,
+                         void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
+                         int batch, void *stream);
+
+/* Whole stack, one token per sequence: embedding gather -> n_layers layers ->
+ * final RMSNorm -> logits -> greedy argmax (lowest index on ties).
+ *   embed [V,D]; layers: HOST array [n_layers]; g_final [D]; w_lm_head packed;
+ *   k_caches, v_caches: HOST arrays [n_layers] of device cache pointers;
+ *   token_ids [B] int32 device; pos, seq_lens [B] int32 device, each advanced by
+ *   one at the end of the step iff advance != 0;
+ *   logits [B,V] float device or NULL (an internal buffer is used);
+ *   next_ids [B] int32 device (may be the same buffer as token_ids). */
+int fasttps_model_decode(fasttps_ctx *ctx, const void *embed, const fasttps_layer_weights *layers,
+                         const void *g_final, const void *w_lm_head,
+                         void *const *k_caches, void *const *v_caches,
+                         const int32_t *token_ids, int32_t *pos, int32_t *seq_lens,
+                         float *logits, int32_t *next_ids, int batch, int advance, void *stream);
+
+/* End-to-end variant with HOST token buffers: copies host_token_ids [B] to the
+ * device, runs fasttps_model_decode(advance = 1) on `stream`, copies next ids
+ * back into host_next_ids [B] and synchronises the stream.  pos/seq_lens stay
+ * on the device. */
+int fasttps_model_decode_host(fasttps_ctx *ctx, const void *embed, const fasttps_layer_weights *layers,
+                              const void *g_final, const void *w_lm_head,
+                              void *const *k_caches, void *const *v_caches,
+                              const int32_t *host_token_ids, int32_t *pos, int32_t *seq_lens,
+                              int32_t *host_next_ids, int batch, void *stream);
+
+/* Synchronises the device and returns the status word (then clears it). */
+int fasttps_get_status(fasttps_ctx *ctx, uint32_t *host_status);
+/* Optional per-launch timing for benchmarks: while enabled, every kernel launch of this
+ * context is bracketed by CUDA events on its stream (up to 8192 launches; not usable during
+ * stream capture).  fasttps_profile_read() synchronises and sums the elapsed time and the
+ * launch count per kernel class into arrays of FASTTPS_PROFILE_CLASSES entries, in the order
+ * qkv projection, attention, output projection, fused MLP, lm_head, embedding gather. */
+#define FASTTPS_PROFILE_CLASSES 6
+int fasttps_profile(fasttps_ctx *ctx, int enable);
+int fasttps_profile_read(fasttps_ctx *ctx, double *ms_per_class, uint64_t *launches_per_class);
+/* Number of kernels this context has launched so far (host counter). */
+uint64_t fasttps_launch_count(const fasttps_ctx *ctx);
+/* Split count the attention kernel would use for this batch (for tests/benchmarks). */
+int fasttps_attn_splits(const fasttps_ctx *ctx, int batch);
+const char *fasttps_strerror(int code);
+/* Text of the last CUDA error seen by this thread inside the library ("" if none). */
+const char *fasttps_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASTTPS_H */

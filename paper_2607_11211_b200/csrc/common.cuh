@@ -1,0 +1,242 @@
+// Shared device helpers and the context layout of the FastTPS decode library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/fasttps.h"
+
+namespace fasttps {
+
+constexpr int kMaxNB = 8;            // batch rows one weight pass serves
+constexpr int kMaxSplits = 32;       // split-KV partitions per (sequence, head)
+constexpr unsigned kFull = 0xffffffffu;
+
+// ------------------------------------------------------------------ context
+
+struct Ctx {
+    fasttps_config cfg;
+    int n_sm;
+    cudaDeviceProp prop;
+    // device workspace
+    float *cos_tab, *sin_tab;        // [max_seq][d/2]
+    float *attn_part;                // [max_batch][Hq][kMaxSplits][d + 2]
+    int *attn_ticket;                // [max_batch][Hq]
+    float *mlp_acc;                  // [max_batch][D] FP32, kept at zero between calls
+    int *mlp_ticket;                 // [1]
+    float *amax_val;                 // [max_batch][n_cta] lm_head argmax partials
+    int *amax_idx;
+    int *amax_ticket;
+    uint32_t *status;                // device status word
+    // activation scratch of the chains
+    __nv_bfloat16 *qkv;              // [max_batch][(Hq+2Hkv) d]
+    __nv_bfloat16 *attn_out;         // [max_batch][Hq d]
+    __nv_bfloat16 *h;                // [max_batch][D]
+    __nv_bfloat16 *xa, *xb;          // [max_batch][D]
+    float *logits;                   // [max_batch][V]
+    int32_t *tok;                    // [max_batch] staging for the host-buffer entry point
+    int32_t *pinned_tok;             // pinned host staging [2][max_batch]
+    uint64_t launches;
+    // optional per-launch timing (CUDA events on the launch stream), off by default
+    bool prof_on;
+    int prof_n;                      // event pairs used
+    cudaEvent_t *prof_ev;            // [2 * kProfMax]
+    unsigned char *prof_cls;         // kernel class of each pair
+};
+
+constexpr int kProfMax = 8192;
+enum ProfClass { kProfQkv = 0, kProfAttn, kProfOproj, kProfMlp, kProfLmHead, kProfEmbed, kProfClasses };
+
+// Brackets one kernel launch with events when profiling is on.
+struct ProfScope {
+    Ctx *c; cudaStream_t st; int slot;
+    ProfScope(Ctx *c_, int cls, cudaStream_t st_) : c(c_), st(st_), slot(-1)
+    {
+        if (c->prof_on && c->prof_n < kProfMax) {
+            slot = c->prof_n++;
+            c->prof_cls[slot] = (unsigned char)cls;
+            cudaEventRecord(c->prof_ev[2 * slot], st);
+        }
+    }
+    ~ProfScope() { if (slot >= 0) cudaEventRecord(c->prof_ev[2 * slot + 1], st); }
+};
+
+void set_last_error(cudaError_t e, const char *where);
+
+#define FT_CUDA(call)                                                   \
+    do {                                                                \
+        cudaError_t e__ = (call);                                       \
+        if (e__ != cudaSuccess) {                                       \
+            ::fasttps::set_last_error(e__, #call);                      \
+            return FASTTPS_CUDA_ERROR;                                  \
+        }                                                               \
+    } while (0)
+
+// --------------------------------------------------------------- bf16 / loads
+
+__device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// 8 bf16 (one 16-byte vector) -> 8 floats
+__device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8])
+{
+    f[0] = bf_lo(v.x); f[1] = bf_hi(v.x);
+    f[2] = bf_lo(v.y); f[3] = bf_hi(v.y);
+    f[4] = bf_lo(v.z); f[5] = bf_hi(v.z);
+    f[6] = bf_lo(v.w); f[7] = bf_hi(v.w);
+}
+
+__device__ __forceinline__ uint32_t pack2(float a, float b)
+{
+    __nv_bfloat162 t = __floats2bfloat162_rn(a, b);   // a -> low half, b -> high half
+    return *reinterpret_cast<uint32_t *>(&t);
+}
+
+__device__ __forceinline__ float bf16_round(float a)
+{
+    return __bfloat162float(__float2bfloat16_rn(a));
+}
+
+// 2^x with the hardware approximation (2 ulp); exp2(-inf) = 0
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// streaming 16-byte load: read-only path, do not keep in L1
+__device__ __forceinline__ uint4 ldg_stream(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// L2-coherent loads for data other CTAs produced in this kernel
+__device__ __forceinline__ float ld_cg_f32(const float *p)
+{
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ int ld_cg_s32(const int *p)
+{
+    int v;
+    asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void red_add_v4(float *p, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+// Programmatic dependent launch: wait for the producers of this kernel's inputs /
+// let the next kernel in the stream start its independent prologue.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// ------------------------------------------------------- warp multi-reduction
+
+// Sums V per-lane values over the 32 lanes of a warp with a halving butterfly.
+// On return v[0] of lane l holds the full sum of value index
+//   which = (l >> (5 - log2 V)) for V <= 32,
+// replicated over the lanes that share it.  V is a power of two, 1 <= V <= 32.
+template <int V>
+__device__ __forceinline__ float warp_multi_reduce(float (&v)[V], int lane)
+{
+    static_assert(V >= 1 && V <= 32 && (V & (V - 1)) == 0, "V must be a power of two <= 32");
+    int s = 16;
+#pragma unroll
+    for (int n = V; n > 1; n >>= 1, s >>= 1) {
+        const int half = n >> 1;
+        const bool upper = (lane & s) != 0;
+#pragma unroll
+        for (int i = 0; i < half; ++i) {
+            float send = upper ? v[i] : v[i + half];
+            float keep = upper ? v[i + half] : v[i];
+            v[i] = keep + __shfl_xor_sync(kFull, send, s);
+        }
+    }
+#pragma unroll
+    for (; s >= 1; s >>= 1) v[0] += __shfl_xor_sync(kFull, v[0], s);
+    return v[0];
+}
+
+template <int V>
+__device__ __forceinline__ int warp_multi_which(int lane)
+{
+    int sh = 5;
+#pragma unroll
+    for (int n = V; n > 1; n >>= 1) --sh;
+    return V == 1 ? 0 : (lane >> sh);
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(kFull, v, s);
+    return v;
+}
+
+// ---------------------------------------------------------------- launchers
+
+struct LinearArgs {
+    const __nv_bfloat16 *x;      // [B][in] rows of stride x_stride
+    int x_stride;
+    const __nv_bfloat16 *g;      // [in] gain or null
+    float eps;
+    const __nv_bfloat16 *w;      // [out][in]
+    const __nv_bfloat16 *res;    // [B][out] (stride res_stride) or null
+    int res_stride;
+    __nv_bfloat16 *out_bf16;     // [B][out] (stride out_stride) or null
+    float *out_f32;              // [B][out] or null
+    int out_stride;
+    int n_in, n_out, batch;
+    // optional greedy argmax over out (lm_head)
+    float *amax_val;
+    int *amax_idx;
+    int *amax_ticket;
+    int32_t *next_ids;
+    int32_t *adv_pos, *adv_len;  // advanced by one by the argmax finaliser when non-null
+    int prof_class;
+};
+
+struct AttnArgs {
+    const __nv_bfloat16 *q, *k_new, *v_new;
+    int q_stride, kv_stride;          // elements between consecutive sequences
+    __nv_bfloat16 *k_cache, *v_cache;
+    const int32_t *pos, *seq_lens;
+    __nv_bfloat16 *out;
+    int out_stride;
+    int batch, n_q_heads, n_kv_heads, head_dim, max_seq, n_splits;
+    const float *cos_tab, *sin_tab;
+    float *part;
+    int *ticket;
+    uint32_t *status;
+};
+
+struct MlpArgs {
+    const __nv_bfloat16 *x;      // [B][D]
+    const __nv_bfloat16 *g;      // [D] gain or null (norm prologue)
+    float eps;
+    const __nv_bfloat16 *w_gu;   // packed [2K][D]
+    const __nv_bfloat16 *w_down; // [K][D]
+    const __nv_bfloat16 *res;    // [B][D] residual or null
+    __nv_bfloat16 *out;          // [B][D]
+    int D, K, batch;
+    float *acc;                  // [B][D] FP32 zero on entry, zero on exit
+    int *ticket;
+};
+
+int launch_linear(Ctx *c, const LinearArgs &a, cudaStream_t st);
+int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st);
+int launch_mlp(Ctx *c, const MlpArgs &a, cudaStream_t st);
+int launch_embed(Ctx *c, const __nv_bfloat16 *embed, const int32_t *ids, __nv_bfloat16 *x, int batch, cudaStream_t st);
+int launch_pack(Ctx *c, int kind, const void *src, void *dst, bool inverse, cudaStream_t st);
+int attn_splits_for(const Ctx *c, int batch);
+
+}  // namespace fasttps

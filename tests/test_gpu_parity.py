@@ -1,0 +1,408 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.
+
+Bars: cache elements not written this step bit-exact; appended K/V rows within 1 bf16 ulp;
+outputs |gpu - oracle| <= 2e-2 + 2e-2 |oracle|; integer-valued cases bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2607_11211_b200 import workload as wl
+from tests.helpers import assert_close_bits, from_bf16_bits as F32, to_bf16_bits as B16, ulp_distance
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fb():
+    from paper_2607_11211_b200 import binding, build
+    build.build()
+    return binding
+
+
+def dev(bits):
+    return wl.from_bits(bits, "cuda")
+
+
+def i32(a):
+    return torch.tensor(np.asarray(a, dtype=np.int32), device="cuda")
+
+
+def make_ctx(fb, dims, max_batch, max_seq, n_layers=None):
+    return fb.Context.from_dims(dims, max_batch, max_seq, n_layers=n_layers)
+
+
+# ------------------------------------------------------------------ packing
+
+@pytest.mark.parametrize("dims", [wl.TINY, wl.SMALL_GQA])
+def test_pack_unpack_round_trip_and_interlace(fb, dims):
+    ctx = make_ctx(fb, dims, 1, 64)
+    w = wl.layer_weights(dims, 0, device="cuda")
+    lm = wl.normal_bf16(1, 2, (dims.vocab, dims.hidden), 0.02, device="cuda")
+    for kind, t in ((fb.W_QKV, w["w_qkv"]), (fb.W_O, w["w_o"]), (fb.W_GATE_UP, w["w_gu"]), (fb.W_DOWN, w["w_down"]),
+                    (fb.W_LM_HEAD, lm)):
+        p = ctx.pack_weight(kind, t)
+        back = ctx.unpack_weight(kind, p, t.shape)
+        assert torch.equal(back.view(torch.int16), t.view(torch.int16)), kind
+    # the packed gate_up rows are the logical columns interlaced in blocks of 8 (gate block, up block)
+    K, D = dims.inter, dims.hidden
+    p = ctx.pack_weight(fb.W_GATE_UP, w["w_gu"]).view(2 * K, D)
+    r = torch.arange(2 * K, device="cuda")
+    col = ((r // 8) % 2) * K + (r // 16) * 8 + r % 8
+    assert torch.equal(p.view(torch.int16), w["w_gu"].t()[col].contiguous().view(torch.int16))
+    assert torch.equal(ctx.pack_weight(fb.W_QKV, w["w_qkv"]).view(-1, D).view(torch.int16),
+                       w["w_qkv"].t().contiguous().view(torch.int16))
+    ctx.close()
+
+
+# ------------------------------------------------------------------- linear
+
+@pytest.mark.parametrize("dims,batch", [(wl.TINY, 1), (wl.SMALL, 3), (wl.SMALL_GQA, 8), (wl.SMALL, 11),
+                                        (wl.PHI3_MINI, 1), (wl.PHI3_MINI, 2)])
+def test_linear_decode_matches_oracle(fb, dims, batch):
+    ctx = make_ctx(fb, dims, batch, 64)
+    w = wl.layer_weights(dims, 0, device="cuda")
+    act = wl.activations(dims, batch, device="cuda")
+    nq = dims.n_q_heads * dims.head_dim
+    # QKV with the norm prologue
+    out = torch.zeros(batch, dims.qkv_out, dtype=torch.bfloat16, device="cuda")
+    ctx.linear_decode(fb.W_QKV, act["x"], w["g_attn"], ctx.pack_weight(fb.W_QKV, w["w_qkv"]), None, out, None)
+    n1 = orc.rmsnorm(wl.bits(act["x"]), wl.bits(w["g_attn"]), dims.rms_eps)
+    want = orc.f64_to_bf16(orc.gemv(n1, wl.bits(w["w_qkv"])))
+    assert_close_bits(wl.bits(out), want, what="qkv")
+    # output projection with residual, input = q activations flattened
+    a_in = act["q"].reshape(batch, nq).contiguous()
+    out = torch.zeros(batch, dims.hidden, dtype=torch.bfloat16, device="cuda")
+    ctx.linear_decode(fb.W_O, a_in, None, ctx.pack_weight(fb.W_O, w["w_o"]), act["x"], out, None)
+    want = orc.f64_to_bf16(orc.gemv(wl.bits(a_in), wl.bits(w["w_o"])) + F32(wl.bits(act["x"])).astype(np.float64))
+    assert_close_bits(wl.bits(out), want, what="o_proj")
+    # logits in FP32
+    if dims.vocab:
+        lm = wl.normal_bf16(wl.MASTER_SEED, wl.tid("w_lm"), (dims.vocab, dims.hidden), 0.02, device="cuda")
+        lg = torch.zeros(batch, dims.vocab, dtype=torch.float32, device="cuda")
+        ctx.linear_decode(fb.W_LM_HEAD, act["x"], w["g_mlp"], ctx.pack_weight(fb.W_LM_HEAD, lm), None, None, lg)
+        nf = orc.rmsnorm(wl.bits(act["x"]), wl.bits(w["g_mlp"]), dims.rms_eps)
+        want = orc.gemv_t(nf, wl.bits(lm))
+        got = lg.cpu().numpy().astype(np.float64)
+        assert (np.abs(got - want) <= 2e-2 + 2e-2 * np.abs(want)).all()
+        assert np.abs(got - want).max() < 1e-3            # FP32 accumulation is far inside the bar
+    assert ctx.get_status() == 0
+    ctx.close()
+
+
+def test_linear_integer_inputs_are_bit_exact(fb):
+    # small integers: every partial sum is exact in FP32 whatever the order of summation
+    dims = wl.SMALL
+    ctx = make_ctx(fb, dims, 4, 64)
+    rng = np.random.default_rng(3)
+    x = B16(rng.integers(-2, 3, (4, dims.hidden)))
+    W = B16(rng.integers(-1, 2, (dims.hidden, dims.qkv_out)))
+    out = torch.zeros(4, dims.qkv_out, dtype=torch.bfloat16, device="cuda")
+    ctx.linear_decode(fb.W_QKV, dev(x), None, ctx.pack_weight(fb.W_QKV, dev(W)), None, out, None)
+    want = orc.f64_to_bf16(orc.gemv(x, W))
+    assert (wl.bits(out) == want).all()
+    # column-index weights catch a permuted packing
+    Wc = B16(np.tile(np.arange(dims.qkv_out) % 7, (dims.hidden, 1)))
+    ctx.linear_decode(fb.W_QKV, dev(x), None, ctx.pack_weight(fb.W_QKV, dev(Wc)), None, out, None)
+    assert (wl.bits(out) == orc.f64_to_bf16(orc.gemv(x, Wc))).all()
+    ctx.close()
+
+
+# ---------------------------------------------------------------- attention
+
+def run_attn_case(fb, dims, lens, max_seq, pos=None, seed=wl.MASTER_SEED, nan_tail=True):
+    batch = len(lens)
+    lens = np.asarray(lens, np.int32)
+    pos = lens if pos is None else np.asarray(pos, np.int32)
+    ctx = make_ctx(fb, dims, batch, max_seq)
+    act = wl.activations(dims, batch, seed, device="cuda")
+    kc, vc = wl.kv_cache(dims, 0, batch, max_seq, seed, device="cuda")
+    if nan_tail:                                   # rows past the new one must never be read
+        for b in range(batch):
+            kc[b, :, lens[b] + 1:] = float("nan")
+            vc[b, :, lens[b] + 1:] = float("nan")
+    k0, v0 = wl.bits(kc), wl.bits(vc)
+    out = torch.zeros(batch, dims.n_q_heads, dims.head_dim, dtype=torch.bfloat16, device="cuda")
+    ctx.attn_decode(act["q"], act["k_new"], act["v_new"], kc, vc, i32(pos), i32(lens), out)
+    torch.cuda.synchronize()
+    assert ctx.get_status() == 0
+    ko, vo = k0.copy(), v0.copy()
+    want = orc.attn_decode(wl.bits(act["q"]), wl.bits(act["k_new"]), wl.bits(act["v_new"]), ko, vo, pos, lens,
+                           dims.rope_theta)
+    kg, vg = wl.bits(kc), wl.bits(vc)
+    # rows not written this step: bit-exact (raw 16-bit compare, NaN payloads included)
+    mask = np.ones(kg.shape, bool)
+    for b in range(batch):
+        mask[b, :, lens[b]] = False
+    assert (kg[mask] == k0[mask]).all() and (vg[mask] == v0[mask]).all()
+    for b in range(batch):
+        assert (vg[b, :, lens[b]] == wl.bits(act["v_new"])[b]).all()               # V row: bit copy
+        assert ulp_distance(kg[b, :, lens[b]], ko[b, :, lens[b]]).max() <= 1       # K row: 1 ulp
+        assert (kg[b, :, lens[b]] == ko[b, :, lens[b]]).mean() > 0.999
+    assert_close_bits(wl.bits(out), want, what=f"attn out lens={lens.tolist()}")
+    rel = np.abs(F32(wl.bits(out)).astype(np.float64) - F32(want)).max() / max(1e-9, np.sqrt((F32(want).astype(np.float64) ** 2).mean()))
+    assert rel < 0.05, rel
+    # a second call with the same inputs rewrites the same row with the same bits
+    out2 = torch.zeros_like(out)
+    ctx.attn_decode(act["q"], act["k_new"], act["v_new"], kc, vc, i32(pos), i32(lens), out2)
+    torch.cuda.synchronize()
+    assert (wl.bits(kc) == kg).all() and (wl.bits(vc) == vg).all()
+    assert_close_bits(wl.bits(out2), want, what="attn second call")
+    ctx.close()
+
+
+@pytest.mark.parametrize("L", [0, 1, 7, 15, 16, 17, 63, 64, 65, 257, 1000])
+def test_attn_decode_lengths_head_dim_32(fb, L):
+    run_attn_case(fb, wl.TINY, [L], 1024 if L < 1000 else 1001)
+
+
+@pytest.mark.parametrize("dims", [wl.SMALL, wl.SMALL_GQA])
+def test_attn_decode_ragged_batches(fb, dims):
+    run_attn_case(fb, dims, [0, 5, 130, 64, 299, 31, 200], 300)
+    run_attn_case(fb, dims, [77, 3], 128, pos=[100, 0])          # position differs from the length
+
+
+@pytest.mark.parametrize("lens", [[256], [4095], [1024, 1, 2500]])
+def test_attn_decode_phi3_shape(fb, lens):
+    run_attn_case(fb, wl.PHI3_MINI, lens, 4096)
+
+
+def test_attn_decode_batch_32_uses_a_single_split_path(fb):
+    run_attn_case(fb, wl.SMALL, list(range(1, 330, 10))[:32], 384)
+
+
+def test_attn_decode_rejects_full_cache_and_bad_position_without_writing(fb):
+    dims, max_seq = wl.TINY, 64
+    ctx = make_ctx(fb, dims, 3, max_seq)
+    act = wl.activations(dims, 3, device="cuda")
+    kc, vc = wl.kv_cache(dims, 0, 3, max_seq, device="cuda")
+    k0, v0 = wl.bits(kc), wl.bits(vc)
+    sentinel = torch.full((3, dims.n_q_heads, dims.head_dim), 7.0, dtype=torch.bfloat16, device="cuda")
+    out = sentinel.clone()
+    lens, pos = [max_seq, 10, 20], [5, -1, 20]
+    ctx.attn_decode(act["q"], act["k_new"], act["v_new"], kc, vc, i32(pos), i32(lens), out)
+    st = ctx.get_status()
+    assert st & fb.DEV_CACHE_FULL and st & fb.DEV_BAD_POSITION
+    kg, vg = wl.bits(kc), wl.bits(vc)
+    assert (kg[:2] == k0[:2]).all() and (vg[:2] == v0[:2]).all()
+    assert torch.equal(out[:2], sentinel[:2])
+    assert not torch.equal(out[2], sentinel[2]) and (kg[2, :, 20] != k0[2, :, 20]).any()
+    assert ctx.get_status() == 0                       # reading clears the word
+    ctx.close()
+
+
+def test_attn_decode_planted_key_and_last_row_of_the_cache(fb):
+    # structured O(1) outputs: one cached key per head is a large multiple of rope(q)
+    dims, max_seq = wl.SMALL, 128
+    L = max_seq - 1                                    # the append lands in the very last row
+    ctx = make_ctx(fb, dims, 2, max_seq)
+    act = wl.activations(dims, 2, device="cuda")
+    kc, vc = wl.kv_cache(dims, 0, 2, max_seq, device="cuda")
+    kb, vb, q = wl.bits(kc), wl.bits(vc), wl.bits(act["q"])
+    for b in range(2):
+        for h in range(dims.n_q_heads):
+            qr = orc.rope(F32(q[b, h]), L)
+            j = (17 * b + 5 * h) % L
+            kb[b, h, j] = B16(qr * (60.0 / float(qr @ qr)) * np.sqrt(dims.head_dim))
+            vb[b, h, j] = B16(np.full(dims.head_dim, 10.0 * (b * dims.n_q_heads + h + 1)))
+    kc, vc = dev(kb), dev(vb)
+    out = torch.zeros(2, dims.n_q_heads, dims.head_dim, dtype=torch.bfloat16, device="cuda")
+    ctx.attn_decode(act["q"], act["k_new"], act["v_new"], kc, vc, i32([L, L]), i32([L, L]), out)
+    want = orc.attn_decode(q, wl.bits(act["k_new"]), wl.bits(act["v_new"]), kb, vb, [L, L], [L, L])
+    assert_close_bits(wl.bits(out), want, what="planted")
+    o = out.float().cpu().numpy()
+    for b in range(2):
+        for h in range(dims.n_q_heads):
+            assert np.allclose(o[b, h], 10.0 * (b * dims.n_q_heads + h + 1), rtol=2e-2)
+    assert (wl.bits(kc)[:, :, L] == kb[:, :, L]).all()
+    ctx.close()
+
+
+# ---------------------------------------------------------------------- MLP
+
+@pytest.mark.parametrize("dims,batch", [(wl.TINY, 1), (wl.SMALL, 2), (wl.SMALL, 3), (wl.SMALL_GQA, 5), (wl.SMALL, 8),
+                                        (wl.SMALL, 9), (wl.SMALL, 19), (wl.PHI3_MINI, 1), (wl.PHI3_MINI, 4)])
+def test_mlp_decode_matches_oracle(fb, dims, batch):
+    ctx = make_ctx(fb, dims, batch, 64)
+    w = wl.layer_weights(dims, 1, device="cuda")
+    x = wl.activations(dims, batch, device="cuda")["x"]
+    # scale the weights up so the outputs are O(1), well above the absolute part of the bar
+    wgu = (w["w_gu"].float() * 4).to(torch.bfloat16)
+    wdn = (w["w_down"].float() * 4).to(torch.bfloat16)
+    pg, pd = ctx.pack_weight(fb.W_GATE_UP, wgu), ctx.pack_weight(fb.W_DOWN, wdn)
+    out = torch.full((batch, dims.hidden), 3.0, dtype=torch.bfloat16, device="cuda")
+    ctx.mlp_decode(x, pg, pd, out)
+    want = orc.mlp_decode(wl.bits(x), wl.bits(wgu), wl.bits(wdn))
+    assert_close_bits(wl.bits(out), want, what="mlp")
+    err = np.abs(F32(wl.bits(out)).astype(np.float64) - F32(want))
+    assert err.max() <= 2.0 ** -7 * max(1.0, np.abs(F32(want)).max())      # about one output rounding
+    # the workspace accumulator is back at zero: a second call gives the same answer
+    out2 = torch.zeros_like(out)
+    ctx.mlp_decode(x, pg, pd, out2)
+    assert_close_bits(wl.bits(out2), want, what="mlp second call")
+    ctx.close()
+
+
+def test_mlp_zero_weights_and_identity_construction(fb):
+    dims = wl.Dims(hidden=64, n_q_heads=2, n_kv_heads=2, head_dim=32, inter=64, vocab=0, n_layers=0)
+    ctx = make_ctx(fb, dims, 2, 64)
+    x = wl.activations(dims, 2, device="cuda")["x"]
+    D = dims.hidden
+    z_gu = torch.zeros(D, 2 * D, dtype=torch.bfloat16, device="cuda")
+    rnd_dn = wl.normal_bf16(5, 6, (D, D), 1.0, device="cuda")
+    out = torch.full((2, D), 3.0, dtype=torch.bfloat16, device="cuda")
+    ctx.mlp_decode(x, ctx.pack_weight(fb.W_GATE_UP, z_gu), ctx.pack_weight(fb.W_DOWN, rnd_dn), out)
+    assert (out == 0).all()
+    # W_gate = 2 I, W_up = W_down = I  =>  y_i = silu(2 x_i) x_i
+    eye = torch.eye(D, device="cuda")
+    gu = torch.cat([2 * eye, eye], dim=1).to(torch.bfloat16)
+    ctx.mlp_decode(x, ctx.pack_weight(fb.W_GATE_UP, gu), ctx.pack_weight(fb.W_DOWN, eye.to(torch.bfloat16)), out)
+    xv = x.double().cpu().numpy()
+    want = (2 * xv) / (1 + np.exp(-2 * xv)) * xv
+    assert_close_bits(wl.bits(out), orc.f64_to_bf16(want), what="identity mlp")
+    assert_close_bits(wl.bits(out), orc.mlp_decode(wl.bits(x), wl.bits(gu), wl.bits(eye.to(torch.bfloat16))))
+    ctx.close()
+
+
+# -------------------------------------------------------------------- layer
+
+def k_rows_ok(got, want, half):
+    """Appended K rows when the projection that feeds them is inside the call: the two sides may
+    round k to different neighbouring bf16 values before the rotation, which moves the rotated pair
+    by up to about one ulp at the magnitude of the pair."""
+    d1 = ulp_distance(got, want) <= 1
+    g, w = F32(got).astype(np.float64), F32(want).astype(np.float64)
+    pair = np.sqrt(w[..., :half] ** 2 + w[..., half:] ** 2)
+    pair = np.concatenate([pair, pair], axis=-1)
+    return d1 | (np.abs(g - w) <= 2.0 ** -7 * pair)
+
+
+def run_layer_case(fb, dims, lens, max_seq, layer=0):
+    batch = len(lens)
+    lens = np.asarray(lens, np.int32)
+    ctx = make_ctx(fb, dims, batch, max_seq)
+    w = wl.layer_weights(dims, layer, device="cuda")
+    pw = ctx.pack_layer(w)
+    x = wl.activations(dims, batch, device="cuda")["x"]
+    kc, vc = wl.kv_cache(dims, layer, batch, max_seq, device="cuda")
+    k0, v0 = wl.bits(kc), wl.bits(vc)
+    xo = torch.zeros_like(x)
+    ctx.layer_decode(pw["struct"], x, xo, kc, vc, i32(lens), i32(lens))
+    torch.cuda.synchronize()
+    assert ctx.get_status() == 0
+    ko, vo = k0.copy(), v0.copy()
+    wb = {k: wl.bits(v) for k, v in w.items()}
+    want = orc.layer_decode(wb, wl.bits(x), ko, vo, lens, lens, dims.rms_eps, dims.rope_theta)
+    kg, vg = wl.bits(kc), wl.bits(vc)
+    mask = np.ones(kg.shape, bool)
+    for b in range(batch):
+        mask[b, :, lens[b]] = False
+    assert (kg[mask] == k0[mask]).all() and (vg[mask] == v0[mask]).all()
+    for b in range(batch):
+        assert ulp_distance(vg[b, :, lens[b]], vo[b, :, lens[b]]).max() <= 1
+        assert k_rows_ok(kg[b, :, lens[b]], ko[b, :, lens[b]], dims.head_dim // 2).all()
+        assert (ulp_distance(kg[b, :, lens[b]], ko[b, :, lens[b]]) <= 1).mean() > 0.99
+    assert_close_bits(wl.bits(xo), want, what=f"layer out lens={lens.tolist()}")
+    # in place (x_out aliases x_in)
+    x2 = x.clone()
+    kc2, vc2 = dev(k0), dev(v0)
+    ctx.layer_decode(pw["struct"], x2, x2, kc2, vc2, i32(lens), i32(lens))
+    assert_close_bits(wl.bits(x2), want, what="layer in place")
+    ctx.close()
+
+
+@pytest.mark.parametrize("dims,lens", [(wl.TINY, [0]), (wl.TINY, [5, 64, 17]), (wl.SMALL, [100, 3, 250, 64, 65]),
+                                       (wl.SMALL_GQA, [9, 200]), (wl.SMALL, list(range(20, 240, 20)))])
+def test_layer_decode_small_shapes(fb, dims, lens):
+    run_layer_case(fb, dims, lens, 256)
+
+
+@pytest.mark.parametrize("lens", [[256], [4095]])
+def test_layer_decode_phi3_single_layer_configs(fb, lens):
+    # the two single-layer workloads: 256 resp. 4095 past tokens, new token at that position
+    run_layer_case(fb, wl.PHI3_MINI, lens, 4096)
+
+
+# -------------------------------------------------------------------- model
+
+def build_model(fb, ctx, dims, batch, max_seq, device="cuda"):
+    mw = wl.model_weights(dims, device=device)
+    packed = [ctx.pack_layer(w) for w in mw["layers"]]
+    caches = [wl.kv_cache(dims, l, batch, max_seq, device=device) for l in range(dims.n_layers)]
+    kcs, vcs = [c[0] for c in caches], [c[1] for c in caches]
+    model = ctx.make_model(mw["embed"], packed, mw["g_final"], ctx.pack_weight(fb.W_LM_HEAD, mw["w_lm"]), kcs, vcs)
+    return mw, model, kcs, vcs
+
+
+@pytest.mark.parametrize("dims,lens", [(wl.SMALL, [40, 7, 100]), (wl.SMALL_GQA, [3]), (wl.TINY, list(range(1, 11)))])
+def test_model_decode_teacher_forced_steps(fb, dims, lens):
+    batch, max_seq, steps = len(lens), 128, 4
+    ctx = make_ctx(fb, dims, batch, max_seq)
+    mw, model, kcs, vcs = build_model(fb, ctx, dims, batch, max_seq)
+    ok = [wl.bits(t) for t in kcs]
+    ov = [wl.bits(t) for t in vcs]
+    ow = [{k: wl.bits(v) for k, v in L.items()} for L in mw["layers"]]
+    ids = wl.token_ids(batch * steps, dims.vocab).reshape(steps, batch)
+    pos = i32(lens)
+    sl = i32(lens)
+    logits = torch.zeros(batch, dims.vocab, dtype=torch.float32, device="cuda")
+    nxt = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    cur = np.asarray(lens, np.int32).copy()
+    for s in range(steps):
+        ctx.model_decode(model, i32(ids[s]), pos, sl, logits, nxt, advance=True)
+        torch.cuda.synchronize()
+        wlog, wnext = orc.model_decode(wl.bits(mw["embed"]), ow, wl.bits(mw["g_final"]), wl.bits(mw["w_lm"]), ok, ov,
+                                       ids[s], cur, cur, dims.rms_eps, dims.rope_theta)
+        got = logits.cpu().numpy().astype(np.float64)
+        assert (np.abs(got - wlog) <= 2e-2 + 2e-2 * np.abs(wlog)).all(), s
+        # the argmax must agree wherever the oracle's top-2 gap exceeds twice the bar
+        top2 = np.sort(wlog, axis=1)[:, -2:]
+        sure = (top2[:, 1] - top2[:, 0]) > 2 * (2e-2 + 2e-2 * np.abs(top2[:, 1]))
+        g = nxt.cpu().numpy()
+        assert (g[sure] == wnext[sure]).all()
+        assert (got[np.arange(batch), g] >= got.max(axis=1) - 1e-6).all()      # a true maximum of its own logits
+        cur += 1
+        assert (pos.cpu().numpy() == cur).all() and (sl.cpu().numpy() == cur).all()
+        # free-running caches stay within the output bar of the oracle's
+        for l in range(dims.n_layers):
+            for b in range(batch):
+                r = cur[b] - 1
+                assert_close_bits(wl.bits(kcs[l])[b, :, r], ok[l][b, :, r], what="k row")
+                assert_close_bits(wl.bits(vcs[l])[b, :, r], ov[l][b, :, r], what="v row")
+    assert ctx.get_status() == 0
+    ctx.close()
+
+
+def test_model_decode_host_buffers_and_greedy_feedback(fb):
+    dims, batch, max_seq = wl.SMALL, 2, 64
+    ctx = make_ctx(fb, dims, batch, max_seq)
+    mw, model, kcs, vcs = build_model(fb, ctx, dims, batch, max_seq)
+    k0 = [t.clone() for t in kcs]
+    v0 = [t.clone() for t in vcs]
+    start = np.array([11, 500], np.int32)
+    # device path with on-device feedback (next ids buffer is the token buffer)
+    pos, sl = i32([5, 9]), i32([5, 9])
+    tok = i32(start)
+    seq_dev = []
+    for _ in range(3):
+        ctx.model_decode(model, tok, pos, sl, None, tok, advance=True)
+        seq_dev.append(tok.cpu().numpy().copy())
+    # host path from the same initial state
+    for l in range(dims.n_layers):
+        kcs[l].copy_(k0[l]); vcs[l].copy_(v0[l])
+    pos, sl = i32([5, 9]), i32([5, 9])
+    h_in, h_out = start.copy(), np.zeros(batch, np.int32)
+    seq_host = []
+    for _ in range(3):
+        ctx.model_decode_host(model, h_in, pos, sl, h_out)
+        seq_host.append(h_out.copy())
+        h_in = h_out.copy()
+    assert (np.array(seq_dev) == np.array(seq_host)).all()
+    assert (pos.cpu().numpy() == [8, 12]).all()
+    assert ctx.launch_count() > 0
+    # a token id outside the vocabulary is reported, not dereferenced
+    ctx.model_decode(model, i32([dims.vocab + 5, 1]), pos, sl, None, tok, advance=False)
+    assert ctx.get_status() & fb.DEV_BAD_TOKEN
+    ctx.close()
