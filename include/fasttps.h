@@ -48,9 +48,9 @@ typedef enum {
 #define FASTTPS_DEV_WAIT_TIMEOUT 4u   /* a bounded wait on an asynchronous copy ran out         */
 #define FASTTPS_DEV_BAD_TOKEN    8u   /* a token id outside [0, vocab): row 0 used instead      */
 
-/* Model shape and limits.  Supported: hidden % 8 == 0, hidden <= 8192;
+/* Model shape and limits.  Supported: hidden % 8 == 0, hidden <= 6144;
  * head_dim in {32, 64, 96, 128}; n_q_heads % n_kv_heads == 0; inter % 8 == 0;
- * (n_q_heads * head_dim) % 8 == 0 and <= 8192; max_batch >= 1; max_seq >= 1.
+ * (n_q_heads * head_dim) % 8 == 0 and <= 6144; max_batch >= 1; max_seq >= 1.
  * vocab and n_layers may be 0 when only the block-level calls are used. */
 typedef struct {
     int hidden;        /* D                                   */

@@ -20,10 +20,10 @@ static bool aligned16(const void *p) { return p != nullptr && (reinterpret_cast<
 
 static bool config_ok(const fasttps_config &f)
 {
-    if (f.hidden <= 0 || f.hidden % 8 || f.hidden > 8192) return false;
+    if (f.hidden <= 0 || f.hidden % 8 || f.hidden > 6144) return false;
     if (f.head_dim != 32 && f.head_dim != 64 && f.head_dim != 96 && f.head_dim != 128) return false;
     if (f.n_q_heads <= 0 || f.n_kv_heads <= 0 || f.n_q_heads % f.n_kv_heads) return false;
-    if ((f.n_q_heads * f.head_dim) % 8 || f.n_q_heads * f.head_dim > 8192) return false;
+    if ((f.n_q_heads * f.head_dim) % 8 || f.n_q_heads * f.head_dim > 6144) return false;
     if (f.inter <= 0 || f.inter % 8) return false;
     if (f.vocab < 0 || f.n_layers < 0 || f.max_batch < 1 || f.max_seq < 1) return false;
     if (!(f.rms_eps >= 0.f) || !(f.rope_theta > 0.f)) return false;
@@ -72,6 +72,11 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     c->cfg = *cfg;
     FT_CUDA(cudaGetDeviceProperties(&c->prop, cfg->device));
     c->n_sm = c->prop.multiProcessorCount;
+    {
+        int rc = configure_linear_kernels();
+        if (rc == FASTTPS_OK) rc = configure_mlp_kernels();
+        if (rc != FASTTPS_OK) { delete c; return rc; }
+    }
 
     const fasttps_config &f = c->cfg;
     const size_t B = f.max_batch, D = f.hidden, half = f.head_dim / 2;
@@ -215,7 +220,7 @@ static int mlp_impl(Ctx *c, const __nv_bfloat16 *x, const __nv_bfloat16 *g, cons
     a.w_down = static_cast<const __nv_bfloat16 *>(w_down);
     a.res = res; a.out = out;
     a.D = c->cfg.hidden; a.K = c->cfg.inter; a.batch = batch;
-    a.acc = c->mlp_acc; a.ticket = c->mlp_ticket;
+    a.acc = c->mlp_acc; a.ticket = c->mlp_ticket; a.status = c->status;
     return launch_mlp(c, a, st);
 }
 
@@ -237,6 +242,7 @@ static int linear_impl(Ctx *c, int n_in, int n_out, const __nv_bfloat16 *x, int 
 {
     LinearArgs a;
     a.prof_class = prof_class;
+    a.status = c->status;
     a.x = x; a.x_stride = x_stride; a.g = g; a.eps = c->cfg.rms_eps;
     a.w = static_cast<const __nv_bfloat16 *>(w);
     a.res = res; a.res_stride = res_stride;

@@ -10,7 +10,7 @@
 // bulk asynchronous copy (cp.async.bulk, the 1-D TMA path) into a ring of shared-memory
 // stages guarded by mbarriers.  The new row never makes a round trip through global
 // memory: it is scored from registers/shared memory and written to the cache once.
-#include "common.cuh"
+#include "async_copy.cuh"
 
 namespace fasttps {
 
@@ -23,55 +23,6 @@ constexpr int kStages = 3;
 constexpr int kLanesPerRow = 4;
 constexpr int kRowsPerPass = 32 / kLanesPerRow;                  // 8 rows per warp pass
 constexpr int kPasses = kTileRows / (kAttnWarps * kRowsPerPass); // passes per warp per tile
-constexpr uint32_t kWaitPolls = 1u << 22;                        // bounded mbarrier polling: poll count ...
-constexpr unsigned long long kWaitNanos = 400ull * 1000 * 1000;  // ... and wall time (0.4 s)
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t *bar, int count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\t"
-                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                 "selp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long v;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(v));
-    return v;
-}
-// Bounded wait: gives up after kWaitPolls polls or kWaitNanos of wall time, whichever comes
-// first, and reports failure instead of spinning forever.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity)
-{
-    unsigned long long t0 = 0;
-    for (uint32_t i = 0; i < kWaitPolls; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 255u) {
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitNanos) return false;
-        }
-    }
-    return false;
-}
-__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-
 template <int DH>
 struct AttnSmem {
     static constexpr int kRowBytes = DH * 2;

@@ -203,6 +203,7 @@ struct LinearArgs {
     int32_t *next_ids;
     int32_t *adv_pos, *adv_len;  // advanced by one by the argmax finaliser when non-null
     int prof_class;
+    uint32_t *status;
 };
 
 struct AttnArgs {
@@ -230,6 +231,7 @@ struct MlpArgs {
     int D, K, batch;
     float *acc;                  // [B][D] FP32 zero on entry, zero on exit
     int *ticket;
+    uint32_t *status;
 };
 
 int launch_linear(Ctx *c, const LinearArgs &a, cudaStream_t st);
@@ -238,5 +240,7 @@ int launch_mlp(Ctx *c, const MlpArgs &a, cudaStream_t st);
 int launch_embed(Ctx *c, const __nv_bfloat16 *embed, const int32_t *ids, __nv_bfloat16 *x, int batch, cudaStream_t st);
 int launch_pack(Ctx *c, int kind, const void *src, void *dst, bool inverse, cudaStream_t st);
 int attn_splits_for(const Ctx *c, int batch);
+int configure_linear_kernels();
+int configure_mlp_kernels();
 
 }  // namespace fasttps

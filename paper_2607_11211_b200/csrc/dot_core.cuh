@@ -2,21 +2,22 @@
 // gate_up half of the fused MLP kernel.
 //
 // Layout: W is [rows][n_in] bf16 with every row (one output feature) contiguous.
-// A CTA of ceil(n_in / 8 / 32) warps owns a contiguous range of rows.  Thread t
-// owns the 16-byte k-slice [8t, 8t+8) of EVERY row, keeps its slice of the
-// activations in registers (FP32, NB batch rows) and streams the rows with
-// 16-byte read-only loads, R rows per group, two groups in flight.  A warp load
-// is 512 contiguous bytes and a group covers R whole rows, so a CTA walks
-// through its slice of the matrix strictly sequentially.  The R*NB partial sums
-// of a group are reduced with a halving butterfly (about one shuffle per
-// value), meet in shared memory (one __syncthreads per group, double buffered)
-// and are handed to the epilogue by the first R*NB threads.
+// A CTA of ceil(n_in / 8 / 32) warps owns a contiguous range of rows, which is one
+// contiguous byte range of the matrix.  The range arrives through the shared-memory
+// weight ring (bulk asynchronous copies, R rows per group, several groups in
+// flight).  Thread t owns the 16-byte k-slice [8t, 8t+8) of EVERY row and keeps its
+// slice of the activations in registers (FP32, NB batch rows).  The R*NB partial sums
+// of a group are reduced with a halving butterfly (about one shuffle per value), meet
+// in shared memory (one block barrier per group, double buffered) and are handed to
+// the epilogue by the first R*NB threads.
 #pragma once
-#include "common.cuh"
+#include "async_copy.cuh"
 
 namespace fasttps {
 
 template <int NB> struct RowsPerGroup { static constexpr int value = (NB <= 4) ? 8 : 4; };
+
+constexpr int kRingBudget = 192 * 1024;     // shared memory given to the weight ring
 
 // Loads this thread's activation slice: x[b][8t .. 8t+8) for NB batch rows, with an
 // optional RMSNorm (gain g, eps) whose result is rounded to bf16 like a stored tensor.
@@ -72,11 +73,12 @@ __device__ __forceinline__ void load_activations(float (&x)[NB][8], const __nv_b
     __syncthreads();   // smem_red may be reused by the caller
 }
 
-// Streams rows [row0, row1) of W and calls epi(row, b, value) for every row and
-// batch row b < NB, from threads 0 .. R*NB-1 (one (row, b) pair per thread and group).
-// smem_red: 2 * nwarps * R * NB floats.  All threads of the CTA must call.
+// Consumes ring groups [g0, g0 + ceil(nrows / R)) = rows [row0, row0 + nrows) of a matrix and
+// calls epi(row, b, value) for every row and batch row b < NB, from threads 0 .. R*NB-1 (one
+// (row, b) pair per thread and group).  smem_red: 2 * nwarps * R * NB floats.  All threads of
+// the CTA must call.  Returns false if a bounded wait ran out (the CTA must then leave).
 template <int NB, class Epi>
-__device__ __forceinline__ void dot_rows(const __nv_bfloat16 *W, int n_in, int row0, int row1,
+__device__ __forceinline__ bool dot_rows(WeightRing &ring, int g0, int n_in, int row0, int nrows,
                                          const float (&x)[NB][8], float *smem_red, Epi epi)
 {
     constexpr int R = RowsPerGroup<NB>::value;
@@ -84,26 +86,17 @@ __device__ __forceinline__ void dot_rows(const __nv_bfloat16 *W, int n_in, int r
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5, nwarps = (blockDim.x + 31) >> 5;
     const bool active = t * 8 < n_in;
     const int nvec = n_in >> 3;
-    const uint4 *Wv = reinterpret_cast<const uint4 *>(W);
-    const int nrows = row1 - row0;
-    if (nrows <= 0) return;
     const int ngroups = (nrows + R - 1) / R;
-
-    auto load_group = [&](uint4 (&w)[R], int g) {
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            int row = row0 + g * R + r;
-            row = row < row1 ? row : row1 - 1;
-            if (active) w[r] = ldg_stream(Wv + (size_t)row * nvec + t);
-            else w[r] = make_uint4(0, 0, 0, 0);
-        }
-    };
-    auto compute_group = [&](const uint4 (&w)[R], int g, int buf) {
+    bool ok = true;
+    for (int g = 0; g < ngroups; ++g) {
+        const int buf = g & 1;
+        const uint4 *slot = reinterpret_cast<const uint4 *>(ring.wait(g0 + g, ok));
         float p[V];
 #pragma unroll
         for (int r = 0; r < R; ++r) {
             float wf[8];
-            unpack8(w[r], wf);
+            const uint4 w = active ? slot[r * nvec + t] : make_uint4(0, 0, 0, 0);
+            unpack8(w, wf);
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
                 float s = 0.f;
@@ -115,25 +108,16 @@ __device__ __forceinline__ void dot_rows(const __nv_bfloat16 *W, int n_in, int r
         const float tot = warp_multi_reduce<V>(p, lane);
         constexpr int rep = 32 / V;                       // lanes sharing one value
         if ((lane & (rep - 1)) == 0) smem_red[(buf * nwarps + warp) * V + warp_multi_which<V>(lane)] = tot;
-        __syncthreads();
+        if (!__syncthreads_and(ok ? 1 : 0)) return false; // every warp is done with the slot
+        if (t == 0) ring.refill(g0 + g);
         if (t < V) {
             float s = 0.f;
             for (int w2 = 0; w2 < nwarps; ++w2) s += smem_red[(buf * nwarps + w2) * V + t];
-            const int row = row0 + g * R + t / NB;
-            if (row < row1) epi(row, t % NB, s);
-        }
-    };
-
-    uint4 wa[R], wb[R];
-    load_group(wa, 0);
-    for (int g = 0; g < ngroups; g += 2) {
-        if (g + 1 < ngroups) load_group(wb, g + 1);
-        compute_group(wa, g, 0);
-        if (g + 1 < ngroups) {
-            if (g + 2 < ngroups) load_group(wa, g + 2);
-            compute_group(wb, g + 1, 1);
+            const int row = g * R + t / NB;
+            if (row < nrows) epi(row0 + row, t % NB, s);
         }
     }
+    return true;
 }
 
 }  // namespace fasttps

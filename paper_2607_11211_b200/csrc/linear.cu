@@ -3,6 +3,7 @@
 // attention output projection and the logits (Figure 1 of the paper; these
 // products are weight-bound GEMVs at decode time).
 #include "dot_core.cuh"
+#include "stream_launch.cuh"
 
 namespace fasttps {
 
@@ -10,30 +11,44 @@ template <int NB, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1) linear_kernel(LinearArgs a)
 {
     constexpr int R = RowsPerGroup<NB>::value;
-    extern __shared__ float smem[];           // [2][nwarps][R*NB] reduction scratch (>= 32*NB floats)
+    extern __shared__ __align__(128) unsigned char dsm[];
     __shared__ float s_best_val[R * NB];
     __shared__ int s_best_idx[R * NB];
     __shared__ int s_last;
 
     const int t = threadIdx.x;
+    const StreamSmemLayout lay = stream_smem_layout(a.n_in, R, NB, (blockDim.x + 31) >> 5);
+    float *smem = reinterpret_cast<float *>(dsm + lay.red_off);
+
     // contiguous, balanced row range of this CTA
     const int base = a.n_out / gridDim.x, rem = a.n_out % gridDim.x;
     const int cta = blockIdx.x;
     const int row0 = cta * base + (cta < rem ? cta : rem);
-    const int row1 = row0 + base + (cta < rem ? 1 : 0);
+    const int nrows = base + (cta < rem ? 1 : 0);
+
+    // the weights do not depend on the activations: start streaming them first
+    WeightRing ring;
+    ring.init(dsm + lay.ring_off, reinterpret_cast<uint64_t *>(dsm + lay.bar_off), lay.nslot, a.n_in * 2, R,
+              a.w + (size_t)row0 * a.n_in, nrows, nullptr, 0);
+    __syncthreads();
+    if (t == 0) ring.start();
 
     float x[NB][8];
     load_activations<NB>(x, a.x, a.x_stride, a.batch, a.n_in, a.g, a.eps, smem);
 
     float best_val = -INFINITY;
     int best_idx = 0x7fffffff;
-    dot_rows<NB>(a.w, a.n_in, row0, row1, x, smem, [&](int row, int b, float v) {
+    const bool ok = dot_rows<NB>(ring, 0, a.n_in, row0, nrows, x, smem, [&](int row, int b, float v) {
         if (b >= a.batch) return;
         if (a.res) v += __bfloat162float(a.res[(size_t)b * a.res_stride + row]);
         if (a.out_bf16) a.out_bf16[(size_t)b * a.out_stride + row] = __float2bfloat16_rn(v);
         if (a.out_f32) a.out_f32[(size_t)b * a.out_stride + row] = v;
         if (v > best_val) { best_val = v; best_idx = row; }       // rows ascend per thread: first max kept
     });
+    if (!ok) {
+        if (t == 0) { atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT); ring.drain(0); }
+        return;
+    }
 
     if (a.next_ids == nullptr) return;
 
@@ -78,23 +93,43 @@ int linear_grid(const Ctx *c, int n_out)
 }
 
 template <int NB>
+static cudaError_t configure_linear_nb()
+{
+    cudaError_t e = allow_big_smem(linear_kernel<NB, 128>);
+    if (e == cudaSuccess) e = allow_big_smem(linear_kernel<NB, 256>);
+    if (e == cudaSuccess) e = allow_big_smem(linear_kernel<NB, 384>);
+    if (e == cudaSuccess) e = allow_big_smem(linear_kernel<NB, 512>);
+    if (e == cudaSuccess) e = allow_big_smem(linear_kernel<NB, 768>);
+    return e;
+}
+
+int configure_linear_kernels()
+{
+    FT_CUDA(configure_linear_nb<1>());
+    FT_CUDA(configure_linear_nb<2>());
+    FT_CUDA(configure_linear_nb<4>());
+    FT_CUDA(configure_linear_nb<8>());
+    return FASTTPS_OK;
+}
+
+template <int NB>
 static int launch_linear_nb(Ctx *c, const LinearArgs &a, cudaStream_t st)
 {
     constexpr int R = RowsPerGroup<NB>::value;
     const int threads = ((a.n_in / 8) + 31) / 32 * 32;
-    const int nwarps = threads / 32;
-    const size_t smem = sizeof(float) * (size_t)(2 * nwarps * R * NB > 32 * NB ? 2 * nwarps * R * NB : 32 * NB);
+    const StreamSmemLayout lay = stream_smem_layout(a.n_in, R, NB, threads / 32);
+    if (lay.nslot < 2) return FASTTPS_INVALID_ARG;
     const int grid = linear_grid(c, a.n_out);
     ProfScope prof(c, a.prof_class, st);
+    int rc;
     // the register budget follows the block size: one instantiation per size class
-    if (threads <= 128) linear_kernel<NB, 128><<<grid, threads, smem, st>>>(a);
-    else if (threads <= 256) linear_kernel<NB, 256><<<grid, threads, smem, st>>>(a);
-    else if (threads <= 384) linear_kernel<NB, 384><<<grid, threads, smem, st>>>(a);
-    else if (threads <= 512) linear_kernel<NB, 512><<<grid, threads, smem, st>>>(a);
-    else linear_kernel<NB, 1024><<<grid, threads, smem, st>>>(a);
+    if (threads <= 128) rc = launch_stream_kernel(linear_kernel<NB, 128>, grid, threads, lay.total, st, &a);
+    else if (threads <= 256) rc = launch_stream_kernel(linear_kernel<NB, 256>, grid, threads, lay.total, st, &a);
+    else if (threads <= 384) rc = launch_stream_kernel(linear_kernel<NB, 384>, grid, threads, lay.total, st, &a);
+    else if (threads <= 512) rc = launch_stream_kernel(linear_kernel<NB, 512>, grid, threads, lay.total, st, &a);
+    else rc = launch_stream_kernel(linear_kernel<NB, 768>, grid, threads, lay.total, st, &a);
     c->launches++;
-    FT_CUDA(cudaGetLastError());
-    return FASTTPS_OK;
+    return rc;
 }
 
 // Batches above kMaxNB are served in tiles of kMaxNB rows (the weights are re-read per tile).

@@ -12,8 +12,11 @@
 //      accumulates y[:, 8t..8t+8) += a_j * W_down[j, 8t..8t+8) in registers,
 //   4. adds its partial y into an FP32 accumulator in global memory (vector red.add); the
 //      CTA that arrives last adds the residual, rounds to bf16 and re-zeroes the accumulator.
-// Both weight streams are strictly sequential per CTA.
+// Both weight slices of a CTA are contiguous byte ranges and go through ONE shared-memory
+// ring of bulk asynchronous copies, so the W_down rows are already in flight while the
+// gate_up reduction and the SiLU step are still running.
 #include "dot_core.cuh"
+#include "stream_launch.cuh"
 
 namespace fasttps {
 
@@ -21,37 +24,48 @@ namespace {
 
 constexpr int kMaxOctetsPerCta = 16;      // bounds the shared-memory intermediate
 
-template <int NB> struct DownUnroll { static constexpr int value = (NB <= 2) ? 8 : 4; };
-
 template <int NB, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1) mlp_decode_kernel(MlpArgs a)
 {
-    constexpr int U = DownUnroll<NB>::value;
-    extern __shared__ float smem[];                         // reduction scratch of dot_rows
+    constexpr int R = RowsPerGroup<NB>::value;               // rows per ring group, both phases
+    extern __shared__ __align__(128) unsigned char dsm[];
     __shared__ float s_gu[kMaxOctetsPerCta * 16][NB];       // gate/up values of this CTA's rows
     __shared__ float s_act[kMaxOctetsPerCta * 8][NB];       // silu(gate) * up
     __shared__ int s_last;
 
     const int t = threadIdx.x;
+    const StreamSmemLayout lay = stream_smem_layout(a.D, R, NB, (blockDim.x + 31) >> 5);
+    float *smem = reinterpret_cast<float *>(dsm + lay.red_off);
+
     const int n_oct = a.K >> 3;
     const int base = n_oct / gridDim.x, rem = n_oct % gridDim.x;
     const int cta = blockIdx.x;
     const int oct0 = cta * base + (cta < rem ? cta : rem);
     const int noct = base + (cta < rem ? 1 : 0);
     const bool active = t * 8 < a.D;
+    const int row0 = oct0 * 16, nrows_gu = noct * 16, nj = noct * 8;
+
+    // both weight slices of this CTA, back to back through one ring
+    WeightRing ring;
+    ring.init(dsm + lay.ring_off, reinterpret_cast<uint64_t *>(dsm + lay.bar_off), lay.nslot, a.D * 2, R,
+              a.w_gu + (size_t)row0 * a.D, nrows_gu, a.w_down + (size_t)oct0 * 8 * a.D, nj);
+    __syncthreads();
+    if (t == 0) ring.start();
 
     // ---- Algorithm 4 step 1 (optional): RMSNorm of the block input ----
     float x[NB][8];
     load_activations<NB>(x, a.x, a.D, a.batch, a.D, a.g, a.eps, smem);
 
     // ---- steps 2-10: interlaced gate_up product for rows [16*oct0, 16*(oct0+noct)) ----
-    const int row0 = oct0 * 16;
-    dot_rows<NB>(a.w_gu, a.D, row0, row0 + noct * 16, x, smem,
-                 [&](int row, int b, float v) { s_gu[row - row0][b] = v; });
+    bool ok = dot_rows<NB>(ring, 0, a.D, 0, nrows_gu, x, smem, [&](int row, int b, float v) { s_gu[row][b] = v; });
+    if (!ok) {
+        if (t == 0) { atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT); ring.drain(0); }
+        return;
+    }
     __syncthreads();
 
     // ---- step 11: siLu_Mul (first half of an interlaced block is gate, second half up) ----
-    for (int i = t; i < noct * 8 * NB; i += blockDim.x) {
+    for (int i = t; i < nj * NB; i += blockDim.x) {
         const int j = i / NB, b = i % NB;
         const int o = j >> 3, c = j & 7;
         const float g = s_gu[o * 16 + c][b], u = s_gu[o * 16 + 8 + c][b];
@@ -66,37 +80,32 @@ __global__ void __launch_bounds__(MAXT, 1) mlp_decode_kernel(MlpArgs a)
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[b][i] = 0.f;
     const int nvec = a.D >> 3;
-    const uint4 *Wd = reinterpret_cast<const uint4 *>(a.w_down) + (size_t)oct0 * 8 * nvec + t;
-    const int nj = noct * 8;                                // multiple of 8, hence of U
-    if (active) {
-        uint4 wa[U], wb[U];
-        auto load = [&](uint4 (&w)[U], int j0) {
+    const int g_down0 = ring.groups0;
+    const int ngroups_down = nj / R;                         // nj is a multiple of 8, hence of R
+    for (int g = 0; g < ngroups_down; ++g) {
+        const uint4 *slot = reinterpret_cast<const uint4 *>(ring.wait(g_down0 + g, ok));
+        if (active) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) w[u] = ldg_stream(Wd + (size_t)(j0 + u) * nvec);
-        };
-        auto fma_rows = [&](const uint4 (&w)[U], int j0) {
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
+            for (int u = 0; u < R; ++u) {
                 float wf[8];
-                unpack8(w[u], wf);
+                unpack8(slot[u * nvec + t], wf);
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
-                    const float av = s_act[j0 + u][b];
+                    const float av = s_act[g * R + u][b];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) acc[b][i] = fmaf(av, wf[i], acc[b][i]);
                 }
             }
-        };
-        if (nj > 0) load(wa, 0);
-        for (int j0 = 0; j0 < nj; j0 += 2 * U) {
-            if (j0 + U < nj) load(wb, j0 + U);
-            fma_rows(wa, j0);
-            if (j0 + U < nj) {
-                if (j0 + 2 * U < nj) load(wa, j0 + 2 * U);
-                fma_rows(wb, j0 + U);
-            }
         }
-        // ---- partial sums of all CTAs meet in the FP32 accumulator ----
+        if (!__syncthreads_and(ok ? 1 : 0)) {
+            if (t == 0) { atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT); ring.drain(g_down0 + g); }
+            return;
+        }
+        if (t == 0) ring.refill(g_down0 + g);
+    }
+
+    // ---- partial sums of all CTAs meet in the FP32 accumulator ----
+    if (active) {
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
             if (b < a.batch) {
@@ -138,28 +147,48 @@ __global__ void __launch_bounds__(MAXT, 1) mlp_decode_kernel(MlpArgs a)
 }
 
 template <int NB>
+cudaError_t configure_mlp_nb()
+{
+    cudaError_t e = allow_big_smem(mlp_decode_kernel<NB, 128>);
+    if (e == cudaSuccess) e = allow_big_smem(mlp_decode_kernel<NB, 256>);
+    if (e == cudaSuccess) e = allow_big_smem(mlp_decode_kernel<NB, 384>);
+    if (e == cudaSuccess) e = allow_big_smem(mlp_decode_kernel<NB, 512>);
+    if (e == cudaSuccess) e = allow_big_smem(mlp_decode_kernel<NB, 768>);
+    return e;
+}
+
+template <int NB>
 int launch_mlp_nb(Ctx *c, const MlpArgs &a, cudaStream_t st)
 {
     constexpr int R = RowsPerGroup<NB>::value;
     const int threads = ((a.D / 8) + 31) / 32 * 32;
-    const int nwarps = threads / 32;
+    const StreamSmemLayout lay = stream_smem_layout(a.D, R, NB, threads / 32);
+    if (lay.nslot < 2) return FASTTPS_INVALID_ARG;
     const int n_oct = a.K / 8;
     int grid = c->n_sm;
     if (grid > n_oct) grid = n_oct;
     while ((n_oct + grid - 1) / grid > kMaxOctetsPerCta) grid *= 2;   // tiny GPUs / huge K only
-    size_t smem = sizeof(float) * (size_t)(2 * nwarps * R * NB > 32 * NB ? 2 * nwarps * R * NB : 32 * NB);
     ProfScope prof(c, kProfMlp, st);
-    if (threads <= 128) mlp_decode_kernel<NB, 128><<<grid, threads, smem, st>>>(a);
-    else if (threads <= 256) mlp_decode_kernel<NB, 256><<<grid, threads, smem, st>>>(a);
-    else if (threads <= 384) mlp_decode_kernel<NB, 384><<<grid, threads, smem, st>>>(a);
-    else if (threads <= 512) mlp_decode_kernel<NB, 512><<<grid, threads, smem, st>>>(a);
-    else mlp_decode_kernel<NB, 1024><<<grid, threads, smem, st>>>(a);
+    int rc;
+    if (threads <= 128) rc = launch_stream_kernel(mlp_decode_kernel<NB, 128>, grid, threads, lay.total, st, &a);
+    else if (threads <= 256) rc = launch_stream_kernel(mlp_decode_kernel<NB, 256>, grid, threads, lay.total, st, &a);
+    else if (threads <= 384) rc = launch_stream_kernel(mlp_decode_kernel<NB, 384>, grid, threads, lay.total, st, &a);
+    else if (threads <= 512) rc = launch_stream_kernel(mlp_decode_kernel<NB, 512>, grid, threads, lay.total, st, &a);
+    else rc = launch_stream_kernel(mlp_decode_kernel<NB, 768>, grid, threads, lay.total, st, &a);
     c->launches++;
-    FT_CUDA(cudaGetLastError());
-    return FASTTPS_OK;
+    return rc;
 }
 
 }  // namespace
+
+int configure_mlp_kernels()
+{
+    FT_CUDA(configure_mlp_nb<1>());
+    FT_CUDA(configure_mlp_nb<2>());
+    FT_CUDA(configure_mlp_nb<4>());
+    FT_CUDA(configure_mlp_nb<8>());
+    return FASTTPS_OK;
+}
 
 // Batches above kMaxNB are served in tiles of kMaxNB rows (the weights are re-read per tile).
 int launch_mlp(Ctx *c, const MlpArgs &a0, cudaStream_t st)
