@@ -1,6 +1,7 @@
 // C ABI of the FastTPS decode library: context, argument checks and the launch chains.
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -16,14 +17,23 @@ void set_last_error(cudaError_t e, const char *where)
     snprintf(g_last_error, sizeof g_last_error, "%s: %s (%s)", where, cudaGetErrorName(e), cudaGetErrorString(e));
 }
 
+bool pdl_enabled()
+{
+    static const bool on = [] {
+        const char *e = getenv("FASTTPS_PDL");
+        return !(e && e[0] == '0');
+    }();
+    return on;
+}
+
 static bool aligned16(const void *p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static bool config_ok(const fasttps_config &f)
 {
-    if (f.hidden <= 0 || f.hidden % 8 || f.hidden > 6144) return false;
+    if (f.hidden <= 0 || f.hidden > 6144 || !reduction_length_ok(f.hidden)) return false;
     if (f.head_dim != 32 && f.head_dim != 64 && f.head_dim != 96 && f.head_dim != 128) return false;
     if (f.n_q_heads <= 0 || f.n_kv_heads <= 0 || f.n_q_heads % f.n_kv_heads) return false;
-    if ((f.n_q_heads * f.head_dim) % 8 || f.n_q_heads * f.head_dim > 6144) return false;
+    if (f.n_q_heads * f.head_dim > 6144 || !reduction_length_ok(f.n_q_heads * f.head_dim)) return false;
     if (f.inter <= 0 || f.inter % 8) return false;
     if (f.vocab < 0 || f.n_layers < 0 || f.max_batch < 1 || f.max_seq < 1) return false;
     if (!(f.rms_eps >= 0.f) || !(f.rope_theta > 0.f)) return false;
@@ -73,7 +83,8 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     FT_CUDA(cudaGetDeviceProperties(&c->prop, cfg->device));
     c->n_sm = c->prop.multiProcessorCount;
     {
-        int rc = configure_linear_kernels();
+        int rc = configure_attn_kernels();
+        if (rc == FASTTPS_OK) rc = configure_linear_kernels();
         if (rc == FASTTPS_OK) rc = configure_mlp_kernels();
         if (rc != FASTTPS_OK) { delete c; return rc; }
     }
@@ -144,16 +155,7 @@ int fasttps_destroy(fasttps_ctx *ctx)
 size_t fasttps_packed_bytes(const fasttps_ctx *ctx, int kind)
 {
     if (!ctx) return 0;
-    const fasttps_config &f = reinterpret_cast<const Ctx *>(ctx)->cfg;
-    const size_t nq = (size_t)f.n_q_heads * f.head_dim, nkv = (size_t)f.n_kv_heads * f.head_dim;
-    switch (kind) {
-    case FASTTPS_W_QKV: return 2 * (size_t)f.hidden * (nq + 2 * nkv);
-    case FASTTPS_W_O: return 2 * nq * f.hidden;
-    case FASTTPS_W_GATE_UP: return 2 * (size_t)f.hidden * 2 * f.inter;
-    case FASTTPS_W_DOWN: return 2 * (size_t)f.inter * f.hidden;
-    case FASTTPS_W_LM_HEAD: return 2 * (size_t)f.vocab * f.hidden;
-    default: return 0;
-    }
+    return 2 * packed_elems(reinterpret_cast<const Ctx *>(ctx)->cfg, kind);
 }
 
 int fasttps_pack_weight(fasttps_ctx *ctx, int kind, const void *src, void *dst, void *stream)

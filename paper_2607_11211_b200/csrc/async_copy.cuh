@@ -22,6 +22,10 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
     uint32_t ok;
@@ -38,13 +42,15 @@ __device__ __forceinline__ unsigned long long global_ns()
     return v;
 }
 // Bounded wait: gives up after kWaitPolls polls or kWaitNanos of wall time, whichever comes
-// first, and reports failure instead of spinning forever.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity)
+// first (or as soon as *abort_flag is set, when given), and reports failure instead of
+// spinning forever.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, const volatile int *abort_flag = nullptr)
 {
     unsigned long long t0 = 0;
     for (uint32_t i = 0; i < kWaitPolls; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 255u) == 255u) {
+            if (abort_flag && *abort_flag) return false;
             const unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
             else if (now - t0 > kWaitNanos) return false;
@@ -58,87 +64,95 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
+// named barrier over the first `nthreads` threads' warps (id 1..15; id 0 is __syncthreads)
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// named barrier that also ANDs a predicate over its participants: every thread gets the same verdict
+__device__ __forceinline__ bool named_bar_and(int id, int nthreads, bool pred)
+{
+    uint32_t out;
+    asm volatile("{\n\t.reg .pred p, q;\n\t"
+                 "setp.ne.u32 q, %1, 0;\n\t"
+                 "bar.red.and.pred p, %2, %3, q;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(out) : "r"(pred ? 1u : 0u), "r"(id), "r"(nthreads) : "memory");
+    return out != 0;
+}
 
 // ----------------------------------------------------------------- weight ring
 //
-// A CTA's share of a weight matrix is a contiguous run of rows (each row = the n_in weights
-// of one output, or one row of W_down).  The ring streams up to two such runs, one after the
-// other, as "groups" of R rows: group g lands in slot g % nslot with ONE bulk copy issued by
-// thread 0, and completes on the slot's mbarrier.  Up to nslot groups (about 190 KB per SM)
-// are in flight at any time, independent of what the consumer warps are doing, which is what
-// keeps HBM busy across reductions, barriers and the switch from one matrix to the next.
-//
-// Protocol: thread 0 calls start() once (after init + __syncthreads), all threads call
-// wait(g) before reading group g, and after a block-wide barrier that follows the last read
-// of group g thread 0 calls refill(g) to reuse its slot for group g + nslot.
+// A CTA's share of a packed weight matrix is one contiguous byte range (two for the fused
+// MLP: its gate_up tiles, then its W_down octets).  A dedicated producer warp streams the
+// ranges, one after the other, in slot-sized pieces: piece g lands in slot g % nslot with
+// ONE bulk copy and completes on the slot's "full" mbarrier.  Each consumer warp arrives on
+// the slot's "empty" mbarrier when it has read its part, and the producer refills the slot
+// as soon as all consumer warps have.  Up to nslot pieces (about 190 KB per SM) are in
+// flight at any time, independent of what the consumer warps are doing, which keeps HBM
+// busy across reductions, barriers and the switch from one matrix to the next.
 struct WeightRing {
     unsigned char *slots;        // nslot * slot_bytes, 128-byte aligned
-    uint64_t *full;              // nslot mbarriers
-    int nslot, slot_bytes, row_bytes, rows_per_group;
+    uint64_t *full, *empty;      // nslot mbarriers each
+    volatile int *abort_flag;    // shared-memory word, set when any bounded wait ran out
+    int nslot, slot_bytes;
     const unsigned char *base0, *base1;
-    int rows0, rows1;            // rows in each run
-    int groups0, groups;         // groups of run 0, of both runs
+    int pieces0, pieces;         // pieces of run 0, of both runs (every run is a whole number of slots)
 
-    __device__ __forceinline__ void init(unsigned char *slots_, uint64_t *full_, int nslot_, int row_bytes_, int R,
-                                         const void *b0, int r0, const void *b1, int r1)
+    // all threads; follow with a block-wide barrier before any other use
+    __device__ __forceinline__ void init(unsigned char *slots_, uint64_t *bars, int *abort_, int nslot_, int slot_bytes_,
+                                         int n_consumer_warps, const void *b0, long long bytes0, const void *b1,
+                                         long long bytes1)
     {
-        slots = slots_; full = full_; nslot = nslot_; row_bytes = row_bytes_; rows_per_group = R;
-        slot_bytes = R * row_bytes_;
-        base0 = static_cast<const unsigned char *>(b0); rows0 = r0;
-        base1 = static_cast<const unsigned char *>(b1); rows1 = r1;
-        groups0 = (r0 + R - 1) / R;
-        groups = groups0 + (r1 + R - 1) / R;
+        slots = slots_; full = bars; empty = bars + nslot_; abort_flag = abort_;
+        nslot = nslot_; slot_bytes = slot_bytes_;
+        base0 = static_cast<const unsigned char *>(b0);
+        base1 = static_cast<const unsigned char *>(b1);
+        pieces0 = (int)(bytes0 / slot_bytes_);
+        pieces = pieces0 + (int)(bytes1 / slot_bytes_);
         if (threadIdx.x == 0) {
-            for (int s = 0; s < nslot; ++s) mbar_init(&full[s], 1);
+            for (int s = 0; s < nslot; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], n_consumer_warps); }
+            *abort_ = 0;
             mbar_fence_init();
         }
     }
-    // thread 0 only
-    __device__ __forceinline__ void issue(int g)
+    // one thread of the producer warp: stream every piece, then return
+    __device__ __forceinline__ void produce()
     {
-        const bool second = g >= groups0;
-        const int gl = second ? g - groups0 : g;
-        int n = (second ? rows1 : rows0) - gl * rows_per_group;
-        n = n < rows_per_group ? n : rows_per_group;
-        const uint32_t bytes = (uint32_t)n * (uint32_t)row_bytes;
-        uint64_t *bar = &full[g % nslot];
-        mbar_expect_tx(bar, bytes);
-        bulk_g2s(slots + (size_t)(g % nslot) * slot_bytes, (second ? base1 : base0) + (size_t)gl * slot_bytes, bytes, bar);
+        for (int g = 0; g < pieces; ++g) {
+            const int s = g % nslot;
+            if (g >= nslot && !mbar_wait_bounded(&empty[s], (uint32_t)(g / nslot - 1) & 1u, abort_flag)) {
+                *abort_flag = 1;
+                return;
+            }
+            const unsigned char *src = g < pieces0 ? base0 + (size_t)g * slot_bytes
+                                                   : base1 + (size_t)(g - pieces0) * slot_bytes;
+            mbar_expect_tx(&full[s], (uint32_t)slot_bytes);
+            bulk_g2s(slots + (size_t)s * slot_bytes, src, (uint32_t)slot_bytes, &full[s]);
+        }
     }
-    __device__ __forceinline__ void start()
-    {
-        for (int g = 0; g < groups && g < nslot; ++g) issue(g);
-    }
-    __device__ __forceinline__ void refill(int g)
-    {
-        if (g + nslot < groups) issue(g + nslot);
-    }
-    // all threads; lane 0 polls, the warp shares the verdict
+    // every lane of a consumer warp; returns the slot holding piece g (ok is cleared on a failed wait)
     __device__ __forceinline__ const unsigned char *wait(int g, bool &ok)
     {
-        bool mine = true;
-        if ((threadIdx.x & 31) == 0) mine = mbar_wait_bounded(&full[g % nslot], (uint32_t)(g / nslot) & 1u);
-        mine = __shfl_sync(kFull, mine ? 1 : 0, 0) != 0;
-        // every lane observes the (already completed) phase itself, so that its reads of the
-        // slot are ordered after the copy; this returns at once
-        if (mine) mine = mbar_try_wait(&full[g % nslot], (uint32_t)(g / nslot) & 1u);
+        bool mine = ok;
+        if (mine) mine = mbar_wait_bounded(&full[g % nslot], (uint32_t)(g / nslot) & 1u, abort_flag);
         mine = __all_sync(kFull, mine);
-        ok = ok && mine;
+        if (!mine && ok) *abort_flag = 1;
+        ok = mine;
         return slots + (size_t)(g % nslot) * slot_bytes;
     }
-    // thread 0, after a failed wait: give the copies still in flight (groups g .. issued) a bounded chance to land
-    __device__ __forceinline__ void drain(int g)
+    // consumer warp, after its last read of piece g
+    __device__ __forceinline__ void release(int g)
     {
-        for (int u = g; u < groups && u < g + nslot; ++u)
-            (void)mbar_wait_bounded(&full[u % nslot], (uint32_t)(u / nslot) & 1u);
+        __syncwarp();
+        if ((threadIdx.x & 31) == 0) mbar_arrive(&empty[g % nslot]);
+    }
+    // producer thread, on the way out after a failure: give the copies in flight a bounded chance to land
+    __device__ __forceinline__ void drain()
+    {
+        for (int s = 0; s < nslot; ++s) (void)mbar_wait_bounded(&full[s], 0, nullptr);
     }
 };
-
-// shared-memory bytes the ring needs for rows of row_bytes, and how many slots fit into `budget`
-__host__ __device__ inline int ring_slots_for(int row_bytes, int R, int budget)
-{
-    int n = budget / (R * row_bytes);
-    return n > 8 ? 8 : n;
-}
 
 }  // namespace fasttps

@@ -73,6 +73,27 @@ void set_last_error(cudaError_t e, const char *where);
         }                                                               \
     } while (0)
 
+// Launch of a decode-path kernel taking one argument struct.  Unless FASTTPS_PDL=0 is set, the
+// launch carries the programmatic-stream-serialization attribute: the kernel may start (and
+// prefetch weights, which no kernel writes) while its predecessor in the stream drains, and
+// orders everything else behind `griddepcontrol.wait`.
+bool pdl_enabled();
+
+template <class Args>
+static int launch_ex(void (*kernel)(Args), dim3 grid, dim3 block, size_t smem, cudaStream_t st, const Args *a)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    void *params[] = {const_cast<Args *>(a)};
+    FT_CUDA(cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(kernel), params));
+    return FASTTPS_OK;
+}
+
 // --------------------------------------------------------------- bf16 / loads
 
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
@@ -240,6 +261,14 @@ int launch_mlp(Ctx *c, const MlpArgs &a, cudaStream_t st);
 int launch_embed(Ctx *c, const __nv_bfloat16 *embed, const int32_t *ids, __nv_bfloat16 *x, int batch, cudaStream_t st);
 int launch_pack(Ctx *c, int kind, const void *src, void *dst, bool inverse, cudaStream_t st);
 int attn_splits_for(const Ctx *c, int batch);
+size_t packed_elems(const fasttps_config &f, int kind);
+// A reduction length the tensor-core kernels can split over their warps: a multiple of 128,
+// at most 3072, or a multiple of 256 from 2048 to 6144.
+inline bool reduction_length_ok(int n)
+{
+    return n > 0 && ((n % 128 == 0 && n / 128 <= 24) || (n >= 2048 && n % 256 == 0 && n / 256 <= 24));
+}
+int configure_attn_kernels();
 int configure_linear_kernels();
 int configure_mlp_kernels();
 

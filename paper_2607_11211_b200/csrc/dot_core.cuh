@@ -1,120 +1,144 @@
-// Weight-streaming dot-product core shared by the projection kernel and the
-// gate_up half of the fused MLP kernel.
+// Tensor-core weight-streaming core shared by the projection kernel and the fused MLP kernel.
 //
-// Layout: W is [rows][n_in] bf16 with every row (one output feature) contiguous.
-// A CTA of ceil(n_in / 8 / 32) warps owns a contiguous range of rows, which is one
-// contiguous byte range of the matrix.  The range arrives through the shared-memory
-// weight ring (bulk asynchronous copies, R rows per group, several groups in
-// flight).  Thread t owns the 16-byte k-slice [8t, 8t+8) of EVERY row and keeps its
-// slice of the activations in registers (FP32, NB batch rows).  The R*NB partial sums
-// of a group are reduced with a halving butterfly (about one shuffle per value), meet
-// in shared memory (one block barrier per group, double buffered) and are handed to
-// the epilogue by the first R*NB threads.
+// Why tensor cores at batch 1: with FP32 FMAs every 16 bytes of bf16 weights cost 8 unpack
+// instructions, 8 FMAs and a share of a cross-lane reduction; at the HBM rate of a B200 that is
+// more warp-instructions than an SM with a handful of warps can issue (measured: issue-bound at
+// ~5.3 TB/s).  One mma.sync.m16n8k16 consumes 512 bytes of weights with one instruction, takes
+// bf16 directly, reduces over k inside the instruction and serves up to 8 batch rows for free.
+//
+// Packed layout ("tiled", written by the packing kernels): an [n_out][n_in] matrix is cut into
+// tiles of 16 rows x 32 k, each tile stored row-major (1 KB), tiles ordered by (row tile, k block).
+// A warp reads a tile with two conflict-free 16-byte shared loads per lane: lane (g = lane / 4,
+// t4 = lane % 4) gets W[row g][8 t4 .. 8 t4 + 8) and W[row g + 8][same k].  Those 8 consecutive k
+// of the two rows are exactly the A fragments of TWO m16n8k16 MMAs if the k index inside the MMA
+// is permuted; the same permutation makes the B fragments of both MMAs one contiguous 16-byte
+// piece x[batch row g][8 t4 .. 8 t4 + 8) of the bf16 activations.
+//
+// Work split inside a CTA: n_in / 32 k blocks per row tile are dealt round-robin to NW consumer
+// warps, IPW blocks each (n_in = 32 * NW * IPW).  A warp keeps the B fragments of its IPW k
+// blocks in registers for the whole kernel, accumulates a 16 x 8 partial tile over its blocks,
+// and the NW partial tiles of a row tile meet in shared memory (one named barrier per 16 rows).
 #pragma once
 #include "async_copy.cuh"
 
 namespace fasttps {
 
-template <int NB> struct RowsPerGroup { static constexpr int value = (NB <= 4) ? 8 : 4; };
-
 constexpr int kRingBudget = 192 * 1024;     // shared memory given to the weight ring
+constexpr int kTileBytes = 1024;            // 16 rows x 32 k bf16
+constexpr int kBlocksPerWarpPerSlot = 2;    // a slot holds 2 k blocks of every consumer warp
 
-// Loads this thread's activation slice: x[b][8t .. 8t+8) for NB batch rows, with an
-// optional RMSNorm (gain g, eps) whose result is rounded to bf16 like a stored tensor.
-// smem_red: at least 32 * NB floats.  All threads of the CTA must call.
-template <int NB>
-__device__ __forceinline__ void load_activations(float (&x)[NB][8], const __nv_bfloat16 *xg, int x_stride,
-                                                 int batch, int n_in, const __nv_bfloat16 *g, float eps,
-                                                 float *smem_red)
+__device__ __forceinline__ void mma_bf16_k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                             uint32_t b0, uint32_t b1)
 {
-    const int t = threadIdx.x;
-    const bool active = t * 8 < n_in;
-#pragma unroll
-    for (int b = 0; b < NB; ++b) {
-        if (active && b < batch) {
-            uint4 v = *reinterpret_cast<const uint4 *>(xg + (size_t)b * x_stride + t * 8);
-            unpack8(v, x[b]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) x[b][i] = 0.f;
-        }
-    }
-    if (g == nullptr) return;
-    const int lane = t & 31, warp = t >> 5, nwarps = (blockDim.x + 31) >> 5;
-    float ss[NB];
-#pragma unroll
-    for (int b = 0; b < NB; ++b) {
-        float s = 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) s += x[b][i] * x[b][i];
-        ss[b] = warp_sum(s);
-    }
-    if (lane == 0) {
-#pragma unroll
-        for (int b = 0; b < NB; ++b) smem_red[warp * NB + b] = ss[b];
-    }
-    __syncthreads();
-    float gv[8];
-    if (active) {
-        uint4 v = *reinterpret_cast<const uint4 *>(g + t * 8);
-        unpack8(v, gv);
-    } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) gv[i] = 0.f;
-    }
-#pragma unroll
-    for (int b = 0; b < NB; ++b) {
-        float tot = 0.f;
-        for (int w = 0; w < nwarps; ++w) tot += smem_red[w * NB + b];
-        const float r = rsqrtf(tot / (float)n_in + eps);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) x[b][i] = bf16_round(x[b][i] * r * gv[i]);
-    }
-    __syncthreads();   // smem_red may be reused by the caller
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_bf16_k8(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0)
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(b0));
 }
 
-// Consumes ring groups [g0, g0 + ceil(nrows / R)) = rows [row0, row0 + nrows) of a matrix and
-// calls epi(row, b, value) for every row and batch row b < NB, from threads 0 .. R*NB-1 (one
-// (row, b) pair per thread and group).  smem_red: 2 * nwarps * R * NB floats.  All threads of
-// the CTA must call.  Returns false if a bounded wait ran out (the CTA must then leave).
-template <int NB, class Epi>
-__device__ __forceinline__ bool dot_rows(WeightRing &ring, int g0, int n_in, int row0, int nrows,
-                                         const float (&x)[NB][8], float *smem_red, Epi epi)
+// How a reduction length n_in maps onto consumer warps: n_in = 32 * nw * ipw, ipw in {4, 8}.
+struct WarpSplit { int nw, ipw; };
+__host__ __device__ inline WarpSplit warp_split(int n_in)
 {
-    constexpr int R = RowsPerGroup<NB>::value;
-    constexpr int V = R * NB;
-    const int t = threadIdx.x, lane = t & 31, warp = t >> 5, nwarps = (blockDim.x + 31) >> 5;
-    const bool active = t * 8 < n_in;
-    const int nvec = n_in >> 3;
-    const int ngroups = (nrows + R - 1) / R;
-    bool ok = true;
-    for (int g = 0; g < ngroups; ++g) {
-        const int buf = g & 1;
-        const uint4 *slot = reinterpret_cast<const uint4 *>(ring.wait(g0 + g, ok));
-        float p[V];
+    WarpSplit s = {0, 0};
+    if (n_in >= 2048 && n_in % 256 == 0 && n_in / 256 <= 24) { s.nw = n_in / 256; s.ipw = 8; }
+    else if (n_in % 128 == 0 && n_in / 128 <= 24) { s.nw = n_in / 128; s.ipw = 4; }
+    return s;
+}
+
+// B fragments of this consumer thread: the bf16 activations x[g][32 (w + nw i) + 8 t4 .. + 8) for its
+// IPW k blocks, batch row g = lane / 4 (zero for g >= batch), optionally RMS-normalised (gain gn, eps)
+// with the result rounded to bf16 like a stored tensor.  Consumer threads only (named barrier 1).
+// smem_red: nw * 8 floats.
+template <int IPW>
+__device__ __forceinline__ void load_b_frags(uint32_t (&bf)[IPW][4], const __nv_bfloat16 *x, int x_stride, int batch,
+                                             int n_in, int nw, const __nv_bfloat16 *gn, float eps, float *smem_red)
+{
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3;
+    const bool live = g < batch;
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            float wf[8];
-            const uint4 w = active ? slot[r * nvec + t] : make_uint4(0, 0, 0, 0);
-            unpack8(w, wf);
+    for (int i = 0; i < IPW; ++i) {
+        const int k = 32 * (w + nw * i) + 8 * t4;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (live) v = *reinterpret_cast<const uint4 *>(x + (size_t)g * x_stride + k);
+        bf[i][0] = v.x; bf[i][1] = v.y; bf[i][2] = v.z; bf[i][3] = v.w;
+    }
+    if (gn == nullptr) return;
+    float ss = 0.f;
 #pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                float s = 0.f;
+    for (int i = 0; i < IPW; ++i)
 #pragma unroll
-                for (int i = 0; i < 8; ++i) s = fmaf(wf[i], x[b][i], s);
-                p[r * NB + b] = s;
-            }
+        for (int j = 0; j < 4; ++j) {
+            const float lo = bf_lo(bf[i][j]), hi = bf_hi(bf[i][j]);
+            ss = fmaf(lo, lo, ss);
+            ss = fmaf(hi, hi, ss);
         }
-        const float tot = warp_multi_reduce<V>(p, lane);
-        constexpr int rep = 32 / V;                       // lanes sharing one value
-        if ((lane & (rep - 1)) == 0) smem_red[(buf * nwarps + warp) * V + warp_multi_which<V>(lane)] = tot;
-        if (!__syncthreads_and(ok ? 1 : 0)) return false; // every warp is done with the slot
-        if (t == 0) ring.refill(g0 + g);
-        if (t < V) {
-            float s = 0.f;
-            for (int w2 = 0; w2 < nwarps; ++w2) s += smem_red[(buf * nwarps + w2) * V + t];
-            const int row = g * R + t / NB;
-            if (row < nrows) epi(row0 + row, t % NB, s);
+    ss += __shfl_xor_sync(kFull, ss, 1);
+    ss += __shfl_xor_sync(kFull, ss, 2);
+    if (t4 == 0) smem_red[w * 8 + g] = ss;
+    named_bar_sync(1, nw * 32);
+    float tot = 0.f;
+    for (int w2 = 0; w2 < nw; ++w2) tot += smem_red[w2 * 8 + g];
+    const float r = rsqrtf(tot / (float)n_in + eps);
+#pragma unroll
+    for (int i = 0; i < IPW; ++i) {
+        const int k = 32 * (w + nw * i) + 8 * t4;
+        const uint4 gv = *reinterpret_cast<const uint4 *>(gn + k);
+        const uint32_t gg[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            bf[i][j] = pack2(bf_lo(bf[i][j]) * r * bf_lo(gg[j]), bf_hi(bf[i][j]) * r * bf_hi(gg[j]));
+    }
+    named_bar_sync(1, nw * 32);   // smem_red may be reused by the caller
+}
+
+// Consumes ring pieces [g0, g0 + ntiles * IPW / 2) = `ntiles` row tiles of a tiled matrix and calls
+// epi(tile, c, b, v_lo, v_hi) from consumer threads 0..63 with the finished sums of rows c and c + 8
+// (c = 0..7) of the tile for batch row b = 0..7.  smem_part: 2 * nw * 128 floats.  Consumer threads
+// only.  Returns false if a bounded wait ran out.
+template <int IPW, class Epi>
+__device__ __forceinline__ bool dot_tiles(WeightRing &ring, int g0, int ntiles, int nw, const uint32_t (&bf)[IPW][4],
+                                          float *smem_part, Epi epi)
+{
+    constexpr int SPT = IPW / kBlocksPerWarpPerSlot;      // ring pieces per row tile
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    bool ok = true;
+    for (int tile = 0; tile < ntiles; ++tile) {
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int q = 0; q < SPT; ++q) {
+            const int piece = g0 + tile * SPT + q;
+            const unsigned char *slot = ring.wait(piece, ok);
+#pragma unroll
+            for (int s = 0; s < kBlocksPerWarpPerSlot; ++s) {
+                const unsigned char *blk = slot + (size_t)(s * nw + w) * kTileBytes + lane * 16;
+                const uint4 lo = *reinterpret_cast<const uint4 *>(blk);          // row g,     k 8 t4 ..
+                const uint4 hi = *reinterpret_cast<const uint4 *>(blk + 512);    // row g + 8, k 8 t4 ..
+                const int i = q * kBlocksPerWarpPerSlot + s;
+                mma_bf16_k16(c, lo.x, hi.x, lo.y, hi.y, bf[i][0], bf[i][1]);
+                mma_bf16_k16(c, lo.z, hi.z, lo.w, hi.w, bf[i][2], bf[i][3]);
+            }
+            ring.release(piece);
+        }
+        // partial 16 x 8 tiles of the nw warps meet in shared memory (double buffered)
+        float *part = smem_part + (size_t)(tile & 1) * nw * 128;
+        *reinterpret_cast<float4 *>(part + (size_t)w * 128 + lane * 4) = make_float4(c[0], c[1], c[2], c[3]);
+        if (!named_bar_and(1, nw * 32, ok)) return false;   // same verdict in every consumer thread
+        for (int u = t; u < 64; u += nw * 32) {
+            // fragment layout: lane (g, t4) holds rows g / g + 8, batch columns 2 t4 / 2 t4 + 1
+            const int cc = u >> 3, b = u & 7;
+            const int idx = (cc * 4 + (b >> 1)) * 4 + (b & 1);
+            float v0 = 0.f, v1 = 0.f;
+            for (int w2 = 0; w2 < nw; ++w2) {
+                v0 += part[(size_t)w2 * 128 + idx];
+                v1 += part[(size_t)w2 * 128 + idx + 2];
+            }
+            epi(tile, cc, b, v0, v1);
         }
     }
     return true;

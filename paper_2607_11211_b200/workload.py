@@ -121,7 +121,7 @@ class Dims:
 
 
 PHI3_MINI = Dims()
-TINY = Dims(hidden=64, n_q_heads=2, n_kv_heads=2, head_dim=32, inter=128, vocab=160, n_layers=2)
+TINY = Dims(hidden=128, n_q_heads=4, n_kv_heads=4, head_dim=32, inter=128, vocab=160, n_layers=2)
 SMALL = Dims(hidden=256, n_q_heads=4, n_kv_heads=4, head_dim=64, inter=640, vocab=1000, n_layers=3)
 SMALL_GQA = Dims(hidden=256, n_q_heads=8, n_kv_heads=2, head_dim=32, inter=384, vocab=520, n_layers=2)
 

@@ -46,14 +46,30 @@ def test_pack_unpack_round_trip_and_interlace(fb, dims):
         p = ctx.pack_weight(kind, t)
         back = ctx.unpack_weight(kind, p, t.shape)
         assert torch.equal(back.view(torch.int16), t.view(torch.int16)), kind
-    # the packed gate_up rows are the logical columns interlaced in blocks of 8 (gate block, up block)
+    # gate_up: logical columns interlaced in blocks of 8 (gate block, up block), then cut into
+    # row-major tiles of 16 rows x 32 k ordered by (row tile, k block)
     K, D = dims.inter, dims.hidden
-    p = ctx.pack_weight(fb.W_GATE_UP, w["w_gu"]).view(2 * K, D)
     r = torch.arange(2 * K, device="cuda")
     col = ((r // 8) % 2) * K + (r // 16) * 8 + r % 8
-    assert torch.equal(p.view(torch.int16), w["w_gu"].t()[col].contiguous().view(torch.int16))
-    assert torch.equal(ctx.pack_weight(fb.W_QKV, w["w_qkv"]).view(-1, D).view(torch.int16),
-                       w["w_qkv"].t().contiguous().view(torch.int16))
+
+    def tiled(rows_by_k):                                    # [n_out, n_in] -> packed order
+        n_out, n_in = rows_by_k.shape
+        return rows_by_k.reshape(n_out // 16, 16, n_in // 32, 32).permute(0, 2, 1, 3).contiguous().view(-1)
+
+    p = ctx.pack_weight(fb.W_GATE_UP, w["w_gu"])
+    assert torch.equal(p.view(torch.int16), tiled(w["w_gu"].t()[col]).view(torch.int16))
+    assert torch.equal(ctx.pack_weight(fb.W_QKV, w["w_qkv"]).view(torch.int16),
+                       tiled(w["w_qkv"].t()).view(torch.int16))
+    # down: per (octet, 32-column block) one 512-byte block of m16n8k8 A fragments
+    pd = ctx.pack_weight(fb.W_DOWN, w["w_down"]).view(K // 8, D // 32, 32, 4, 2)
+    lane = torch.arange(32, device="cuda")
+    g, t4 = lane // 4, lane % 4
+    wd = w["w_down"].view(K // 8, 8, D // 32, 32)            # [o, j8, nb, n32]
+    for q in range(4):
+        for jj in range(2):
+            want = wd[:, 2 * t4 + jj][:, :, :, :].permute(0, 2, 1, 3)      # [o, nb, lane, n32]
+            want = want[:, :, lane, g + 8 * q]
+            assert torch.equal(pd[:, :, :, q, jj].view(torch.int16), want.contiguous().view(torch.int16))
     ctx.close()
 
 
@@ -246,7 +262,7 @@ def test_mlp_decode_matches_oracle(fb, dims, batch):
 
 
 def test_mlp_zero_weights_and_identity_construction(fb):
-    dims = wl.Dims(hidden=64, n_q_heads=2, n_kv_heads=2, head_dim=32, inter=64, vocab=0, n_layers=0)
+    dims = wl.Dims(hidden=128, n_q_heads=4, n_kv_heads=4, head_dim=32, inter=128, vocab=0, n_layers=0)
     ctx = make_ctx(fb, dims, 2, 64)
     x = wl.activations(dims, 2, device="cuda")["x"]
     D = dims.hidden

@@ -40,7 +40,7 @@ def test_moments_and_recipes():
     z = wl.normal_f32(3, 4, 0, 1 << 20).double()
     assert abs(z.mean()) < 5e-3 and abs(z.std() - 1) < 5e-3 and z.abs().max() < 4.9
     w = wl.layer_weights(wl.TINY, 0)
-    assert w["w_qkv"].shape == (64, 192) and w["w_gu"].shape == (64, 256) and w["w_down"].shape == (128, 64)
+    assert w["w_qkv"].shape == (128, 384) and w["w_gu"].shape == (128, 256) and w["w_down"].shape == (128, 128)
     assert abs(w["w_gu"].float().std() - 0.02) < 2e-3
     assert abs(w["g_attn"].float().mean() - 1.0) < 2e-2
     L = wl.ragged_lengths(8, 512, 4096)
