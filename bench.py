@@ -35,6 +35,8 @@ UNIT = "tok/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one mlp_decode_kernel launch (Phi-3 shape,
 # batch 1) from the ncu capture summarised in profiles/; None until a capture exists.
 NCU_MLP_TRAFFIC_BYTES = None
+# the same for one decode step inside a decode_step_kernel launch (cfg3 shape)
+NCU_STEP_TRAFFIC_BYTES_PER_STEP = None
 
 
 def parse_args():
@@ -45,6 +47,9 @@ def parse_args():
     ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--graph", type=int, default=1, help="replay the step as a CUDA graph (1) or launch eagerly (0)")
+    ap.add_argument("--step-kernel", type=int, default=0,
+                    help="1: whole decode steps in the persistent cooperative kernel (batch <= 8)")
+    ap.add_argument("--l2-ahead", type=int, default=0, help="lookahead of the step kernel's L2 prefetch warp (pieces)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -210,6 +215,8 @@ def run_ours(args):
     n_sets = 8 if not W.full_stack else 1            # single-layer cases rotate weight sets to defeat L2
 
     ctx = fb.Context.from_dims(dm, B, max_seq, device=local, n_layers=W.n_layers)
+    ctx.set_option("step_kernel", args.step_kernel)
+    ctx.set_option("l2_ahead", args.l2_ahead)
     seed = wl.MASTER_SEED + 1000 * rank
 
     def packed_layer(idx):
@@ -230,6 +237,8 @@ def run_ours(args):
         model = ctx.make_model(embed, layers, g_final, w_lm, [c[0] for c in caches], [c[1] for c in caches])
         tok0 = torch.tensor(wl.token_ids(B, dm.vocab, seed), device=dev)
         tok = tok0.clone()
+
+        out_ids = torch.zeros(max(K, Wm), B, dtype=torch.int32, device=dev)
 
         def step(i):
             ctx.model_decode(model, tok, pos, sl, None, tok, advance=advance, stream=stream)
@@ -256,7 +265,9 @@ def run_ours(args):
 
     # optional CUDA graph of one step (pos/seq_lens/token live on the device, so one graph serves every step)
     graphs = None
-    use_graph = bool(args.graph)
+    # the greedy multi-token workload is ONE call: all steps run inside one launch of the persistent kernel
+    one_call = advance and B <= 8 and bool(args.step_kernel)
+    use_graph = bool(args.graph) and not one_call
     if use_graph:
         try:
             with torch.cuda.stream(stream):
@@ -277,6 +288,9 @@ def run_ours(args):
 
     def run_steps(n):
         with torch.cuda.stream(stream):
+            if one_call:
+                ctx.model_generate(model, tok, pos, sl, out_ids[:n], stream=stream)
+                return
             for i in range(n):
                 if graphs is not None:
                     graphs[i % n_sets].replay()
@@ -309,29 +323,45 @@ def run_ours(args):
     # kernels per step: count one eager step
     reset_state()
     c0 = ctx.launch_count()
-    with torch.cuda.stream(stream):
-        step(0)
+    if one_call:
+        run_steps(K)
+    else:
+        with torch.cuda.stream(stream):
+            step(0)
     stream.synchronize()
-    launches_per_step = ctx.launch_count() - c0
+    launches_total = (ctx.launch_count() - c0) * (1 if one_call else K)
 
-    # ---- roofline pass: per-kernel CUDA events on the launch stream, same K steps, eager ----
+    # ---- roofline pass: CUDA events around every launch on the launch stream, same steps, eager ----
     reset_state()
     ctx.profile(True)
-    with torch.cuda.stream(stream):
-        for i in range(min(K, 48)):
-            step(i)
+    n_prof = K if one_call else min(K, 48)
+    if one_call:
+        run_steps(n_prof)
+    else:
+        with torch.cuda.stream(stream):
+            for i in range(n_prof):
+                step(i)
     stream.synchronize()
     prof = ctx.profile_read()
     ctx.profile(False)
-    mlp_ms, mlp_n = prof["mlp"]
     total_prof_ms = sum(v[0] for v in prof.values())
+    dom = max(prof, key=lambda k: prof[k][0])                 # the kernel class with the largest share of the time
+    dom_ms, dom_n = prof[dom]
     mlp_bytes = 2 * (dm.hidden * 2 * dm.inter + dm.inter * dm.hidden) + B * dm.hidden * 2 * 2
+    if dom == "step":                                         # one launch = n_steps whole decode steps
+        steps_per_launch = n_prof if one_call else 1
+        dom_bytes = float(sum(W.algorithmic_bytes(s if advance else 0) for s in range(steps_per_launch)))
+        dom_name = "decode_step_kernel"
+        ncu_traffic = NCU_STEP_TRAFFIC_BYTES_PER_STEP * steps_per_launch if NCU_STEP_TRAFFIC_BYTES_PER_STEP else None
+    else:
+        dom, (dom_ms, dom_n) = "mlp", prof["mlp"]
+        dom_bytes, dom_name, ncu_traffic = float(mlp_bytes), "mlp_decode_kernel", NCU_MLP_TRAFFIC_BYTES
     peak, peak_kind = measured_peaks()
-    achieved = mlp_bytes / (mlp_ms / mlp_n * 1e-3) / 1e9 if mlp_n else None
-    roofline = {"bound": "hbm", "kernel": "mlp_decode_kernel", "achieved": achieved, "peak": peak,
+    achieved = dom_bytes / (dom_ms / dom_n * 1e-3) / 1e9 if dom_n else None
+    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_source": f"of {peak_kind}",
-                "traffic": NCU_MLP_TRAFFIC_BYTES, "bytes_per_launch": mlp_bytes,
-                "avg_launch_us": mlp_ms / mlp_n * 1e3 if mlp_n else None,
+                "traffic": ncu_traffic, "bytes_per_launch": dom_bytes,
+                "avg_launch_us": dom_ms / dom_n * 1e3 if dom_n else None,
                 "kernel_share": {k: round(v[0] / total_prof_ms, 4) for k, v in prof.items()} if total_prof_ms else None,
                 "kernel_avg_us": {k: round(v[0] / v[1] * 1e3, 2) for k, v in prof.items() if v[1]},
                 "how": "CUDA events around every launch on the launch stream, separate eager pass of the same steps"}
@@ -398,14 +428,15 @@ def run_ours(args):
                 "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic",
                 "config": {"workload": args.workload, "batch": B, "n_layers": W.n_layers, "full_stack": W.full_stack,
                            "past_lens": lens0.tolist()[:8], "max_seq": max_seq,
-                           "launch": "cuda_graph_replay" if use_graph else "eager",
+                           "launch": "one persistent-kernel launch for all steps" if one_call else
+                                     ("cuda_graph_replay" if use_graph else "eager"),
                            "l2": "inputs larger than L2: every step streams %.2f GB of weights and KV" % (step_bytes / 1e9)
                                  if W.full_stack else "rotates over 8 weight/cache sets (1.8 GB) so no operand stays in L2",
                            "parallelism": "replicas" if world > 1 else "single"},
                 "algorithmic_bytes_per_step": float(step_bytes),
                 "hbm_gbs_whole_step": float(step_bytes) / (ms_max / K * 1e-3) / 1e9,
                 "hbm_frac_whole_step": float(step_bytes) / (ms_max / K * 1e-3) / 1e9 / peak,
-                "gpu_launches": int(launches_per_step * K), "launches_per_step": int(launches_per_step),
+                "gpu_launches": int(launches_total),
                 "device_status": status, "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu}
         print(json.dumps(line), flush=True)
     ctx.close()

@@ -150,12 +150,31 @@ int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const
  *   token_ids [B] int32 device; pos, seq_lens [B] int32 device, each advanced by
  *   one at the end of the step iff advance != 0;
  *   logits [B,V] float device or NULL (an internal buffer is used);
- *   next_ids [B] int32 device (may be the same buffer as token_ids). */
+ *   next_ids [B] int32 device (may be the same buffer as token_ids).
+ * For batch <= 8 (and n_q_heads * head_dim == hidden) the whole step is ONE cooperative
+ * launch of a persistent kernel (one CTA per SM, grid-wide barriers between the products,
+ * weights and K/V streamed ahead through shared memory across all boundaries); larger
+ * batches run one kernel per product, chained with programmatic dependent launch.  A
+ * context serves one model at a time: the layer pointers are cached on the device and
+ * re-uploaded (asynchronously, on `stream`) whenever the arrays passed here change. */
 int fasttps_model_decode(fasttps_ctx *ctx, const void *embed, const fasttps_layer_weights *layers,
                          const void *g_final, const void *w_lm_head,
                          void *const *k_caches, void *const *v_caches,
                          const int32_t *token_ids, int32_t *pos, int32_t *seq_lens,
                          float *logits, int32_t *next_ids, int batch, int advance, void *stream);
+
+/* Greedy decode of n_steps consecutive tokens per sequence without returning to the host:
+ * step 0 consumes token_ids [B], every later step the argmax of the step before it.
+ *   out_ids [n_steps, B] int32 device: the token chosen at every step;
+ *   pos, seq_lens are advanced by n_steps (sequences that would outgrow max_seq are
+ *   reported in the status word and stop contributing at that point).
+ * For batch <= 8 all steps run inside one launch of the persistent kernel, so the weight
+ * stream never stops between tokens. */
+int fasttps_model_generate(fasttps_ctx *ctx, const void *embed, const fasttps_layer_weights *layers,
+                           const void *g_final, const void *w_lm_head,
+                           void *const *k_caches, void *const *v_caches,
+                           const int32_t *token_ids, int32_t *pos, int32_t *seq_lens,
+                           int32_t *out_ids, int n_steps, int batch, void *stream);
 
 /* End-to-end variant with HOST token buffers: copies host_token_ids [B] to the
  * device, runs fasttps_model_decode(advance = 1) on `stream`, copies next ids
@@ -167,16 +186,32 @@ int fasttps_model_decode_host(fasttps_ctx *ctx, const void *embed, const fasttps
                               const int32_t *host_token_ids, int32_t *pos, int32_t *seq_lens,
                               int32_t *host_next_ids, int batch, void *stream);
 
+/* Tuning switches of a context (host side, take effect at the next call):
+ *   "step_kernel" 0/1  route model calls with batch <= 8 through the persistent step kernel
+ *                      (default: environment variable FASTTPS_STEP_KERNEL, else 0);
+ *   "l2_ahead"    n    ring pieces the step kernel's L2 prefetch warp may run ahead (0 = off;
+ *                      default: FASTTPS_L2_AHEAD, else 0).
+ * Unknown names return FASTTPS_INVALID_ARG. */
+int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value);
+
 /* Synchronises the device and returns the status word (then clears it). */
 int fasttps_get_status(fasttps_ctx *ctx, uint32_t *host_status);
 /* Optional per-launch timing for benchmarks: while enabled, every kernel launch of this
  * context is bracketed by CUDA events on its stream (up to 8192 launches; not usable during
  * stream capture).  fasttps_profile_read() synchronises and sums the elapsed time and the
  * launch count per kernel class into arrays of FASTTPS_PROFILE_CLASSES entries, in the order
- * qkv projection, attention, output projection, fused MLP, lm_head, embedding gather. */
-#define FASTTPS_PROFILE_CLASSES 6
+ * qkv projection, attention, output projection, fused MLP, lm_head, embedding gather,
+ * persistent step kernel. */
+#define FASTTPS_PROFILE_CLASSES 7
 int fasttps_profile(fasttps_ctx *ctx, int enable);
 int fasttps_profile_read(fasttps_ctx *ctx, double *ms_per_class, uint64_t *launches_per_class);
+/* Phase timeline of the last launch of the persistent step kernel, for profiling: the first and
+ * the last CTA stamp the GPU global timer (ns) immediately before and after every grid-wide
+ * barrier (order per step: embedding, then per layer QKV, attention, output projection, MLP,
+ * then logits and argmax).  Synchronises, copies up to max_per_cta stamps of each of the two CTAs
+ * into stamps[0 .. max_per_cta) and stamps[max_per_cta .. 2 max_per_cta), returns the number
+ * of slots copied per CTA (slots past the launch's last stamp hold older or zero values). */
+int fasttps_trace_read(fasttps_ctx *ctx, uint64_t *stamps, int max_per_cta);
 /* Number of kernels this context has launched so far (host counter). */
 uint64_t fasttps_launch_count(const fasttps_ctx *ctx);
 /* Split count the attention kernel would use for this batch (for tests/benchmarks). */

@@ -61,6 +61,8 @@ def load_library() -> C.CDLL:
                                          ip, ip, ip, vp, ip, i, i, vp]
     lib.fasttps_model_decode_host.argtypes = [vp, vp, C.POINTER(LayerWeights), vp, vp, C.POINTER(vp), C.POINTER(vp),
                                               vp, ip, ip, vp, i, vp]
+    lib.fasttps_model_generate.argtypes = [vp, vp, C.POINTER(LayerWeights), vp, vp, C.POINTER(vp), C.POINTER(vp),
+                                           ip, ip, ip, ip, i, i, vp]
     lib.fasttps_get_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.fasttps_profile.argtypes = [vp, i]
     lib.fasttps_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
@@ -192,6 +194,14 @@ class Context:
                                              _ptr(next_ids), token_ids.shape[0], 1 if advance else 0,
                                              _stream(stream)), "fasttps_model_decode")
 
+    def model_generate(self, model, token_ids, pos, seq_lens, out_ids, stream=None):
+        """out_ids: int32 device tensor [n_steps, B]; pos/seq_lens are advanced by n_steps."""
+        n_steps, batch = out_ids.shape
+        _check(self.lib.fasttps_model_generate(self.handle, _ptr(model["embed"]), model["layers"],
+                                               _ptr(model["g_final"]), _ptr(model["w_lm"]), model["kc"], model["vc"],
+                                               _ptr(token_ids), _ptr(pos), _ptr(seq_lens), _ptr(out_ids), n_steps,
+                                               batch, _stream(stream)), "fasttps_model_generate")
+
     def model_decode_host(self, model, host_token_ids, pos, seq_lens, host_next_ids, stream=None):
         """host_token_ids / host_next_ids: numpy int32 arrays in host memory."""
         batch = int(host_token_ids.size)
@@ -206,17 +216,31 @@ class Context:
         _check(self.lib.fasttps_get_status(self.handle, C.byref(st)), "fasttps_get_status")
         return int(st.value)
 
-    PROFILE_CLASSES = ("qkv", "attn", "o_proj", "mlp", "lm_head", "embed")
+    PROFILE_CLASSES = ("qkv", "attn", "o_proj", "mlp", "lm_head", "embed", "step")
 
     def profile(self, enable: bool):
         _check(self.lib.fasttps_profile(self.handle, 1 if enable else 0), "fasttps_profile")
 
     def profile_read(self) -> dict:
         """{class: (total_ms, launches)} of the launches recorded since profile(True)."""
-        ms = (C.c_double * 6)()
-        n = (C.c_uint64 * 6)()
+        ms = (C.c_double * 7)()
+        n = (C.c_uint64 * 7)()
         _check(self.lib.fasttps_profile_read(self.handle, ms, n), "fasttps_profile_read")
         return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(self.PROFILE_CLASSES)}
+
+    def set_option(self, name: str, value: int):
+        self.lib.fasttps_set_option.argtypes = [C.c_void_p, C.c_char_p, C.c_int]
+        _check(self.lib.fasttps_set_option(self.handle, name.encode(), int(value)), "fasttps_set_option")
+
+    def trace_read(self, n: int = 4096):
+        """(first_cta, last_cta) numpy uint64 arrays of global-timer stamps around the grid barriers."""
+        import numpy as np
+        buf = np.zeros(2 * n, dtype=np.uint64)
+        self.lib.fasttps_trace_read.argtypes = [C.c_void_p, C.c_void_p, C.c_int]
+        got = self.lib.fasttps_trace_read(self.handle, buf.ctypes.data, n)
+        if got < 0:
+            _check(got, "fasttps_trace_read")
+        return buf[:got], buf[n:n + got]
 
     def launch_count(self) -> int:
         return int(self.lib.fasttps_launch_count(self.handle))

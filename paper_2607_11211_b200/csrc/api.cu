@@ -53,8 +53,10 @@ static void free_all(Ctx *c)
     cudaFree(c->cos_tab); cudaFree(c->sin_tab); cudaFree(c->attn_part); cudaFree(c->attn_ticket);
     cudaFree(c->mlp_acc); cudaFree(c->mlp_ticket); cudaFree(c->amax_val); cudaFree(c->amax_idx);
     cudaFree(c->amax_ticket); cudaFree(c->status); cudaFree(c->qkv); cudaFree(c->attn_out);
-    cudaFree(c->h); cudaFree(c->xa); cudaFree(c->xb); cudaFree(c->logits); cudaFree(c->tok);
+    cudaFree(c->h); cudaFree(c->xa); cudaFree(c->xb); cudaFree(c->logits); cudaFree(c->tok); cudaFree(c->tok2);
     if (c->pinned_tok) cudaFreeHost(c->pinned_tok);
+    cudaFree(c->grid_bar); cudaFree(c->d_layers); cudaFree(c->trace);
+    if (c->pin_layers) cudaFreeHost(c->pin_layers);
     if (c->prof_ev) {
         for (int i = 0; i < 2 * kProfMax; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
         delete[] c->prof_ev;
@@ -83,6 +85,12 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     FT_CUDA(cudaGetDeviceProperties(&c->prop, cfg->device));
     c->n_sm = c->prop.multiProcessorCount;
     {
+        const char *e = getenv("FASTTPS_STEP_KERNEL");
+        c->opt_step_kernel = (e && *e) ? atoi(e) != 0 : 0;
+        e = getenv("FASTTPS_L2_AHEAD");
+        c->opt_l2_ahead = (e && *e) ? atoi(e) : 0;
+    }
+    {
         int rc = configure_attn_kernels();
         if (rc == FASTTPS_OK) rc = configure_linear_kernels();
         if (rc == FASTTPS_OK) rc = configure_mlp_kernels();
@@ -98,7 +106,12 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     A(dev_alloc(&c->sin_tab, (size_t)f.max_seq * half, false));
     A(dev_alloc(&c->attn_part, B * f.n_q_heads * kMaxSplits * (f.head_dim + 2), true));
     A(dev_alloc(&c->attn_ticket, B * f.n_q_heads, true));
-    A(dev_alloc(&c->mlp_acc, B * D, true));
+    A(dev_alloc(&c->mlp_acc, 2 * B * D, true));
+    A(dev_alloc(&c->grid_bar, 128, true));
+    A(dev_alloc(&c->trace, 2 * (size_t)kTraceLen, true));
+    A(dev_alloc(&c->d_layers, (size_t)(f.n_layers > 0 ? f.n_layers : 1), true));
+    if (e == cudaSuccess)
+        e = cudaMallocHost(reinterpret_cast<void **>(&c->pin_layers), sizeof(LayerPtrs) * (size_t)(f.n_layers > 0 ? f.n_layers : 1));
     A(dev_alloc(&c->mlp_ticket, 1, true));
     A(dev_alloc(&c->amax_val, (size_t)kMaxNB * 1024, true));
     A(dev_alloc(&c->amax_idx, (size_t)kMaxNB * 1024, true));
@@ -111,6 +124,7 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     A(dev_alloc(&c->xb, B * D, true));
     A(dev_alloc(&c->logits, B * (size_t)f.vocab, true));
     A(dev_alloc(&c->tok, B, true));
+    A(dev_alloc(&c->tok2, B, true));
     if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void **>(&c->pinned_tok), 2 * B * sizeof(int32_t));
     if (e != cudaSuccess) {
         set_last_error(e, "fasttps_create: workspace allocation");
@@ -191,6 +205,7 @@ static int attn_impl(Ctx *c, const __nv_bfloat16 *q, const __nv_bfloat16 *k, con
     a.batch = batch; a.n_q_heads = f.n_q_heads; a.n_kv_heads = f.n_kv_heads;
     a.head_dim = f.head_dim; a.max_seq = f.max_seq;
     a.n_splits = attn_splits_for(c, batch);
+    a.len_add = 0;
     a.cos_tab = c->cos_tab; a.sin_tab = c->sin_tab;
     a.part = c->attn_part; a.ticket = c->attn_ticket; a.status = c->status;
     return launch_attn(c, a, st);
@@ -322,23 +337,100 @@ int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const
                       v_cache, pos, seq_lens, batch, static_cast<cudaStream_t>(stream));
 }
 
+static bool use_step_kernel(const Ctx *c, int batch)
+{
+    return c->opt_step_kernel != 0 && step_kernel_supported(c, batch);
+}
+
+int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value)
+{
+    if (!ctx || !name) return FASTTPS_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (strcmp(name, "step_kernel") == 0) c->opt_step_kernel = value != 0;
+    else if (strcmp(name, "l2_ahead") == 0) c->opt_l2_ahead = value < 0 ? 0 : (value > 64 ? 64 : value);
+    else return FASTTPS_INVALID_ARG;
+    return FASTTPS_OK;
+}
+
+static int model_args_ok(const Ctx *c, const void *embed, const fasttps_layer_weights *layers, const void *g_final,
+                         const void *w_lm_head, void *const *k_caches, void *const *v_caches, const int32_t *token_ids,
+                         const int32_t *pos, const int32_t *seq_lens, int batch)
+{
+    const fasttps_config &f = c->cfg;
+    if (batch < 1 || batch > f.max_batch || f.vocab < 1 || f.n_layers < 1) return FASTTPS_INVALID_ARG;
+    if (!aligned16(embed) || !layers || !aligned16(g_final) || !aligned16(w_lm_head) || !k_caches || !v_caches ||
+        !token_ids || !pos || !seq_lens)
+        return FASTTPS_INVALID_ARG;
+    for (int l = 0; l < f.n_layers; ++l)
+        if (!layer_ok(&layers[l]) || !aligned16(k_caches[l]) || !aligned16(v_caches[l])) return FASTTPS_INVALID_ARG;
+    return FASTTPS_OK;
+}
+
+// n_steps consecutive tokens in one launch of the persistent step kernel (batch <= 8)
+static int step_impl(Ctx *c, const void *embed, const fasttps_layer_weights *layers, const void *g_final,
+                     const void *w_lm_head, void *const *k_caches, void *const *v_caches, const int32_t *token_ids,
+                     int32_t *pos, int32_t *seq_lens, float *logits, int32_t *next_ids, int32_t *out_ids, int batch,
+                     int n_steps, int advance, cudaStream_t st)
+{
+    const fasttps_config &f = c->cfg;
+    // the device table of layer pointers is refreshed only when the caller's arrays change
+    bool same = c->layers_uploaded == f.n_layers;
+    for (int l = 0; l < f.n_layers; ++l) {
+        LayerPtrs lp;
+        lp.g_attn = static_cast<const __nv_bfloat16 *>(layers[l].g_attn_norm);
+        lp.w_qkv = static_cast<const __nv_bfloat16 *>(layers[l].w_qkv);
+        lp.w_o = static_cast<const __nv_bfloat16 *>(layers[l].w_o);
+        lp.g_mlp = static_cast<const __nv_bfloat16 *>(layers[l].g_mlp_norm);
+        lp.w_gu = static_cast<const __nv_bfloat16 *>(layers[l].w_gate_up);
+        lp.w_down = static_cast<const __nv_bfloat16 *>(layers[l].w_down);
+        lp.k_cache = static_cast<__nv_bfloat16 *>(k_caches[l]);
+        lp.v_cache = static_cast<__nv_bfloat16 *>(v_caches[l]);
+        if (!same || memcmp(&c->pin_layers[l], &lp, sizeof lp) != 0) {
+            same = false;
+            c->pin_layers[l] = lp;
+        }
+    }
+    if (!same) {
+        FT_CUDA(cudaMemcpyAsync(c->d_layers, c->pin_layers, sizeof(LayerPtrs) * f.n_layers, cudaMemcpyHostToDevice, st));
+        c->layers_uploaded = f.n_layers;
+    }
+    StepArgs a;
+    a.embed = static_cast<const __nv_bfloat16 *>(embed);
+    a.layers = c->d_layers;
+    a.g_final = static_cast<const __nv_bfloat16 *>(g_final);
+    a.w_lm = static_cast<const __nv_bfloat16 *>(w_lm_head);
+    a.token_ids = token_ids; a.pos = pos; a.seq_lens = seq_lens;
+    a.logits = logits; a.next_ids = next_ids; a.out_ids = out_ids;
+    a.batch = batch; a.n_steps = n_steps; a.advance = advance; a.n_layers = f.n_layers;
+    a.D = f.hidden; a.n_q_heads = f.n_q_heads; a.n_kv_heads = f.n_kv_heads; a.head_dim = f.head_dim;
+    a.K = f.inter; a.V = f.vocab; a.max_seq = f.max_seq; a.eps = f.rms_eps;
+    a.cos_tab = c->cos_tab; a.sin_tab = c->sin_tab;
+    a.x0 = c->xa; a.qkv = c->qkv; a.attn_out = c->attn_out; a.h = c->h;
+    a.acc = c->mlp_acc; a.attn_part = c->attn_part; a.attn_ticket = c->attn_ticket;
+    a.amax_val = c->amax_val; a.amax_idx = c->amax_idx; a.tok = c->tok2;
+    a.bar = c->grid_bar; a.status = c->status;
+    a.trace = c->trace; a.trace_len = kTraceLen;
+    a.l2_ahead = c->opt_l2_ahead;
+    return launch_step(c, a, st);
+}
+
 int fasttps_model_decode(fasttps_ctx *ctx, const void *embed, const fasttps_layer_weights *layers,
                          const void *g_final, const void *w_lm_head,
                          void *const *k_caches, void *const *v_caches,
                          const int32_t *token_ids, int32_t *pos, int32_t *seq_lens,
                          float *logits, int32_t *next_ids, int batch, int advance, void *stream)
 {
-    if (!ctx) return FASTTPS_INVALID_ARG;
+    if (!ctx || !next_ids) return FASTTPS_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);
     const fasttps_config &f = c->cfg;
-    if (batch < 1 || batch > f.max_batch || f.vocab < 1 || f.n_layers < 1) return FASTTPS_INVALID_ARG;
-    if (!aligned16(embed) || !layers || !aligned16(g_final) || !aligned16(w_lm_head) || !k_caches || !v_caches ||
-        !token_ids || !pos || !seq_lens || !next_ids)
-        return FASTTPS_INVALID_ARG;
-    for (int l = 0; l < f.n_layers; ++l)
-        if (!layer_ok(&layers[l]) || !aligned16(k_caches[l]) || !aligned16(v_caches[l])) return FASTTPS_INVALID_ARG;
+    int rc = model_args_ok(c, embed, layers, g_final, w_lm_head, k_caches, v_caches, token_ids, pos, seq_lens, batch);
+    if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int rc = launch_embed(c, static_cast<const __nv_bfloat16 *>(embed), token_ids, c->xa, batch, st);
+    if (use_step_kernel(c, batch))
+        return step_impl(c, embed, layers, g_final, w_lm_head, k_caches, v_caches, token_ids, pos, seq_lens, logits,
+                         next_ids, nullptr, batch, 1, advance, st);
+    // larger batches: one kernel per product, chained with programmatic dependent launch
+    rc = launch_embed(c, static_cast<const __nv_bfloat16 *>(embed), token_ids, c->xa, batch, st);
     if (rc) return rc;
     __nv_bfloat16 *cur = c->xa, *nxt = c->xb;
     for (int l = 0; l < f.n_layers; ++l) {
@@ -350,6 +442,29 @@ int fasttps_model_decode(fasttps_ctx *ctx, const void *embed, const fasttps_laye
     return linear_impl(c, f.hidden, f.vocab, cur, f.hidden, static_cast<const __nv_bfloat16 *>(g_final), w_lm_head,
                        nullptr, 0, nullptr, lg, f.vocab, batch, next_ids, advance ? pos : nullptr,
                        advance ? seq_lens : nullptr, kProfLmHead, st);
+}
+
+int fasttps_model_generate(fasttps_ctx *ctx, const void *embed, const fasttps_layer_weights *layers,
+                           const void *g_final, const void *w_lm_head,
+                           void *const *k_caches, void *const *v_caches,
+                           const int32_t *token_ids, int32_t *pos, int32_t *seq_lens,
+                           int32_t *out_ids, int n_steps, int batch, void *stream)
+{
+    if (!ctx || !out_ids || n_steps < 1) return FASTTPS_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    int rc = model_args_ok(c, embed, layers, g_final, w_lm_head, k_caches, v_caches, token_ids, pos, seq_lens, batch);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (use_step_kernel(c, batch))
+        return step_impl(c, embed, layers, g_final, w_lm_head, k_caches, v_caches, token_ids, pos, seq_lens, nullptr,
+                         out_ids + (size_t)(n_steps - 1) * batch, out_ids, batch, n_steps, 1, st);
+    for (int s = 0; s < n_steps; ++s) {
+        rc = fasttps_model_decode(ctx, embed, layers, g_final, w_lm_head, k_caches, v_caches,
+                                  s == 0 ? token_ids : out_ids + (size_t)(s - 1) * batch, pos, seq_lens, nullptr,
+                                  out_ids + (size_t)s * batch, batch, 1, stream);
+        if (rc) return rc;
+    }
+    return FASTTPS_OK;
 }
 
 int fasttps_model_decode_host(fasttps_ctx *ctx, const void *embed, const fasttps_layer_weights *layers,
@@ -413,6 +528,18 @@ int fasttps_profile_read(fasttps_ctx *ctx, double *ms_per_class, uint64_t *launc
         launches_per_class[c->prof_cls[i]] += 1;
     }
     return FASTTPS_OK;
+}
+
+int fasttps_trace_read(fasttps_ctx *ctx, uint64_t *stamps, int max_per_cta)
+{
+    if (!ctx || !stamps || max_per_cta < 1) return FASTTPS_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    const int n = max_per_cta < kTraceLen ? max_per_cta : kTraceLen;
+    FT_CUDA(cudaDeviceSynchronize());
+    for (int k = 0; k < 2; ++k)
+        FT_CUDA(cudaMemcpy(stamps + (size_t)k * max_per_cta, c->trace + (size_t)k * kTraceLen, sizeof(uint64_t) * n,
+                           cudaMemcpyDeviceToHost));
+    return n;
 }
 
 uint64_t fasttps_launch_count(const fasttps_ctx *ctx)

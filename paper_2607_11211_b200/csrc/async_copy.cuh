@@ -117,19 +117,41 @@ struct WeightRing {
             mbar_fence_init();
         }
     }
-    // one thread of the producer warp: stream every piece, then return
+    // producer thread: wait until the slot of piece g is free again (false after a failed bounded wait)
+    __device__ __forceinline__ bool acquire(int g)
+    {
+        if (g >= nslot && !mbar_wait_bounded(&empty[g % nslot], (uint32_t)(g / nslot - 1) & 1u, abort_flag)) {
+            *abort_flag = 1;
+            return false;
+        }
+        return true;
+    }
+    // producer thread: piece g = `bytes` contiguous bytes at src
+    __device__ __forceinline__ bool put(int g, const void *src, uint32_t bytes)
+    {
+        if (!acquire(g)) return false;
+        const int s = g % nslot;
+        mbar_expect_tx(&full[s], bytes);
+        bulk_g2s(slots + (size_t)s * slot_bytes, src, bytes, &full[s]);
+        return true;
+    }
+    // producer thread: piece g = two blocks of `bytes` each, the second landing at offset off1 of the slot
+    __device__ __forceinline__ bool put2(int g, const void *src0, const void *src1, uint32_t bytes, uint32_t off1)
+    {
+        if (!acquire(g)) return false;
+        const int s = g % nslot;
+        mbar_expect_tx(&full[s], 2 * bytes);
+        bulk_g2s(slots + (size_t)s * slot_bytes, src0, bytes, &full[s]);
+        bulk_g2s(slots + (size_t)s * slot_bytes + off1, src1, bytes, &full[s]);
+        return true;
+    }
+    // one thread of the producer warp: stream every piece of the two runs given to init(), then return
     __device__ __forceinline__ void produce()
     {
         for (int g = 0; g < pieces; ++g) {
-            const int s = g % nslot;
-            if (g >= nslot && !mbar_wait_bounded(&empty[s], (uint32_t)(g / nslot - 1) & 1u, abort_flag)) {
-                *abort_flag = 1;
-                return;
-            }
             const unsigned char *src = g < pieces0 ? base0 + (size_t)g * slot_bytes
                                                    : base1 + (size_t)(g - pieces0) * slot_bytes;
-            mbar_expect_tx(&full[s], (uint32_t)slot_bytes);
-            bulk_g2s(slots + (size_t)s * slot_bytes, src, (uint32_t)slot_bytes, &full[s]);
+            if (!put(g, src, (uint32_t)slot_bytes)) return;
         }
     }
     // every lane of a consumer warp; returns the slot holding piece g (ok is cleared on a failed wait)

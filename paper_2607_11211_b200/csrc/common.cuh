@@ -15,7 +15,16 @@ constexpr unsigned kFull = 0xffffffffu;
 
 // ------------------------------------------------------------------ context
 
+struct LayerPtrs;
+
 struct Ctx {
+    // persistent step kernel: grid barrier words, device table of layer pointers and its pinned shadow
+    unsigned *grid_bar;
+    unsigned long long *trace;       // [2][kTraceLen] phase timeline of the last step-kernel launch
+    LayerPtrs *d_layers, *pin_layers;
+    int layers_uploaded;             // number of valid entries in pin_layers / d_layers
+    int opt_step_kernel;             // 1: model calls with batch <= 8 use the persistent step kernel
+    int opt_l2_ahead;                // lookahead of its L2 prefetch warp in ring pieces (0 = off)
     fasttps_config cfg;
     int n_sm;
     cudaDeviceProp prop;
@@ -36,6 +45,7 @@ struct Ctx {
     __nv_bfloat16 *xa, *xb;          // [max_batch][D]
     float *logits;                   // [max_batch][V]
     int32_t *tok;                    // [max_batch] staging for the host-buffer entry point
+    int32_t *tok2;                   // [max_batch] current tokens inside the persistent step kernel
     int32_t *pinned_tok;             // pinned host staging [2][max_batch]
     uint64_t launches;
     // optional per-launch timing (CUDA events on the launch stream), off by default
@@ -46,7 +56,8 @@ struct Ctx {
 };
 
 constexpr int kProfMax = 8192;
-enum ProfClass { kProfQkv = 0, kProfAttn, kProfOproj, kProfMlp, kProfLmHead, kProfEmbed, kProfClasses };
+constexpr int kTraceLen = 4096;      // global-timer stamps kept per traced CTA of the step kernel
+enum ProfClass { kProfQkv = 0, kProfAttn, kProfOproj, kProfMlp, kProfLmHead, kProfEmbed, kProfStep, kProfClasses };
 
 // Brackets one kernel launch with events when profiling is on.
 struct ProfScope {
@@ -150,6 +161,25 @@ __device__ __forceinline__ int ld_cg_s32(const int *p)
     return v;
 }
 
+__device__ __forceinline__ __nv_bfloat16 ld_cg_bf16(const __nv_bfloat16 *p)
+{
+    unsigned short v;
+    asm volatile("ld.global.cg.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return __ushort_as_bfloat16(v);
+}
+__device__ __forceinline__ uint4 ld_cg_u4(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float4 ld_cg_f4(const float *p)
+{
+    float4 v;
+    asm volatile("ld.global.cg.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+
 __device__ __forceinline__ void red_add_v4(float *p, float a, float b, float c, float d)
 {
     asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
@@ -235,6 +265,7 @@ struct AttnArgs {
     __nv_bfloat16 *out;
     int out_stride;
     int batch, n_q_heads, n_kv_heads, head_dim, max_seq, n_splits;
+    int len_add;                      // added to every seq_lens / pos entry (step index of a multi-step launch)
     const float *cos_tab, *sin_tab;
     float *part;
     int *ticket;
@@ -255,7 +286,43 @@ struct MlpArgs {
     uint32_t *status;
 };
 
+// One layer's packed weights and caches, as the persistent step kernel reads them (device table).
+struct LayerPtrs {
+    const __nv_bfloat16 *g_attn, *w_qkv, *w_o, *g_mlp, *w_gu, *w_down;
+    __nv_bfloat16 *k_cache, *v_cache;
+};
+
+struct StepArgs {
+    const __nv_bfloat16 *embed;      // [V][D]
+    const LayerPtrs *layers;         // device table [n_layers]
+    const __nv_bfloat16 *g_final, *w_lm;
+    const int32_t *token_ids;        // [B] tokens of the first step
+    int32_t *pos, *seq_lens;         // [B]; advanced by n_steps at the end iff advance
+    float *logits;                   // [B][V] of the last step, or null
+    int32_t *next_ids;               // [B] argmax of the last step
+    int32_t *out_ids;                // [n_steps][B] argmax of every step, or null
+    int batch, n_steps, advance, n_layers;
+    int D, n_q_heads, n_kv_heads, head_dim, K, V, max_seq;
+    float eps;
+    const float *cos_tab, *sin_tab;
+    // workspace
+    __nv_bfloat16 *x0, *qkv, *attn_out, *h;
+    float *acc;                      // [2][B][D] FP32, zero on entry and on exit
+    float *attn_part;
+    int *attn_ticket;
+    float *amax_val;
+    int *amax_idx;
+    int32_t *tok;                    // [B] current tokens
+    unsigned *bar;                   // grid barrier: [0] arrivals, [32] abort flag, [64] generation
+    uint32_t *status;
+    unsigned long long *trace;       // [2][trace_len] global-timer stamps of the first and last CTA, or null
+    int trace_len;
+    int l2_ahead;                    // ring pieces the optional L2 prefetch warp may lead the producer by (0 = off)
+};
+
 int launch_linear(Ctx *c, const LinearArgs &a, cudaStream_t st);
+bool step_kernel_supported(const Ctx *c, int batch);
+int launch_step(Ctx *c, const StepArgs &a, cudaStream_t st);
 int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st);
 int launch_mlp(Ctx *c, const MlpArgs &a, cudaStream_t st);
 int launch_embed(Ctx *c, const __nv_bfloat16 *embed, const int32_t *ids, __nv_bfloat16 *x, int batch, cudaStream_t st);

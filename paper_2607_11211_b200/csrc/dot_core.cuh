@@ -54,10 +54,13 @@ __host__ __device__ inline WarpSplit warp_split(int n_in)
 // B fragments of this consumer thread: the bf16 activations x[g][32 (w + nw i) + 8 t4 .. + 8) for its
 // IPW k blocks, batch row g = lane / 4 (zero for g >= batch), optionally RMS-normalised (gain gn, eps)
 // with the result rounded to bf16 like a stored tensor.  Consumer threads only (named barrier 1).
-// smem_red: nw * 8 floats.
+// smem_red: nw * 8 floats.  If `add` is given (FP32 [batch][n_in], e.g. the MLP partial sums of the
+// previous layer), the activation is bf16(x + add).  All loads bypass L1: inside a persistent kernel the
+// activations were written by other SMs.
 template <int IPW>
 __device__ __forceinline__ void load_b_frags(uint32_t (&bf)[IPW][4], const __nv_bfloat16 *x, int x_stride, int batch,
-                                             int n_in, int nw, const __nv_bfloat16 *gn, float eps, float *smem_red)
+                                             int n_in, int nw, const __nv_bfloat16 *gn, float eps, float *smem_red,
+                                             const float *add = nullptr)
 {
     const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3;
     const bool live = g < batch;
@@ -65,7 +68,14 @@ __device__ __forceinline__ void load_b_frags(uint32_t (&bf)[IPW][4], const __nv_
     for (int i = 0; i < IPW; ++i) {
         const int k = 32 * (w + nw * i) + 8 * t4;
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (live) v = *reinterpret_cast<const uint4 *>(x + (size_t)g * x_stride + k);
+        if (live) v = ld_cg_u4(x + (size_t)g * x_stride + k);
+        if (live && add) {
+            const float4 a0 = ld_cg_f4(add + (size_t)g * n_in + k), a1 = ld_cg_f4(add + (size_t)g * n_in + k + 4);
+            v.x = pack2(bf_lo(v.x) + a0.x, bf_hi(v.x) + a0.y);
+            v.y = pack2(bf_lo(v.y) + a0.z, bf_hi(v.y) + a0.w);
+            v.z = pack2(bf_lo(v.z) + a1.x, bf_hi(v.z) + a1.y);
+            v.w = pack2(bf_lo(v.w) + a1.z, bf_hi(v.w) + a1.w);
+        }
         bf[i][0] = v.x; bf[i][1] = v.y; bf[i][2] = v.z; bf[i][3] = v.w;
     }
     if (gn == nullptr) return;

@@ -1,0 +1,493 @@
+// Persistent decode-step kernel: the whole token phase of the model -- embedding gather, then for
+// every layer RMSNorm -> QKV -> attention (Algorithm 3) -> output projection -> RMSNorm -> fused MLP
+// (Algorithm 4), then the final norm, the logits and the greedy argmax -- in ONE cooperative launch,
+// for one or several consecutive tokens.
+//
+// Why: at batch 1 a layer is ~40 us of HBM streaming cut into four dependent products.  As separate
+// kernels each of them pays a launch, a cold start of its copy pipeline and a drain (~5 us, more for
+// attention), during which HBM idles.  Here one CTA per SM stays resident; a producer warp walks the
+// CTA's share of EVERY weight matrix and K/V tile of the step in order and keeps the shared-memory
+// ring (~190 KB per SM) full, never waiting for anything but free slots; the consumer warps meet at
+// a grid-wide barrier after each product.  While they wait there, or run the latency-bound parts of
+// attention, the bytes of the next product keep arriving, so HBM stays busy across all boundaries.
+//
+// Grid barrier: sense-reversing counter in global memory, bounded wait, abort flag (no CTA ever
+// spins forever; the launch is cooperative, so all CTAs are resident).
+#include "attn_core.cuh"
+#include "mlp_core.cuh"
+#include "stream_launch.cuh"
+
+namespace fasttps {
+
+namespace {
+
+constexpr unsigned long long kGridWaitNanos = 500ull * 1000 * 1000;   // 0.5 s per barrier at most
+constexpr int kMegaThreadsMax = 448;                                   // up to 12 consumer warps + producer + prefetcher
+
+// the 32 lanes of the prefetch warp ask L2 for the 128-byte lines of [p, p + bytes)
+__device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
+{
+    const unsigned char *q = static_cast<const unsigned char *>(p);
+    for (uint32_t off = (threadIdx.x & 31) * 128u; off < bytes; off += 32u * 128u)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(q + off));
+}
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+struct GridBarrier {
+    unsigned *count;  // arrivals since the launch (zeroed by the host before every launch)
+    int *abort;
+    unsigned target;  // arrivals that complete the barrier this CTA waits at next
+    int ncta;
+    int *s_go;        // shared-memory word
+};
+
+// All consumer threads of every CTA.  `ok` = this thread saw no failed wait.  Returns the same verdict in
+// every thread of the grid that gets past it: false means "leave now".  One atomic per CTA and barrier;
+// the waiters poll the arrival counter itself.
+__device__ __forceinline__ bool grid_sync(GridBarrier &gb, int nct, bool ok)
+{
+    const bool all_ok = named_bar_and(1, nct, ok);       // CTA verdict; all global writes of the phase are issued
+    if (threadIdx.x == 0) {
+        int go = 1;
+        if (!all_ok) { atomicExch(gb.abort, 1); go = 0; }
+        __threadfence();
+        atomicAdd(gb.count, 1u);
+        unsigned long long t0 = 0;
+        for (unsigned it = 1; ld_acquire_u32(gb.count) < gb.target; ++it) {
+            if ((it & 63u) == 0) {                       // now and then: has anybody given up? have we waited too long?
+                if (ld_cg_s32(gb.abort)) { go = 0; break; }
+                const unsigned long long now = global_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > kGridWaitNanos) { atomicExch(gb.abort, 1); go = 0; break; }
+            }
+        }
+        if (!all_ok || ld_cg_s32(gb.abort)) go = 0;
+        *gb.s_go = go;
+    }
+    named_bar_sync(1, nct);
+    gb.target += (unsigned)gb.ncta;
+    return *gb.s_go != 0;
+}
+
+__host__ __device__ inline void cta_range(int n_units, int cta, int ncta, int &u0, int &n)
+{
+    const int base = n_units / ncta, rem = n_units % ncta;
+    u0 = cta * base + (cta < rem ? cta : rem);
+    n = base + (cta < rem ? 1 : 0);
+}
+
+struct MegaLayout {
+    int nw, ipw, nslot, slot_stride, wpiece;
+    size_t ring_off, bar_off, abort_off, part_off, red_off, scratch_off, total;
+};
+
+template <int DH>
+__host__ __device__ inline MegaLayout mega_layout(int D)
+{
+    MegaLayout l;
+    const WarpSplit s = warp_split(D);
+    l.nw = s.nw; l.ipw = s.ipw;
+    l.wpiece = kBlocksPerWarpPerSlot * (s.nw > 0 ? s.nw : 1) * kTileBytes;
+    l.slot_stride = l.wpiece > AttnTile<DH>::kPieceBytes ? l.wpiece : AttnTile<DH>::kPieceBytes;
+    l.nslot = kRingBudget / l.slot_stride;
+    if (l.nslot > 8) l.nslot = 8;
+    l.ring_off = 0;
+    l.bar_off = (size_t)l.nslot * l.slot_stride;
+    l.abort_off = l.bar_off + 2 * 8 * 8;
+    l.part_off = l.abort_off + 16;
+    l.red_off = l.part_off + sizeof(float) * 2 * (size_t)s.nw * 128;
+    l.scratch_off = (l.red_off + sizeof(float) * (size_t)s.nw * 8 + 15) & ~(size_t)15;
+    l.total = l.scratch_off + sizeof(AttnScratch<DH>);
+    return l;
+}
+
+__device__ __forceinline__ AttnArgs attn_args_of(const StepArgs &a, const LayerPtrs &lp, int step, int ncta_attn)
+{
+    AttnArgs aa;
+    const int nq = a.n_q_heads * a.head_dim, nkv = a.n_kv_heads * a.head_dim;
+    aa.q = a.qkv; aa.k_new = a.qkv + nq; aa.v_new = a.qkv + nq + nkv;
+    aa.q_stride = nq + 2 * nkv; aa.kv_stride = nq + 2 * nkv;
+    aa.k_cache = lp.k_cache; aa.v_cache = lp.v_cache;
+    aa.pos = a.pos; aa.seq_lens = a.seq_lens;
+    aa.out = a.attn_out; aa.out_stride = nq;
+    aa.batch = a.batch; aa.n_q_heads = a.n_q_heads; aa.n_kv_heads = a.n_kv_heads;
+    aa.head_dim = a.head_dim; aa.max_seq = a.max_seq; aa.n_splits = ncta_attn; aa.len_add = step;
+    aa.cos_tab = a.cos_tab; aa.sin_tab = a.sin_tab;
+    aa.part = a.attn_part; aa.ticket = a.attn_ticket; aa.status = a.status;
+    return aa;
+}
+
+template <int IPW, int DH>
+__global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArgs a)
+{
+    extern __shared__ __align__(128) unsigned char dsm[];
+    __shared__ __align__(16) ActTile s_hi[kMaxOctetsPerCta];
+    __shared__ __align__(16) ActTile s_lo[kMaxOctetsPerCta];
+    __shared__ float s_best_val[64];
+    __shared__ int s_best_idx[64];
+    __shared__ int s_go;
+    __shared__ int s_steps_done;
+    __shared__ int s_prod_piece;      // pieces the producer has issued so far (read by the prefetcher)
+
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    const int cta = blockIdx.x, ncta = gridDim.x;
+    if (t == 0) { s_steps_done = 0; s_prod_piece = 0; }
+    const MegaLayout lay = mega_layout<DH>(a.D);
+    const int nw = lay.nw, nct = nw * 32;
+    float *smem_part = reinterpret_cast<float *>(dsm + lay.part_off);
+    float *smem_red = reinterpret_cast<float *>(dsm + lay.red_off);
+    AttnScratch<DH> &scratch = *reinterpret_cast<AttnScratch<DH> *>(dsm + lay.scratch_off);
+
+    const int D = a.D, B = a.batch;
+    const int nq = a.n_q_heads * a.head_dim, nkv = a.n_kv_heads * a.head_dim, nqkv = nq + 2 * nkv;
+    constexpr int SPT = IPW / kBlocksPerWarpPerSlot;      // ring pieces per 16-row tile
+    constexpr int PPO = IPW / 4;                          // ring pieces per W_down octet
+    const size_t tile_bytes = (size_t)D * 32;             // 16 rows x D (every reduction length here is D)
+    const size_t oct_bytes = (size_t)D * 16;
+
+    // this CTA's share of every product (the same for every layer)
+    int q0, qn, o0, on, m0, mn, l0, ln;
+    cta_range((nqkv + 15) >> 4, cta, ncta, q0, qn);
+    cta_range((D + 15) >> 4, cta, ncta, o0, on);
+    cta_range(a.K >> 3, cta, ncta, m0, mn);
+    cta_range((a.V + 15) >> 4, cta, ncta, l0, ln);
+    int ncta_attn = (kMaxSplits - 2) * a.n_q_heads;
+    if (ncta_attn > ncta) ncta_attn = ncta;
+
+    WeightRing ring;
+    ring.init(dsm + lay.ring_off, reinterpret_cast<uint64_t *>(dsm + lay.bar_off),
+              reinterpret_cast<int *>(dsm + lay.abort_off), lay.nslot, lay.slot_stride, nw, nullptr, 0, nullptr, 0);
+    if (t < 64) { s_best_val[t] = -INFINITY; s_best_idx[t] = 0x7fffffff; }
+    __syncthreads();
+
+    // =========================================================================== producer and prefetch warps
+    // Both walk the SAME schedule: this CTA's share of every weight matrix and K/V tile of every step, in
+    // the order the consumers need it.  The producer copies piece after piece into the shared-memory ring
+    // and blocks only on free slots.  The optional prefetcher (l2_ahead > 0) runs further ahead and only asks
+    // L2 for the lines (prefetch.global.L2 through the load path, so the copy engine stays free), so that HBM
+    // keeps streaming while the consumers sit in barriers or in the latency-bound parts of attention; it
+    // stays at most l2_ahead pieces in front of the producer.  All its lanes walk the schedule in lockstep.
+    if (w >= nw) {
+        const bool is_prefetcher = (w == nw + 1);
+        if (w > nw + 1 || (is_prefetcher ? a.l2_ahead <= 0 : lane != 0)) return;
+        const int kPrefetchAhead = a.l2_ahead;
+        const uint32_t wp = (uint32_t)lay.wpiece;
+        int piece = 0;
+        // throttle of the prefetcher: wait (bounded) until the producer is within kPrefetchAhead pieces
+        auto throttle = [&]() -> bool {
+            if (piece - *reinterpret_cast<volatile int *>(&s_prod_piece) <= kPrefetchAhead) return true;
+            const unsigned long long t0 = global_ns();
+            while (piece - *reinterpret_cast<volatile int *>(&s_prod_piece) > kPrefetchAhead) {
+                if (*ring.abort_flag || global_ns() - t0 > kGridWaitNanos) return false;
+                __nanosleep(200);
+            }
+            return true;
+        };
+        auto weights = [&](const void *base, size_t first_byte, int npieces) -> bool {
+            const unsigned char *p = static_cast<const unsigned char *>(base) + first_byte;
+            for (int i = 0; i < npieces; ++i, ++piece) {
+                if (is_prefetcher) {
+                    if (!throttle()) return false;
+                    prefetch_l2(p + (size_t)i * wp, wp);
+                } else {
+                    if (!ring.put(piece, p + (size_t)i * wp, wp)) return false;
+                    *reinterpret_cast<volatile int *>(&s_prod_piece) = piece + 1;
+                }
+            }
+            return true;
+        };
+        for (int step = 0; step < a.n_steps; ++step) {
+            for (int l = 0; l < a.n_layers; ++l) {
+                const LayerPtrs lp = a.layers[l];
+                if (!weights(lp.w_qkv, (size_t)q0 * tile_bytes, qn * SPT)) return;
+                if (!is_prefetcher && step > 0 && l == 0) {
+                    // K/V tiles of this step include the rows appended by the step before it: they may be
+                    // copied only once that step is complete grid-wide (weights are never held back).  For
+                    // all but toy models the flag is set long before the producer gets here.
+                    const unsigned long long t0 = global_ns();
+                    while (*reinterpret_cast<volatile int *>(&s_steps_done) < step) {
+                        if (*ring.abort_flag || global_ns() - t0 > kGridWaitNanos) { *ring.abort_flag = 1; return; }
+                        __nanosleep(64);
+                    }
+                }
+                const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
+                const bool kv_ok = attn_for_each_tile<DH>(aa, cta, ncta_attn, [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
+                    if (is_prefetcher) {
+                        if (!throttle()) return false;
+                        prefetch_l2(k, bytes);
+                        prefetch_l2(v, bytes);
+                        ++piece;
+                        return true;
+                    }
+                    const bool r = ring.put2(piece, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
+                    *reinterpret_cast<volatile int *>(&s_prod_piece) = ++piece;
+                    return r;
+                });
+                if (!kv_ok) return;
+                if (!weights(lp.w_o, (size_t)o0 * tile_bytes, on * SPT)) return;
+                if (!weights(lp.w_gu, (size_t)m0 * tile_bytes, mn * SPT)) return;
+                if (!weights(lp.w_down, (size_t)m0 * oct_bytes, mn * PPO)) return;
+            }
+            if (!weights(a.w_lm, (size_t)l0 * tile_bytes, ln * SPT)) return;
+        }
+        return;
+    }
+
+    // =========================================================================== consumer warps
+    GridBarrier gb;
+    // arrivals and abort flag in two different 128-byte lines
+    gb.count = a.bar; gb.abort = reinterpret_cast<int *>(a.bar + 32);
+    gb.ncta = ncta; gb.s_go = &s_go;
+    gb.target = (unsigned)ncta;
+    if (cta == 0 && t == 0) {
+        // sequences that cannot be served for all steps are reported once and contribute no rows
+        for (int bb = 0; bb < B; ++bb) {
+            const int L = a.seq_lens[bb], p = a.pos[bb];
+            if (L < 0 || L + a.n_steps > a.max_seq) atomicOr(a.status, FASTTPS_DEV_CACHE_FULL);
+            else if (p < 0 || p + a.n_steps > a.max_seq) atomicOr(a.status, FASTTPS_DEV_BAD_POSITION);
+        }
+    }
+
+    // gathers the embedding rows of the current tokens into x0 (CTA 0 only)
+    auto embed_rows = [&](const int32_t *ids) {
+        for (int idx = t; idx < B * (D >> 3); idx += nct) {
+            const int b = idx / (D >> 3), j = idx - b * (D >> 3);
+            int id = ld_cg_s32(ids + b);
+            if (id < 0 || id >= a.V) { if (j == 0) atomicOr(a.status, FASTTPS_DEV_BAD_TOKEN); id = 0; }
+            reinterpret_cast<uint4 *>(a.x0 + (size_t)b * D)[j] = reinterpret_cast<const uint4 *>(a.embed + (size_t)id * D)[j];
+        }
+    };
+
+    uint32_t bf[IPW][4];
+    int piece = 0;
+    bool ok = true;
+
+    // optional timeline for profiling: the first and the last CTA stamp the global timer before and
+    // after every grid barrier
+    int n_stamp = 0;
+    auto stamp = [&]() {
+        if (a.trace && t == 0 && (cta == 0 || cta == ncta - 1) && n_stamp < a.trace_len)
+            a.trace[(size_t)(cta ? 1 : 0) * a.trace_len + n_stamp] = global_ns();
+        ++n_stamp;
+    };
+    auto sync_phase = [&]() -> bool {
+        stamp();
+        const bool go = grid_sync(gb, nct, /*ok=*/ok);
+        stamp();
+        return go;
+    };
+
+    if (cta == 0) embed_rows(a.token_ids);
+    if (!sync_phase()) return;
+
+    for (int step = 0; step < a.n_steps; ++step) {
+        for (int l = 0; l < a.n_layers; ++l) {
+            const LayerPtrs lp = a.layers[l];
+            const float *y_prev = l > 0 ? a.acc + (size_t)((l - 1) & 1) * B * D : nullptr;   // MLP sums of layer l - 1
+            const __nv_bfloat16 *x_base = l > 0 ? a.h : a.x0;                             // x_l = bf16(x_base + y_prev)
+
+            // ---- RMSNorm -> QKV ----
+            load_b_frags<IPW>(bf, x_base, D, B, D, nw, lp.g_attn, a.eps, smem_red, y_prev);
+            ok = dot_tiles<IPW>(ring, piece, qn, nw, bf, smem_part, [&](int tile, int cc, int b, float v0, float v1) {
+                if (b >= B) return;
+                const int row = (q0 + tile) * 16 + cc;
+                if (row < nqkv) a.qkv[(size_t)b * nqkv + row] = __float2bfloat16_rn(v0);
+                if (row + 8 < nqkv) a.qkv[(size_t)b * nqkv + row + 8] = __float2bfloat16_rn(v1);
+            }) && ok;
+            piece += qn * SPT;
+            if (!sync_phase()) return;
+
+            // ---- attention (Algorithm 3) ----
+            {
+                const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
+                ok = attn_consume<DH>(aa, ring, piece, cta, ncta_attn, scratch, nw) && ok;
+            }
+            if (!sync_phase()) return;
+
+            // ---- output projection + residual: h = x_l + attn . W_o ----
+            load_b_frags<IPW>(bf, a.attn_out, nq, B, D, nw, nullptr, a.eps, smem_red);
+            ok = dot_tiles<IPW>(ring, piece, on, nw, bf, smem_part, [&](int tile, int cc, int b, float v0, float v1) {
+                if (b >= B) return;
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int row = (o0 + tile) * 16 + cc + 8 * hh;
+                    if (row >= D) continue;
+                    float x = __bfloat162float(ld_cg_bf16(x_base + (size_t)b * D + row));
+                    if (y_prev) x = bf16_round(x + ld_cg_f32(y_prev + (size_t)b * D + row));
+                    a.h[(size_t)b * D + row] = __float2bfloat16_rn(x + (hh ? v1 : v0));
+                }
+            }) && ok;
+            piece += on * SPT;
+            if (!sync_phase()) return;
+
+            // ---- RMSNorm -> fused MLP (Algorithm 4); the sums of all CTAs meet in acc[l & 1] ----
+            float *y_cur = a.acc + (size_t)(l & 1) * B * D;
+            load_b_frags<IPW>(bf, a.h, D, B, D, nw, lp.g_mlp, a.eps, smem_red);
+            ok = mlp_gate_up_phase<IPW>(ring, piece, mn, nw, bf, smem_part, s_hi, s_lo) && ok;
+            piece += mn * SPT;
+            if (cta == 0 && y_prev) {
+                // layer l - 1's sums have been consumed by everyone (two barriers ago): zero them for layer l + 1
+                float *z = a.acc + (size_t)((l - 1) & 1) * B * D;
+                for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            named_bar_sync(1, nct);
+            {
+                float acc[IPW][2][4];
+#pragma unroll
+                for (int i = 0; i < IPW; ++i)
+#pragma unroll
+                    for (int m = 0; m < 2; ++m)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) acc[i][m][e] = 0.f;
+                mlp_down_phase<IPW>(ring, piece, mn, nw, s_hi, s_lo, acc, ok);
+                piece += mn * PPO;
+                mlp_scatter_add<IPW>(acc, smem_part, y_cur, B, D, nw);
+            }
+            if (!sync_phase()) return;
+        }
+
+        // ---- final norm -> logits -> greedy argmax ----
+        {
+            const int L = a.n_layers;
+            const float *y_last = a.acc + (size_t)((L - 1) & 1) * B * D;
+            load_b_frags<IPW>(bf, a.h, D, B, D, nw, a.g_final, a.eps, smem_red, y_last);
+            for (int u = t; u < 64; u += nct) { s_best_val[u] = -INFINITY; s_best_idx[u] = 0x7fffffff; }
+            named_bar_sync(1, nct);
+            ok = dot_tiles<IPW>(ring, piece, ln, nw, bf, smem_part, [&](int tile, int cc, int b, float v0, float v1) {
+                if (b >= B) return;
+                const int u = cc * 8 + b;
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int row = (l0 + tile) * 16 + cc + 8 * hh;
+                    if (row >= a.V) continue;
+                    const float v = hh ? v1 : v0;
+                    if (a.logits) a.logits[(size_t)b * a.V + row] = v;
+                    if (v > s_best_val[u]) { s_best_val[u] = v; s_best_idx[u] = row; }   // rows ascend: first max kept
+                }
+            }) && ok;
+            piece += ln * SPT;
+            named_bar_sync(1, nct);
+            if (t < 8 && t < B) {
+                float bv = -INFINITY; int bi = 0x7fffffff;
+                for (int cc = 0; cc < 8; ++cc) {
+                    const float v = s_best_val[cc * 8 + t]; const int i = s_best_idx[cc * 8 + t];
+                    if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+                }
+                a.amax_val[(size_t)t * ncta + cta] = bv;
+                a.amax_idx[(size_t)t * ncta + cta] = bi;
+            }
+            if (!sync_phase()) return;
+
+            if (cta == 0) {
+                // every thread fetches its share of the per-CTA candidates at once, then warps and the CTA reduce
+                for (int b = 0; b < B; ++b) {
+                    float bv = -INFINITY; int bi = 0x7fffffff;
+                    for (int c = t; c < ncta; c += nct) {
+                        const float v = ld_cg_f32(a.amax_val + (size_t)b * ncta + c);
+                        const int i = ld_cg_s32(a.amax_idx + (size_t)b * ncta + c);
+                        if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+                    }
+#pragma unroll
+                    for (int s = 16; s >= 1; s >>= 1) {
+                        const float ov = __shfl_xor_sync(kFull, bv, s);
+                        const int oi = __shfl_xor_sync(kFull, bi, s);
+                        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+                    }
+                    if (lane == 0) { s_best_val[w] = bv; s_best_idx[w] = bi; }
+                    named_bar_sync(1, nct);
+                    if (t == 0) {
+                        for (int w2 = 0; w2 < nw; ++w2) {
+                            const float v = s_best_val[w2]; const int i = s_best_idx[w2];
+                            if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+                        }
+                        if (bi == 0x7fffffff) bi = 0;      // all-NaN row: fall back to index 0
+                        a.tok[b] = bi;
+                        if (a.out_ids) a.out_ids[(size_t)step * B + b] = bi;
+                        if (step == a.n_steps - 1) {
+                            a.next_ids[b] = bi;
+                            if (a.advance) { a.pos[b] += a.n_steps; a.seq_lens[b] += a.n_steps; }
+                        }
+                    }
+                    named_bar_sync(1, nct);
+                }
+                // the last layer's MLP sums are consumed: back to zero (the other buffer was zeroed in the last MLP phase)
+                float *z = a.acc + (size_t)((L - 1) & 1) * B * D;
+                for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (step + 1 < a.n_steps) {
+                    __threadfence();
+                    named_bar_sync(1, nct);
+                    embed_rows(a.tok);
+                }
+            }
+            if (step + 1 < a.n_steps) {
+                if (!sync_phase()) return;
+                if (t == 0) atomicExch(&s_steps_done, step + 1);    // the producer may fetch the new K/V rows now
+            }
+        }
+    }
+}
+
+}  // namespace
+
+template <int IPW, int DH>
+static int launch_step_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
+{
+    const MegaLayout lay = mega_layout<DH>(a.D);
+    auto kernel = decode_step_kernel<IPW, DH>;
+    static bool configured[16] = {};
+    if (!configured[c->cfg.device & 15]) {
+        FT_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemMax));
+        int per_sm = 0;
+        FT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, (lay.nw + 2) * 32, lay.total));
+        if (per_sm < 1) return FASTTPS_INVALID_ARG;
+        configured[c->cfg.device & 15] = true;
+    }
+    // barrier counter and abort flag start from zero every launch (the generation may be anything)
+    FT_CUDA(cudaMemsetAsync(c->grid_bar, 0, 64 * sizeof(unsigned), st));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(c->n_sm); cfg.blockDim = dim3((lay.nw + 2) * 32); cfg.dynamicSmemBytes = lay.total; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    void *params[] = {const_cast<StepArgs *>(&a)};
+    ProfScope prof(c, kProfStep, st);
+    FT_CUDA(cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(kernel), params));
+    c->launches++;
+    return FASTTPS_OK;
+}
+
+// True when the persistent kernel can serve this model shape and batch.
+bool step_kernel_supported(const Ctx *c, int batch)
+{
+    const fasttps_config &f = c->cfg;
+    const WarpSplit s = warp_split(f.hidden);
+    if (batch < 1 || batch > kMaxNB) return false;
+    if (f.n_q_heads * f.head_dim != f.hidden) return false;      // one reduction length for every product
+    if (s.nw < 1 || s.nw > 12) return false;
+    if (f.vocab < 1 || f.n_layers < 1) return false;
+    return true;
+}
+
+int launch_step(Ctx *c, const StepArgs &a, cudaStream_t st)
+{
+    const int ipw = warp_split(a.D).ipw;
+#define FT_STEP(DHV)                                                                          \
+    case DHV: return ipw == 8 ? launch_step_inst<8, DHV>(c, a, st) : launch_step_inst<4, DHV>(c, a, st)
+    switch (a.head_dim) {
+        FT_STEP(32);
+        FT_STEP(64);
+        FT_STEP(96);
+        FT_STEP(128);
+    default: return FASTTPS_INVALID_ARG;
+    }
+#undef FT_STEP
+}
+
+}  // namespace fasttps

@@ -16,23 +16,22 @@
 // Both weight slices of a CTA are contiguous byte ranges and go through ONE shared-memory
 // ring fed by a producer warp, so the W_down octets are already in flight while the gate_up
 // reduction and the SiLU step are still running.
+#include "mlp_core.cuh"
 #include "stream_launch.cuh"
 
 namespace fasttps {
 
 namespace {
 
-constexpr int kMaxOctetsPerCta = 16;      // bounds the shared-memory intermediate
-
 template <int IPW, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1) mlp_decode_kernel(MlpArgs a)
 {
     extern __shared__ __align__(128) unsigned char dsm[];
-    __shared__ __align__(16) __nv_bfloat16 s_hi[kMaxOctetsPerCta][8][8];   // [octet][batch row][j in octet]
-    __shared__ __align__(16) __nv_bfloat16 s_lo[kMaxOctetsPerCta][8][8];
+    __shared__ __align__(16) ActTile s_hi[kMaxOctetsPerCta];   // [octet][batch row][j in octet]
+    __shared__ __align__(16) ActTile s_lo[kMaxOctetsPerCta];
     __shared__ int s_last;
 
-    const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3;
+    const int t = threadIdx.x;
     const StreamSmemLayout lay = stream_smem_layout(a.D);
     const int nw = lay.nw, nct = nw * 32;
     float *smem_part = reinterpret_cast<float *>(dsm + lay.part_off);
@@ -67,12 +66,7 @@ __global__ void __launch_bounds__(MAXT, 1) mlp_decode_kernel(MlpArgs a)
     load_b_frags<IPW>(bf, a.x, a.D, a.batch, a.D, nw, a.g, a.eps, smem_red);
 
     // ---- steps 2-11: interlaced gate_up product, then siLu_Mul on the finished sums ----
-    bool ok = dot_tiles<IPW>(ring, 0, noct, nw, bf, smem_part, [&](int tile, int cc, int b, float gate, float up) {
-        const float act = gate / (1.f + __expf(-gate)) * up;
-        const __nv_bfloat16 hi = __float2bfloat16_rn(act);
-        s_hi[tile][b][cc] = hi;
-        s_lo[tile][b][cc] = __float2bfloat16_rn(act - __bfloat162float(hi));
-    });
+    bool ok = mlp_gate_up_phase<IPW>(ring, 0, noct, nw, bf, smem_part, s_hi, s_lo);
     if (!ok) {
         if (t == 0) atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT);
         return;
@@ -87,49 +81,13 @@ __global__ void __launch_bounds__(MAXT, 1) mlp_decode_kernel(MlpArgs a)
         for (int m = 0; m < 2; ++m)
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[i][m][e] = 0.f;
-    constexpr int PPO = IPW / 4;                            // ring pieces per octet
-    const int piece0 = ring.pieces0;
-    for (int o = 0; o < noct; ++o) {
-        const uint32_t bh = *reinterpret_cast<const uint32_t *>(&s_hi[o][g][2 * t4]);
-        const uint32_t bl = *reinterpret_cast<const uint32_t *>(&s_lo[o][g][2 * t4]);
-#pragma unroll
-        for (int q = 0; q < PPO; ++q) {
-            const int piece = piece0 + o * PPO + q;
-            const unsigned char *slot = ring.wait(piece, ok);
-#pragma unroll
-            for (int s = 0; s < 4; ++s) {
-                const uint4 r = *reinterpret_cast<const uint4 *>(slot + (size_t)(s * nw + w) * 512 + lane * 16);
-                const int i = q * 4 + s;
-                mma_bf16_k8(acc[i][0], r.x, r.y, bh);
-                mma_bf16_k8(acc[i][0], r.x, r.y, bl);
-                mma_bf16_k8(acc[i][1], r.z, r.w, bh);
-                mma_bf16_k8(acc[i][1], r.z, r.w, bl);
-            }
-            ring.release(piece);
-        }
-    }
+    mlp_down_phase<IPW>(ring, ring.pieces0, noct, nw, s_hi, s_lo, acc, ok);
     if (!named_bar_and(1, nct, ok)) {                       // also: every warp is done with the ring
         if (t == 0) atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT);
         return;
     }
-
-    // ---- y^T fragments -> [batch][D] in shared memory (the ring is idle now) -> vector red.add ----
-    float *out_s = reinterpret_cast<float *>(dsm + lay.ring_off);
-#pragma unroll
-    for (int i = 0; i < IPW; ++i)
-#pragma unroll
-        for (int m = 0; m < 2; ++m) {
-            const int n = 32 * (w + nw * i) + 16 * m + g;
-            const int b0 = 2 * t4;
-            if (b0 < a.batch) { out_s[(size_t)b0 * a.D + n] = acc[i][m][0]; out_s[(size_t)b0 * a.D + n + 8] = acc[i][m][2]; }
-            if (b0 + 1 < a.batch) { out_s[(size_t)(b0 + 1) * a.D + n] = acc[i][m][1]; out_s[(size_t)(b0 + 1) * a.D + n + 8] = acc[i][m][3]; }
-        }
-    named_bar_sync(1, nct);
-    const int nvec4 = a.batch * (a.D >> 2);
-    for (int idx = t; idx < nvec4; idx += nct) {
-        const float4 v = *reinterpret_cast<const float4 *>(out_s + (size_t)idx * 4);
-        red_add_v4(a.acc + (size_t)idx * 4, v.x, v.y, v.z, v.w);
-    }
+    // ---- partial y -> shared memory -> vector red.add ----
+    mlp_scatter_add<IPW>(acc, smem_part, a.acc, a.batch, a.D, nw);
     __threadfence();
     named_bar_sync(1, nct);
     if (t == 0) s_last = (atomicAdd(a.ticket, 1) == (int)gridDim.x - 1);

@@ -353,9 +353,11 @@ def build_model(fb, ctx, dims, batch, max_seq, device="cuda"):
 
 
 @pytest.mark.parametrize("dims,lens", [(wl.SMALL, [40, 7, 100]), (wl.SMALL_GQA, [3]), (wl.TINY, list(range(1, 11)))])
-def test_model_decode_teacher_forced_steps(fb, dims, lens):
+@pytest.mark.parametrize("step_kernel", [0, 1])
+def test_model_decode_teacher_forced_steps(fb, dims, lens, step_kernel):
     batch, max_seq, steps = len(lens), 128, 4
     ctx = make_ctx(fb, dims, batch, max_seq)
+    ctx.set_option("step_kernel", step_kernel)     # one kernel per product, or the persistent step kernel
     mw, model, kcs, vcs = build_model(fb, ctx, dims, batch, max_seq)
     ok = [wl.bits(t) for t in kcs]
     ov = [wl.bits(t) for t in vcs]
@@ -391,9 +393,11 @@ def test_model_decode_teacher_forced_steps(fb, dims, lens):
     ctx.close()
 
 
-def test_model_decode_host_buffers_and_greedy_feedback(fb):
+@pytest.mark.parametrize("step_kernel", [0, 1])
+def test_model_decode_host_buffers_and_greedy_feedback(fb, step_kernel):
     dims, batch, max_seq = wl.SMALL, 2, 64
     ctx = make_ctx(fb, dims, batch, max_seq)
+    ctx.set_option("step_kernel", step_kernel)
     mw, model, kcs, vcs = build_model(fb, ctx, dims, batch, max_seq)
     k0 = [t.clone() for t in kcs]
     v0 = [t.clone() for t in vcs]
@@ -421,4 +425,50 @@ def test_model_decode_host_buffers_and_greedy_feedback(fb):
     # a token id outside the vocabulary is reported, not dereferenced
     ctx.model_decode(model, i32([dims.vocab + 5, 1]), pos, sl, None, tok, advance=False)
     assert ctx.get_status() & fb.DEV_BAD_TOKEN
+    ctx.close()
+
+
+@pytest.mark.parametrize("dims,lens", [(wl.SMALL, [30, 5]), (wl.TINY, [9]), (wl.SMALL_GQA, [12, 40, 3])])
+@pytest.mark.parametrize("step_kernel,l2_ahead", [(0, 0), (1, 0), (1, 6)])
+def test_model_generate_multi_step_greedy(fb, dims, lens, step_kernel, l2_ahead):
+    """Several greedy tokens inside one launch: same tokens as the oracle's greedy loop wherever its
+    argmax is beyond doubt, caches and counters advanced by n_steps."""
+    batch, max_seq, steps = len(lens), 96, 5
+    ctx = make_ctx(fb, dims, batch, max_seq)
+    ctx.set_option("step_kernel", step_kernel)
+    ctx.set_option("l2_ahead", l2_ahead)
+    mw, model, kcs, vcs = build_model(fb, ctx, dims, batch, max_seq)
+    ok = [wl.bits(t) for t in kcs]
+    ov = [wl.bits(t) for t in vcs]
+    ow = [{k: wl.bits(v) for k, v in L.items()} for L in mw["layers"]]
+    start = wl.token_ids(batch, dims.vocab)
+    pos, sl = i32(lens), i32(lens)
+    out = torch.zeros(steps, batch, dtype=torch.int32, device="cuda")
+    ctx.model_generate(model, i32(start), pos, sl, out)
+    torch.cuda.synchronize()
+    assert ctx.get_status() == 0
+    got = out.cpu().numpy()
+    cur = np.asarray(lens, np.int32).copy()
+    tok = start.copy()
+    alive = np.ones(batch, bool)                    # sequences whose history still equals the oracle's
+    compared = 0
+    for s in range(steps):
+        wlog, wnext = orc.model_decode(wl.bits(mw["embed"]), ow, wl.bits(mw["g_final"]), wl.bits(mw["w_lm"]), ok, ov,
+                                       tok, cur, cur, dims.rms_eps, dims.rope_theta)
+        top2 = np.sort(wlog, axis=1)[:, -2:]
+        sure = (top2[:, 1] - top2[:, 0]) > 2 * (2e-2 + 2e-2 * np.abs(top2[:, 1]))
+        chk = alive & sure
+        assert (got[s][chk] == wnext[chk]).all(), s
+        compared += int(chk.sum())
+        alive &= (got[s] == wnext)
+        tok = wnext.astype(np.int32)
+        cur += 1
+    assert compared >= batch                        # at least the first step of every sequence
+    assert (pos.cpu().numpy() == np.asarray(lens) + steps).all() and (sl.cpu().numpy() == np.asarray(lens) + steps).all()
+    # the appended rows of the sequences that stayed on the oracle's path are within the output bar
+    for l in range(dims.n_layers):
+        for b in np.flatnonzero(alive):
+            r = slice(lens[b], lens[b] + steps)
+            assert_close_bits(wl.bits(kcs[l])[b, :, r], ok[l][b, :, r], what="k rows")
+            assert_close_bits(wl.bits(vcs[l])[b, :, r], ov[l][b, :, r], what="v rows")
     ctx.close()
