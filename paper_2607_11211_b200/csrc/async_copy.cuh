@@ -44,7 +44,8 @@ __device__ __forceinline__ unsigned long long global_ns()
 // Bounded wait: gives up after kWaitPolls polls or kWaitNanos of wall time, whichever comes
 // first (or as soon as *abort_flag is set, when given), and reports failure instead of
 // spinning forever.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, const volatile int *abort_flag = nullptr)
+// The polling loop is kept out of line so that the hot loops that call it stay small.
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, const volatile int *abort_flag)
 {
     unsigned long long t0 = 0;
     for (uint32_t i = 0; i < kWaitPolls; ++i) {
@@ -57,6 +58,11 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
         }
     }
     return false;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, const volatile int *abort_flag = nullptr)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag);
 }
 // global -> shared bulk copy; dst, src 16-byte aligned, bytes a multiple of 16; completes on `bar`
 __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar)

@@ -286,149 +286,147 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     if (cta == 0) embed_rows(a.token_ids);
     if (!sync_phase()) return;
 
+    // One loop over all products of a step.  Every matrix product (QKV, output projection, gate_up, logits)
+    // goes through the SAME copy of the B-fragment prologue and of the tile loop, selected by `kind`: the hot
+    // code of the kernel stays small enough to live in the instruction cache from one product to the next.
+    enum { kQkv = 0, kAttn = 1, kOproj = 2, kMlp = 3, kHead = 4 };
+    const int L = a.n_layers;
     for (int step = 0; step < a.n_steps; ++step) {
-        for (int l = 0; l < a.n_layers; ++l) {
-            const LayerPtrs lp = a.layers[l];
-            const float *y_prev = l > 0 ? a.acc + (size_t)((l - 1) & 1) * B * D : nullptr;   // MLP sums of layer l - 1
-            const __nv_bfloat16 *x_base = l > 0 ? a.h : a.x0;                             // x_l = bf16(x_base + y_prev)
+        for (int ph = 0; ph <= 4 * L; ++ph) {
+            const int l = ph >> 2;
+            const int kind = ph == 4 * L ? kHead : (ph & 3);
+            const LayerPtrs lp = a.layers[l < L ? l : L - 1];
+            const int lprev = (kind == kHead ? L : l) - 1;                               // layer whose MLP sums feed x
+            const float *y_prev = lprev >= 0 ? a.acc + (size_t)(lprev & 1) * B * D : nullptr;
+            const __nv_bfloat16 *x_base = lprev >= 0 ? a.h : a.x0;                      // x = bf16(x_base + y_prev)
 
-            // ---- RMSNorm -> QKV ----
-            load_b_frags<IPW>(bf, x_base, D, B, D, nw, lp.g_attn, a.eps, smem_red, y_prev);
-            ok = dot_tiles<IPW>(ring, piece, qn, nw, bf, smem_part, [&](int tile, int cc, int b, float v0, float v1) {
-                if (b >= B) return;
-                const int row = (q0 + tile) * 16 + cc;
-                if (row < nqkv) a.qkv[(size_t)b * nqkv + row] = __float2bfloat16_rn(v0);
-                if (row + 8 < nqkv) a.qkv[(size_t)b * nqkv + row + 8] = __float2bfloat16_rn(v1);
-            }) && ok;
-            piece += qn * SPT;
-            if (!sync_phase()) return;
-
-            // ---- attention (Algorithm 3) ----
-            {
+            if (kind == kAttn) {
+                // ---- attention (Algorithm 3) ----
                 const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
                 ok = attn_consume<DH>(aa, ring, piece, cta, ncta_attn, scratch, nw) && ok;
-            }
-            if (!sync_phase()) return;
-
-            // ---- output projection + residual: h = x_l + attn . W_o ----
-            load_b_frags<IPW>(bf, a.attn_out, nq, B, D, nw, nullptr, a.eps, smem_red);
-            ok = dot_tiles<IPW>(ring, piece, on, nw, bf, smem_part, [&](int tile, int cc, int b, float v0, float v1) {
-                if (b >= B) return;
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int row = (o0 + tile) * 16 + cc + 8 * hh;
-                    if (row >= D) continue;
-                    float x = __bfloat162float(ld_cg_bf16(x_base + (size_t)b * D + row));
-                    if (y_prev) x = bf16_round(x + ld_cg_f32(y_prev + (size_t)b * D + row));
-                    a.h[(size_t)b * D + row] = __float2bfloat16_rn(x + (hh ? v1 : v0));
+            } else {
+                // ---- a matrix product: B fragments, then this CTA's row tiles ----
+                const __nv_bfloat16 *src = x_base, *gain = nullptr;
+                const float *add = y_prev;
+                int tile0 = 0, ntile = 0;
+                if (kind == kQkv) { gain = lp.g_attn; tile0 = q0; ntile = qn; }
+                else if (kind == kOproj) { src = a.attn_out; add = nullptr; tile0 = o0; ntile = on; }
+                else if (kind == kMlp) { src = a.h; add = nullptr; gain = lp.g_mlp; tile0 = m0; ntile = mn; }
+                else { gain = a.g_final; tile0 = l0; ntile = ln; }
+                load_b_frags<IPW>(bf, src, D, B, D, nw, gain, a.eps, smem_red, add);
+                if (kind == kHead) {
+                    for (int u = t; u < 64; u += nct) { s_best_val[u] = -INFINITY; s_best_idx[u] = 0x7fffffff; }
+                    named_bar_sync(1, nct);
                 }
-            }) && ok;
-            piece += on * SPT;
-            if (!sync_phase()) return;
+                ok = dot_tiles<IPW>(ring, piece, ntile, nw, bf, smem_part, [&](int tile, int cc, int b, float v0, float v1) {
+                    if (kind == kMlp) {                      // siLu_Mul: rows cc / cc + 8 are a gate value and its up value
+                        const float act = v0 / (1.f + __expf(-v0)) * v1;
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(act);
+                        s_hi[tile][b][cc] = hi;
+                        s_lo[tile][b][cc] = __float2bfloat16_rn(act - __bfloat162float(hi));
+                        return;
+                    }
+                    if (b >= B) return;
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int row = (tile0 + tile) * 16 + cc + 8 * hh;
+                        const float v = hh ? v1 : v0;
+                        if (kind == kQkv) {
+                            if (row < nqkv) a.qkv[(size_t)b * nqkv + row] = __float2bfloat16_rn(v);
+                        } else if (kind == kOproj) {         // h = x_l + attn . W_o
+                            if (row < D) {
+                                float x = __bfloat162float(ld_cg_bf16(x_base + (size_t)b * D + row));
+                                if (y_prev) x = bf16_round(x + ld_cg_f32(y_prev + (size_t)b * D + row));
+                                a.h[(size_t)b * D + row] = __float2bfloat16_rn(x + v);
+                            }
+                        } else if (row < a.V) {              // logits and the running argmax of this thread's rows
+                            const int u = cc * 8 + b;
+                            if (a.logits) a.logits[(size_t)b * a.V + row] = v;
+                            if (v > s_best_val[u]) { s_best_val[u] = v; s_best_idx[u] = row; }
+                        }
+                    }
+                }) && ok;
+                piece += ntile * SPT;
 
-            // ---- RMSNorm -> fused MLP (Algorithm 4); the sums of all CTAs meet in acc[l & 1] ----
-            float *y_cur = a.acc + (size_t)(l & 1) * B * D;
-            load_b_frags<IPW>(bf, a.h, D, B, D, nw, lp.g_mlp, a.eps, smem_red);
-            ok = mlp_gate_up_phase<IPW>(ring, piece, mn, nw, bf, smem_part, s_hi, s_lo) && ok;
-            piece += mn * SPT;
-            if (cta == 0 && y_prev) {
-                // layer l - 1's sums have been consumed by everyone (two barriers ago): zero them for layer l + 1
-                float *z = a.acc + (size_t)((l - 1) & 1) * B * D;
-                for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            named_bar_sync(1, nct);
-            {
-                float acc[IPW][2][4];
+                if (kind == kMlp) {
+                    // ---- down projection of this CTA's octets; the sums of all CTAs meet in acc[l & 1] ----
+                    if (cta == 0 && y_prev) {
+                        // layer l - 1's sums have been consumed by everyone (two barriers ago): zero them for layer l + 1
+                        float *z = a.acc + (size_t)((l - 1) & 1) * B * D;
+                        for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    named_bar_sync(1, nct);
+                    float acc[IPW][2][4];
 #pragma unroll
-                for (int i = 0; i < IPW; ++i)
+                    for (int i = 0; i < IPW; ++i)
 #pragma unroll
-                    for (int m = 0; m < 2; ++m)
+                        for (int m = 0; m < 2; ++m)
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) acc[i][m][e] = 0.f;
-                mlp_down_phase<IPW>(ring, piece, mn, nw, s_hi, s_lo, acc, ok);
-                piece += mn * PPO;
-                mlp_scatter_add<IPW>(acc, smem_part, y_cur, B, D, nw);
+                            for (int e = 0; e < 4; ++e) acc[i][m][e] = 0.f;
+                    mlp_down_phase<IPW>(ring, piece, mn, nw, s_hi, s_lo, acc, ok);
+                    piece += mn * PPO;
+                    mlp_scatter_add<IPW>(acc, smem_part, a.acc + (size_t)(l & 1) * B * D, B, D, nw);
+                } else if (kind == kHead) {
+                    named_bar_sync(1, nct);
+                    if (t < 8 && t < B) {
+                        float bv = -INFINITY; int bi = 0x7fffffff;
+                        for (int cc = 0; cc < 8; ++cc) {
+                            const float v = s_best_val[cc * 8 + t]; const int i = s_best_idx[cc * 8 + t];
+                            if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+                        }
+                        a.amax_val[(size_t)t * ncta + cta] = bv;
+                        a.amax_idx[(size_t)t * ncta + cta] = bi;
+                    }
+                }
             }
             if (!sync_phase()) return;
         }
 
-        // ---- final norm -> logits -> greedy argmax ----
-        {
-            const int L = a.n_layers;
-            const float *y_last = a.acc + (size_t)((L - 1) & 1) * B * D;
-            load_b_frags<IPW>(bf, a.h, D, B, D, nw, a.g_final, a.eps, smem_red, y_last);
-            for (int u = t; u < 64; u += nct) { s_best_val[u] = -INFINITY; s_best_idx[u] = 0x7fffffff; }
-            named_bar_sync(1, nct);
-            ok = dot_tiles<IPW>(ring, piece, ln, nw, bf, smem_part, [&](int tile, int cc, int b, float v0, float v1) {
-                if (b >= B) return;
-                const int u = cc * 8 + b;
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int row = (l0 + tile) * 16 + cc + 8 * hh;
-                    if (row >= a.V) continue;
-                    const float v = hh ? v1 : v0;
-                    if (a.logits) a.logits[(size_t)b * a.V + row] = v;
-                    if (v > s_best_val[u]) { s_best_val[u] = v; s_best_idx[u] = row; }   // rows ascend: first max kept
-                }
-            }) && ok;
-            piece += ln * SPT;
-            named_bar_sync(1, nct);
-            if (t < 8 && t < B) {
+        // ---- CTA 0 finishes the greedy argmax, advances the state and gathers the next embedding rows ----
+        if (cta == 0) {
+            // every thread fetches its share of the per-CTA candidates at once, then warps and the CTA reduce
+            for (int b = 0; b < B; ++b) {
                 float bv = -INFINITY; int bi = 0x7fffffff;
-                for (int cc = 0; cc < 8; ++cc) {
-                    const float v = s_best_val[cc * 8 + t]; const int i = s_best_idx[cc * 8 + t];
+                for (int c = t; c < ncta; c += nct) {
+                    const float v = ld_cg_f32(a.amax_val + (size_t)b * ncta + c);
+                    const int i = ld_cg_s32(a.amax_idx + (size_t)b * ncta + c);
                     if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
                 }
-                a.amax_val[(size_t)t * ncta + cta] = bv;
-                a.amax_idx[(size_t)t * ncta + cta] = bi;
-            }
-            if (!sync_phase()) return;
-
-            if (cta == 0) {
-                // every thread fetches its share of the per-CTA candidates at once, then warps and the CTA reduce
-                for (int b = 0; b < B; ++b) {
-                    float bv = -INFINITY; int bi = 0x7fffffff;
-                    for (int c = t; c < ncta; c += nct) {
-                        const float v = ld_cg_f32(a.amax_val + (size_t)b * ncta + c);
-                        const int i = ld_cg_s32(a.amax_idx + (size_t)b * ncta + c);
+#pragma unroll
+                for (int s = 16; s >= 1; s >>= 1) {
+                    const float ov = __shfl_xor_sync(kFull, bv, s);
+                    const int oi = __shfl_xor_sync(kFull, bi, s);
+                    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+                }
+                if (lane == 0) { s_best_val[w] = bv; s_best_idx[w] = bi; }
+                named_bar_sync(1, nct);
+                if (t == 0) {
+                    for (int w2 = 0; w2 < nw; ++w2) {
+                        const float v = s_best_val[w2]; const int i = s_best_idx[w2];
                         if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
                     }
-#pragma unroll
-                    for (int s = 16; s >= 1; s >>= 1) {
-                        const float ov = __shfl_xor_sync(kFull, bv, s);
-                        const int oi = __shfl_xor_sync(kFull, bi, s);
-                        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+                    if (bi == 0x7fffffff) bi = 0;      // all-NaN row: fall back to index 0
+                    a.tok[b] = bi;
+                    if (a.out_ids) a.out_ids[(size_t)step * B + b] = bi;
+                    if (step == a.n_steps - 1) {
+                        a.next_ids[b] = bi;
+                        if (a.advance) { a.pos[b] += a.n_steps; a.seq_lens[b] += a.n_steps; }
                     }
-                    if (lane == 0) { s_best_val[w] = bv; s_best_idx[w] = bi; }
-                    named_bar_sync(1, nct);
-                    if (t == 0) {
-                        for (int w2 = 0; w2 < nw; ++w2) {
-                            const float v = s_best_val[w2]; const int i = s_best_idx[w2];
-                            if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
-                        }
-                        if (bi == 0x7fffffff) bi = 0;      // all-NaN row: fall back to index 0
-                        a.tok[b] = bi;
-                        if (a.out_ids) a.out_ids[(size_t)step * B + b] = bi;
-                        if (step == a.n_steps - 1) {
-                            a.next_ids[b] = bi;
-                            if (a.advance) { a.pos[b] += a.n_steps; a.seq_lens[b] += a.n_steps; }
-                        }
-                    }
-                    named_bar_sync(1, nct);
                 }
-                // the last layer's MLP sums are consumed: back to zero (the other buffer was zeroed in the last MLP phase)
-                float *z = a.acc + (size_t)((L - 1) & 1) * B * D;
-                for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (step + 1 < a.n_steps) {
-                    __threadfence();
-                    named_bar_sync(1, nct);
-                    embed_rows(a.tok);
-                }
+                named_bar_sync(1, nct);
             }
+            // the last layer's MLP sums are consumed: back to zero (the other buffer was zeroed in the last MLP phase)
+            float *z = a.acc + (size_t)((L - 1) & 1) * B * D;
+            for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (step + 1 < a.n_steps) {
-                if (!sync_phase()) return;
-                if (t == 0) atomicExch(&s_steps_done, step + 1);    // the producer may fetch the new K/V rows now
+                __threadfence();
+                named_bar_sync(1, nct);
+                embed_rows(a.tok);
             }
+        }
+        if (step + 1 < a.n_steps) {
+            if (!sync_phase()) return;
+            if (t == 0) atomicExch(&s_steps_done, step + 1);    // the producer may fetch the new K/V rows now
         }
     }
 }
