@@ -49,7 +49,6 @@ def parse_args():
     ap.add_argument("--graph", type=int, default=1, help="replay the step as a CUDA graph (1) or launch eagerly (0)")
     ap.add_argument("--step-kernel", type=int, default=0,
                     help="1: whole decode steps in the persistent cooperative kernel (batch <= 8)")
-    ap.add_argument("--l2-ahead", type=int, default=0, help="lookahead of the step kernel's L2 prefetch warp (pieces)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -216,7 +215,6 @@ def run_ours(args):
 
     ctx = fb.Context.from_dims(dm, B, max_seq, device=local, n_layers=W.n_layers)
     ctx.set_option("step_kernel", args.step_kernel)
-    ctx.set_option("l2_ahead", args.l2_ahead)
     seed = wl.MASTER_SEED + 1000 * rank
 
     def packed_layer(idx):

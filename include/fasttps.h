@@ -96,12 +96,22 @@ int fasttps_destroy(fasttps_ctx *ctx);
 /* One-time weight packing, outside the decode path: the offline re-layout of
  * Section 3.2 item 1 ("interlaced layout of gate-up weights").  `src` is the
  * logical row-major bf16 matrix described at fasttps_weight_kind, `dst` a
- * device buffer of fasttps_packed_bytes(kind) bytes.  Packed layouts:
- *   QKV, O, LM_HEAD: [out, in] (each output's weights contiguous);
- *   GATE_UP: [2K, D] rows interlaced in blocks of 8: for j-octet J the rows
- *            16J..16J+7 are gate columns 8J..8J+7 and 16J+8..16J+15 the matching
- *            up columns, so a gate value and its up value meet in one CTA;
- *   DOWN: [K, D] unchanged. */
+ * device buffer of fasttps_packed_bytes(kind) bytes.  Packed layouts (bf16):
+ *   QKV, O, LM_HEAD: the transposed matrix W^T [out, in], with `out` padded up to a
+ *            multiple of 16 by zero rows, cut into tiles of 16 output rows x 32 inputs;
+ *            a tile is stored row-major (1 KB), tiles are ordered by (row tile, input
+ *            block), so that the share of a CTA -- a run of row tiles -- is one contiguous
+ *            byte range and one tile is the A operand of two tensor-core instructions;
+ *   GATE_UP: the same tiling of a [2K, D] matrix whose rows are interlaced in blocks of
+ *            8: for j-octet J the rows 16J..16J+7 are gate columns 8J..8J+7 and
+ *            16J+8..16J+15 the matching up columns, so a gate value and its up value
+ *            come out of the same tile;
+ *   DOWN:    for every j-octet J (8 rows of the logical [K, D] matrix) and block of 32
+ *            output columns one 512-byte block holding W_down[8J..8J+7, 32c..32c+31] in
+ *            the register order of an m16n8k8 A operand; blocks ordered by (J, c), so a
+ *            CTA's octets are again one contiguous byte range.
+ * Limits: D and H_q d multiples of 128 up to 3072 or multiples of 256 from 2048 to 6144;
+ * K a multiple of 8. */
 size_t fasttps_packed_bytes(const fasttps_ctx *ctx, int kind);
 int fasttps_pack_weight(fasttps_ctx *ctx, int kind, const void *src, void *dst, void *stream);
 /* Inverse of fasttps_pack_weight (for round-trip checks). */
@@ -188,9 +198,7 @@ int fasttps_model_decode_host(fasttps_ctx *ctx, const void *embed, const fasttps
 
 /* Tuning switches of a context (host side, take effect at the next call):
  *   "step_kernel" 0/1  route model calls with batch <= 8 through the persistent step kernel
- *                      (default: environment variable FASTTPS_STEP_KERNEL, else 0);
- *   "l2_ahead"    n    ring pieces the step kernel's L2 prefetch warp may run ahead (0 = off;
- *                      default: FASTTPS_L2_AHEAD, else 0).
+ *                      (default: environment variable FASTTPS_STEP_KERNEL, else 0).
  * Unknown names return FASTTPS_INVALID_ARG. */
 int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value);
 

@@ -34,11 +34,12 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
     objdir = PKG / "build"
     objdir.mkdir(exist_ok=True)
     nvcc = _nvcc()
+    extra = os.environ.get("FASTTPS_NVCC_EXTRA", "").split()      # e.g. -DFASTTPS_FINE_TRACE for a development build
     jobs = []
     for s in SOURCES:
         src, obj = CSRC / s, objdir / (s + ".o")
         if force or _stale(obj, [src, *headers]):
-            cmd = [nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if ptxas_info else []), "-c", str(src), "-o", str(obj)]
+            cmd = [nvcc, *NVCC_FLAGS, *extra, *(["-Xptxas", "-v"] if ptxas_info else []), "-c", str(src), "-o", str(obj)]
             jobs.append(cmd)
 
     def run(cmd):

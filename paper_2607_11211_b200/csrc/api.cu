@@ -87,8 +87,8 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     {
         const char *e = getenv("FASTTPS_STEP_KERNEL");
         c->opt_step_kernel = (e && *e) ? atoi(e) != 0 : 0;
-        e = getenv("FASTTPS_L2_AHEAD");
-        c->opt_l2_ahead = (e && *e) ? atoi(e) : 0;
+        e = getenv("FASTTPS_RING_INFLIGHT");
+        c->opt_ring_inflight = (e && *e) ? atoi(e) : 0;
     }
     {
         int rc = configure_attn_kernels();
@@ -104,7 +104,7 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     auto A = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
     A(dev_alloc(&c->cos_tab, (size_t)f.max_seq * half, false));
     A(dev_alloc(&c->sin_tab, (size_t)f.max_seq * half, false));
-    A(dev_alloc(&c->attn_part, B * f.n_q_heads * kMaxSplits * (f.head_dim + 2), true));
+    A(dev_alloc(&c->attn_part, B * f.n_q_heads * kMaxSplits * (f.head_dim + 4), true));
     A(dev_alloc(&c->attn_ticket, B * f.n_q_heads, true));
     A(dev_alloc(&c->mlp_acc, 2 * B * D, true));
     A(dev_alloc(&c->grid_bar, 128, true));
@@ -347,7 +347,7 @@ int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value)
     if (!ctx || !name) return FASTTPS_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);
     if (strcmp(name, "step_kernel") == 0) c->opt_step_kernel = value != 0;
-    else if (strcmp(name, "l2_ahead") == 0) c->opt_l2_ahead = value < 0 ? 0 : (value > 64 ? 64 : value);
+    else if (strcmp(name, "ring_inflight") == 0) c->opt_ring_inflight = value < 0 ? 0 : value;
     else return FASTTPS_INVALID_ARG;
     return FASTTPS_OK;
 }
@@ -410,7 +410,7 @@ static int step_impl(Ctx *c, const void *embed, const fasttps_layer_weights *lay
     a.amax_val = c->amax_val; a.amax_idx = c->amax_idx; a.tok = c->tok2;
     a.bar = c->grid_bar; a.status = c->status;
     a.trace = c->trace; a.trace_len = kTraceLen;
-    a.l2_ahead = c->opt_l2_ahead;
+    a.max_inflight = c->opt_ring_inflight;
     return launch_step(c, a, st);
 }
 

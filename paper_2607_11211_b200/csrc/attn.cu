@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a
             else if (p < 0 || p >= a.max_seq) atomicOr(a.status, FASTTPS_DEV_BAD_POSITION);
         }
     }
-    if (!attn_consume<DH>(a, ring, piece, blockIdx.x, gridDim.x, sm.scratch, kAttnWarps) && t == 0)
+    if (!attn_consume<DH, false>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x), sm.scratch, kAttnWarps) && t == 0)
         atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT);
 }
 

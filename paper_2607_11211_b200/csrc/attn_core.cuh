@@ -62,11 +62,24 @@ struct ShareWalk {
     {
         seq_lens = sl; pos = ps; add = add_; B = B_; H = H_; max_seq = max_seq_;
         T = 0;
-        for (int bb = 0; bb < B; ++bb) T += (long long)H * rows_of(bb);
+        int live = 0, rows0 = 0;
+        bool uniform = true;
+        for (int bb = 0; bb < B; ++bb) {
+            const int r = rows_of(bb);
+            T += (long long)H * r;
+            if (r > 0) {
+                if (live == 0) rows0 = r;
+                else if (r != rows0) uniform = false;
+                ++live;
+            }
+        }
         // only as many CTAs take part as can get at least 16 rows each: every share is then
         // non-empty, so the CTAs that share a head are exactly first_cta .. first_cta + n_cta - 1
         const long long want = T / 16;
         ncta = want < 1 ? 1 : (want < ncta_ ? (int)want : ncta_);
+        // equal lengths and no more heads than CTAs: a whole number of CTAs per head, so that every share
+        // is ONE segment and every head has the same, small number of partials
+        if (uniform && live > 0 && live * H <= ncta) ncta = live * H * (ncta / (live * H));
         const bool in = T > 0 && cta < ncta;
         f = in ? share_begin(cta) : 0;
         f_end = in ? share_begin(cta + 1) : 0;
@@ -124,14 +137,41 @@ template <int DH> struct AttnTile {
 
 // Calls f(k_tile, v_tile, bytes_each) for every K/V tile of this CTA's share, in walk order; stops and
 // returns false as soon as f does.
-template <int DH, class F>
-__device__ __forceinline__ bool attn_for_each_tile(const AttnArgs &a, int cta, int ncta, F f)
+// A share as a list of segments kept in shared memory (the persistent kernel computes it once per step
+// and uses it for every layer).
+constexpr int kMaxSegments = 20;
+struct SegmentList {
+    int n;
+    Segment seg[kMaxSegments];
+};
+
+// Segment sources: `bool next(Segment &)`.
+struct WalkSource {
+    ShareWalk walk;
+    __device__ __forceinline__ WalkSource(const AttnArgs &a, int cta, int ncta)
+    {
+        walk.init(a.seq_lens, a.pos, a.len_add, a.batch, a.n_q_heads, a.max_seq, cta, ncta);
+    }
+    __device__ __forceinline__ bool next(Segment &s) { return walk.next(s); }
+};
+struct ListSource {
+    const SegmentList *list;
+    int i;
+    __device__ __forceinline__ explicit ListSource(const SegmentList *l) : list(l), i(0) {}
+    __device__ __forceinline__ bool next(Segment &s)
+    {
+        if (i >= list->n) return false;
+        s = list->seg[i++];
+        return true;
+    }
+};
+
+template <int DH, class Src, class F>
+__device__ __forceinline__ bool attn_for_each_tile(const AttnArgs &a, Src src, F f)
 {
     const int G = a.n_q_heads / a.n_kv_heads;
-    ShareWalk walk;
-    walk.init(a.seq_lens, a.pos, a.len_add, a.batch, a.n_q_heads, a.max_seq, cta, ncta);
     Segment sg;
-    while (walk.next(sg)) {
+    while (src.next(sg)) {
         const int c1 = sg.r1 < sg.L ? sg.r1 : sg.L;              // cached rows of the segment: [r0, c1)
         const size_t slab = ((size_t)sg.b * a.n_kv_heads + sg.h / G) * (size_t)a.max_seq * DH;
         for (int r = sg.r0; r < c1; r += kAttnTileRows) {
@@ -148,7 +188,7 @@ __device__ __forceinline__ bool attn_for_each_tile(const AttnArgs &a, int cta, i
 template <int DH>
 __device__ __forceinline__ bool attn_produce(const AttnArgs &a, WeightRing &ring, int &piece, int cta, int ncta)
 {
-    return attn_for_each_tile<DH>(a, cta, ncta, [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
+    return attn_for_each_tile<DH>(a, WalkSource(a, cta, ncta), [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
         return ring.put2(piece++, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
     });
 }
@@ -156,14 +196,17 @@ __device__ __forceinline__ bool attn_produce(const AttnArgs &a, WeightRing &ring
 // Consumer warps (nwc of them, threads 0 .. 32 nwc - 1, synchronised by named barrier 1): the attention
 // of this CTA's share.  The first min(nwc, 8) warps score rows; the others only keep the ring protocol.
 // Returns false (in every consumer thread alike) if a bounded wait ran out.
-template <int DH>
-__device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring, int &piece, int cta, int ncta,
+// DEFER: the partial of every segment is published (even when the CTA owns the whole head) and nobody
+// merges here; the reader of the attention output merges on the fly (load_b_frags_attn).
+template <int DH, bool DEFER, class Src>
+__device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring, int &piece, int cta, Src src,
                                              AttnScratch<DH> &sm, int nwc)
 {
     constexpr int EPL = DH / kLanesPerRow;      // elements per lane of a row
     constexpr int VPL = EPL / 8;                // 16-byte vectors per lane
     constexpr int HALF = DH / 2;
     constexpr int kRowBytes = AttnTile<DH>::kRowBytes;
+    constexpr int kPartStride = DH + 4;         // partial = o[DH], max, sum, pad (16-byte aligned records)
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int nct = nwc * 32;
     const int nwork = nwc < kAttnMaxWorkers ? nwc : kAttnMaxWorkers;
@@ -174,10 +217,8 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
     bool ok = true;
 
-    ShareWalk walk;
-    walk.init(a.seq_lens, a.pos, a.len_add, a.batch, a.n_q_heads, a.max_seq, cta, ncta);
     Segment sg;
-    while (walk.next(sg)) {
+    while (src.next(sg)) {
         const int hq = sg.h, hk = hq / G, b = sg.b, L = sg.L;
         const bool has_new = sg.r1 > L;
         const int c1 = has_new ? L : sg.r1;
@@ -301,8 +342,9 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
         float M = -INFINITY;
         for (int w = 0; w < nwork; ++w) M = fmaxf(M, sm.wm[w]);
         __nv_bfloat16 *outp = a.out + (size_t)b * a.out_stride + (size_t)hq * DH;
-        float *hp = a.part + ((size_t)b * a.n_q_heads + hq) * kMaxSplits * (DH + 2);
-        float *part = hp + (size_t)(cta - sg.first_cta) * (DH + 2);
+        float *hp = a.part + ((size_t)b * a.n_q_heads + hq) * kMaxSplits * kPartStride;
+        float *part = hp + (size_t)(cta - sg.first_cta) * kPartStride;
+        const bool whole = !DEFER && sg.n_cta == 1;      // this CTA alone finishes the head right here
         for (int i = t; i < DH; i += nct) {
             float o = 0.f, l = 0.f;
             for (int w = 0; w < nwork; ++w) {
@@ -310,13 +352,13 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
                 o += f * sm.wo[w][i];
                 l += f * sm.wl[w];
             }
-            if (sg.n_cta == 1) outp[i] = __float2bfloat16_rn(o / l);
+            if (whole) outp[i] = __float2bfloat16_rn(o / l);
             else {
-                part[2 + i] = o;
-                if (i == 0) { part[0] = M; part[1] = l; }
+                part[i] = o;
+                if (i == 0) { part[DH] = M; part[DH + 1] = l; }
             }
         }
-        if (sg.n_cta > 1) {
+        if (!DEFER && sg.n_cta > 1) {
             // ---- several CTAs share the head: the partial is published, the last one merges ----
             __threadfence();
             named_bar_sync(1, nct);
@@ -328,8 +370,8 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
                 // all loads of the merge are issued side by side: one lane per partial for (max, sum) ...
                 if (warp == 0) {
                     const bool have = lane < sg.n_cta;
-                    const float ms = have ? ld_cg_f32(hp + (size_t)lane * (DH + 2)) : -INFINITY;
-                    const float ls = have ? ld_cg_f32(hp + (size_t)lane * (DH + 2) + 1) : 0.f;
+                    const float ms = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH) : -INFINITY;
+                    const float ls = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH + 1) : 0.f;
                     float MM = ms;
 #pragma unroll
                     for (int s = 16; s >= 1; s >>= 1) MM = fmaxf(MM, __shfl_xor_sync(kFull, MM, s));
@@ -346,7 +388,7 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
                         float v[8];
 #pragma unroll
                         for (int u = 0; u < 8; ++u)
-                            v[u] = (s0 + u < sg.n_cta) ? ld_cg_f32(hp + (size_t)(s0 + u) * (DH + 2) + 2 + i) : 0.f;
+                            v[u] = (s0 + u < sg.n_cta) ? ld_cg_f32(hp + (size_t)(s0 + u) * kPartStride + i) : 0.f;
 #pragma unroll
                         for (int u = 0; u < 8; ++u) oo = fmaf(sm.mf[(s0 + u) & (kMaxSplits - 1)], v[u], oo);
                     }
@@ -358,6 +400,85 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
         named_bar_sync(1, nct);                          // the scratch is reused by the next segment
     }
     return true;
+}
+
+// Tensor-core B fragments of the attention output, merged on the fly from the partials that
+// attn_consume<DH, true> published.  A consumer thread (g = lane / 4, t4 = lane % 4) needs, for each of its
+// IPW k blocks, the 8 elements k = 32 (w + nw i) + 8 t4 .. + 8 of batch row g (as in load_b_frags of
+// dot_core.cuh).  The warp's batch * IPW * 4 chunks are first dealt to its lanes 32 at a time, so that at
+// batch 1 all lanes fetch and merge instead of four; a lane reads its chunk from every partial of the head
+// the chunk belongs to (four partials in flight at a time), combines them with the softmax merge
+//   out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s,
+// rounds to bf16 (the attention output is a bf16 tensor), and the packed chunks are then handed to the lanes
+// that need them with shuffles.  head_n[b * Hq + h] = number of partials of head (b, h).  All loads
+// bypass L1 (the partials were written by other SMs).
+template <int IPW, int DH>
+__device__ __forceinline__ void load_b_frags_attn(uint32_t (&bf)[IPW][4], const float *part, const unsigned char *head_n,
+                                                  int batch, int n_q_heads, int nw)
+{
+    constexpr int PS = DH + 4;
+    constexpr int CPB = IPW * 4;                     // chunks per batch row and warp
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, g = lane >> 2, t4 = lane & 3;
+    const int total = batch * CPB;
+#pragma unroll
+    for (int i = 0; i < IPW; ++i) bf[i][0] = bf[i][1] = bf[i][2] = bf[i][3] = 0u;
+    for (int j = 0; j * 32 < total; ++j) {
+        const int c = j * 32 + lane;
+        uint32_t r[4] = {0u, 0u, 0u, 0u};
+        if (c < total) {
+            const int b = c / CPB, ci = (c % CPB) >> 2, ct = c & 3;
+            const int k = 32 * (w + nw * ci) + 8 * ct;
+            const int hq = k / DH, c0 = k - hq * DH;
+            const int n = head_n[b * n_q_heads + hq];
+            const float *hp = part + ((size_t)b * n_q_heads + hq) * kMaxSplits * PS;
+            float M = -INFINITY, den = 0.f, o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int s0 = 0; s0 < n; s0 += 4) {
+                float ms[4], ls[4];
+                float4 a0[4], a1[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const bool have = s0 + u < n;
+                    const float *p = hp + (size_t)(have ? s0 + u : 0) * PS;
+                    ms[u] = ld_cg_f32(p + DH);
+                    ls[u] = ld_cg_f32(p + DH + 1);
+                    a0[u] = ld_cg_f4(p + c0);
+                    a1[u] = ld_cg_f4(p + c0 + 4);
+                    if (!have) ms[u] = -INFINITY;
+                }
+                float Mn = M;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) Mn = fmaxf(Mn, ms[u]);
+                const float corr = fast_exp2(M - Mn);        // 0 on the first round (M = -inf)
+                den *= corr;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) o[e] *= corr;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float f = ms[u] == -INFINITY ? 0.f : fast_exp2(ms[u] - Mn);
+                    den = fmaf(f, ls[u], den);
+                    o[0] = fmaf(f, a0[u].x, o[0]); o[1] = fmaf(f, a0[u].y, o[1]);
+                    o[2] = fmaf(f, a0[u].z, o[2]); o[3] = fmaf(f, a0[u].w, o[3]);
+                    o[4] = fmaf(f, a1[u].x, o[4]); o[5] = fmaf(f, a1[u].y, o[5]);
+                    o[6] = fmaf(f, a1[u].z, o[6]); o[7] = fmaf(f, a1[u].w, o[7]);
+                }
+                M = Mn;
+            }
+            const float inv = n > 0 ? 1.f / den : 0.f;       // n = 0: a skipped sequence, output zero
+            r[0] = pack2(o[0] * inv, o[1] * inv);
+            r[1] = pack2(o[2] * inv, o[3] * inv);
+            r[2] = pack2(o[4] * inv, o[5] * inv);
+            r[3] = pack2(o[6] * inv, o[7] * inv);
+        }
+        // hand the chunks of this round to the lanes whose fragments they are
+#pragma unroll
+        for (int i = 0; i < IPW; ++i) {
+            const int need = g * CPB + i * 4 + t4;
+            const int src = need & 31;
+            const uint32_t v0 = __shfl_sync(kFull, r[0], src), v1 = __shfl_sync(kFull, r[1], src);
+            const uint32_t v2 = __shfl_sync(kFull, r[2], src), v3 = __shfl_sync(kFull, r[3], src);
+            if ((need >> 5) == j && g < batch) { bf[i][0] = v0; bf[i][1] = v1; bf[i][2] = v2; bf[i][3] = v3; }
+        }
+    }
 }
 
 }  // namespace fasttps

@@ -64,21 +64,42 @@ __device__ __forceinline__ void load_b_frags(uint32_t (&bf)[IPW][4], const __nv_
 {
     const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3;
     const bool live = g < batch;
+    // Every load is issued unconditionally (rows beyond the batch read row 0 and are zeroed afterwards): with
+    // no branch around them all loads of a thread go out back to back and cost ONE round trip to L2.
+    const int gr = live ? g : 0;
 #pragma unroll
     for (int i = 0; i < IPW; ++i) {
-        const int k = 32 * (w + nw * i) + 8 * t4;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (live) v = ld_cg_u4(x + (size_t)g * x_stride + k);
-        if (live && add) {
-            const float4 a0 = ld_cg_f4(add + (size_t)g * n_in + k), a1 = ld_cg_f4(add + (size_t)g * n_in + k + 4);
-            v.x = pack2(bf_lo(v.x) + a0.x, bf_hi(v.x) + a0.y);
-            v.y = pack2(bf_lo(v.y) + a0.z, bf_hi(v.y) + a0.w);
-            v.z = pack2(bf_lo(v.z) + a1.x, bf_hi(v.z) + a1.y);
-            v.w = pack2(bf_lo(v.w) + a1.z, bf_hi(v.w) + a1.w);
-        }
+        const uint4 v = ld_cg_u4(x + (size_t)gr * x_stride + 32 * (w + nw * i) + 8 * t4);
         bf[i][0] = v.x; bf[i][1] = v.y; bf[i][2] = v.z; bf[i][3] = v.w;
     }
+    if (add) {
+#pragma unroll
+        for (int h = 0; h < IPW; h += 4) {                  // four k blocks (32 registers) of addends in flight
+            float4 a0[4], a1[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float *p = add + (size_t)gr * n_in + 32 * (w + nw * (h + u)) + 8 * t4;
+                a0[u] = ld_cg_f4(p);
+                a1[u] = ld_cg_f4(p + 4);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                uint32_t(&v)[4] = bf[h + u];
+                v[0] = pack2(bf_lo(v[0]) + a0[u].x, bf_hi(v[0]) + a0[u].y);
+                v[1] = pack2(bf_lo(v[1]) + a0[u].z, bf_hi(v[1]) + a0[u].w);
+                v[2] = pack2(bf_lo(v[2]) + a1[u].x, bf_hi(v[2]) + a1[u].y);
+                v[3] = pack2(bf_lo(v[3]) + a1[u].z, bf_hi(v[3]) + a1[u].w);
+            }
+        }
+    }
+    if (!live) {
+#pragma unroll
+        for (int i = 0; i < IPW; ++i) bf[i][0] = bf[i][1] = bf[i][2] = bf[i][3] = 0u;
+    }
     if (gn == nullptr) return;
+    uint4 gv[IPW];                      // the gains are fetched before the reduction, not after its barrier
+#pragma unroll
+    for (int i = 0; i < IPW; ++i) gv[i] = *reinterpret_cast<const uint4 *>(gn + 32 * (w + nw * i) + 8 * t4);
     float ss = 0.f;
 #pragma unroll
     for (int i = 0; i < IPW; ++i)
@@ -97,9 +118,7 @@ __device__ __forceinline__ void load_b_frags(uint32_t (&bf)[IPW][4], const __nv_
     const float r = rsqrtf(tot / (float)n_in + eps);
 #pragma unroll
     for (int i = 0; i < IPW; ++i) {
-        const int k = 32 * (w + nw * i) + 8 * t4;
-        const uint4 gv = *reinterpret_cast<const uint4 *>(gn + k);
-        const uint32_t gg[4] = {gv.x, gv.y, gv.z, gv.w};
+        const uint32_t gg[4] = {gv[i].x, gv[i].y, gv[i].z, gv[i].w};
 #pragma unroll
         for (int j = 0; j < 4; ++j)
             bf[i][j] = pack2(bf_lo(bf[i][j]) * r * bf_lo(gg[j]), bf_hi(bf[i][j]) * r * bf_hi(gg[j]));

@@ -22,15 +22,30 @@ namespace fasttps {
 namespace {
 
 constexpr unsigned long long kGridWaitNanos = 500ull * 1000 * 1000;   // 0.5 s per barrier at most
-constexpr int kMegaThreadsMax = 448;                                   // up to 12 consumer warps + producer + prefetcher
+// Up to 12 consumer warps + the producer warp = 13 warps, so one of the four SM sub-partitions (16 K
+// registers each) hosts four warps: 128 registers per thread is the most a CTA of this size can be given.
+constexpr int kMegaThreadsMax = 416;
+constexpr int kMaxStepLayers = 48;                                     // layers the shared-memory layer table holds
+constexpr int kMaxStepHeads = 128;                                     // query heads the per-step head table holds
 
-// the 32 lanes of the prefetch warp ask L2 for the 128-byte lines of [p, p + bytes)
-__device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
-{
-    const unsigned char *q = static_cast<const unsigned char *>(p);
-    for (uint32_t off = (threadIdx.x & 31) * 128u; off < bytes; off += 32u * 128u)
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(q + off));
-}
+// The attention share of a CTA for one step: the segment list when it fits (computed once per step, used
+// by the producer and the consumers for every layer), else the walk itself.
+struct StepSource {
+    const SegmentList *list;
+    int i;
+    ShareWalk walk;
+    __device__ __forceinline__ StepSource(const SegmentList *l, const AttnArgs &a, int cta, int ncta) : list(l), i(0)
+    {
+        if (l->n < 0) walk.init(a.seq_lens, a.pos, a.len_add, a.batch, a.n_q_heads, a.max_seq, cta, ncta);
+    }
+    __device__ __forceinline__ bool next(Segment &s)
+    {
+        if (list->n < 0) return walk.next(s);
+        if (i >= list->n) return false;
+        s = list->seg[i++];
+        return true;
+    }
+};
 
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
 {
@@ -133,11 +148,13 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     __shared__ int s_best_idx[64];
     __shared__ int s_go;
     __shared__ int s_steps_done;
-    __shared__ int s_prod_piece;      // pieces the producer has issued so far (read by the prefetcher)
+    __shared__ LayerPtrs s_layers[kMaxStepLayers];               // the layer table: no global round trip per phase
+    __shared__ SegmentList s_segs;                               // this CTA's attention share for the current step
+    __shared__ unsigned char s_head_n[kMaxNB * kMaxStepHeads];   // CTAs that share head (b, h) in the current step
 
     const int t = threadIdx.x, lane = t & 31, w = t >> 5;
     const int cta = blockIdx.x, ncta = gridDim.x;
-    if (t == 0) { s_steps_done = 0; s_prod_piece = 0; }
+    if (t == 0) s_steps_done = 0;
     const MegaLayout lay = mega_layout<DH>(a.D);
     const int nw = lay.nw, nct = nw * 32;
     float *smem_part = reinterpret_cast<float *>(dsm + lay.part_off);
@@ -164,70 +181,74 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     ring.init(dsm + lay.ring_off, reinterpret_cast<uint64_t *>(dsm + lay.bar_off),
               reinterpret_cast<int *>(dsm + lay.abort_off), lay.nslot, lay.slot_stride, nw, nullptr, 0, nullptr, 0);
     if (t < 64) { s_best_val[t] = -INFINITY; s_best_idx[t] = 0x7fffffff; }
+    for (int i = t; i < a.n_layers * (int)(sizeof(LayerPtrs) / 8); i += blockDim.x)
+        reinterpret_cast<unsigned long long *>(s_layers)[i] = reinterpret_cast<const unsigned long long *>(a.layers)[i];
+
+    // Per-step attention tables (the lengths grow by one per step, so the split changes with the step, but
+    // not with the layer): the segments of this CTA's share, and for every head the number of CTAs that
+    // publish a partial for it.  Threads [0, nthr) take part.
+    auto build_step_tables = [&](int step, int nthr) {
+        ShareWalk wk;
+        wk.init(a.seq_lens, a.pos, step, B, a.n_q_heads, a.max_seq, cta, ncta_attn);
+        if (t == 0) {
+            int n = 0;
+            Segment sg;
+            while (wk.next(sg)) {
+                if (n < kMaxSegments) s_segs.seg[n] = sg;
+                ++n;
+            }
+            s_segs.n = n <= kMaxSegments ? n : -1;               // -1: too many short segments, walk every time
+        } else {
+            long long head0 = 0;
+            int b = 0, rows = wk.rows_of(0);
+            for (int idx = t - 1; idx < B * a.n_q_heads; idx += nthr - 1) {
+                const int bb = idx / a.n_q_heads, hh = idx - bb * a.n_q_heads;
+                while (b < bb) { head0 += (long long)a.n_q_heads * rows; ++b; rows = wk.rows_of(b); }
+                const long long h0 = head0 + (long long)hh * rows;
+                s_head_n[idx] = rows > 0 ? (unsigned char)(wk.owner_of(h0 + rows - 1) - wk.owner_of(h0) + 1) : 0;
+            }
+        }
+    };
+    build_step_tables(0, blockDim.x);
     __syncthreads();
 
-    // =========================================================================== producer and prefetch warps
-    // Both walk the SAME schedule: this CTA's share of every weight matrix and K/V tile of every step, in
-    // the order the consumers need it.  The producer copies piece after piece into the shared-memory ring
-    // and blocks only on free slots.  The optional prefetcher (l2_ahead > 0) runs further ahead and only asks
-    // L2 for the lines (prefetch.global.L2 through the load path, so the copy engine stays free), so that HBM
-    // keeps streaming while the consumers sit in barriers or in the latency-bound parts of attention; it
-    // stays at most l2_ahead pieces in front of the producer.  All its lanes walk the schedule in lockstep.
+    // =========================================================================== producer warp
+    // One thread walks this CTA's share of every weight matrix and K/V tile of every step, in the order the
+    // consumers need it, copies piece after piece into the shared-memory ring and blocks only on free slots.
     if (w >= nw) {
-        const bool is_prefetcher = (w == nw + 1);
-        if (w > nw + 1 || (is_prefetcher ? a.l2_ahead <= 0 : lane != 0)) return;
-        const int kPrefetchAhead = a.l2_ahead;
+        if (w > nw || lane != 0) return;
         const uint32_t wp = (uint32_t)lay.wpiece;
         int piece = 0;
-        // throttle of the prefetcher: wait (bounded) until the producer is within kPrefetchAhead pieces
-        auto throttle = [&]() -> bool {
-            if (piece - *reinterpret_cast<volatile int *>(&s_prod_piece) <= kPrefetchAhead) return true;
-            const unsigned long long t0 = global_ns();
-            while (piece - *reinterpret_cast<volatile int *>(&s_prod_piece) > kPrefetchAhead) {
-                if (*ring.abort_flag || global_ns() - t0 > kGridWaitNanos) return false;
-                __nanosleep(200);
-            }
-            return true;
-        };
+        // Copies in flight are limited separately from pieces buffered: every other memory access of the SM
+        // (the barrier, the activations of a prologue) queues behind the bulk copies already issued.
+        const int inflight = (a.max_inflight > 0 && a.max_inflight < lay.nslot) ? a.max_inflight : 0;   // 0: no separate limit
         auto weights = [&](const void *base, size_t first_byte, int npieces) -> bool {
             const unsigned char *p = static_cast<const unsigned char *>(base) + first_byte;
-            for (int i = 0; i < npieces; ++i, ++piece) {
-                if (is_prefetcher) {
-                    if (!throttle()) return false;
-                    prefetch_l2(p + (size_t)i * wp, wp);
-                } else {
-                    if (!ring.put(piece, p + (size_t)i * wp, wp)) return false;
-                    *reinterpret_cast<volatile int *>(&s_prod_piece) = piece + 1;
-                }
-            }
+            for (int i = 0; i < npieces; ++i, ++piece)
+                if ((inflight && !ring.landed(piece - inflight)) || !ring.put(piece, p + (size_t)i * wp, wp)) return false;
             return true;
         };
         for (int step = 0; step < a.n_steps; ++step) {
             for (int l = 0; l < a.n_layers; ++l) {
-                const LayerPtrs lp = a.layers[l];
+                const LayerPtrs &lp = s_layers[l];
                 if (!weights(lp.w_qkv, (size_t)q0 * tile_bytes, qn * SPT)) return;
-                if (!is_prefetcher && step > 0 && l == 0) {
-                    // K/V tiles of this step include the rows appended by the step before it: they may be
-                    // copied only once that step is complete grid-wide (weights are never held back).  For
-                    // all but toy models the flag is set long before the producer gets here.
+                if (step > 0 && l == 0) {
+                    // K/V tiles of this step include the rows appended by the step before it, and the share
+                    // table is rebuilt per step: both are ready once that step is complete grid-wide
+                    // (weights are never held back).  For all but toy models the flag is set long before
+                    // the producer gets here.
                     const unsigned long long t0 = global_ns();
                     while (*reinterpret_cast<volatile int *>(&s_steps_done) < step) {
                         if (*ring.abort_flag || global_ns() - t0 > kGridWaitNanos) { *ring.abort_flag = 1; return; }
                         __nanosleep(64);
                     }
+                    __threadfence_block();
                 }
                 const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
-                const bool kv_ok = attn_for_each_tile<DH>(aa, cta, ncta_attn, [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
-                    if (is_prefetcher) {
-                        if (!throttle()) return false;
-                        prefetch_l2(k, bytes);
-                        prefetch_l2(v, bytes);
-                        ++piece;
-                        return true;
-                    }
-                    const bool r = ring.put2(piece, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
-                    *reinterpret_cast<volatile int *>(&s_prod_piece) = ++piece;
-                    return r;
+                const bool kv_ok = attn_for_each_tile<DH>(aa, StepSource(&s_segs, aa, cta, ncta_attn),
+                                                          [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
+                    if (inflight && !ring.landed(piece - inflight)) return false;
+                    return ring.put2(piece++, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
                 });
                 if (!kv_ok) return;
                 if (!weights(lp.w_o, (size_t)o0 * tile_bytes, on * SPT)) return;
@@ -272,10 +293,26 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     // after every grid barrier
     int n_stamp = 0;
     auto stamp = [&]() {
+#ifdef FASTTPS_FINE_TRACE
+        if (a.trace && t == 0 && cta == 0 && n_stamp < a.trace_len)
+#else
         if (a.trace && t == 0 && (cta == 0 || cta == ncta - 1) && n_stamp < a.trace_len)
+#endif
             a.trace[(size_t)(cta ? 1 : 0) * a.trace_len + n_stamp] = global_ns();
         ++n_stamp;
     };
+#ifdef FASTTPS_FINE_TRACE
+    // development build: CTA 0 also stamps, into the second half of the buffer, the end of every product's
+    // prologue and of its tile loop (two stamps per product phase, none for attention)
+    int n_fine = 0;
+    auto fine = [&]() {
+        if (a.trace && t == 0 && cta == 0 && n_fine < a.trace_len) a.trace[(size_t)a.trace_len + n_fine] = global_ns();
+        ++n_fine;
+    };
+#define FT_FINE() fine()
+#else
+#define FT_FINE() ((void)0)
+#endif
     auto sync_phase = [&]() -> bool {
         stamp();
         const bool go = grid_sync(gb, nct, /*ok=*/ok);
@@ -295,7 +332,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
         for (int ph = 0; ph <= 4 * L; ++ph) {
             const int l = ph >> 2;
             const int kind = ph == 4 * L ? kHead : (ph & 3);
-            const LayerPtrs lp = a.layers[l < L ? l : L - 1];
+            const LayerPtrs &lp = s_layers[l < L ? l : L - 1];
             const int lprev = (kind == kHead ? L : l) - 1;                               // layer whose MLP sums feed x
             const float *y_prev = lprev >= 0 ? a.acc + (size_t)(lprev & 1) * B * D : nullptr;
             const __nv_bfloat16 *x_base = lprev >= 0 ? a.h : a.x0;                      // x = bf16(x_base + y_prev)
@@ -303,17 +340,41 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
             if (kind == kAttn) {
                 // ---- attention (Algorithm 3) ----
                 const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
-                ok = attn_consume<DH>(aa, ring, piece, cta, ncta_attn, scratch, nw) && ok;
+                // every CTA publishes the partial (max, sum, output) of each of its segments; nobody merges
+                // here: the output projection merges while it builds its B fragments
+                ok = attn_consume<DH, true>(aa, ring, piece, cta, StepSource(&s_segs, aa, cta, ncta_attn), scratch, nw) && ok;
             } else {
                 // ---- a matrix product: B fragments, then this CTA's row tiles ----
                 const __nv_bfloat16 *src = x_base, *gain = nullptr;
                 const float *add = y_prev;
                 int tile0 = 0, ntile = 0;
                 if (kind == kQkv) { gain = lp.g_attn; tile0 = q0; ntile = qn; }
-                else if (kind == kOproj) { src = a.attn_out; add = nullptr; tile0 = o0; ntile = on; }
+                else if (kind == kOproj) { tile0 = o0; ntile = on; }
                 else if (kind == kMlp) { src = a.h; add = nullptr; gain = lp.g_mlp; tile0 = m0; ntile = mn; }
                 else { gain = a.g_final; tile0 = l0; ntile = ln; }
-                load_b_frags<IPW>(bf, src, D, B, D, nw, gain, a.eps, smem_red, add);
+                // residual of the output projection for the first two tiles (all there are on a full grid),
+                // fetched by the epilogue threads now instead of in the epilogue, where the tile loop would wait
+                float res[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+                const bool res_pre = kind == kOproj && nct >= 64 && t < 64 && (t & 7) < B;
+                if (res_pre) {
+                    __nv_bfloat16 xb[2][2];
+                    float ya[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        int row = (o0 + (q >> 1)) * 16 + (t >> 3) + 8 * (q & 1);
+                        if (row >= D) row = D - 1;
+                        xb[q >> 1][q & 1] = ld_cg_bf16(x_base + (size_t)(t & 7) * D + row);
+                        if (y_prev) ya[q >> 1][q & 1] = ld_cg_f32(y_prev + (size_t)(t & 7) * D + row);
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float x = __bfloat162float(xb[q >> 1][q & 1]);
+                        res[q >> 1][q & 1] = y_prev ? bf16_round(x + ya[q >> 1][q & 1]) : x;
+                    }
+                }
+                if (kind == kOproj) load_b_frags_attn<IPW, DH>(bf, a.attn_part, s_head_n, B, a.n_q_heads, nw);
+                else load_b_frags<IPW>(bf, src, D, B, D, nw, gain, a.eps, smem_red, add);
+                FT_FINE();
                 if (kind == kHead) {
                     for (int u = t; u < 64; u += nct) { s_best_val[u] = -INFINITY; s_best_idx[u] = 0x7fffffff; }
                     named_bar_sync(1, nct);
@@ -335,8 +396,12 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                             if (row < nqkv) a.qkv[(size_t)b * nqkv + row] = __float2bfloat16_rn(v);
                         } else if (kind == kOproj) {         // h = x_l + attn . W_o
                             if (row < D) {
-                                float x = __bfloat162float(ld_cg_bf16(x_base + (size_t)b * D + row));
-                                if (y_prev) x = bf16_round(x + ld_cg_f32(y_prev + (size_t)b * D + row));
+                                float x;
+                                if (res_pre && tile < 2) x = tile == 0 ? res[0][hh] : res[1][hh];
+                                else {
+                                    x = __bfloat162float(ld_cg_bf16(x_base + (size_t)b * D + row));
+                                    if (y_prev) x = bf16_round(x + ld_cg_f32(y_prev + (size_t)b * D + row));
+                                }
                                 a.h[(size_t)b * D + row] = __float2bfloat16_rn(x + v);
                             }
                         } else if (row < a.V) {              // logits and the running argmax of this thread's rows
@@ -347,6 +412,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                     }
                 }) && ok;
                 piece += ntile * SPT;
+                FT_FINE();
 
                 if (kind == kMlp) {
                     // ---- down projection of this CTA's octets; the sums of all CTAs meet in acc[l & 1] ----
@@ -426,7 +492,12 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
         }
         if (step + 1 < a.n_steps) {
             if (!sync_phase()) return;
-            if (t == 0) atomicExch(&s_steps_done, step + 1);    // the producer may fetch the new K/V rows now
+            build_step_tables(step + 1, nct);
+            named_bar_sync(1, nct);
+            if (t == 0) {
+                __threadfence_block();
+                atomicExch(&s_steps_done, step + 1);            // the producer may fetch the new K/V rows now
+            }
         }
     }
 }
@@ -442,14 +513,14 @@ static int launch_step_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
     if (!configured[c->cfg.device & 15]) {
         FT_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemMax));
         int per_sm = 0;
-        FT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, (lay.nw + 2) * 32, lay.total));
+        FT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, (lay.nw + 1) * 32, lay.total));
         if (per_sm < 1) return FASTTPS_INVALID_ARG;
         configured[c->cfg.device & 15] = true;
     }
     // barrier counter and abort flag start from zero every launch (the generation may be anything)
     FT_CUDA(cudaMemsetAsync(c->grid_bar, 0, 64 * sizeof(unsigned), st));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(c->n_sm); cfg.blockDim = dim3((lay.nw + 2) * 32); cfg.dynamicSmemBytes = lay.total; cfg.stream = st;
+    cfg.gridDim = dim3(c->n_sm); cfg.blockDim = dim3((lay.nw + 1) * 32); cfg.dynamicSmemBytes = lay.total; cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
@@ -469,6 +540,7 @@ bool step_kernel_supported(const Ctx *c, int batch)
     if (batch < 1 || batch > kMaxNB) return false;
     if (f.n_q_heads * f.head_dim != f.hidden) return false;      // one reduction length for every product
     if (s.nw < 1 || s.nw > 12) return false;
+    if (f.n_q_heads > kMaxStepHeads || f.n_layers > kMaxStepLayers) return false;
     if (f.vocab < 1 || f.n_layers < 1) return false;
     return true;
 }

@@ -64,30 +64,39 @@ __device__ __forceinline__ void mlp_down_phase(WeightRing &ring, int piece0, int
 
 // y^T fragments -> FP32 accumulator `acc_g` [batch][D] in global memory with vector red.add, staged
 // through shared memory in IPW chunks of 32 * nw output columns (the columns the warps own for one
-// value of i are one contiguous chunk).  stage: 8 * 32 * nw floats that are idle (the partial-tile
-// scratch of the gate_up phase).  Consumer threads only (named barrier 1).
+// value of i are one contiguous chunk), several chunks per round when the batch is small.  stage:
+// 8 * 32 * nw floats that are idle (the partial-tile scratch of the gate_up phase).  Consumer threads
+// only (named barrier 1).
 template <int IPW>
 __device__ __forceinline__ void mlp_scatter_add(const float (&acc)[IPW][2][4], float *stage, float *acc_g, int batch,
                                                 int D, int nw)
 {
     const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3, nct = nw * 32;
     const int cw = 32 * nw;                                  // chunk width in columns
+    // chunks staged per round: as many as the stage holds (all 8 at batch 1: one barrier instead of fifteen)
+    const int R = batch <= 1 ? 8 : (batch <= 2 ? 4 : (batch <= 4 ? 2 : 1));
+    const int per_row = cw >> 2;
 #pragma unroll
     for (int i = 0; i < IPW; ++i) {
-        if (i > 0) named_bar_sync(1, nct);                   // the previous chunk has been read
+        const int ir = i % R;                                // slot of chunk i inside the round
+        if (ir == 0 && i > 0) named_bar_sync(1, nct);        // the previous round has been read
+        float *st = stage + (size_t)ir * batch * cw;
 #pragma unroll
         for (int m = 0; m < 2; ++m) {
             const int n = 32 * w + 16 * m + g;
             const int b0 = 2 * t4;
-            if (b0 < batch) { stage[b0 * cw + n] = acc[i][m][0]; stage[b0 * cw + n + 8] = acc[i][m][2]; }
-            if (b0 + 1 < batch) { stage[(b0 + 1) * cw + n] = acc[i][m][1]; stage[(b0 + 1) * cw + n + 8] = acc[i][m][3]; }
+            if (b0 < batch) { st[b0 * cw + n] = acc[i][m][0]; st[b0 * cw + n + 8] = acc[i][m][2]; }
+            if (b0 + 1 < batch) { st[(b0 + 1) * cw + n] = acc[i][m][1]; st[(b0 + 1) * cw + n + 8] = acc[i][m][3]; }
         }
-        named_bar_sync(1, nct);
-        const int per_row = cw >> 2;
-        for (int idx = t; idx < batch * per_row; idx += nct) {
-            const int b = idx / per_row, j = idx - b * per_row;
-            const float4 v = *reinterpret_cast<const float4 *>(stage + b * cw + 4 * j);
-            red_add_v4(acc_g + (size_t)b * D + (size_t)cw * i + 4 * j, v.x, v.y, v.z, v.w);
+        if (ir == R - 1 || i == IPW - 1) {
+            named_bar_sync(1, nct);
+            const int i0 = i - ir, nchunk = ir + 1;
+            for (int idx = t; idx < nchunk * batch * per_row; idx += nct) {
+                const int cb = idx / per_row, j = idx - cb * per_row;      // cb = chunk * batch + b
+                const int ch = cb / batch, b = cb - ch * batch;
+                const float4 v = *reinterpret_cast<const float4 *>(stage + (size_t)cb * cw + 4 * j);
+                red_add_v4(acc_g + (size_t)b * D + (size_t)cw * (i0 + ch) + 4 * j, v.x, v.y, v.z, v.w);
+            }
         }
     }
 }
