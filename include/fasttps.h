@@ -138,6 +138,22 @@ int fasttps_attn_decode(fasttps_ctx *ctx, const void *q, const void *k_new, cons
 int fasttps_mlp_decode(fasttps_ctx *ctx, const void *x, const void *w_gate_up, const void *w_down,
                        void *out, int batch, void *stream);
 
+/* Variant of fasttps_mlp_decode that uses no workspace memory and allocates nothing.  The paper has
+ * no counterpart: the arithmetic and the kernel are those of fasttps_mlp_decode; only the scratch of
+ * the kernel (the FP32 accumulator of batch x hidden partial sums and its arrival counter) lives in a
+ * fixed array in the library's own device data segment instead of the context workspace.  It is for
+ * callers that may not allocate device memory where they call (a frozen memory pool, an allocator
+ * lock held elsewhere) and do not want to depend on a workspace they did not size.
+ *   Limits: batch <= 8 and hidden <= 6144 (192 KB of accumulator); larger requests return
+ *   FASTTPS_INVALID_ARG with a message in fasttps_last_error() and launch nothing.
+ *   Set-up: the first call on a device looks the array's address up once (this may load the module);
+ *   make it during initialisation, before capturing a stream.  No call allocates or frees.
+ *   Every call clears the counter and the accumulator rows it uses, on `stream`, before the kernel.
+ *   The array is one per device and process: calls that overlap in time (other streams or threads)
+ *   race on it; calls on one stream are ordered. */
+int fasttps_mlp_decode_static(fasttps_ctx *ctx, const void *x, const void *w_gate_up, const void *w_down,
+                              void *out, int batch, void *stream);
+
 /* Building block of the chain (QKV, output projection, lm_head; Figure 1):
  *   out[b,n] = (g_norm ? rmsnorm(x[b], g_norm) : x[b]) . W[n,:] (+ residual[b,n])
  *   x [B,in]; w packed [out,in]; residual [B,out] or NULL; out_bf16 [B,out] or NULL;

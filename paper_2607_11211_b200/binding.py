@@ -55,6 +55,7 @@ def load_library() -> C.CDLL:
     lib.fasttps_unpack_weight.argtypes = [vp, i, vp, vp, vp]
     lib.fasttps_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, vp, i, vp]
     lib.fasttps_mlp_decode.argtypes = [vp, vp, vp, vp, vp, i, vp]
+    lib.fasttps_mlp_decode_static.argtypes = [vp, vp, vp, vp, vp, i, vp]
     lib.fasttps_linear_decode.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, i, vp]
     lib.fasttps_layer_decode.argtypes = [vp, C.POINTER(LayerWeights), vp, vp, vp, vp, ip, ip, i, vp]
     lib.fasttps_model_decode.argtypes = [vp, vp, C.POINTER(LayerWeights), vp, vp, C.POINTER(vp), C.POINTER(vp),
@@ -165,6 +166,12 @@ class Context:
     def mlp_decode(self, x, w_gate_up, w_down, out, stream=None):
         _check(self.lib.fasttps_mlp_decode(self.handle, _ptr(x), _ptr(w_gate_up), _ptr(w_down), _ptr(out),
                                            x.shape[0], _stream(stream)), "fasttps_mlp_decode")
+        return out
+
+    def mlp_decode_static(self, x, w_gate_up, w_down, out, stream=None):
+        """fasttps_mlp_decode with the kernel's scratch in the library's fixed device array (no workspace)."""
+        _check(self.lib.fasttps_mlp_decode_static(self.handle, _ptr(x), _ptr(w_gate_up), _ptr(w_down), _ptr(out),
+                                                  x.shape[0], _stream(stream)), "fasttps_mlp_decode_static")
         return out
 
     def linear_decode(self, kind, x, g_norm, w, residual, out_bf16, out_f32, stream=None):

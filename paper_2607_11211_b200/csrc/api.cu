@@ -17,6 +17,8 @@ void set_last_error(cudaError_t e, const char *where)
     snprintf(g_last_error, sizeof g_last_error, "%s: %s (%s)", where, cudaGetErrorName(e), cudaGetErrorString(e));
 }
 
+void set_last_error_text(const char *msg) { snprintf(g_last_error, sizeof g_last_error, "%s", msg); }
+
 bool pdl_enabled()
 {
     static const bool on = [] {

@@ -74,6 +74,7 @@ struct ProfScope {
 };
 
 void set_last_error(cudaError_t e, const char *where);
+void set_last_error_text(const char *msg);
 
 #define FT_CUDA(call)                                                   \
     do {                                                                \
