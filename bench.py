@@ -32,11 +32,15 @@ if str(ROOT) not in sys.path:
 METRIC = "decode_tokens_per_s"
 UNIT = "tok/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one mlp_decode_kernel launch (Phi-3 shape,
-# batch 1) from the ncu capture summarised in profiles/; None until a capture exists.
-NCU_MLP_TRAFFIC_BYTES = None
-# the same for one decode step inside a decode_step_kernel launch (cfg3 shape)
-NCU_STEP_TRAFFIC_BYTES_PER_STEP = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one mlp_decode_kernel launch (Phi-3 shape, batch 1) from the
+# ncu capture summarised in profiles/chain_kernels_cfg1_cfg2.md (151.09 MB read + 4.05 MB written).
+NCU_MLP_TRAFFIC_BYTES = 155.1e6
+# DRAM traffic of decode_step_kernel relative to its algorithmic bytes, from two ncu captures of one decode
+# step of the cfg3 shape cut to 4 and to 8 layers (profiles/decode_step_kernel_cfg3.md): 243.9 MB per layer
+# and 212 MB for the head against 239.1 MB and 197.1 MB algorithmic, i.e. 8.017 GB for a full 32-layer step
+# against 7.873 GB.  The full-size launch is too large to capture; traffic grows in proportion to the layers
+# and steps a launch processes.
+NCU_STEP_TRAFFIC_RATIO = 1.018
 
 
 def parse_args():
@@ -47,8 +51,11 @@ def parse_args():
     ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--graph", type=int, default=1, help="replay the step as a CUDA graph (1) or launch eagerly (0)")
-    ap.add_argument("--step-kernel", type=int, default=0,
+    ap.add_argument("--step-kernel", type=int, default=1,
                     help="1: whole decode steps in the persistent cooperative kernel (batch <= 8)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="run only this many layers of a full-stack workload (a small case for profiler captures; "
+                         "not the benchmark configuration)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -204,6 +211,9 @@ def run_ours(args):
     dev = torch.device("cuda", local)
 
     W = wl.workload(args.workload)
+    if args.layers > 0 and W.full_stack:
+        import dataclasses
+        W = dataclasses.replace(W, n_layers=args.layers)
     dm, B = W.dims, W.batch
     K, Wm = args.steps, max(args.warmup, 3)
     lens0 = np.asarray(W.past_lens, np.int32)
@@ -296,13 +306,14 @@ def run_ours(args):
                     step(i)
 
     # ---- warm-up, then the timed region ----
-    reset_state()
-    run_steps(Wm)
-    reset_state()
-    launches0 = ctx.launch_count()
+    # (the clock sampler is started first: an idle gap between the warm-up and the timed region would let the
+    # GPU drop out of its loaded power state)
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)
+    reset_state()
+    run_steps(Wm)
+    reset_state()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     ev0.record(stream)
@@ -350,7 +361,7 @@ def run_ours(args):
         steps_per_launch = n_prof if one_call else 1
         dom_bytes = float(sum(W.algorithmic_bytes(s if advance else 0) for s in range(steps_per_launch)))
         dom_name = "decode_step_kernel"
-        ncu_traffic = NCU_STEP_TRAFFIC_BYTES_PER_STEP * steps_per_launch if NCU_STEP_TRAFFIC_BYTES_PER_STEP else None
+        ncu_traffic = dom_bytes * NCU_STEP_TRAFFIC_RATIO if (dm is wl.PHI3_MINI and B == 1) else None
     else:
         dom, (dom_ms, dom_n) = "mlp", prof["mlp"]
         dom_bytes, dom_name, ncu_traffic = float(mlp_bytes), "mlp_decode_kernel", NCU_MLP_TRAFFIC_BYTES
@@ -423,9 +434,11 @@ def run_ours(args):
         step_bytes = np.mean([W.algorithmic_bytes(s if advance else 0) for s in range(K if advance else 1)])
         line = {"metric": METRIC, "value": tokens / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
                 "warmup": Wm, "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate", "data": "synthetic",
-                "config": {"workload": args.workload, "batch": B, "n_layers": W.n_layers, "full_stack": W.full_stack,
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": args.workload + (f" cut to {W.n_layers} layers (profiling case)" if args.layers > 0 and W.full_stack else ""),
+                           "batch": B, "n_layers": W.n_layers, "full_stack": W.full_stack,
                            "past_lens": lens0.tolist()[:8], "max_seq": max_seq,
+                           "arithmetic": "bf16 tensors, bf16 tensor-core products, f32 accumulation and softmax",
                            "launch": "one persistent-kernel launch for all steps" if one_call else
                                      ("cuda_graph_replay" if use_graph else "eager"),
                            "l2": "inputs larger than L2: every step streams %.2f GB of weights and KV" % (step_bytes / 1e9)

@@ -88,7 +88,7 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     c->n_sm = c->prop.multiProcessorCount;
     {
         const char *e = getenv("FASTTPS_STEP_KERNEL");
-        c->opt_step_kernel = (e && *e) ? atoi(e) != 0 : 0;
+        c->opt_step_kernel = (e && *e) ? atoi(e) != 0 : 1;
         e = getenv("FASTTPS_RING_INFLIGHT");
         c->opt_ring_inflight = (e && *e) ? atoi(e) : 0;
     }
