@@ -36,11 +36,11 @@ UNIT = "tok/s"
 # ncu capture summarised in profiles/chain_kernels_cfg1_cfg2.md (151.09 MB read + 4.05 MB written).
 NCU_MLP_TRAFFIC_BYTES = 155.1e6
 # DRAM traffic of decode_step_kernel relative to its algorithmic bytes, from two ncu captures of one decode
-# step of the cfg3 shape cut to 4 and to 8 layers (profiles/decode_step_kernel_cfg3.md): 243.9 MB per layer
-# and 212 MB for the head against 239.1 MB and 197.1 MB algorithmic, i.e. 8.017 GB for a full 32-layer step
+# step of the cfg3 shape cut to 4 and to 8 layers (profiles/decode_step_kernel_cfg3.md): 245.3 MB per layer
+# and 206 MB for the head against 239.1 MB and 197.1 MB algorithmic, i.e. 8.06 GB for a full 32-layer step
 # against 7.873 GB.  The full-size launch is too large to capture; traffic grows in proportion to the layers
 # and steps a launch processes.
-NCU_STEP_TRAFFIC_RATIO = 1.018
+NCU_STEP_TRAFFIC_RATIO = 1.023
 
 
 def parse_args():
@@ -188,6 +188,29 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------- replicas (N > 1)
+
+def replica_seed(master_seed: int, rank: int) -> int:
+    """Every replica generates its own weights, caches and token ids."""
+    return master_seed + 1000 * rank
+
+
+def max_over_ranks(x: float, device, world: int) -> float:
+    """Slowest rank's time: the only data the replicas exchange (besides the barrier)."""
+    if world == 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: int, world: int, seconds_max: float) -> float:
+    """Whole-job throughput: the units all ranks processed over the slowest rank's time."""
+    return world * units_per_rank / seconds_max
+
+
 # ------------------------------------------------------------------ our arm
 
 def run_ours(args):
@@ -225,7 +248,7 @@ def run_ours(args):
 
     ctx = fb.Context.from_dims(dm, B, max_seq, device=local, n_layers=W.n_layers)
     ctx.set_option("step_kernel", args.step_kernel)
-    seed = wl.MASTER_SEED + 1000 * rank
+    seed = replica_seed(wl.MASTER_SEED, rank)
 
     def packed_layer(idx):
         w = wl.layer_weights(dm, idx, seed, device=dev)
@@ -323,10 +346,7 @@ def run_ours(args):
     barrier()
     ms = ev0.elapsed_time(ev1)
     clocks = sampler.stop()
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max = float(t.item())
+    ms_max = max_over_ranks(ms, dev, world)
     status = ctx.get_status()
 
     # kernels per step: count one eager step
@@ -417,10 +437,7 @@ def run_ours(args):
                     stream.synchronize()
             el = time.perf_counter() - t0
             bi = bo = B * dm.hidden * 2
-        te = torch.tensor([el], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * B * K / float(te.item()), "unit": UNIT, "h2d_bytes_per_step": bi,
+        e2e = {"value": whole_job_rate(B * K, world, max_over_ranks(el, dev, world)), "unit": UNIT, "h2d_bytes_per_step": bi,
                "d2h_bytes_per_step": bo, "timing": "host wall clock around K calls that each synchronise"}
 
     # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1 only) ----
@@ -430,9 +447,8 @@ def run_ours(args):
         cpu = {"value": B / per_step, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
 
     if rank == 0:
-        tokens = world * B * K
         step_bytes = np.mean([W.algorithmic_bytes(s if advance else 0) for s in range(K if advance else 1)])
-        line = {"metric": METRIC, "value": tokens / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        line = {"metric": METRIC, "value": whole_job_rate(B * K, world, ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
                 "warmup": Wm, "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": args.workload + (f" cut to {W.n_layers} layers (profiling case)" if args.layers > 0 and W.full_stack else ""),
