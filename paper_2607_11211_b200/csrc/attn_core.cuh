@@ -137,12 +137,18 @@ template <int DH> struct AttnTile {
 
 // Calls f(k_tile, v_tile, bytes_each) for every K/V tile of this CTA's share, in walk order; stops and
 // returns false as soon as f does.
-// A share as a list of segments kept in shared memory (the persistent kernel computes it once per step
-// and uses it for every layer).
-constexpr int kMaxSegments = 20;
+// A share as a list of segments kept in shared memory (the persistent kernel computes it once per step and
+// uses it for every layer).  12 bytes per segment; lengths and positions of the step sit beside the list.
+constexpr int kMaxSegments = 257;            // a share touches at most batch * n_q_heads heads (<= 256 here)
+struct PackedSegment {
+    int r0, r1;
+    unsigned short bh;                       // b * n_q_heads + h
+    unsigned char first_cta, n_cta;
+};
 struct SegmentList {
-    int n;
-    Segment seg[kMaxSegments];
+    int n, n_q_heads;
+    int len[kMaxNB], pos[kMaxNB];            // cached rows and rotary position of every sequence in this step
+    PackedSegment seg[kMaxSegments];
 };
 
 // Segment sources: `bool next(Segment &)`.
@@ -161,7 +167,10 @@ struct ListSource {
     __device__ __forceinline__ bool next(Segment &s)
     {
         if (i >= list->n) return false;
-        s = list->seg[i++];
+        const PackedSegment p = list->seg[i++];
+        s.b = p.bh / list->n_q_heads; s.h = p.bh - s.b * list->n_q_heads;
+        s.L = list->len[s.b]; s.pos = list->pos[s.b];
+        s.r0 = p.r0; s.r1 = p.r1; s.first_cta = p.first_cta; s.n_cta = p.n_cta;
         return true;
     }
 };

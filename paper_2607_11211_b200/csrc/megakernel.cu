@@ -28,25 +28,6 @@ constexpr int kMegaThreadsMax = 416;
 constexpr int kMaxStepLayers = 48;                                     // layers the shared-memory layer table holds
 constexpr int kMaxStepHeads = 128;                                     // query heads the per-step head table holds
 
-// The attention share of a CTA for one step: the segment list when it fits (computed once per step, used
-// by the producer and the consumers for every layer), else the walk itself.
-struct StepSource {
-    const SegmentList *list;
-    int i;
-    ShareWalk walk;
-    __device__ __forceinline__ StepSource(const SegmentList *l, const AttnArgs &a, int cta, int ncta) : list(l), i(0)
-    {
-        if (l->n < 0) walk.init(a.seq_lens, a.pos, a.len_add, a.batch, a.n_q_heads, a.max_seq, cta, ncta);
-    }
-    __device__ __forceinline__ bool next(Segment &s)
-    {
-        if (list->n < 0) return walk.next(s);
-        if (i >= list->n) return false;
-        s = list->seg[i++];
-        return true;
-    }
-};
-
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
 {
     unsigned v;
@@ -138,7 +119,12 @@ __device__ __forceinline__ AttnArgs attn_args_of(const StepArgs &a, const LayerP
     return aa;
 }
 
-template <int IPW, int DH>
+// DEFER: where the softmax merge of a head shared by several CTAs happens.  true (batch <= 2): every CTA only
+// publishes its partials and the prologue of the output projection merges them on the fly -- no ticket chain in
+// the short attention phase.  false: the CTA that finishes a head last merges it, hidden behind the long
+// attention phase of a larger batch, where the merge loads of the prologue would serialise.  Two kernels
+// rather than a run-time switch: code that does not run still costs instruction-cache reach and registers.
+template <int IPW, int DH, bool DEFER>
 __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArgs a)
 {
     extern __shared__ __align__(128) unsigned char dsm[];
@@ -147,14 +133,14 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     __shared__ float s_best_val[64];
     __shared__ int s_best_idx[64];
     __shared__ int s_go;
-    __shared__ int s_steps_done;
+    __shared__ int s_tables_ready;                               // steps whose attention tables are built
     __shared__ LayerPtrs s_layers[kMaxStepLayers];               // the layer table: no global round trip per phase
     __shared__ SegmentList s_segs;                               // this CTA's attention share for the current step
-    __shared__ unsigned char s_head_n[kMaxNB * kMaxStepHeads];   // CTAs that share head (b, h) in the current step
+    __shared__ unsigned char s_head_n[kMaxSegments];               // CTAs that share head (b, h) in the current step
 
     const int t = threadIdx.x, lane = t & 31, w = t >> 5;
     const int cta = blockIdx.x, ncta = gridDim.x;
-    if (t == 0) s_steps_done = 0;
+    if (t == 0) s_tables_ready = 0;
     const MegaLayout lay = mega_layout<DH>(a.D);
     const int nw = lay.nw, nct = nw * 32;
     float *smem_part = reinterpret_cast<float *>(dsm + lay.part_off);
@@ -186,22 +172,26 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
 
     // Per-step attention tables (the lengths grow by one per step, so the split changes with the step, but
     // not with the layer): the segments of this CTA's share, and for every head the number of CTAs that
-    // publish a partial for it.  Threads [0, nthr) take part.
-    auto build_step_tables = [&](int step, int nthr) {
+    // publish a partial for it.  Built by the consumer threads at the top of every step, after the barrier that
+    // ends the step before; the producer waits for s_tables_ready before it fetches the step's first K/V tile.
+    auto build_step_tables = [&](int step) {
         ShareWalk wk;
         wk.init(a.seq_lens, a.pos, step, B, a.n_q_heads, a.max_seq, cta, ncta_attn);
         if (t == 0) {
             int n = 0;
             Segment sg;
-            while (wk.next(sg)) {
-                if (n < kMaxSegments) s_segs.seg[n] = sg;
-                ++n;
+            while (wk.next(sg) && n < kMaxSegments) {
+                PackedSegment p;
+                p.r0 = sg.r0; p.r1 = sg.r1; p.bh = (unsigned short)(sg.b * a.n_q_heads + sg.h);
+                p.first_cta = (unsigned char)sg.first_cta; p.n_cta = (unsigned char)sg.n_cta;
+                s_segs.seg[n++] = p;
             }
-            s_segs.n = n <= kMaxSegments ? n : -1;               // -1: too many short segments, walk every time
+            s_segs.n = n; s_segs.n_q_heads = a.n_q_heads;
+            for (int bb = 0; bb < B; ++bb) { s_segs.len[bb] = wk.rows_of(bb) - 1; s_segs.pos[bb] = a.pos[bb] + step; }
         } else {
             long long head0 = 0;
             int b = 0, rows = wk.rows_of(0);
-            for (int idx = t - 1; idx < B * a.n_q_heads; idx += nthr - 1) {
+            for (int idx = t - 1; idx < B * a.n_q_heads; idx += nct - 1) {
                 const int bb = idx / a.n_q_heads, hh = idx - bb * a.n_q_heads;
                 while (b < bb) { head0 += (long long)a.n_q_heads * rows; ++b; rows = wk.rows_of(b); }
                 const long long h0 = head0 + (long long)hh * rows;
@@ -209,7 +199,6 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
             }
         }
     };
-    build_step_tables(0, blockDim.x);
     __syncthreads();
 
     // =========================================================================== producer warp
@@ -232,20 +221,20 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
             for (int l = 0; l < a.n_layers; ++l) {
                 const LayerPtrs &lp = s_layers[l];
                 if (!weights(lp.w_qkv, (size_t)q0 * tile_bytes, qn * SPT)) return;
-                if (step > 0 && l == 0) {
+                if (l == 0) {
                     // K/V tiles of this step include the rows appended by the step before it, and the share
-                    // table is rebuilt per step: both are ready once that step is complete grid-wide
-                    // (weights are never held back).  For all but toy models the flag is set long before
-                    // the producer gets here.
+                    // table is rebuilt per step: both are ready once the consumers have passed the barrier
+                    // that ends that step and built the table (weights are never held back).  For all but
+                    // toy models the flag is set long before the producer gets here.
                     const unsigned long long t0 = global_ns();
-                    while (*reinterpret_cast<volatile int *>(&s_steps_done) < step) {
+                    while (*reinterpret_cast<volatile int *>(&s_tables_ready) <= step) {
                         if (*ring.abort_flag || global_ns() - t0 > kGridWaitNanos) { *ring.abort_flag = 1; return; }
                         __nanosleep(64);
                     }
                     __threadfence_block();
                 }
                 const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
-                const bool kv_ok = attn_for_each_tile<DH>(aa, StepSource(&s_segs, aa, cta, ncta_attn),
+                const bool kv_ok = attn_for_each_tile<DH>(aa, ListSource(&s_segs),
                                                           [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
                     if (inflight && !ring.landed(piece - inflight)) return false;
                     return ring.put2(piece++, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
@@ -329,6 +318,12 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     enum { kQkv = 0, kAttn = 1, kOproj = 2, kMlp = 3, kHead = 4 };
     const int L = a.n_layers;
     for (int step = 0; step < a.n_steps; ++step) {
+        build_step_tables(step);
+        named_bar_sync(1, nct);
+        if (t == 0) {
+            __threadfence_block();
+            atomicExch(&s_tables_ready, step + 1);              // the producer may fetch this step's K/V rows now
+        }
         for (int ph = 0; ph <= 4 * L; ++ph) {
             const int l = ph >> 2;
             const int kind = ph == 4 * L ? kHead : (ph & 3);
@@ -342,14 +337,14 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                 const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
                 // every CTA publishes the partial (max, sum, output) of each of its segments; nobody merges
                 // here: the output projection merges while it builds its B fragments
-                ok = attn_consume<DH, true>(aa, ring, piece, cta, StepSource(&s_segs, aa, cta, ncta_attn), scratch, nw) && ok;
+                ok = attn_consume<DH, DEFER>(aa, ring, piece, cta, ListSource(&s_segs), scratch, nw) && ok;
             } else {
                 // ---- a matrix product: B fragments, then this CTA's row tiles ----
                 const __nv_bfloat16 *src = x_base, *gain = nullptr;
                 const float *add = y_prev;
                 int tile0 = 0, ntile = 0;
                 if (kind == kQkv) { gain = lp.g_attn; tile0 = q0; ntile = qn; }
-                else if (kind == kOproj) { tile0 = o0; ntile = on; }
+                else if (kind == kOproj) { src = a.attn_out; add = nullptr; tile0 = o0; ntile = on; }
                 else if (kind == kMlp) { src = a.h; add = nullptr; gain = lp.g_mlp; tile0 = m0; ntile = mn; }
                 else { gain = a.g_final; tile0 = l0; ntile = ln; }
                 // residual of the output projection for the first two tiles (all there are on a full grid),
@@ -372,7 +367,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                         res[q >> 1][q & 1] = y_prev ? bf16_round(x + ya[q >> 1][q & 1]) : x;
                     }
                 }
-                if (kind == kOproj) load_b_frags_attn<IPW, DH>(bf, a.attn_part, s_head_n, B, a.n_q_heads, nw);
+                if (DEFER && kind == kOproj) load_b_frags_attn<IPW, DH>(bf, a.attn_part, s_head_n, B, a.n_q_heads, nw);
                 else load_b_frags<IPW>(bf, src, D, B, D, nw, gain, a.eps, smem_red, add);
                 FT_FINE();
                 if (kind == kHead) {
@@ -490,25 +485,17 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                 embed_rows(a.tok);
             }
         }
-        if (step + 1 < a.n_steps) {
-            if (!sync_phase()) return;
-            build_step_tables(step + 1, nct);
-            named_bar_sync(1, nct);
-            if (t == 0) {
-                __threadfence_block();
-                atomicExch(&s_steps_done, step + 1);            // the producer may fetch the new K/V rows now
-            }
-        }
+        if (step + 1 < a.n_steps && !sync_phase()) return;
     }
 }
 
 }  // namespace
 
-template <int IPW, int DH>
+template <int IPW, int DH, bool DEFER>
 static int launch_step_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
 {
     const MegaLayout lay = mega_layout<DH>(a.D);
-    auto kernel = decode_step_kernel<IPW, DH>;
+    auto kernel = decode_step_kernel<IPW, DH, DEFER>;
     static bool configured[16] = {};
     if (!configured[c->cfg.device & 15]) {
         FT_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemMax));
@@ -541,6 +528,7 @@ bool step_kernel_supported(const Ctx *c, int batch)
     if (f.n_q_heads * f.head_dim != f.hidden) return false;      // one reduction length for every product
     if (s.nw < 1 || s.nw > 12) return false;
     if (f.n_q_heads > kMaxStepHeads || f.n_layers > kMaxStepLayers) return false;
+    if (batch * f.n_q_heads >= kMaxSegments || c->n_sm > 255) return false;   // segment table: capacity, 8-bit CTA index
     if (f.vocab < 1 || f.n_layers < 1) return false;
     return true;
 }
@@ -548,8 +536,11 @@ bool step_kernel_supported(const Ctx *c, int batch)
 int launch_step(Ctx *c, const StepArgs &a, cudaStream_t st)
 {
     const int ipw = warp_split(a.D).ipw;
-#define FT_STEP(DHV)                                                                          \
-    case DHV: return ipw == 8 ? launch_step_inst<8, DHV>(c, a, st) : launch_step_inst<4, DHV>(c, a, st)
+    const bool defer = a.batch <= 2;
+#define FT_STEP(DHV)                                                                                     \
+    case DHV:                                                                                            \
+        if (defer) return ipw == 8 ? launch_step_inst<8, DHV, true>(c, a, st) : launch_step_inst<4, DHV, true>(c, a, st); \
+        return ipw == 8 ? launch_step_inst<8, DHV, false>(c, a, st) : launch_step_inst<4, DHV, false>(c, a, st)
     switch (a.head_dim) {
         FT_STEP(32);
         FT_STEP(64);
