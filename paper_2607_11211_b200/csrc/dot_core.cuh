@@ -137,6 +137,7 @@ __device__ __forceinline__ bool dot_tiles(WeightRing &ring, int g0, int ntiles, 
     constexpr int SPT = IPW / kBlocksPerWarpPerSlot;      // ring pieces per row tile
     const int t = threadIdx.x, lane = t & 31, w = t >> 5;
     bool ok = true;
+#pragma unroll 1
     for (int tile = 0; tile < ntiles; ++tile) {
         float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll

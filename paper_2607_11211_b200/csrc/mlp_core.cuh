@@ -41,6 +41,7 @@ __device__ __forceinline__ void mlp_down_phase(WeightRing &ring, int piece0, int
 {
     constexpr int PPO = IPW / 4;                            // ring pieces per octet
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, g = lane >> 2, t4 = lane & 3;
+#pragma unroll 1
     for (int o = 0; o < noct; ++o) {
         const uint32_t bh = *reinterpret_cast<const uint32_t *>(&s_hi[o][g][2 * t4]);
         const uint32_t bl = *reinterpret_cast<const uint32_t *>(&s_lo[o][g][2 * t4]);
@@ -62,6 +63,21 @@ __device__ __forceinline__ void mlp_down_phase(WeightRing &ring, int piece0, int
     }
 }
 
+// One round of mlp_scatter_add: the staged chunks i0 .. i0 + nchunk - 1 go to global memory.  Out of line: the
+// caller is unrolled over the chunks and would carry a copy of this loop for each of them.
+static __device__ __noinline__ void mlp_scatter_drain(const float *stage, float *acc_g, int i0, int nchunk, int batch, int D,
+                                                      int cw, int nct)
+{
+    const int t = threadIdx.x, per_row = cw >> 2;
+    named_bar_sync(1, nct);
+    for (int idx = t; idx < nchunk * batch * per_row; idx += nct) {
+        const int cb = idx / per_row, j = idx - cb * per_row;      // cb = chunk * batch + b
+        const int ch = cb / batch, b = cb - ch * batch;
+        const float4 v = *reinterpret_cast<const float4 *>(stage + (size_t)cb * cw + 4 * j);
+        red_add_v4(acc_g + (size_t)b * D + (size_t)cw * (i0 + ch) + 4 * j, v.x, v.y, v.z, v.w);
+    }
+}
+
 // y^T fragments -> FP32 accumulator `acc_g` [batch][D] in global memory with vector red.add, staged
 // through shared memory in IPW chunks of 32 * nw output columns (the columns the warps own for one
 // value of i are one contiguous chunk), several chunks per round when the batch is small.  stage:
@@ -75,7 +91,6 @@ __device__ __forceinline__ void mlp_scatter_add(const float (&acc)[IPW][2][4], f
     const int cw = 32 * nw;                                  // chunk width in columns
     // chunks staged per round: as many as the stage holds (all 8 at batch 1: one barrier instead of fifteen)
     const int R = batch <= 1 ? 8 : (batch <= 2 ? 4 : (batch <= 4 ? 2 : 1));
-    const int per_row = cw >> 2;
 #pragma unroll
     for (int i = 0; i < IPW; ++i) {
         const int ir = i % R;                                // slot of chunk i inside the round
@@ -88,16 +103,7 @@ __device__ __forceinline__ void mlp_scatter_add(const float (&acc)[IPW][2][4], f
             if (b0 < batch) { st[b0 * cw + n] = acc[i][m][0]; st[b0 * cw + n + 8] = acc[i][m][2]; }
             if (b0 + 1 < batch) { st[(b0 + 1) * cw + n] = acc[i][m][1]; st[(b0 + 1) * cw + n + 8] = acc[i][m][3]; }
         }
-        if (ir == R - 1 || i == IPW - 1) {
-            named_bar_sync(1, nct);
-            const int i0 = i - ir, nchunk = ir + 1;
-            for (int idx = t; idx < nchunk * batch * per_row; idx += nct) {
-                const int cb = idx / per_row, j = idx - cb * per_row;      // cb = chunk * batch + b
-                const int ch = cb / batch, b = cb - ch * batch;
-                const float4 v = *reinterpret_cast<const float4 *>(stage + (size_t)cb * cw + 4 * j);
-                red_add_v4(acc_g + (size_t)b * D + (size_t)cw * (i0 + ch) + 4 * j, v.x, v.y, v.z, v.w);
-            }
-        }
+        if (ir == R - 1 || i == IPW - 1) mlp_scatter_drain(stage, acc_g, i - ir, ir + 1, batch, D, cw, nct);
     }
 }
 
