@@ -214,9 +214,7 @@ int fasttps_model_decode_host(fasttps_ctx *ctx, const void *embed, const fasttps
 
 /* Tuning switches of a context (host side, take effect at the next call):
  *   "step_kernel" 0/1  route model calls with batch <= 8 through the persistent step kernel
- *                      (default: environment variable FASTTPS_STEP_KERNEL, else 1);
- *   "ring_inflight" n  ring pieces whose copies the step kernel's producer keeps in flight at most
- *                      (0 = as many as the ring has slots; default: FASTTPS_RING_INFLIGHT, else 0).
+ *                      (default: environment variable FASTTPS_STEP_KERNEL, else 1).
  * Unknown names return FASTTPS_INVALID_ARG. */
 int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value);
 

@@ -89,8 +89,6 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     {
         const char *e = getenv("FASTTPS_STEP_KERNEL");
         c->opt_step_kernel = (e && *e) ? atoi(e) != 0 : 1;
-        e = getenv("FASTTPS_RING_INFLIGHT");
-        c->opt_ring_inflight = (e && *e) ? atoi(e) : 0;
     }
     {
         int rc = configure_attn_kernels();
@@ -349,7 +347,6 @@ int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value)
     if (!ctx || !name) return FASTTPS_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);
     if (strcmp(name, "step_kernel") == 0) c->opt_step_kernel = value != 0;
-    else if (strcmp(name, "ring_inflight") == 0) c->opt_ring_inflight = value < 0 ? 0 : value;
     else return FASTTPS_INVALID_ARG;
     return FASTTPS_OK;
 }
@@ -412,7 +409,6 @@ static int step_impl(Ctx *c, const void *embed, const fasttps_layer_weights *lay
     a.amax_val = c->amax_val; a.amax_idx = c->amax_idx; a.tok = c->tok2;
     a.bar = c->grid_bar; a.status = c->status;
     a.trace = c->trace; a.trace_len = kTraceLen;
-    a.max_inflight = c->opt_ring_inflight;
     return launch_step(c, a, st);
 }
 

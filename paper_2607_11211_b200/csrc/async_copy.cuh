@@ -132,15 +132,6 @@ struct WeightRing {
         }
         return true;
     }
-    // producer thread: bounded wait until the copies of piece g (issued earlier, slot not reused since) have landed
-    __device__ __forceinline__ bool landed(int g)
-    {
-        if (g >= 0 && !mbar_wait_bounded(&full[g % nslot], (uint32_t)(g / nslot) & 1u, abort_flag)) {
-            *abort_flag = 1;
-            return false;
-        }
-        return true;
-    }
     // producer thread: piece g = `bytes` contiguous bytes at src
     __device__ __forceinline__ bool put(int g, const void *src, uint32_t bytes)
     {

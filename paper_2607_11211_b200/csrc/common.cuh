@@ -24,7 +24,6 @@ struct Ctx {
     LayerPtrs *d_layers, *pin_layers;
     int layers_uploaded;             // number of valid entries in pin_layers / d_layers
     int opt_step_kernel;             // 1: model calls with batch <= 8 use the persistent step kernel
-    int opt_ring_inflight;           // ring pieces the step kernel's producer keeps in flight at most (0 = all slots)
     fasttps_config cfg;
     int n_sm;
     cudaDeviceProp prop;
@@ -318,7 +317,6 @@ struct StepArgs {
     uint32_t *status;
     unsigned long long *trace;       // [2][trace_len] global-timer stamps of the first and last CTA, or null
     int trace_len;
-    int max_inflight;                // ring pieces whose copies may be in flight at a time (0 = as many as slots)
 };
 
 int launch_linear(Ctx *c, const LinearArgs &a, cudaStream_t st);

@@ -208,13 +208,10 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
         if (w > nw || lane != 0) return;
         const uint32_t wp = (uint32_t)lay.wpiece;
         int piece = 0;
-        // Copies in flight are limited separately from pieces buffered: every other memory access of the SM
-        // (the barrier, the activations of a prologue) queues behind the bulk copies already issued.
-        const int inflight = (a.max_inflight > 0 && a.max_inflight < lay.nslot) ? a.max_inflight : 0;   // 0: no separate limit
         auto weights = [&](const void *base, size_t first_byte, int npieces) -> bool {
             const unsigned char *p = static_cast<const unsigned char *>(base) + first_byte;
             for (int i = 0; i < npieces; ++i, ++piece)
-                if ((inflight && !ring.landed(piece - inflight)) || !ring.put(piece, p + (size_t)i * wp, wp)) return false;
+                if (!ring.put(piece, p + (size_t)i * wp, wp)) return false;
             return true;
         };
         for (int step = 0; step < a.n_steps; ++step) {
@@ -236,7 +233,6 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                 const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
                 const bool kv_ok = attn_for_each_tile<DH>(aa, ListSource(&s_segs),
                                                           [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
-                    if (inflight && !ring.landed(piece - inflight)) return false;
                     return ring.put2(piece++, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
                 });
                 if (!kv_ok) return;
