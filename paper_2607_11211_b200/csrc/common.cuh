@@ -313,7 +313,7 @@ struct StepArgs {
     float *amax_val;
     int *amax_idx;
     int32_t *tok;                    // [B] current tokens
-    unsigned *bar;                   // grid barrier: [0] arrivals, [32] abort flag, [64] generation
+    unsigned *bar;                   // grid barrier: [0] arrivals since the launch (zeroed by the host)
     uint32_t *status;
     unsigned long long *trace;       // [2][trace_len] global-timer stamps of the first and last CTA, or null
     int trace_len;

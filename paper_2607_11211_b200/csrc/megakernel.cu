@@ -35,35 +35,38 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
     return v;
 }
 
+// A CTA that gives up (a bounded wait ran out) adds this instead of 1: the count is then beyond every target, so
+// all waiters are released at once and see from the count itself that the launch is being abandoned.
+constexpr unsigned kBarAbort = 0x40000000u;
+
 struct GridBarrier {
     unsigned *count;  // arrivals since the launch (zeroed by the host before every launch)
-    int *abort;
-    unsigned target;  // arrivals that complete the barrier this CTA waits at next
+    uint32_t *status; // device status word
+    unsigned target;  // arrivals that complete the barrier this CTA waits at next (always < kBarAbort)
     int ncta;
     int *s_go;        // shared-memory word
 };
 
 // All consumer threads of every CTA.  `ok` = this thread saw no failed wait.  Returns the same verdict in
 // every thread of the grid that gets past it: false means "leave now".  One atomic per CTA and barrier;
-// the waiters poll the arrival counter itself.
+// the waiters poll the arrival counter itself, and nothing else is read on the way out.
 __device__ __forceinline__ bool grid_sync(GridBarrier &gb, int nct, bool ok)
 {
     const bool all_ok = named_bar_and(1, nct, ok);       // CTA verdict; all global writes of the phase are issued
     if (threadIdx.x == 0) {
-        int go = 1;
-        if (!all_ok) { atomicExch(gb.abort, 1); go = 0; }
         __threadfence();
-        atomicAdd(gb.count, 1u);
+        atomicAdd(gb.count, all_ok ? 1u : kBarAbort);
+        unsigned v;
         unsigned long long t0 = 0;
-        for (unsigned it = 1; ld_acquire_u32(gb.count) < gb.target; ++it) {
-            if ((it & 63u) == 0) {                       // now and then: has anybody given up? have we waited too long?
-                if (ld_cg_s32(gb.abort)) { go = 0; break; }
+        for (unsigned it = 1; (v = ld_acquire_u32(gb.count)) < gb.target; ++it) {
+            if ((it & 63u) == 0) {                       // now and then: have we waited too long?
                 const unsigned long long now = global_ns();
                 if (t0 == 0) t0 = now;
-                else if (now - t0 > kGridWaitNanos) { atomicExch(gb.abort, 1); go = 0; break; }
+                else if (now - t0 > kGridWaitNanos) { atomicAdd(gb.count, kBarAbort); v = kBarAbort; break; }
             }
         }
-        if (!all_ok || ld_cg_s32(gb.abort)) go = 0;
+        const int go = all_ok && v < kBarAbort;
+        if (!go) atomicOr(gb.status, FASTTPS_DEV_WAIT_TIMEOUT);
         *gb.s_go = go;
     }
     named_bar_sync(1, nct);
@@ -247,8 +250,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
 
     // =========================================================================== consumer warps
     GridBarrier gb;
-    // arrivals and abort flag in two different 128-byte lines
-    gb.count = a.bar; gb.abort = reinterpret_cast<int *>(a.bar + 32);
+    gb.count = a.bar; gb.status = a.status;
     gb.ncta = ncta; gb.s_go = &s_go;
     gb.target = (unsigned)ncta;
     if (cta == 0 && t == 0) {
@@ -328,6 +330,12 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
             const float *y_prev = lprev >= 0 ? a.acc + (size_t)(lprev & 1) * B * D : nullptr;
             const __nv_bfloat16 *x_base = lprev >= 0 ? a.h : a.x0;                      // x = bf16(x_base + y_prev)
 
+            // The gains of the norm two phases ahead are asked from L2 now (they come from HBM once per step):
+            // one CTA, one thread per 128-byte line.
+            if (cta == ncta - 1 && (kind == kAttn || kind == kMlp) && t * 64 < D) {
+                const __nv_bfloat16 *gnext = kind == kAttn ? lp.g_mlp : (l + 1 < L ? s_layers[l + 1].g_attn : a.g_final);
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(gnext + t * 64));
+            }
             if (kind == kAttn) {
                 // ---- attention (Algorithm 3) ----
                 const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
@@ -500,7 +508,9 @@ static int launch_step_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
         if (per_sm < 1) return FASTTPS_INVALID_ARG;
         configured[c->cfg.device & 15] = true;
     }
-    // barrier counter and abort flag start from zero every launch (the generation may be anything)
+    if ((unsigned long long)(4 * a.n_layers + 3) * (unsigned long long)a.n_steps * (unsigned long long)c->n_sm >= kBarAbort)
+        return FASTTPS_INVALID_ARG;                      // the arrival counter must stay below the abort mark
+    // the barrier counter starts from zero every launch
     FT_CUDA(cudaMemsetAsync(c->grid_bar, 0, 64 * sizeof(unsigned), st));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c->n_sm); cfg.blockDim = dim3((lay.nw + 1) * 32); cfg.dynamicSmemBytes = lay.total; cfg.stream = st;
