@@ -111,10 +111,17 @@ __device__ __forceinline__ void load_b_frags(uint32_t (&bf)[IPW][4], const __nv_
         }
     ss += __shfl_xor_sync(kFull, ss, 1);
     ss += __shfl_xor_sync(kFull, ss, 2);
-    if (t4 == 0) smem_red[w * 8 + g] = ss;
+    if (t4 == 0) smem_red[g * nw + w] = ss;             // [row][warp]: a row's partial sums are contiguous
     named_bar_sync(1, nw * 32);
     float tot = 0.f;
-    for (int w2 = 0; w2 < nw; ++w2) tot += smem_red[w2 * 8 + g];
+    if ((nw & 3) == 0) {
+        for (int w4 = 0; w4 < nw; w4 += 4) {
+            const float4 p = *reinterpret_cast<const float4 *>(smem_red + g * nw + w4);
+            tot += (p.x + p.y) + (p.z + p.w);
+        }
+    } else {
+        for (int w2 = 0; w2 < nw; ++w2) tot += smem_red[g * nw + w2];
+    }
     const float r = rsqrtf(tot / (float)n_in + eps);
 #pragma unroll
     for (int i = 0; i < IPW; ++i) {
