@@ -430,7 +430,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                             for (int e = 0; e < 4; ++e) acc[i][m][e] = 0.f;
                     mlp_down_phase<IPW>(ring, piece, mn, nw, s_hi, s_lo, acc, ok);
                     piece += mn * PPO;
-                    mlp_scatter_add<IPW>(acc, smem_part, a.acc + (size_t)(l & 1) * B * D, B, D, nw);
+                    mlp_scatter_add<IPW, !DEFER>(acc, smem_part, a.acc + (size_t)(l & 1) * B * D, B, D, nw);
                 } else if (kind == kHead) {
                     named_bar_sync(1, nct);
                     if (t < 8 && t < B) {

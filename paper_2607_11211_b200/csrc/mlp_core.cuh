@@ -84,7 +84,7 @@ static __device__ __noinline__ void mlp_scatter_drain(const float *stage, float 
 // 8 * 32 * nw floats that are idle (the partial-tile scratch of the gate_up phase).  Consumer threads
 // only (named barrier 1).
 template <int IPW>
-__device__ __forceinline__ void mlp_scatter_add(const float (&acc)[IPW][2][4], float *stage, float *acc_g, int batch,
+__device__ __forceinline__ void mlp_scatter_add_block(const float (&acc)[IPW][2][4], float *stage, float *acc_g, int batch,
                                                 int D, int nw)
 {
     const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3, nct = nw * 32;
@@ -105,6 +105,57 @@ __device__ __forceinline__ void mlp_scatter_add(const float (&acc)[IPW][2][4], f
         }
         if (ir == R - 1 || i == IPW - 1) mlp_scatter_drain(stage, acc_g, i - ir, ir + 1, batch, D, cw, nct);
     }
+}
+
+
+// The same scatter for larger batches, where the block-wide version would need two block-wide barriers per
+// value of i.  For a given i a
+// warp owns 32 contiguous output columns, 32 (nw i + w) .. + 32, so the transposition from fragment order to
+// rows of 4 consecutive columns is private to the warp: it goes through the warp's own 1 KB of `stage`
+// (8 * 32 * nw floats that are idle: the partial-tile scratch of the gate_up phase) with no block-wide barrier.
+// The region holds R = 8 / batch' values of i at a time as rows [chunk][batch row][32 columns]; the eight
+// 4-column groups of a row are XOR-swizzled with the row index, which makes both the fragment-order writes and
+// the 16-byte row reads free of bank conflicts.
+template <int IPW>
+__device__ __forceinline__ void mlp_scatter_add_warp(const float (&acc)[IPW][2][4], float *stage, float *acc_g, int batch,
+                                                int D, int nw)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, g = lane >> 2, t4 = lane & 3;
+    const int R = batch <= 1 ? 8 : (batch <= 2 ? 4 : (batch <= 4 ? 2 : 1));
+    float *st = stage + w * 256;
+#pragma unroll
+    for (int i = 0; i < IPW; ++i) {
+        const int ir = i % R;                                // slot of chunk i inside the round
+        if (ir == 0 && i > 0) __syncwarp();                  // the previous round has been read
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int b = 2 * t4 + (e & 1), n = 16 * m + g + 8 * (e >> 1);
+                const int row = ir * batch + b;
+                if (b < batch) st[row * 32 + ((((n >> 2) ^ row) & 7) << 2) + (n & 3)] = acc[i][m][e];
+            }
+        }
+        if (ir == R - 1 || i == IPW - 1) {
+            __syncwarp();
+            const int i0 = i - ir, nrow = (ir + 1) * batch;
+            for (int idx = lane; idx < nrow * 8; idx += 32) {
+                const int row = idx >> 3, j = idx & 7;
+                const int ch = row / batch, b = row - ch * batch;
+                const float4 v = *reinterpret_cast<const float4 *>(st + row * 32 + (((j ^ row) & 7) << 2));
+                red_add_v4(acc_g + (size_t)b * D + 32 * (nw * (i0 + ch) + w) + 4 * j, v.x, v.y, v.z, v.w);
+            }
+        }
+    }
+}
+
+// WARP_PRIVATE: which of the two a caller wants (small batches: block-wide, one barrier in all; larger: per warp).
+template <int IPW, bool WARP_PRIVATE>
+__device__ __forceinline__ void mlp_scatter_add(const float (&acc)[IPW][2][4], float *stage, float *acc_g, int batch,
+                                                int D, int nw)
+{
+    if (WARP_PRIVATE) mlp_scatter_add_warp<IPW>(acc, stage, acc_g, batch, D, nw);
+    else mlp_scatter_add_block<IPW>(acc, stage, acc_g, batch, D, nw);
 }
 
 }  // namespace fasttps
