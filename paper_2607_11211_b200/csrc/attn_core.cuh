@@ -135,8 +135,6 @@ template <int DH> struct AttnTile {
     static constexpr int kPieceBytes = 2 * kAttnTileRows * kRowBytes;     // K tile then V tile
 };
 
-// Calls f(k_tile, v_tile, bytes_each) for every K/V tile of this CTA's share, in walk order; stops and
-// returns false as soon as f does.
 // A share as a list of segments kept in shared memory (the persistent kernel computes it once per step and
 // uses it for every layer).  12 bytes per segment; lengths and positions of the step sit beside the list.
 constexpr int kMaxSegments = 257;            // a share touches at most batch * n_q_heads heads (<= 256 here)
@@ -175,6 +173,8 @@ struct ListSource {
     }
 };
 
+// Calls f(k_tile, v_tile, bytes_each) for every K/V tile of this CTA's share, in walk order; stops and
+// returns false as soon as f does.
 template <int DH, class Src, class F>
 __device__ __forceinline__ bool attn_for_each_tile(const AttnArgs &a, Src src, F f)
 {

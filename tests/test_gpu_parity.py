@@ -471,3 +471,49 @@ def test_model_generate_multi_step_greedy(fb, dims, lens, step_kernel):
             assert_close_bits(wl.bits(kcs[l])[b, :, r], ok[l][b, :, r], what="k rows")
             assert_close_bits(wl.bits(vcs[l])[b, :, r], ov[l][b, :, r], what="v rows")
     ctx.close()
+
+
+@pytest.mark.parametrize("step_kernel", [0, 1])
+def test_model_decode_reports_a_full_cache_and_serves_the_other_sequences(fb, step_kernel):
+    """One sequence of the batch has no free row: the status word says so, its caches are left alone, and the
+    other sequences get the same logits as the oracle computes for them alone."""
+    dims, max_seq = wl.SMALL, 48
+    lens = np.array([20, max_seq, 7], np.int32)          # sequence 1 is full
+    batch = len(lens)
+    ctx = make_ctx(fb, dims, batch, max_seq)
+    ctx.set_option("step_kernel", step_kernel)
+    mw, model, kcs, vcs = build_model(fb, ctx, dims, batch, max_seq)
+    k0 = [t.clone() for t in kcs]
+    v0 = [t.clone() for t in vcs]
+    ids = wl.token_ids(batch, dims.vocab)
+    logits = torch.zeros(batch, dims.vocab, dtype=torch.float32, device="cuda")
+    nxt = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    ctx.model_decode(model, i32(ids), i32(lens), i32(lens), logits, nxt, advance=False)
+    assert ctx.get_status() & fb.DEV_CACHE_FULL
+    for l in range(dims.n_layers):
+        assert torch.equal(kcs[l][1].view(torch.int16), k0[l][1].view(torch.int16))
+        assert torch.equal(vcs[l][1].view(torch.int16), v0[l][1].view(torch.int16))
+    good = [0, 2]
+    ok = [wl.bits(t[good]) for t in k0]
+    ov = [wl.bits(t[good]) for t in v0]
+    ow = [{k: wl.bits(v) for k, v in L.items()} for L in mw["layers"]]
+    wlog, _ = orc.model_decode(wl.bits(mw["embed"]), ow, wl.bits(mw["g_final"]), wl.bits(mw["w_lm"]), ok, ov,
+                               ids[good], lens[good].copy(), lens[good].copy(), dims.rms_eps, dims.rope_theta)
+    got = logits.cpu().numpy().astype(np.float64)[good]
+    assert (np.abs(got - wlog) <= 2e-2 + 2e-2 * np.abs(wlog)).all()
+    ctx.close()
+
+
+def test_model_generate_stops_at_the_end_of_the_cache(fb):
+    """A multi-token launch that would outgrow the cache is reported before anything is written beyond it."""
+    dims, max_seq = wl.TINY, 16
+    ctx = make_ctx(fb, dims, 1, max_seq)
+    mw, model, kcs, vcs = build_model(fb, ctx, dims, 1, max_seq)
+    k0 = [t.clone() for t in kcs]
+    out = torch.zeros(6, 1, dtype=torch.int32, device="cuda")
+    pos, sl = i32([12]), i32([12])
+    ctx.model_generate(model, i32([3]), pos, sl, out)   # rows 12..17 would be needed, 16 exist
+    assert ctx.get_status() & fb.DEV_CACHE_FULL
+    for l in range(dims.n_layers):                       # nothing outside the rows this launch may touch has changed
+        assert torch.equal(kcs[l][:, :, :12].view(torch.int16), k0[l][:, :, :12].view(torch.int16))
+    ctx.close()
