@@ -11,8 +11,13 @@
 // a grid-wide barrier after each product.  While they wait there, or run the latency-bound parts of
 // attention, the bytes of the next product keep arriving, so HBM stays busy across all boundaries.
 //
-// Grid barrier: sense-reversing counter in global memory, bounded wait, abort flag (no CTA ever
-// spins forever; the launch is cooperative, so all CTAs are resident).
+// Grid barrier: one arrival counter in global memory that only grows during a launch (the host zeroes it
+// before the launch); every wait is bounded, and a CTA that gives up pushes the counter beyond every target so
+// that nobody spins forever (the launch is cooperative, so all CTAs are resident).
+//
+// Two variants are compiled (template parameter DEFER, chosen by batch size at launch): where the softmax
+// merge of a head shared by several CTAs happens, and how the MLP partial sums are staged.  Code that does not
+// run is kept out of each variant: the kernel is sensitive to its instruction footprint and register pressure.
 #include "attn_core.cuh"
 #include "mlp_core.cuh"
 #include "stream_launch.cuh"
