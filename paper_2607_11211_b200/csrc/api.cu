@@ -57,7 +57,7 @@ static void free_all(Ctx *c)
     cudaFree(c->amax_ticket); cudaFree(c->status); cudaFree(c->qkv); cudaFree(c->attn_out);
     cudaFree(c->h); cudaFree(c->xa); cudaFree(c->xb); cudaFree(c->logits); cudaFree(c->tok); cudaFree(c->tok2);
     if (c->pinned_tok) cudaFreeHost(c->pinned_tok);
-    cudaFree(c->grid_bar); cudaFree(c->d_layers); cudaFree(c->trace);
+    cudaFree(c->grid_bar); cudaFree(c->hacc); cudaFree(c->d_layers); cudaFree(c->trace);
     if (c->pin_layers) cudaFreeHost(c->pin_layers);
     if (c->prof_ev) {
         for (int i = 0; i < 2 * kProfMax; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
@@ -107,7 +107,8 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     A(dev_alloc(&c->attn_part, B * f.n_q_heads * kMaxSplits * (f.head_dim + 4), true));
     A(dev_alloc(&c->attn_ticket, B * f.n_q_heads, true));
     A(dev_alloc(&c->mlp_acc, 2 * B * D, true));
-    A(dev_alloc(&c->grid_bar, 128, true));
+    A(dev_alloc(&c->grid_bar, kGridBarWords, true));
+    A(dev_alloc(&c->hacc, 2 * D, true));
     A(dev_alloc(&c->trace, 2 * (size_t)kTraceLen, true));
     A(dev_alloc(&c->d_layers, (size_t)(f.n_layers > 0 ? f.n_layers : 1), true));
     if (e == cudaSuccess)
@@ -346,7 +347,7 @@ int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value)
 {
     if (!ctx || !name) return FASTTPS_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);
-    if (strcmp(name, "step_kernel") == 0) c->opt_step_kernel = value != 0;
+    if (strcmp(name, "step_kernel") == 0) c->opt_step_kernel = value < 0 ? 0 : (value > 2 ? 2 : value);
     else return FASTTPS_INVALID_ARG;
     return FASTTPS_OK;
 }
@@ -405,10 +406,11 @@ static int step_impl(Ctx *c, const void *embed, const fasttps_layer_weights *lay
     a.K = f.inter; a.V = f.vocab; a.max_seq = f.max_seq; a.eps = f.rms_eps;
     a.cos_tab = c->cos_tab; a.sin_tab = c->sin_tab;
     a.x0 = c->xa; a.qkv = c->qkv; a.attn_out = c->attn_out; a.h = c->h;
-    a.acc = c->mlp_acc; a.attn_part = c->attn_part; a.attn_ticket = c->attn_ticket;
+    a.acc = c->mlp_acc; a.hacc = c->hacc; a.attn_part = c->attn_part; a.attn_ticket = c->attn_ticket;
     a.amax_val = c->amax_val; a.amax_idx = c->amax_idx; a.tok = c->tok2;
     a.bar = c->grid_bar; a.status = c->status;
     a.trace = c->trace; a.trace_len = kTraceLen;
+    if (c->opt_step_kernel == 1 && step_b1_supported(c, batch)) return launch_step_b1(c, a, st);
     return launch_step(c, a, st);
 }
 

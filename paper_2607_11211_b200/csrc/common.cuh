@@ -20,10 +20,11 @@ struct LayerPtrs;
 struct Ctx {
     // persistent step kernel: grid barrier words, device table of layer pointers and its pinned shadow
     unsigned *grid_bar;
+    float *hacc;
     unsigned long long *trace;       // [2][kTraceLen] phase timeline of the last step-kernel launch
     LayerPtrs *d_layers, *pin_layers;
     int layers_uploaded;             // number of valid entries in pin_layers / d_layers
-    int opt_step_kernel;             // 1: model calls with batch <= 8 use the persistent step kernel
+    int opt_step_kernel;             // 0: one kernel per product; 1: persistent step kernels (batch <= 8); 2: the general one also at batch 1
     fasttps_config cfg;
     int n_sm;
     cudaDeviceProp prop;
@@ -55,7 +56,8 @@ struct Ctx {
 };
 
 constexpr int kProfMax = 8192;
-constexpr int kTraceLen = 4096;      // global-timer stamps kept per traced CTA of the step kernel
+constexpr int kTraceLen = 4096;             // global-timer stamps kept per traced CTA of the step kernel
+constexpr int kGridBarWords = 256;          // barrier counter + one group counter per query head (<= 128)
 enum ProfClass { kProfQkv = 0, kProfAttn, kProfOproj, kProfMlp, kProfLmHead, kProfEmbed, kProfStep, kProfClasses };
 
 // Brackets one kernel launch with events when profiling is on.
@@ -308,12 +310,13 @@ struct StepArgs {
     // workspace
     __nv_bfloat16 *x0, *qkv, *attn_out, *h;
     float *acc;                      // [2][B][D] FP32, zero on entry and on exit
+    float *hacc;                     // [2][D] FP32 sums of the output projection (batch-1 kernel), zero on entry and exit
     float *attn_part;
     int *attn_ticket;
     float *amax_val;
     int *amax_idx;
     int32_t *tok;                    // [B] current tokens
-    unsigned *bar;                   // grid barrier: [0] arrivals since the launch (zeroed by the host)
+    unsigned *bar;                   // [kGridBarWords], zeroed by the host per launch: [0] grid barrier arrivals, [64 + h] group arrivals of head h
     uint32_t *status;
     unsigned long long *trace;       // [2][trace_len] global-timer stamps of the first and last CTA, or null
     int trace_len;
@@ -322,6 +325,8 @@ struct StepArgs {
 int launch_linear(Ctx *c, const LinearArgs &a, cudaStream_t st);
 bool step_kernel_supported(const Ctx *c, int batch);
 int launch_step(Ctx *c, const StepArgs &a, cudaStream_t st);
+bool step_b1_supported(const Ctx *c, int batch);
+int launch_step_b1(Ctx *c, const StepArgs &a, cudaStream_t st);
 int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st);
 int launch_mlp(Ctx *c, const MlpArgs &a, cudaStream_t st);
 int launch_embed(Ctx *c, const __nv_bfloat16 *embed, const int32_t *ids, __nv_bfloat16 *x, int batch, cudaStream_t st);

@@ -55,12 +55,14 @@ __host__ __device__ inline WarpSplit warp_split(int n_in)
 // IPW k blocks, batch row g = lane / 4 (zero for g >= batch), optionally RMS-normalised (gain gn, eps)
 // with the result rounded to bf16 like a stored tensor.  Consumer threads only (named barrier 1).
 // smem_red: nw * 8 floats.  If `add` is given (FP32 [batch][n_in], e.g. the MLP partial sums of the
-// previous layer), the activation is bf16(x + add).  All loads bypass L1: inside a persistent kernel the
-// activations were written by other SMs.
+// previous layer), the activation is bf16(x + add); if `store` is given, that activation (before the norm) is
+// also written out, one share of its 16-byte chunks per CTA.  All loads bypass L1: inside a persistent kernel
+// the activations were written by other SMs.
 template <int IPW>
 __device__ __forceinline__ void load_b_frags(uint32_t (&bf)[IPW][4], const __nv_bfloat16 *x, int x_stride, int batch,
                                              int n_in, int nw, const __nv_bfloat16 *gn, float eps, float *smem_red,
-                                             const float *add = nullptr)
+                                             const float *add = nullptr, __nv_bfloat16 *store = nullptr,
+                                             int store_rem = 0, int store_mod = 1)
 {
     const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3;
     const bool live = g < batch;
@@ -95,6 +97,16 @@ __device__ __forceinline__ void load_b_frags(uint32_t (&bf)[IPW][4], const __nv_
     if (!live) {
 #pragma unroll
         for (int i = 0; i < IPW; ++i) bf[i][0] = bf[i][1] = bf[i][2] = bf[i][3] = 0u;
+    }
+    if (store != nullptr && live) {
+        // the activation before normalisation is kept as a tensor: of the grid's CTAs, which all hold it, the one
+        // with number store_rem (of store_mod) writes every store_mod-th 16-byte chunk
+#pragma unroll
+        for (int i = 0; i < IPW; ++i) {
+            const int k = 32 * (w + nw * i) + 8 * t4;
+            if ((k >> 3) % store_mod == store_rem)
+                *reinterpret_cast<uint4 *>(store + (size_t)g * x_stride + k) = make_uint4(bf[i][0], bf[i][1], bf[i][2], bf[i][3]);
+        }
     }
     if (gn == nullptr) return;
     uint4 gv[IPW];                      // the gains are fetched before the reduction, not after its barrier

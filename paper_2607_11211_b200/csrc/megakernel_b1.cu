@@ -1,0 +1,493 @@
+// Persistent decode-step kernel for ONE sequence (batch 1): the same token phase as megakernel.cu --
+// embedding, per layer RMSNorm -> QKV -> attention (Algorithm 3) -> output projection -> RMSNorm -> fused MLP
+// (Algorithm 4), final norm, logits, greedy argmax -- with THREE grid-wide phase boundaries per layer
+// instead of four.
+//
+// At batch 1 a layer is ~37 us of streaming and every grid-wide boundary costs 4-5 us of dependent latency
+// (barrier, activation loads, norm).  Here the attention and the output projection are one phase: every query
+// head belongs to a fixed group of m0 = n_sm / H_q CTAs.  The group's CTAs split the rows of the head's cache
+// (Algorithm 3 on each share, partial (max, sum, output) published), meet at a counter of their own -- a wait
+// for at most m0 - 1 neighbours instead of the whole grid --, each merges the head's partials, and each then
+// multiplies the merged head output with ITS slice of the output-projection rows: for row tile r the d / 32
+// k blocks of the head are d KB contiguous in the packed W_o, so a ring piece is a handful of such runs.  The
+// products of the 32 heads meet in an FP32 accumulator (red.add); the residual add h = x + attn W_o moves into
+// the prologue of the MLP phase, which also writes h out (one share of its chunks per CTA), as the QKV
+// prologue does for x = h + y of the layer before.
+#include "step_core.cuh"
+
+namespace fasttps {
+
+namespace {
+
+struct OneSegment {
+    Segment sg;
+    int n;                       // 0 or 1
+};
+struct OneSource {
+    const OneSegment *p;
+    int i;
+    __device__ __forceinline__ explicit OneSource(const OneSegment *p_) : p(p_), i(0) {}
+    __device__ __forceinline__ bool next(Segment &s)
+    {
+        if (i >= p->n) return false;
+        s = p->sg;
+        ++i;
+        return true;
+    }
+};
+
+template <int IPW, int DH>
+__global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(StepArgs a)
+{
+    extern __shared__ __align__(128) unsigned char dsm[];
+    __shared__ __align__(16) ActTile s_hi[kMaxOctetsPerCta];
+    __shared__ __align__(16) ActTile s_lo[kMaxOctetsPerCta];
+    __shared__ float s_best_val[64];
+    __shared__ int s_best_idx[64];
+    __shared__ int s_go;
+    __shared__ int s_tables_ready;                               // steps whose attention share is known
+    __shared__ LayerPtrs s_layers[kMaxStepLayers];               // the layer table: no global round trip per phase
+    __shared__ OneSegment s_one;                                 // this CTA's attention share for the current step
+    __shared__ int s_mprime;                                     // CTAs of a group that hold rows in the current step
+    __shared__ __align__(16) __nv_bfloat16 s_outh[DH];           // the merged output of this CTA's head
+
+    constexpr int KB = DH / 32;                                  // k blocks of a head in the output projection
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3;
+    const int cta = blockIdx.x, ncta = gridDim.x;
+    if (t == 0) s_tables_ready = 0;
+    const MegaLayout lay = mega_layout<DH>(a.D);
+    const int nw = lay.nw, nct = nw * 32;
+    float *smem_part = reinterpret_cast<float *>(dsm + lay.part_off);
+    float *smem_red = reinterpret_cast<float *>(dsm + lay.red_off);
+    AttnScratch<DH> &scratch = *reinterpret_cast<AttnScratch<DH> *>(dsm + lay.scratch_off);
+
+    const int D = a.D;
+    const int nq = a.n_q_heads * a.head_dim, nkv = a.n_kv_heads * a.head_dim, nqkv = nq + 2 * nkv;
+    constexpr int SPT = IPW / kBlocksPerWarpPerSlot;      // ring pieces per 16-row tile
+    constexpr int PPO = IPW / 4;                          // ring pieces per W_down octet
+    const size_t tile_bytes = (size_t)D * 32;             // 16 rows x D (every reduction length here is D)
+    const size_t oct_bytes = (size_t)D * 16;
+
+    // this CTA's share of every grid-wide product (the same for every layer)
+    int q0, qn, m0, mn, l0, ln;
+    cta_range((nqkv + 15) >> 4, cta, ncta, q0, qn);
+    cta_range(a.K >> 3, cta, ncta, m0, mn);
+    cta_range((a.V + 15) >> 4, cta, ncta, l0, ln);
+    // head groups: CTA (head, gs) of gm CTAs per head; the CTAs beyond n_q_heads * gm sit the fused phase out
+    int gm = ncta / a.n_q_heads;
+    if (gm > kMaxSplits) gm = kMaxSplits;
+    const int head = cta / gm, gs = cta - head * gm;
+    const bool in_group = head < a.n_q_heads;
+    int ot0 = 0, ont = 0;                                  // this CTA's row tiles of the output projection
+    if (in_group) cta_range((D + 15) >> 4, gs, gm, ot0, ont);
+    int TP = lay.slot_stride / (KB * kTileBytes);          // row tiles of the output projection per ring piece
+    if (TP > nw) TP = nw;
+    unsigned *grp = a.bar + 64 + (in_group ? head : 0);    // arrivals of this group's partials since the launch
+    float *hacc = a.hacc;                                  // [2][D] FP32 sums of the output projection
+    __nv_bfloat16 *xbuf = a.attn_out;                      // x of the current layer (the attention output tensor is not needed here)
+
+    WeightRing ring;
+    ring.init(dsm + lay.ring_off, reinterpret_cast<uint64_t *>(dsm + lay.bar_off),
+              reinterpret_cast<int *>(dsm + lay.abort_off), lay.nslot, lay.slot_stride, nw, nullptr, 0, nullptr, 0);
+    if (t < 64) { s_best_val[t] = -INFINITY; s_best_idx[t] = 0x7fffffff; }
+    for (int i = t; i < a.n_layers * (int)(sizeof(LayerPtrs) / 8); i += blockDim.x)
+        reinterpret_cast<unsigned long long *>(s_layers)[i] = reinterpret_cast<const unsigned long long *>(a.layers)[i];
+    __syncthreads();
+
+    // =========================================================================== producer warp
+    if (w >= nw) {
+        if (w > nw || lane != 0) return;
+        const uint32_t wp = (uint32_t)lay.wpiece;
+        int piece = 0;
+        auto weights = [&](const void *base, size_t first_byte, int npieces) -> bool {
+            const unsigned char *p = static_cast<const unsigned char *>(base) + first_byte;
+            for (int i = 0; i < npieces; ++i, ++piece)
+                if (!ring.put(piece, p + (size_t)i * wp, wp)) return false;
+            return true;
+        };
+        for (int step = 0; step < a.n_steps; ++step) {
+            for (int l = 0; l < a.n_layers; ++l) {
+                const LayerPtrs &lp = s_layers[l];
+                if (!weights(lp.w_qkv, (size_t)q0 * tile_bytes, qn * SPT)) return;
+                if (l == 0) {
+                    // K/V tiles of this step include the row appended by the step before it, and the share is
+                    // recomputed per step: both are ready once the consumers have passed the barrier that ends
+                    // that step (weights are never held back)
+                    const unsigned long long t0 = global_ns();
+                    while (*reinterpret_cast<volatile int *>(&s_tables_ready) <= step) {
+                        if (*ring.abort_flag || global_ns() - t0 > kGridWaitNanos) { *ring.abort_flag = 1; return; }
+                        __nanosleep(64);
+                    }
+                    __threadfence_block();
+                }
+                const AttnArgs aa = attn_args_of(a, lp, step, gm * a.n_q_heads);
+                const bool kv_ok = attn_for_each_tile<DH>(aa, OneSource(&s_one),
+                                                          [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
+                    return ring.put2(piece++, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
+                });
+                if (!kv_ok) return;
+                // this CTA's rows of the output projection, the head's k blocks only: KB KB per row tile
+                const unsigned char *wo = reinterpret_cast<const unsigned char *>(lp.w_o);
+                for (int p0 = 0; p0 < ont; p0 += TP, ++piece) {
+                    const int nt = ont - p0 < TP ? ont - p0 : TP;
+                    if (!ring.acquire(piece)) return;
+                    const int sl = piece % ring.nslot;
+                    mbar_expect_tx(&ring.full[sl], (uint32_t)(nt * KB * kTileBytes));
+                    for (int j = 0; j < nt; ++j)
+                        bulk_g2s(ring.slots + (size_t)sl * ring.slot_bytes + (size_t)j * KB * kTileBytes,
+                                 wo + ((size_t)(ot0 + p0 + j) * (nq / 32) + (size_t)head * KB) * kTileBytes,
+                                 (uint32_t)(KB * kTileBytes), &ring.full[sl]);
+                }
+                if (!weights(lp.w_gu, (size_t)m0 * tile_bytes, mn * SPT)) return;
+                if (!weights(lp.w_down, (size_t)m0 * oct_bytes, mn * PPO)) return;
+            }
+            if (!weights(a.w_lm, (size_t)l0 * tile_bytes, ln * SPT)) return;
+        }
+        return;
+    }
+
+    // =========================================================================== consumer warps
+    GridBarrier gb;
+    gb.count = a.bar; gb.status = a.status;
+    gb.ncta = ncta; gb.s_go = &s_go;
+    gb.target = (unsigned)ncta;
+    unsigned grp_target = 0;
+    if (cta == 0 && t == 0) {
+        const int L = a.seq_lens[0], p = a.pos[0];
+        if (L < 0 || L + a.n_steps > a.max_seq) atomicOr(a.status, FASTTPS_DEV_CACHE_FULL);
+        else if (p < 0 || p + a.n_steps > a.max_seq) atomicOr(a.status, FASTTPS_DEV_BAD_POSITION);
+    }
+
+    // gathers the embedding row of the current token into x0 (CTA 0 only)
+    auto embed_row = [&](const int32_t *ids) {
+        for (int j = t; j < (D >> 3); j += nct) {
+            int id = ld_cg_s32(ids);
+            if (id < 0 || id >= a.V) { if (j == 0) atomicOr(a.status, FASTTPS_DEV_BAD_TOKEN); id = 0; }
+            reinterpret_cast<uint4 *>(a.x0)[j] = reinterpret_cast<const uint4 *>(a.embed + (size_t)id * D)[j];
+        }
+    };
+
+    uint32_t bf[IPW][4];
+    int piece = 0;
+    bool ok = true;
+
+    // optional timeline for profiling: the first and the last CTA stamp the global timer before and
+    // after every grid barrier
+    int n_stamp = 0;
+    auto stamp = [&]() {
+        if (a.trace && t == 0 && (cta == 0 || cta == ncta - 1) && n_stamp < a.trace_len)
+            a.trace[(size_t)(cta ? 1 : 0) * a.trace_len + n_stamp] = global_ns();
+        ++n_stamp;
+    };
+    auto sync_phase = [&]() -> bool {
+        stamp();
+        const bool go = grid_sync(gb, nct, /*ok=*/ok);
+        stamp();
+        return go;
+    };
+
+    if (cta == 0) embed_row(a.token_ids);
+    if (!sync_phase()) return;
+
+    enum { kQkv = 0, kAttn = 1, kMlp = 2, kHead = 3 };
+    const int L = a.n_layers;
+    for (int step = 0; step < a.n_steps; ++step) {
+        // ---- this step's attention share: rows [R gs / m', R (gs + 1) / m') of the head, m' CTAs of the group ----
+        if (t == 0) {
+            const int Ls = a.seq_lens[0] + step, ps = a.pos[0] + step;
+            const bool valid = !(Ls < step || Ls >= a.max_seq || ps < step || ps >= a.max_seq);
+            const int R = valid ? Ls + 1 : 0;
+            int mp = R / 16;                                   // at least 16 rows per CTA, at most the group
+            mp = R == 0 ? 0 : (mp < 1 ? 1 : (mp > gm ? gm : mp));
+            s_mprime = mp;
+            s_one.n = (in_group && gs < mp) ? 1 : 0;
+            Segment &sg = s_one.sg;
+            sg.b = 0; sg.h = in_group ? head : 0; sg.L = Ls; sg.pos = ps;
+            sg.r0 = mp ? (int)((long long)R * gs / mp) : 0;
+            sg.r1 = mp ? (int)((long long)R * (gs + 1) / mp) : 0;
+            sg.first_cta = head * gm; sg.n_cta = mp;
+        }
+        named_bar_sync(1, nct);
+        if (t == 0) {
+            __threadfence_block();
+            atomicExch(&s_tables_ready, step + 1);              // the producer may fetch this step's K/V rows now
+        }
+        const int mprime = s_mprime;
+
+        for (int ph = 0; ph <= 3 * L; ++ph) {
+            const int l = ph / 3;
+            const int kind = ph == 3 * L ? kHead : ph - 3 * l;
+            const LayerPtrs &lp = s_layers[l < L ? l : L - 1];
+
+            // The gains of the norm after next are asked from L2 now (they come from HBM once per step)
+            if (cta == ncta - 1 && (kind == kQkv || kind == kAttn) && t * 64 < D) {
+                const __nv_bfloat16 *gnext = kind == kQkv ? lp.g_mlp : (l + 1 < L ? s_layers[l + 1].g_attn : a.g_final);
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(gnext + t * 64));
+            }
+
+            if (kind == kAttn) {
+                // ---- attention (Algorithm 3) on this CTA's rows of its head; the partial is published ----
+                const AttnArgs aa = attn_args_of(a, lp, step, gm * a.n_q_heads);
+                ok = attn_consume<DH, true>(aa, ring, piece, cta, OneSource(&s_one), scratch, nw) && ok;
+                grp_target += (unsigned)mprime;
+                if (in_group) {
+                    // ---- the group meets: every CTA of it needs the merged output of the head ----
+                    __threadfence();
+                    named_bar_sync(1, nct);
+                    if (t == 0) {
+                        if (s_one.n && ok) atomicAdd(grp, 1u);
+                        int met = 1;
+                        unsigned long long t0 = 0;
+                        for (unsigned it = 1; ld_acquire_u32(grp) < grp_target; ++it) {
+                            if ((it & 63u) == 0) {
+                                const unsigned long long now = global_ns();
+                                if (t0 == 0) t0 = now;
+                                else if (now - t0 > kGridWaitNanos) { met = 0; break; }
+                            }
+                        }
+                        s_go = met;
+                    }
+                    named_bar_sync(1, nct);
+                    if (!s_go) ok = false;
+                    // ---- softmax merge of the head's partials: out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s ----
+                    constexpr int PS = DH + 4;
+                    const float *hp = a.attn_part + (size_t)head * kMaxSplits * PS;
+                    for (int i = t; i < DH; i += nct) {
+                        float M = -INFINITY, den = 0.f, o = 0.f;
+                        for (int s0 = 0; s0 < mprime; s0 += 4) {
+                            float ms[4], ls[4], os[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const bool have = s0 + u < mprime;
+                                const float *p = hp + (size_t)(have ? s0 + u : 0) * PS;
+                                ms[u] = ld_cg_f32(p + DH);
+                                ls[u] = ld_cg_f32(p + DH + 1);
+                                os[u] = ld_cg_f32(p + i);
+                                if (!have) ms[u] = -INFINITY;
+                            }
+                            float Mn = M;
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) Mn = fmaxf(Mn, ms[u]);
+                            const float corr = fast_exp2(M - Mn);        // 0 in the first round (M = -inf)
+                            den *= corr; o *= corr;
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const float f = ms[u] == -INFINITY ? 0.f : fast_exp2(ms[u] - Mn);
+                                den = fmaf(f, ls[u], den);
+                                o = fmaf(f, os[u], o);
+                            }
+                            M = Mn;
+                        }
+                        s_outh[i] = __float2bfloat16_rn(mprime > 0 && ok ? o / den : 0.f);
+                    }
+                    named_bar_sync(1, nct);
+                    // ---- this CTA's row tiles of the output projection, k = the head: sums go to hacc[l & 1] ----
+                    uint4 bh[KB];
+#pragma unroll
+                    for (int j = 0; j < KB; ++j)
+                        bh[j] = g == 0 ? *reinterpret_cast<const uint4 *>(s_outh + 32 * j + 8 * t4) : make_uint4(0u, 0u, 0u, 0u);
+                    float *hsum = hacc + (size_t)(l & 1) * D;
+                    for (int p0 = 0; p0 < ont; p0 += TP, ++piece) {
+                        const int nt = ont - p0 < TP ? ont - p0 : TP;
+                        const unsigned char *slot = ring.wait(piece, ok);
+                        if (w < nt) {
+                            float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                            for (int j = 0; j < KB; ++j) {
+                                const unsigned char *blk = slot + (size_t)(w * KB + j) * kTileBytes + lane * 16;
+                                const uint4 lo = *reinterpret_cast<const uint4 *>(blk);
+                                const uint4 hi = *reinterpret_cast<const uint4 *>(blk + 512);
+                                mma_bf16_k16(c, lo.x, hi.x, lo.y, hi.y, bh[j].x, bh[j].y);
+                                mma_bf16_k16(c, lo.z, hi.z, lo.w, hi.w, bh[j].z, bh[j].w);
+                            }
+                            const int row = (ot0 + p0 + w) * 16 + g;
+                            if (t4 == 0 && ok) {                 // accumulator column 0 = the one batch row
+                                if (row < D) atomicAdd(hsum + row, c[0]);
+                                if (row + 8 < D) atomicAdd(hsum + row + 8, c[2]);
+                            }
+                        }
+                        ring.release(piece);
+                    }
+                }
+            } else {
+                // ---- a grid-wide matrix product: B fragments, then this CTA's row tiles ----
+                const __nv_bfloat16 *src, *gain;
+                const float *add;
+                __nv_bfloat16 *store = nullptr;
+                int tile0, ntile;
+                if (kind == kQkv) {                          // x_l = h_{l-1} + y_{l-1} (layer 0: the embedding row)
+                    src = l == 0 ? a.x0 : a.h; add = l == 0 ? nullptr : a.acc + (size_t)((l - 1) & 1) * D;
+                    gain = lp.g_attn; store = l == 0 ? nullptr : xbuf; tile0 = q0; ntile = qn;
+                } else if (kind == kMlp) {                   // h_l = x_l + attn . W_o
+                    src = l == 0 ? a.x0 : xbuf; add = hacc + (size_t)(l & 1) * D;
+                    gain = lp.g_mlp; store = a.h; tile0 = m0; ntile = mn;
+                } else {                                     // x_L = h_{L-1} + y_{L-1}
+                    src = a.h; add = a.acc + (size_t)((L - 1) & 1) * D;
+                    gain = a.g_final; tile0 = l0; ntile = ln;
+                }
+                // the sums of the output projection of the layer before are consumed: back to zero
+                if (cta == ncta - 1 && ((kind == kQkv && l > 0) || kind == kHead)) {
+                    float *z = hacc + (size_t)((l - 1) & 1) * D;   // (head: l = L)
+                    for (int idx = t; idx < (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                load_b_frags<IPW>(bf, src, D, 1, D, nw, gain, a.eps, smem_red, add, store, cta, ncta);
+                if (kind == kHead) {
+                    for (int u = t; u < 64; u += nct) { s_best_val[u] = -INFINITY; s_best_idx[u] = 0x7fffffff; }
+                    named_bar_sync(1, nct);
+                }
+                ok = dot_tiles<IPW>(ring, piece, ntile, nw, bf, smem_part, [&](int tile, int cc, int b, float v0, float v1) {
+                    if (kind == kMlp) {                      // siLu_Mul: rows cc / cc + 8 are a gate value and its up value
+                        const float act = v0 / (1.f + __expf(-v0)) * v1;
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(act);
+                        s_hi[tile][b][cc] = hi;
+                        s_lo[tile][b][cc] = __float2bfloat16_rn(act - __bfloat162float(hi));
+                        return;
+                    }
+                    if (b >= 1) return;
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int row = (tile0 + tile) * 16 + cc + 8 * hh;
+                        const float v = hh ? v1 : v0;
+                        if (kind == kQkv) {
+                            if (row < nqkv) a.qkv[row] = __float2bfloat16_rn(v);
+                        } else if (row < a.V) {              // logits and the running argmax of this thread's rows
+                            const int u = cc * 8;
+                            if (a.logits) a.logits[row] = v;
+                            if (v > s_best_val[u]) { s_best_val[u] = v; s_best_idx[u] = row; }
+                        }
+                    }
+                }) && ok;
+                piece += ntile * SPT;
+
+                if (kind == kMlp) {
+                    // ---- down projection of this CTA's octets; the sums of all CTAs meet in acc[l & 1] ----
+                    if (cta == 0 && l > 0) {
+                        // layer l - 1's sums were consumed by the QKV prologue of this layer: zero them for layer l + 1
+                        float *z = a.acc + (size_t)((l - 1) & 1) * D;
+                        for (int idx = t; idx < (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    named_bar_sync(1, nct);
+                    float acc[IPW][2][4];
+#pragma unroll
+                    for (int i = 0; i < IPW; ++i)
+#pragma unroll
+                        for (int m = 0; m < 2; ++m)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) acc[i][m][e] = 0.f;
+                    mlp_down_phase<IPW>(ring, piece, mn, nw, s_hi, s_lo, acc, ok);
+                    piece += mn * PPO;
+                    mlp_scatter_add<IPW, false>(acc, smem_part, a.acc + (size_t)(l & 1) * D, 1, D, nw);
+                } else if (kind == kHead) {
+                    named_bar_sync(1, nct);
+                    if (t == 0) {
+                        float bv = -INFINITY; int bi = 0x7fffffff;
+                        for (int cc = 0; cc < 8; ++cc) {
+                            const float v = s_best_val[cc * 8]; const int i = s_best_idx[cc * 8];
+                            if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+                        }
+                        a.amax_val[cta] = bv;
+                        a.amax_idx[cta] = bi;
+                    }
+                }
+            }
+            if (!sync_phase()) return;
+        }
+
+        // ---- CTA 0 finishes the greedy argmax, advances the state and gathers the next embedding row ----
+        if (cta == 0) {
+            float bv = -INFINITY; int bi = 0x7fffffff;
+            for (int c = t; c < ncta; c += nct) {
+                const float v = ld_cg_f32(a.amax_val + c);
+                const int i = ld_cg_s32(a.amax_idx + c);
+                if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+            }
+#pragma unroll
+            for (int s = 16; s >= 1; s >>= 1) {
+                const float ov = __shfl_xor_sync(kFull, bv, s);
+                const int oi = __shfl_xor_sync(kFull, bi, s);
+                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+            }
+            if (lane == 0) { s_best_val[w] = bv; s_best_idx[w] = bi; }
+            named_bar_sync(1, nct);
+            if (t == 0) {
+                for (int w2 = 0; w2 < nw; ++w2) {
+                    const float v = s_best_val[w2]; const int i = s_best_idx[w2];
+                    if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+                }
+                if (bi == 0x7fffffff) bi = 0;          // all-NaN row: fall back to index 0
+                a.tok[0] = bi;
+                if (a.out_ids) a.out_ids[step] = bi;
+                if (step == a.n_steps - 1) {
+                    a.next_ids[0] = bi;
+                    if (a.advance) { a.pos[0] += a.n_steps; a.seq_lens[0] += a.n_steps; }
+                }
+            }
+            named_bar_sync(1, nct);
+            // the last layer's MLP sums are consumed: back to zero (the other buffer was zeroed in the last MLP phase)
+            float *z = a.acc + (size_t)((L - 1) & 1) * D;
+            for (int idx = t; idx < (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (step + 1 < a.n_steps) {
+                __threadfence();
+                named_bar_sync(1, nct);
+                embed_row(a.tok);
+            }
+        }
+        if (step + 1 < a.n_steps && !sync_phase()) return;
+    }
+}
+
+}  // namespace
+
+template <int IPW, int DH>
+static int launch_step_b1_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
+{
+    const MegaLayout lay = mega_layout<DH>(a.D);
+    auto kernel = decode_step_b1_kernel<IPW, DH>;
+    static bool configured[16] = {};
+    if (!configured[c->cfg.device & 15]) {
+        FT_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemMax));
+        int per_sm = 0;
+        FT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, (lay.nw + 1) * 32, lay.total));
+        if (per_sm < 1) return FASTTPS_INVALID_ARG;
+        configured[c->cfg.device & 15] = true;
+    }
+    if ((unsigned long long)(3 * a.n_layers + 3) * (unsigned long long)a.n_steps * (unsigned long long)c->n_sm >= kBarAbort)
+        return FASTTPS_INVALID_ARG;                      // the arrival counter must stay below the abort mark
+    // the barrier counter and the group counters start from zero every launch
+    FT_CUDA(cudaMemsetAsync(c->grid_bar, 0, kGridBarWords * sizeof(unsigned), st));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(c->n_sm); cfg.blockDim = dim3((lay.nw + 1) * 32); cfg.dynamicSmemBytes = lay.total; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    void *params[] = {const_cast<StepArgs *>(&a)};
+    ProfScope prof(c, kProfStep, st);
+    FT_CUDA(cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(kernel), params));
+    c->launches++;
+    return FASTTPS_OK;
+}
+
+// True when the batch-1 kernel can serve this model shape (the general step kernel's conditions, and a group of
+// at least one CTA per query head).
+bool step_b1_supported(const Ctx *c, int batch)
+{
+    return batch == 1 && step_kernel_supported(c, batch) && c->cfg.n_q_heads <= c->n_sm;
+}
+
+int launch_step_b1(Ctx *c, const StepArgs &a, cudaStream_t st)
+{
+    const int ipw = warp_split(a.D).ipw;
+#define FT_STEP_B1(DHV) \
+    case DHV: return ipw == 8 ? launch_step_b1_inst<8, DHV>(c, a, st) : launch_step_b1_inst<4, DHV>(c, a, st)
+    switch (a.head_dim) {
+        FT_STEP_B1(32);
+        FT_STEP_B1(64);
+        FT_STEP_B1(96);
+        FT_STEP_B1(128);
+    default: return FASTTPS_INVALID_ARG;
+    }
+#undef FT_STEP_B1
+}
+
+}  // namespace fasttps

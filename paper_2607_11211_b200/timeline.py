@@ -25,12 +25,16 @@ def main():
     ap.add_argument("--past", type=int, default=1024)
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--steps", type=int, default=4)
+    ap.add_argument("--step-kernel", type=int, default=1, help="1: batch-1 kernel at batch 1, general step kernel otherwise; 2: general")
     args = ap.parse_args()
     dm, B, NL, NS = wl.PHI3_MINI, args.batch, args.layers, args.steps
     dev = torch.device("cuda", 0)
     max_seq = args.past + NS + 2
     ctx = fb.Context.from_dims(dm, B, max_seq, n_layers=NL)
-    ctx.set_option("step_kernel", 1)
+    ctx.set_option("step_kernel", args.step_kernel)
+    # the batch-1 kernel has three phases per layer (attention and output projection are one), the general one four
+    names = ("qkv", "attn+o_proj", "mlp") if (B == 1 and args.step_kernel == 1) else ("qkv", "attn", "o_proj", "mlp")
+    P = len(names)
     seed = wl.MASTER_SEED
     layers = [ctx.pack_layer(wl.layer_weights(dm, i, seed, device=dev)) for i in range(NL)]
     caches = [wl.kv_cache(dm, i, B, max_seq, seed, device=dev) for i in range(NL)]
@@ -52,9 +56,9 @@ def main():
         ms = e0.elapsed_time(e1)
     status = ctx.get_status()
     first, last = ctx.trace_read()
-    # stamps: 2 for the barrier after the embedding gather, then per step 2 per phase (4 per layer + logits)
+    # stamps: 2 for the barrier after the embedding gather, then per step 2 per phase (P per layer + logits)
     # and 2 for the barrier that ends the step (absent after the last step)
-    per_step = 2 * (4 * NL + 2)
+    per_step = 2 * (P * NL + 2)
     report = {"batch": B, "past": args.past, "layers": NL, "steps": NS, "launch_ms": ms, "ms_per_step": ms / NS,
               "device_status": status}
     for name, stamps in (("first_cta", first), ("last_cta", last)):
@@ -65,12 +69,12 @@ def main():
         prev_after = np.concatenate([[s[base - 1]], after[:-1]])
         busy = (before - prev_after) / 1e3
         wait = (after - before) / 1e3
-        b4, w4 = busy[:4 * NL].reshape(NL, 4), wait[:4 * NL].reshape(NL, 4)
+        b4, w4 = busy[:P * NL].reshape(NL, P), wait[:P * NL].reshape(NL, P)
         report[name] = {
             "step_us": float(st[-1] - s[base - 1]) / 1e3,
-            "mean_busy_us": dict(zip(("qkv", "attn", "o_proj", "mlp"), np.round(b4.mean(0), 2).tolist())),
-            "mean_barrier_wait_us": dict(zip(("qkv", "attn", "o_proj", "mlp"), np.round(w4.mean(0), 2).tolist())),
-            "logits_busy_us": round(float(busy[4 * NL]), 2), "logits_barrier_wait_us": round(float(wait[4 * NL]), 2),
+            "mean_busy_us": dict(zip(names, np.round(b4.mean(0), 2).tolist())),
+            "mean_barrier_wait_us": dict(zip(names, np.round(w4.mean(0), 2).tolist())),
+            "logits_busy_us": round(float(busy[P * NL]), 2), "logits_barrier_wait_us": round(float(wait[P * NL]), 2),
         }
     print(json.dumps(report, indent=1))
     ctx.close()
