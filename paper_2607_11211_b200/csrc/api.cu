@@ -108,7 +108,7 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     A(dev_alloc(&c->attn_ticket, B * f.n_q_heads, true));
     A(dev_alloc(&c->mlp_acc, 2 * B * D, true));
     A(dev_alloc(&c->grid_bar, kGridBarWords, true));
-    A(dev_alloc(&c->hacc, 2 * D, true));
+    A(dev_alloc(&c->hacc, 2 * B * D, true));
     A(dev_alloc(&c->trace, 2 * (size_t)kTraceLen, true));
     A(dev_alloc(&c->d_layers, (size_t)(f.n_layers > 0 ? f.n_layers : 1), true));
     if (e == cudaSuccess)

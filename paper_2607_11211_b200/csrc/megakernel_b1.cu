@@ -1,11 +1,12 @@
-// Persistent decode-step kernel for ONE sequence (batch 1): the same token phase as megakernel.cu --
+// Persistent decode-step kernel with per-head CTA groups (batch <= 8): the same token phase as megakernel.cu --
 // embedding, per layer RMSNorm -> QKV -> attention (Algorithm 3) -> output projection -> RMSNorm -> fused MLP
 // (Algorithm 4), final norm, logits, greedy argmax -- with THREE grid-wide phase boundaries per layer
 // instead of four.
 //
 // At batch 1 a layer is ~37 us of streaming and every grid-wide boundary costs 4-5 us of dependent latency
 // (barrier, activation loads, norm).  Here the attention and the output projection are one phase: every query
-// head belongs to a fixed group of m0 = n_sm / H_q CTAs.  The group's CTAs split the rows of the head's cache
+// head belongs to a fixed group of m0 = n_sm / H_q CTAs.  The group's CTAs split the rows of the head's caches,
+// all sequences of the batch laid end to end, into equal shares whatever the mix of lengths
 // (Algorithm 3 on each share, partial (max, sum, output) published), meet at a counter of their own -- a wait
 // for at most m0 - 1 neighbours instead of the whole grid --, each merges the head's partials, and each then
 // multiplies the merged head output with ITS slice of the output-projection rows: for row tile r the d / 32
@@ -19,25 +20,27 @@ namespace fasttps {
 
 namespace {
 
-struct OneSegment {
-    Segment sg;
-    int n;                       // 0 or 1
+// A CTA's share of its head: at most one segment per sequence.
+struct GroupSegs {
+    int n;
+    Segment seg[kMaxNB];
 };
-struct OneSource {
-    const OneSegment *p;
+struct GroupSource {
+    const GroupSegs *p;
     int i;
-    __device__ __forceinline__ explicit OneSource(const OneSegment *p_) : p(p_), i(0) {}
+    __device__ __forceinline__ explicit GroupSource(const GroupSegs *p_) : p(p_), i(0) {}
     __device__ __forceinline__ bool next(Segment &s)
     {
         if (i >= p->n) return false;
-        s = p->sg;
-        ++i;
+        s = p->seg[i++];
         return true;
     }
 };
 
-template <int IPW, int DH>
-__global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(StepArgs a)
+// BC: batch class.  0: batch 1 (the batch loops fold away at compile time), 1: batch 2, 2: batches 3 to 8 (which
+// also selects the staging of the MLP scatter; see mlp_core.cuh).
+template <int IPW, int DH, int BC>
+__global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_groups_kernel(StepArgs a)
 {
     extern __shared__ __align__(128) unsigned char dsm[];
     __shared__ __align__(16) ActTile s_hi[kMaxOctetsPerCta];
@@ -47,9 +50,10 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
     __shared__ int s_go;
     __shared__ int s_tables_ready;                               // steps whose attention share is known
     __shared__ LayerPtrs s_layers[kMaxStepLayers];               // the layer table: no global round trip per phase
-    __shared__ OneSegment s_one;                                 // this CTA's attention share for the current step
+    __shared__ GroupSegs s_segs;                                 // this CTA's attention share for the current step
     __shared__ int s_mprime;                                     // CTAs of a group that hold rows in the current step
-    __shared__ __align__(16) __nv_bfloat16 s_outh[DH];           // the merged output of this CTA's head
+    __shared__ int s_ncta[kMaxNB];                               // partials of (sequence b, this head) in the current step
+    __shared__ __align__(16) __nv_bfloat16 s_outh[kMaxNB * DH];  // the merged outputs of this CTA's head, per sequence
 
     constexpr int KB = DH / 32;                                  // k blocks of a head in the output projection
     const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3;
@@ -61,7 +65,8 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
     float *smem_red = reinterpret_cast<float *>(dsm + lay.red_off);
     AttnScratch<DH> &scratch = *reinterpret_cast<AttnScratch<DH> *>(dsm + lay.scratch_off);
 
-    const int D = a.D;
+    const int D = a.D, B = BC == 0 ? 1 : a.batch;
+    constexpr bool BIG = BC == 2;
     const int nq = a.n_q_heads * a.head_dim, nkv = a.n_kv_heads * a.head_dim, nqkv = nq + 2 * nkv;
     constexpr int SPT = IPW / kBlocksPerWarpPerSlot;      // ring pieces per 16-row tile
     constexpr int PPO = IPW / 4;                          // ring pieces per W_down octet
@@ -121,7 +126,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
                     __threadfence_block();
                 }
                 const AttnArgs aa = attn_args_of(a, lp, step, gm * a.n_q_heads);
-                const bool kv_ok = attn_for_each_tile<DH>(aa, OneSource(&s_one),
+                const bool kv_ok = attn_for_each_tile<DH>(aa, GroupSource(&s_segs),
                                                           [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
                     return ring.put2(piece++, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
                 });
@@ -153,17 +158,21 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
     gb.target = (unsigned)ncta;
     unsigned grp_target = 0;
     if (cta == 0 && t == 0) {
-        const int L = a.seq_lens[0], p = a.pos[0];
-        if (L < 0 || L + a.n_steps > a.max_seq) atomicOr(a.status, FASTTPS_DEV_CACHE_FULL);
-        else if (p < 0 || p + a.n_steps > a.max_seq) atomicOr(a.status, FASTTPS_DEV_BAD_POSITION);
+        // sequences that cannot be served for all steps are reported once and contribute no rows
+        for (int bb = 0; bb < B; ++bb) {
+            const int L = a.seq_lens[bb], p = a.pos[bb];
+            if (L < 0 || L + a.n_steps > a.max_seq) atomicOr(a.status, FASTTPS_DEV_CACHE_FULL);
+            else if (p < 0 || p + a.n_steps > a.max_seq) atomicOr(a.status, FASTTPS_DEV_BAD_POSITION);
+        }
     }
 
-    // gathers the embedding row of the current token into x0 (CTA 0 only)
+    // gathers the embedding rows of the current tokens into x0 (CTA 0 only)
     auto embed_row = [&](const int32_t *ids) {
-        for (int j = t; j < (D >> 3); j += nct) {
-            int id = ld_cg_s32(ids);
+        for (int idx = t; idx < B * (D >> 3); idx += nct) {
+            const int b = idx / (D >> 3), j = idx - b * (D >> 3);
+            int id = ld_cg_s32(ids + b);
             if (id < 0 || id >= a.V) { if (j == 0) atomicOr(a.status, FASTTPS_DEV_BAD_TOKEN); id = 0; }
-            reinterpret_cast<uint4 *>(a.x0)[j] = reinterpret_cast<const uint4 *>(a.embed + (size_t)id * D)[j];
+            reinterpret_cast<uint4 *>(a.x0 + (size_t)b * D)[j] = reinterpret_cast<const uint4 *>(a.embed + (size_t)id * D)[j];
         }
     };
 
@@ -192,20 +201,45 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
     enum { kQkv = 0, kAttn = 1, kMlp = 2, kHead = 3 };
     const int L = a.n_layers;
     for (int step = 0; step < a.n_steps; ++step) {
-        // ---- this step's attention share: rows [R gs / m', R (gs + 1) / m') of the head, m' CTAs of the group ----
+        // ---- this step's attention share: the rows of the head, all sequences end to end, are cut into m'
+        // equal shares, one per CTA of the group (at least 16 rows each) ----
         if (t == 0) {
-            const int Ls = a.seq_lens[0] + step, ps = a.pos[0] + step;
-            const bool valid = !(Ls < step || Ls >= a.max_seq || ps < step || ps >= a.max_seq);
-            const int R = valid ? Ls + 1 : 0;
-            int mp = R / 16;                                   // at least 16 rows per CTA, at most the group
-            mp = R == 0 ? 0 : (mp < 1 ? 1 : (mp > gm ? gm : mp));
+            int R[kMaxNB];
+            long long T = 0;
+            for (int bb = 0; bb < B; ++bb) {
+                const int Ls = a.seq_lens[bb] + step, ps = a.pos[bb] + step;
+                const bool valid = !(Ls < step || Ls >= a.max_seq || ps < step || ps >= a.max_seq);
+                R[bb] = valid ? Ls + 1 : 0;
+                T += R[bb];
+            }
+            int mp = (int)(T / 16 < gm ? T / 16 : gm);
+            mp = T == 0 ? 0 : (mp < 1 ? 1 : mp);
             s_mprime = mp;
-            s_one.n = (in_group && gs < mp) ? 1 : 0;
-            Segment &sg = s_one.sg;
-            sg.b = 0; sg.h = in_group ? head : 0; sg.L = Ls; sg.pos = ps;
-            sg.r0 = mp ? (int)((long long)R * gs / mp) : 0;
-            sg.r1 = mp ? (int)((long long)R * (gs + 1) / mp) : 0;
-            sg.first_cta = head * gm; sg.n_cta = mp;
+            const long long f0 = mp ? T * gs / mp : 0, f1 = (mp && gs < mp) ? T * (gs + 1) / mp : f0;
+            auto owner = [&](long long x) {                    // the share that holds row x of the head
+                int c = 0;
+                while (c + 1 < mp && T * (c + 1) / mp <= x) ++c;
+                return c;
+            };
+            int n = 0;
+            long long off = 0;
+            for (int bb = 0; bb < B; ++bb) {
+                const int rb = R[bb];
+                s_ncta[bb] = 0;
+                if (rb > 0) {
+                    const int first = owner(off), last = owner(off + rb - 1);
+                    s_ncta[bb] = last - first + 1;
+                    const long long lo = f0 > off ? f0 : off, hi = f1 < off + rb ? f1 : off + rb;
+                    if (in_group && lo < hi) {
+                        Segment &sg = s_segs.seg[n++];
+                        sg.b = bb; sg.h = head; sg.L = rb - 1; sg.pos = a.pos[bb] + step;
+                        sg.r0 = (int)(lo - off); sg.r1 = (int)(hi - off);
+                        sg.first_cta = head * gm + first; sg.n_cta = last - first + 1;
+                    }
+                }
+                off += rb;
+            }
+            s_segs.n = n;
         }
         named_bar_sync(1, nct);
         if (t == 0) {
@@ -228,14 +262,14 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
             if (kind == kAttn) {
                 // ---- attention (Algorithm 3) on this CTA's rows of its head; the partial is published ----
                 const AttnArgs aa = attn_args_of(a, lp, step, gm * a.n_q_heads);
-                ok = attn_consume<DH, true>(aa, ring, piece, cta, OneSource(&s_one), scratch, nw) && ok;
+                ok = attn_consume<DH, true>(aa, ring, piece, cta, GroupSource(&s_segs), scratch, nw) && ok;
                 grp_target += (unsigned)mprime;
                 if (in_group) {
                     // ---- the group meets: every CTA of it needs the merged output of the head ----
                     __threadfence();
                     named_bar_sync(1, nct);
                     if (t == 0) {
-                        if (s_one.n && ok) atomicAdd(grp, 1u);
+                        if (s_segs.n && ok) atomicAdd(grp, 1u);
                         int met = 1;
                         unsigned long long t0 = 0;
                         for (unsigned it = 1; ld_acquire_u32(grp) < grp_target; ++it) {
@@ -251,14 +285,16 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
                     if (!s_go) ok = false;
                     // ---- softmax merge of the head's partials: out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s ----
                     constexpr int PS = DH + 4;
-                    const float *hp = a.attn_part + (size_t)head * kMaxSplits * PS;
-                    for (int i = t; i < DH; i += nct) {
+                    for (int idx = t; idx < B * DH; idx += nct) {
+                        const int b = idx / DH, i = idx - b * DH;
+                        const int np = s_ncta[b];
+                        const float *hp = a.attn_part + ((size_t)b * a.n_q_heads + head) * kMaxSplits * PS;
                         float M = -INFINITY, den = 0.f, o = 0.f;
-                        for (int s0 = 0; s0 < mprime; s0 += 4) {
+                        for (int s0 = 0; s0 < np; s0 += 4) {
                             float ms[4], ls[4], os[4];
 #pragma unroll
                             for (int u = 0; u < 4; ++u) {
-                                const bool have = s0 + u < mprime;
+                                const bool have = s0 + u < np;
                                 const float *p = hp + (size_t)(have ? s0 + u : 0) * PS;
                                 ms[u] = ld_cg_f32(p + DH);
                                 ls[u] = ld_cg_f32(p + DH + 1);
@@ -278,15 +314,15 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
                             }
                             M = Mn;
                         }
-                        s_outh[i] = __float2bfloat16_rn(mprime > 0 && ok ? o / den : 0.f);
+                        s_outh[idx] = __float2bfloat16_rn(np > 0 && ok ? o / den : 0.f);
                     }
                     named_bar_sync(1, nct);
                     // ---- this CTA's row tiles of the output projection, k = the head: sums go to hacc[l & 1] ----
                     uint4 bh[KB];
 #pragma unroll
                     for (int j = 0; j < KB; ++j)
-                        bh[j] = g == 0 ? *reinterpret_cast<const uint4 *>(s_outh + 32 * j + 8 * t4) : make_uint4(0u, 0u, 0u, 0u);
-                    float *hsum = hacc + (size_t)(l & 1) * D;
+                        bh[j] = g < B ? *reinterpret_cast<const uint4 *>(s_outh + g * DH + 32 * j + 8 * t4) : make_uint4(0u, 0u, 0u, 0u);
+                    float *hsum = hacc + (size_t)(l & 1) * B * D;
                     for (int p0 = 0; p0 < ont; p0 += TP, ++piece) {
                         const int nt = ont - p0 < TP ? ont - p0 : TP;
                         const unsigned char *slot = ring.wait(piece, ok);
@@ -300,10 +336,15 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
                                 mma_bf16_k16(c, lo.x, hi.x, lo.y, hi.y, bh[j].x, bh[j].y);
                                 mma_bf16_k16(c, lo.z, hi.z, lo.w, hi.w, bh[j].z, bh[j].w);
                             }
-                            const int row = (ot0 + p0 + w) * 16 + g;
-                            if (t4 == 0 && ok) {                 // accumulator column 0 = the one batch row
-                                if (row < D) atomicAdd(hsum + row, c[0]);
-                                if (row + 8 < D) atomicAdd(hsum + row + 8, c[2]);
+                            // accumulator fragment: rows g / g + 8 of the tile, batch rows 2 t4 / 2 t4 + 1
+                            const int row = (ot0 + p0 + w) * 16 + g, b0 = 2 * t4;
+                            if (ok && b0 < B) {
+                                if (row < D) atomicAdd(hsum + (size_t)b0 * D + row, c[0]);
+                                if (row + 8 < D) atomicAdd(hsum + (size_t)b0 * D + row + 8, c[2]);
+                            }
+                            if (ok && b0 + 1 < B) {
+                                if (row < D) atomicAdd(hsum + (size_t)(b0 + 1) * D + row, c[1]);
+                                if (row + 8 < D) atomicAdd(hsum + (size_t)(b0 + 1) * D + row + 8, c[3]);
                             }
                         }
                         ring.release(piece);
@@ -316,21 +357,21 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
                 __nv_bfloat16 *store = nullptr;
                 int tile0, ntile;
                 if (kind == kQkv) {                          // x_l = h_{l-1} + y_{l-1} (layer 0: the embedding row)
-                    src = l == 0 ? a.x0 : a.h; add = l == 0 ? nullptr : a.acc + (size_t)((l - 1) & 1) * D;
+                    src = l == 0 ? a.x0 : a.h; add = l == 0 ? nullptr : a.acc + (size_t)((l - 1) & 1) * B * D;
                     gain = lp.g_attn; store = l == 0 ? nullptr : xbuf; tile0 = q0; ntile = qn;
                 } else if (kind == kMlp) {                   // h_l = x_l + attn . W_o
-                    src = l == 0 ? a.x0 : xbuf; add = hacc + (size_t)(l & 1) * D;
+                    src = l == 0 ? a.x0 : xbuf; add = hacc + (size_t)(l & 1) * B * D;
                     gain = lp.g_mlp; store = a.h; tile0 = m0; ntile = mn;
                 } else {                                     // x_L = h_{L-1} + y_{L-1}
-                    src = a.h; add = a.acc + (size_t)((L - 1) & 1) * D;
+                    src = a.h; add = a.acc + (size_t)((L - 1) & 1) * B * D;
                     gain = a.g_final; tile0 = l0; ntile = ln;
                 }
                 // the sums of the output projection of the layer before are consumed: back to zero
                 if (cta == ncta - 1 && ((kind == kQkv && l > 0) || kind == kHead)) {
-                    float *z = hacc + (size_t)((l - 1) & 1) * D;   // (head: l = L)
-                    for (int idx = t; idx < (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float *z = hacc + (size_t)((l - 1) & 1) * B * D;   // (head: l = L)
+                    for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
-                load_b_frags<IPW>(bf, src, D, 1, D, nw, gain, a.eps, smem_red, add, store, cta, ncta);
+                load_b_frags<IPW>(bf, src, D, B, D, nw, gain, a.eps, smem_red, add, store, cta, ncta);
                 if (kind == kHead) {
                     for (int u = t; u < 64; u += nct) { s_best_val[u] = -INFINITY; s_best_idx[u] = 0x7fffffff; }
                     named_bar_sync(1, nct);
@@ -343,16 +384,16 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
                         s_lo[tile][b][cc] = __float2bfloat16_rn(act - __bfloat162float(hi));
                         return;
                     }
-                    if (b >= 1) return;
+                    if (b >= B) return;
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh) {
                         const int row = (tile0 + tile) * 16 + cc + 8 * hh;
                         const float v = hh ? v1 : v0;
                         if (kind == kQkv) {
-                            if (row < nqkv) a.qkv[row] = __float2bfloat16_rn(v);
+                            if (row < nqkv) a.qkv[(size_t)b * nqkv + row] = __float2bfloat16_rn(v);
                         } else if (row < a.V) {              // logits and the running argmax of this thread's rows
-                            const int u = cc * 8;
-                            if (a.logits) a.logits[row] = v;
+                            const int u = cc * 8 + b;
+                            if (a.logits) a.logits[(size_t)b * a.V + row] = v;
                             if (v > s_best_val[u]) { s_best_val[u] = v; s_best_idx[u] = row; }
                         }
                     }
@@ -363,8 +404,8 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
                     // ---- down projection of this CTA's octets; the sums of all CTAs meet in acc[l & 1] ----
                     if (cta == 0 && l > 0) {
                         // layer l - 1's sums were consumed by the QKV prologue of this layer: zero them for layer l + 1
-                        float *z = a.acc + (size_t)((l - 1) & 1) * D;
-                        for (int idx = t; idx < (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        float *z = a.acc + (size_t)((l - 1) & 1) * B * D;
+                        for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                     named_bar_sync(1, nct);
                     float acc[IPW][2][4];
@@ -376,56 +417,59 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
                             for (int e = 0; e < 4; ++e) acc[i][m][e] = 0.f;
                     mlp_down_phase<IPW>(ring, piece, mn, nw, s_hi, s_lo, acc, ok);
                     piece += mn * PPO;
-                    mlp_scatter_add<IPW, false>(acc, smem_part, a.acc + (size_t)(l & 1) * D, 1, D, nw);
+                    mlp_scatter_add<IPW, BIG>(acc, smem_part, a.acc + (size_t)(l & 1) * B * D, B, D, nw);
                 } else if (kind == kHead) {
                     named_bar_sync(1, nct);
-                    if (t == 0) {
+                    if (t < 8 && t < B) {
                         float bv = -INFINITY; int bi = 0x7fffffff;
                         for (int cc = 0; cc < 8; ++cc) {
-                            const float v = s_best_val[cc * 8]; const int i = s_best_idx[cc * 8];
+                            const float v = s_best_val[cc * 8 + t]; const int i = s_best_idx[cc * 8 + t];
                             if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
                         }
-                        a.amax_val[cta] = bv;
-                        a.amax_idx[cta] = bi;
+                        a.amax_val[(size_t)t * ncta + cta] = bv;
+                        a.amax_idx[(size_t)t * ncta + cta] = bi;
                     }
                 }
             }
             if (!sync_phase()) return;
         }
 
-        // ---- CTA 0 finishes the greedy argmax, advances the state and gathers the next embedding row ----
+        // ---- CTA 0 finishes the greedy argmax, advances the state and gathers the next embedding rows ----
         if (cta == 0) {
-            float bv = -INFINITY; int bi = 0x7fffffff;
-            for (int c = t; c < ncta; c += nct) {
-                const float v = ld_cg_f32(a.amax_val + c);
-                const int i = ld_cg_s32(a.amax_idx + c);
-                if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
-            }
-#pragma unroll
-            for (int s = 16; s >= 1; s >>= 1) {
-                const float ov = __shfl_xor_sync(kFull, bv, s);
-                const int oi = __shfl_xor_sync(kFull, bi, s);
-                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-            }
-            if (lane == 0) { s_best_val[w] = bv; s_best_idx[w] = bi; }
-            named_bar_sync(1, nct);
-            if (t == 0) {
-                for (int w2 = 0; w2 < nw; ++w2) {
-                    const float v = s_best_val[w2]; const int i = s_best_idx[w2];
+            // every thread fetches its share of the per-CTA candidates at once, then warps and the CTA reduce
+            for (int b = 0; b < B; ++b) {
+                float bv = -INFINITY; int bi = 0x7fffffff;
+                for (int c = t; c < ncta; c += nct) {
+                    const float v = ld_cg_f32(a.amax_val + (size_t)b * ncta + c);
+                    const int i = ld_cg_s32(a.amax_idx + (size_t)b * ncta + c);
                     if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
                 }
-                if (bi == 0x7fffffff) bi = 0;          // all-NaN row: fall back to index 0
-                a.tok[0] = bi;
-                if (a.out_ids) a.out_ids[step] = bi;
-                if (step == a.n_steps - 1) {
-                    a.next_ids[0] = bi;
-                    if (a.advance) { a.pos[0] += a.n_steps; a.seq_lens[0] += a.n_steps; }
+#pragma unroll
+                for (int s = 16; s >= 1; s >>= 1) {
+                    const float ov = __shfl_xor_sync(kFull, bv, s);
+                    const int oi = __shfl_xor_sync(kFull, bi, s);
+                    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
                 }
+                if (lane == 0) { s_best_val[w] = bv; s_best_idx[w] = bi; }
+                named_bar_sync(1, nct);
+                if (t == 0) {
+                    for (int w2 = 0; w2 < nw; ++w2) {
+                        const float v = s_best_val[w2]; const int i = s_best_idx[w2];
+                        if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+                    }
+                    if (bi == 0x7fffffff) bi = 0;      // all-NaN row: fall back to index 0
+                    a.tok[b] = bi;
+                    if (a.out_ids) a.out_ids[(size_t)step * B + b] = bi;
+                    if (step == a.n_steps - 1) {
+                        a.next_ids[b] = bi;
+                        if (a.advance) { a.pos[b] += a.n_steps; a.seq_lens[b] += a.n_steps; }
+                    }
+                }
+                named_bar_sync(1, nct);
             }
-            named_bar_sync(1, nct);
             // the last layer's MLP sums are consumed: back to zero (the other buffer was zeroed in the last MLP phase)
-            float *z = a.acc + (size_t)((L - 1) & 1) * D;
-            for (int idx = t; idx < (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+            float *z = a.acc + (size_t)((L - 1) & 1) * B * D;
+            for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (step + 1 < a.n_steps) {
                 __threadfence();
                 named_bar_sync(1, nct);
@@ -438,11 +482,11 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_b1_kernel(Step
 
 }  // namespace
 
-template <int IPW, int DH>
+template <int IPW, int DH, int BC>
 static int launch_step_b1_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
 {
     const MegaLayout lay = mega_layout<DH>(a.D);
-    auto kernel = decode_step_b1_kernel<IPW, DH>;
+    auto kernel = decode_step_groups_kernel<IPW, DH, BC>;
     static bool configured[16] = {};
     if (!configured[c->cfg.device & 15]) {
         FT_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemMax));
@@ -468,18 +512,22 @@ static int launch_step_b1_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
     return FASTTPS_OK;
 }
 
-// True when the batch-1 kernel can serve this model shape (the general step kernel's conditions, and a group of
-// at least one CTA per query head).
+// True when the kernel with head groups can serve this model shape and batch (the general step kernel's
+// conditions, and a group of at least one CTA per query head).
 bool step_b1_supported(const Ctx *c, int batch)
 {
-    return batch == 1 && step_kernel_supported(c, batch) && c->cfg.n_q_heads <= c->n_sm;
+    return step_kernel_supported(c, batch) && c->cfg.n_q_heads <= c->n_sm;
 }
 
 int launch_step_b1(Ctx *c, const StepArgs &a, cudaStream_t st)
 {
     const int ipw = warp_split(a.D).ipw;
-#define FT_STEP_B1(DHV) \
-    case DHV: return ipw == 8 ? launch_step_b1_inst<8, DHV>(c, a, st) : launch_step_b1_inst<4, DHV>(c, a, st)
+    const int bc = a.batch == 1 ? 0 : (a.batch == 2 ? 1 : 2);
+#define FT_STEP_B1(DHV)                                                                                  \
+    case DHV:                                                                                            \
+        if (bc == 2) return ipw == 8 ? launch_step_b1_inst<8, DHV, 2>(c, a, st) : launch_step_b1_inst<4, DHV, 2>(c, a, st); \
+        if (bc == 1) return ipw == 8 ? launch_step_b1_inst<8, DHV, 1>(c, a, st) : launch_step_b1_inst<4, DHV, 1>(c, a, st); \
+        return ipw == 8 ? launch_step_b1_inst<8, DHV, 0>(c, a, st) : launch_step_b1_inst<4, DHV, 0>(c, a, st)
     switch (a.head_dim) {
         FT_STEP_B1(32);
         FT_STEP_B1(64);

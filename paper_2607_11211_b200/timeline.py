@@ -25,15 +25,15 @@ def main():
     ap.add_argument("--past", type=int, default=1024)
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--steps", type=int, default=4)
-    ap.add_argument("--step-kernel", type=int, default=1, help="1: batch-1 kernel at batch 1, general step kernel otherwise; 2: general")
+    ap.add_argument("--step-kernel", type=int, default=1, help="1: step kernel with head groups; 2: general step kernel")
     args = ap.parse_args()
     dm, B, NL, NS = wl.PHI3_MINI, args.batch, args.layers, args.steps
     dev = torch.device("cuda", 0)
     max_seq = args.past + NS + 2
     ctx = fb.Context.from_dims(dm, B, max_seq, n_layers=NL)
     ctx.set_option("step_kernel", args.step_kernel)
-    # the batch-1 kernel has three phases per layer (attention and output projection are one), the general one four
-    names = ("qkv", "attn+o_proj", "mlp") if (B == 1 and args.step_kernel == 1) else ("qkv", "attn", "o_proj", "mlp")
+    # the kernel with head groups has three phases per layer (attention and output projection are one), the general one four
+    names = ("qkv", "attn+o_proj", "mlp") if args.step_kernel == 1 else ("qkv", "attn", "o_proj", "mlp")
     P = len(names)
     seed = wl.MASTER_SEED
     layers = [ctx.pack_layer(wl.layer_weights(dm, i, seed, device=dev)) for i in range(NL)]
