@@ -347,7 +347,7 @@ int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value)
 {
     if (!ctx || !name) return FASTTPS_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);
-    if (strcmp(name, "step_kernel") == 0) c->opt_step_kernel = value < 0 ? 0 : (value > 2 ? 2 : value);
+    if (strcmp(name, "step_kernel") == 0) c->opt_step_kernel = value != 0;
     else return FASTTPS_INVALID_ARG;
     return FASTTPS_OK;
 }
@@ -410,7 +410,6 @@ static int step_impl(Ctx *c, const void *embed, const fasttps_layer_weights *lay
     a.amax_val = c->amax_val; a.amax_idx = c->amax_idx; a.tok = c->tok2;
     a.bar = c->grid_bar; a.status = c->status;
     a.trace = c->trace; a.trace_len = kTraceLen;
-    if (c->opt_step_kernel == 1 && step_b1_supported(c, batch)) return launch_step_b1(c, a, st);
     return launch_step(c, a, st);
 }
 

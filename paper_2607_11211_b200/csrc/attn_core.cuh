@@ -135,20 +135,6 @@ template <int DH> struct AttnTile {
     static constexpr int kPieceBytes = 2 * kAttnTileRows * kRowBytes;     // K tile then V tile
 };
 
-// A share as a list of segments kept in shared memory (the persistent kernel computes it once per step and
-// uses it for every layer).  12 bytes per segment; lengths and positions of the step sit beside the list.
-constexpr int kMaxSegments = 257;            // a share touches at most batch * n_q_heads heads (<= 256 here)
-struct PackedSegment {
-    int r0, r1;
-    unsigned short bh;                       // b * n_q_heads + h
-    unsigned char first_cta, n_cta;
-};
-struct SegmentList {
-    int n, n_q_heads;
-    int len[kMaxNB], pos[kMaxNB];            // cached rows and rotary position of every sequence in this step
-    PackedSegment seg[kMaxSegments];
-};
-
 // Segment sources: `bool next(Segment &)`.
 struct WalkSource {
     ShareWalk walk;
@@ -158,21 +144,6 @@ struct WalkSource {
     }
     __device__ __forceinline__ bool next(Segment &s) { return walk.next(s); }
 };
-struct ListSource {
-    const SegmentList *list;
-    int i;
-    __device__ __forceinline__ explicit ListSource(const SegmentList *l) : list(l), i(0) {}
-    __device__ __forceinline__ bool next(Segment &s)
-    {
-        if (i >= list->n) return false;
-        const PackedSegment p = list->seg[i++];
-        s.b = p.bh / list->n_q_heads; s.h = p.bh - s.b * list->n_q_heads;
-        s.L = list->len[s.b]; s.pos = list->pos[s.b];
-        s.r0 = p.r0; s.r1 = p.r1; s.first_cta = p.first_cta; s.n_cta = p.n_cta;
-        return true;
-    }
-};
-
 // Calls f(k_tile, v_tile, bytes_each) for every K/V tile of this CTA's share, in walk order; stops and
 // returns false as soon as f does.
 template <int DH, class Src, class F>
@@ -206,7 +177,7 @@ __device__ __forceinline__ bool attn_produce(const AttnArgs &a, WeightRing &ring
 // of this CTA's share.  The first min(nwc, 8) warps score rows; the others only keep the ring protocol.
 // Returns false (in every consumer thread alike) if a bounded wait ran out.
 // DEFER: the partial of every segment is published (even when the CTA owns the whole head) and nobody
-// merges here; the reader of the attention output merges on the fly (load_b_frags_attn).
+// merges here; the caller merges the partials of a head itself (the persistent step kernel does, per group).
 template <int DH, bool DEFER, class Src>
 __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring, int &piece, int cta, Src src,
                                              AttnScratch<DH> &sm, int nwc)
@@ -409,85 +380,6 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
         named_bar_sync(1, nct);                          // the scratch is reused by the next segment
     }
     return true;
-}
-
-// Tensor-core B fragments of the attention output, merged on the fly from the partials that
-// attn_consume<DH, true> published.  A consumer thread (g = lane / 4, t4 = lane % 4) needs, for each of its
-// IPW k blocks, the 8 elements k = 32 (w + nw i) + 8 t4 .. + 8 of batch row g (as in load_b_frags of
-// dot_core.cuh).  The warp's batch * IPW * 4 chunks are first dealt to its lanes 32 at a time, so that at
-// batch 1 all lanes fetch and merge instead of four; a lane reads its chunk from every partial of the head
-// the chunk belongs to (four partials in flight at a time), combines them with the softmax merge
-//   out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s,
-// rounds to bf16 (the attention output is a bf16 tensor), and the packed chunks are then handed to the lanes
-// that need them with shuffles.  head_n[b * Hq + h] = number of partials of head (b, h).  All loads
-// bypass L1 (the partials were written by other SMs).
-template <int IPW, int DH>
-__device__ __forceinline__ void load_b_frags_attn(uint32_t (&bf)[IPW][4], const float *part, const unsigned char *head_n,
-                                                  int batch, int n_q_heads, int nw)
-{
-    constexpr int PS = DH + 4;
-    constexpr int CPB = IPW * 4;                     // chunks per batch row and warp
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, g = lane >> 2, t4 = lane & 3;
-    const int total = batch * CPB;
-#pragma unroll
-    for (int i = 0; i < IPW; ++i) bf[i][0] = bf[i][1] = bf[i][2] = bf[i][3] = 0u;
-    for (int j = 0; j * 32 < total; ++j) {
-        const int c = j * 32 + lane;
-        uint32_t r[4] = {0u, 0u, 0u, 0u};
-        if (c < total) {
-            const int b = c / CPB, ci = (c % CPB) >> 2, ct = c & 3;
-            const int k = 32 * (w + nw * ci) + 8 * ct;
-            const int hq = k / DH, c0 = k - hq * DH;
-            const int n = head_n[b * n_q_heads + hq];
-            const float *hp = part + ((size_t)b * n_q_heads + hq) * kMaxSplits * PS;
-            float M = -INFINITY, den = 0.f, o[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            for (int s0 = 0; s0 < n; s0 += 4) {
-                float ms[4], ls[4];
-                float4 a0[4], a1[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const bool have = s0 + u < n;
-                    const float *p = hp + (size_t)(have ? s0 + u : 0) * PS;
-                    ms[u] = ld_cg_f32(p + DH);
-                    ls[u] = ld_cg_f32(p + DH + 1);
-                    a0[u] = ld_cg_f4(p + c0);
-                    a1[u] = ld_cg_f4(p + c0 + 4);
-                    if (!have) ms[u] = -INFINITY;
-                }
-                float Mn = M;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) Mn = fmaxf(Mn, ms[u]);
-                const float corr = fast_exp2(M - Mn);        // 0 on the first round (M = -inf)
-                den *= corr;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) o[e] *= corr;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float f = ms[u] == -INFINITY ? 0.f : fast_exp2(ms[u] - Mn);
-                    den = fmaf(f, ls[u], den);
-                    o[0] = fmaf(f, a0[u].x, o[0]); o[1] = fmaf(f, a0[u].y, o[1]);
-                    o[2] = fmaf(f, a0[u].z, o[2]); o[3] = fmaf(f, a0[u].w, o[3]);
-                    o[4] = fmaf(f, a1[u].x, o[4]); o[5] = fmaf(f, a1[u].y, o[5]);
-                    o[6] = fmaf(f, a1[u].z, o[6]); o[7] = fmaf(f, a1[u].w, o[7]);
-                }
-                M = Mn;
-            }
-            const float inv = n > 0 ? 1.f / den : 0.f;       // n = 0: a skipped sequence, output zero
-            r[0] = pack2(o[0] * inv, o[1] * inv);
-            r[1] = pack2(o[2] * inv, o[3] * inv);
-            r[2] = pack2(o[4] * inv, o[5] * inv);
-            r[3] = pack2(o[6] * inv, o[7] * inv);
-        }
-        // hand the chunks of this round to the lanes whose fragments they are
-#pragma unroll
-        for (int i = 0; i < IPW; ++i) {
-            const int need = g * CPB + i * 4 + t4;
-            const int src = need & 31;
-            const uint32_t v0 = __shfl_sync(kFull, r[0], src), v1 = __shfl_sync(kFull, r[1], src);
-            const uint32_t v2 = __shfl_sync(kFull, r[2], src), v3 = __shfl_sync(kFull, r[3], src);
-            if ((need >> 5) == j && g < batch) { bf[i][0] = v0; bf[i][1] = v1; bf[i][2] = v2; bf[i][3] = v3; }
-        }
-    }
 }
 
 }  // namespace fasttps

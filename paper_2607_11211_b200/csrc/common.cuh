@@ -24,7 +24,7 @@ struct Ctx {
     unsigned long long *trace;       // [2][kTraceLen] phase timeline of the last step-kernel launch
     LayerPtrs *d_layers, *pin_layers;
     int layers_uploaded;             // number of valid entries in pin_layers / d_layers
-    int opt_step_kernel;             // 0: one kernel per product; 1: persistent step kernels (batch <= 8); 2: the general one also at batch 1
+    int opt_step_kernel;             // 1: model calls with batch <= 8 use the persistent step kernel
     fasttps_config cfg;
     int n_sm;
     cudaDeviceProp prop;
@@ -310,7 +310,7 @@ struct StepArgs {
     // workspace
     __nv_bfloat16 *x0, *qkv, *attn_out, *h;
     float *acc;                      // [2][B][D] FP32, zero on entry and on exit
-    float *hacc;                     // [2][D] FP32 sums of the output projection (batch-1 kernel), zero on entry and exit
+    float *hacc;                     // [2][B][D] FP32 sums of the output projection, zero on entry and on exit
     float *attn_part;
     int *attn_ticket;
     float *amax_val;
@@ -325,8 +325,6 @@ struct StepArgs {
 int launch_linear(Ctx *c, const LinearArgs &a, cudaStream_t st);
 bool step_kernel_supported(const Ctx *c, int batch);
 int launch_step(Ctx *c, const StepArgs &a, cudaStream_t st);
-bool step_b1_supported(const Ctx *c, int batch);
-int launch_step_b1(Ctx *c, const StepArgs &a, cudaStream_t st);
 int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st);
 int launch_mlp(Ctx *c, const MlpArgs &a, cudaStream_t st);
 int launch_embed(Ctx *c, const __nv_bfloat16 *embed, const int32_t *ids, __nv_bfloat16 *x, int batch, cudaStream_t st);

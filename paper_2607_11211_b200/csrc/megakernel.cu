@@ -1,35 +1,53 @@
-// Persistent decode-step kernel: the whole token phase of the model -- embedding gather, then for
-// every layer RMSNorm -> QKV -> attention (Algorithm 3) -> output projection -> RMSNorm -> fused MLP
-// (Algorithm 4), then the final norm, the logits and the greedy argmax -- in ONE cooperative launch,
-// for one or several consecutive tokens.
+// Persistent decode-step kernel (batch <= 8): the whole token phase of the model -- embedding gather, then
+// for every layer RMSNorm -> QKV -> attention (Algorithm 3) -> output projection -> RMSNorm -> fused MLP
+// (Algorithm 4), then the final norm, the logits and the greedy argmax -- in ONE cooperative launch, for one or
+// several consecutive tokens.
 //
-// Why: at batch 1 a layer is ~40 us of HBM streaming cut into four dependent products.  As separate
-// kernels each of them pays a launch, a cold start of its copy pipeline and a drain (~5 us, more for
-// attention), during which HBM idles.  Here one CTA per SM stays resident; a producer warp walks the
-// CTA's share of EVERY weight matrix and K/V tile of the step in order and keeps the shared-memory
-// ring (~190 KB per SM) full, never waiting for anything but free slots; the consumer warps meet at
-// a grid-wide barrier after each product.  While they wait there, or run the latency-bound parts of
-// attention, the bytes of the next product keep arriving, so HBM stays busy across all boundaries.
+// Why: at batch 1 a layer is ~37 us of HBM streaming cut into dependent products.  As separate kernels each of
+// them pays a launch, a cold start of its copy pipeline and a drain, during which HBM idles.  Here one CTA per SM
+// stays resident; a producer warp walks the CTA's share of EVERY weight matrix and K/V tile of the step in
+// order and keeps the shared-memory ring (~190 KB per SM) full, never waiting for anything but free slots; the
+// consumer warps meet at a grid-wide barrier after each phase (one arrival counter in global memory that only
+// grows during a launch; every wait is bounded, and a CTA that gives up pushes the counter beyond every
+// target, so nobody spins forever; the launch is cooperative, so all CTAs are resident).
 //
-// Grid barrier: one arrival counter in global memory that only grows during a launch (the host zeroes it
-// before the launch); every wait is bounded, and a CTA that gives up pushes the counter beyond every target so
-// that nobody spins forever (the launch is cooperative, so all CTAs are resident).
-//
-// Two variants are compiled (template parameter DEFER, chosen by batch size at launch): where the softmax
-// merge of a head shared by several CTAs happens, and how the MLP partial sums are staged.  Code that does not
-// run is kept out of each variant: the kernel is sensitive to its instruction footprint and register pressure.
+// Every grid-wide boundary still costs 4-5 us of dependent latency (barrier, activation loads, norm), so there
+// are THREE per layer, not four: the attention and the output projection are one phase.  Every query
+// head belongs to a fixed group of m0 = n_sm / H_q CTAs.  The group's CTAs split the rows of the head's caches,
+// all sequences of the batch laid end to end, into equal shares whatever the mix of lengths
+// (Algorithm 3 on each share, partial (max, sum, output) published), meet at a counter of their own -- a wait
+// for at most m0 - 1 neighbours instead of the whole grid --, each merges the head's partials, and each then
+// multiplies the merged head output with ITS slice of the output-projection rows: for row tile r the d / 32
+// k blocks of the head are d KB contiguous in the packed W_o, so a ring piece is a handful of such runs.  The
+// products of the 32 heads meet in an FP32 accumulator (red.add); the residual add h = x + attn W_o moves into
+// the prologue of the MLP phase, which also writes h out (one share of its chunks per CTA), as the QKV
+// prologue does for x = h + y of the layer before.
 #include "step_core.cuh"
 
 namespace fasttps {
 
 namespace {
 
-// DEFER: where the softmax merge of a head shared by several CTAs happens.  true (batch <= 2): every CTA only
-// publishes its partials and the prologue of the output projection merges them on the fly -- no ticket chain in
-// the short attention phase.  false: the CTA that finishes a head last merges it, hidden behind the long
-// attention phase of a larger batch, where the merge loads of the prologue would serialise.  Two kernels
-// rather than a run-time switch: code that does not run still costs instruction-cache reach and registers.
-template <int IPW, int DH, bool DEFER>
+// A CTA's share of its head: at most one segment per sequence.
+struct GroupSegs {
+    int n;
+    Segment seg[kMaxNB];
+};
+struct GroupSource {
+    const GroupSegs *p;
+    int i;
+    __device__ __forceinline__ explicit GroupSource(const GroupSegs *p_) : p(p_), i(0) {}
+    __device__ __forceinline__ bool next(Segment &s)
+    {
+        if (i >= p->n) return false;
+        s = p->seg[i++];
+        return true;
+    }
+};
+
+// BC: batch class.  0: batch 1 (the batch loops fold away at compile time), 1: batch 2, 2: batches 3 to 8 (which
+// also selects the staging of the MLP scatter; see mlp_core.cuh).
+template <int IPW, int DH, int BC>
 __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArgs a)
 {
     extern __shared__ __align__(128) unsigned char dsm[];
@@ -38,12 +56,15 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     __shared__ float s_best_val[64];
     __shared__ int s_best_idx[64];
     __shared__ int s_go;
-    __shared__ int s_tables_ready;                               // steps whose attention tables are built
+    __shared__ int s_tables_ready;                               // steps whose attention share is known
     __shared__ LayerPtrs s_layers[kMaxStepLayers];               // the layer table: no global round trip per phase
-    __shared__ SegmentList s_segs;                               // this CTA's attention share for the current step
-    __shared__ unsigned char s_head_n[kMaxSegments];               // CTAs that share head (b, h) in the current step
+    __shared__ GroupSegs s_segs;                                 // this CTA's attention share for the current step
+    __shared__ int s_mprime;                                     // CTAs of a group that hold rows in the current step
+    __shared__ int s_ncta[kMaxNB];                               // partials of (sequence b, this head) in the current step
+    __shared__ __align__(16) __nv_bfloat16 s_outh[kMaxNB * DH];  // the merged outputs of this CTA's head, per sequence
 
-    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    constexpr int KB = DH / 32;                                  // k blocks of a head in the output projection
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3;
     const int cta = blockIdx.x, ncta = gridDim.x;
     if (t == 0) s_tables_ready = 0;
     const MegaLayout lay = mega_layout<DH>(a.D);
@@ -52,21 +73,31 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     float *smem_red = reinterpret_cast<float *>(dsm + lay.red_off);
     AttnScratch<DH> &scratch = *reinterpret_cast<AttnScratch<DH> *>(dsm + lay.scratch_off);
 
-    const int D = a.D, B = a.batch;
+    const int D = a.D, B = BC == 0 ? 1 : a.batch;
+    constexpr bool BIG = BC == 2;
     const int nq = a.n_q_heads * a.head_dim, nkv = a.n_kv_heads * a.head_dim, nqkv = nq + 2 * nkv;
     constexpr int SPT = IPW / kBlocksPerWarpPerSlot;      // ring pieces per 16-row tile
     constexpr int PPO = IPW / 4;                          // ring pieces per W_down octet
     const size_t tile_bytes = (size_t)D * 32;             // 16 rows x D (every reduction length here is D)
     const size_t oct_bytes = (size_t)D * 16;
 
-    // this CTA's share of every product (the same for every layer)
-    int q0, qn, o0, on, m0, mn, l0, ln;
+    // this CTA's share of every grid-wide product (the same for every layer)
+    int q0, qn, m0, mn, l0, ln;
     cta_range((nqkv + 15) >> 4, cta, ncta, q0, qn);
-    cta_range((D + 15) >> 4, cta, ncta, o0, on);
     cta_range(a.K >> 3, cta, ncta, m0, mn);
     cta_range((a.V + 15) >> 4, cta, ncta, l0, ln);
-    int ncta_attn = (kMaxSplits - 2) * a.n_q_heads;
-    if (ncta_attn > ncta) ncta_attn = ncta;
+    // head groups: CTA (head, gs) of gm CTAs per head; the CTAs beyond n_q_heads * gm sit the fused phase out
+    int gm = ncta / a.n_q_heads;
+    if (gm > kMaxSplits) gm = kMaxSplits;
+    const int head = cta / gm, gs = cta - head * gm;
+    const bool in_group = head < a.n_q_heads;
+    int ot0 = 0, ont = 0;                                  // this CTA's row tiles of the output projection
+    if (in_group) cta_range((D + 15) >> 4, gs, gm, ot0, ont);
+    int TP = lay.slot_stride / (KB * kTileBytes);          // row tiles of the output projection per ring piece
+    if (TP > nw) TP = nw;
+    unsigned *grp = a.bar + 64 + (in_group ? head : 0);    // arrivals of this group's partials since the launch
+    float *hacc = a.hacc;                                  // [2][D] FP32 sums of the output projection
+    __nv_bfloat16 *xbuf = a.attn_out;                      // x of the current layer (the attention output tensor is not needed here)
 
     WeightRing ring;
     ring.init(dsm + lay.ring_off, reinterpret_cast<uint64_t *>(dsm + lay.bar_off),
@@ -74,41 +105,9 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     if (t < 64) { s_best_val[t] = -INFINITY; s_best_idx[t] = 0x7fffffff; }
     for (int i = t; i < a.n_layers * (int)(sizeof(LayerPtrs) / 8); i += blockDim.x)
         reinterpret_cast<unsigned long long *>(s_layers)[i] = reinterpret_cast<const unsigned long long *>(a.layers)[i];
-
-    // Per-step attention tables (the lengths grow by one per step, so the split changes with the step, but
-    // not with the layer): the segments of this CTA's share, and for every head the number of CTAs that
-    // publish a partial for it.  Built by the consumer threads at the top of every step, after the barrier that
-    // ends the step before; the producer waits for s_tables_ready before it fetches the step's first K/V tile.
-    auto build_step_tables = [&](int step) {
-        ShareWalk wk;
-        wk.init(a.seq_lens, a.pos, step, B, a.n_q_heads, a.max_seq, cta, ncta_attn);
-        if (t == 0) {
-            int n = 0;
-            Segment sg;
-            while (wk.next(sg) && n < kMaxSegments) {
-                PackedSegment p;
-                p.r0 = sg.r0; p.r1 = sg.r1; p.bh = (unsigned short)(sg.b * a.n_q_heads + sg.h);
-                p.first_cta = (unsigned char)sg.first_cta; p.n_cta = (unsigned char)sg.n_cta;
-                s_segs.seg[n++] = p;
-            }
-            s_segs.n = n; s_segs.n_q_heads = a.n_q_heads;
-            for (int bb = 0; bb < B; ++bb) { s_segs.len[bb] = wk.rows_of(bb) - 1; s_segs.pos[bb] = a.pos[bb] + step; }
-        } else {
-            long long head0 = 0;
-            int b = 0, rows = wk.rows_of(0);
-            for (int idx = t - 1; idx < B * a.n_q_heads; idx += nct - 1) {
-                const int bb = idx / a.n_q_heads, hh = idx - bb * a.n_q_heads;
-                while (b < bb) { head0 += (long long)a.n_q_heads * rows; ++b; rows = wk.rows_of(b); }
-                const long long h0 = head0 + (long long)hh * rows;
-                s_head_n[idx] = rows > 0 ? (unsigned char)(wk.owner_of(h0 + rows - 1) - wk.owner_of(h0) + 1) : 0;
-            }
-        }
-    };
     __syncthreads();
 
     // =========================================================================== producer warp
-    // One thread walks this CTA's share of every weight matrix and K/V tile of every step, in the order the
-    // consumers need it, copies piece after piece into the shared-memory ring and blocks only on free slots.
     if (w >= nw) {
         if (w > nw || lane != 0) return;
         const uint32_t wp = (uint32_t)lay.wpiece;
@@ -124,10 +123,9 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                 const LayerPtrs &lp = s_layers[l];
                 if (!weights(lp.w_qkv, (size_t)q0 * tile_bytes, qn * SPT)) return;
                 if (l == 0) {
-                    // K/V tiles of this step include the rows appended by the step before it, and the share
-                    // table is rebuilt per step: both are ready once the consumers have passed the barrier
-                    // that ends that step and built the table (weights are never held back).  For all but
-                    // toy models the flag is set long before the producer gets here.
+                    // K/V tiles of this step include the row appended by the step before it, and the share is
+                    // recomputed per step: both are ready once the consumers have passed the barrier that ends
+                    // that step (weights are never held back)
                     const unsigned long long t0 = global_ns();
                     while (*reinterpret_cast<volatile int *>(&s_tables_ready) <= step) {
                         if (*ring.abort_flag || global_ns() - t0 > kGridWaitNanos) { *ring.abort_flag = 1; return; }
@@ -135,13 +133,24 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                     }
                     __threadfence_block();
                 }
-                const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
-                const bool kv_ok = attn_for_each_tile<DH>(aa, ListSource(&s_segs),
+                const AttnArgs aa = attn_args_of(a, lp, step, gm * a.n_q_heads);
+                const bool kv_ok = attn_for_each_tile<DH>(aa, GroupSource(&s_segs),
                                                           [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
                     return ring.put2(piece++, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
                 });
                 if (!kv_ok) return;
-                if (!weights(lp.w_o, (size_t)o0 * tile_bytes, on * SPT)) return;
+                // this CTA's rows of the output projection, the head's k blocks only: KB KB per row tile
+                const unsigned char *wo = reinterpret_cast<const unsigned char *>(lp.w_o);
+                for (int p0 = 0; p0 < ont; p0 += TP, ++piece) {
+                    const int nt = ont - p0 < TP ? ont - p0 : TP;
+                    if (!ring.acquire(piece)) return;
+                    const int sl = piece % ring.nslot;
+                    mbar_expect_tx(&ring.full[sl], (uint32_t)(nt * KB * kTileBytes));
+                    for (int j = 0; j < nt; ++j)
+                        bulk_g2s(ring.slots + (size_t)sl * ring.slot_bytes + (size_t)j * KB * kTileBytes,
+                                 wo + ((size_t)(ot0 + p0 + j) * (nq / 32) + (size_t)head * KB) * kTileBytes,
+                                 (uint32_t)(KB * kTileBytes), &ring.full[sl]);
+                }
                 if (!weights(lp.w_gu, (size_t)m0 * tile_bytes, mn * SPT)) return;
                 if (!weights(lp.w_down, (size_t)m0 * oct_bytes, mn * PPO)) return;
             }
@@ -155,6 +164,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     gb.count = a.bar; gb.status = a.status;
     gb.ncta = ncta; gb.s_go = &s_go;
     gb.target = (unsigned)ncta;
+    unsigned grp_target = 0;
     if (cta == 0 && t == 0) {
         // sequences that cannot be served for all steps are reported once and contribute no rows
         for (int bb = 0; bb < B; ++bb) {
@@ -165,7 +175,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     }
 
     // gathers the embedding rows of the current tokens into x0 (CTA 0 only)
-    auto embed_rows = [&](const int32_t *ids) {
+    auto embed_row = [&](const int32_t *ids) {
         for (int idx = t; idx < B * (D >> 3); idx += nct) {
             const int b = idx / (D >> 3), j = idx - b * (D >> 3);
             int id = ld_cg_s32(ids + b);
@@ -182,26 +192,10 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     // after every grid barrier
     int n_stamp = 0;
     auto stamp = [&]() {
-#ifdef FASTTPS_FINE_TRACE
-        if (a.trace && t == 0 && cta == 0 && n_stamp < a.trace_len)
-#else
         if (a.trace && t == 0 && (cta == 0 || cta == ncta - 1) && n_stamp < a.trace_len)
-#endif
             a.trace[(size_t)(cta ? 1 : 0) * a.trace_len + n_stamp] = global_ns();
         ++n_stamp;
     };
-#ifdef FASTTPS_FINE_TRACE
-    // development build: CTA 0 also stamps, into the second half of the buffer, the end of every product's
-    // prologue and of its tile loop (two stamps per product phase, none for attention)
-    int n_fine = 0;
-    auto fine = [&]() {
-        if (a.trace && t == 0 && cta == 0 && n_fine < a.trace_len) a.trace[(size_t)a.trace_len + n_fine] = global_ns();
-        ++n_fine;
-    };
-#define FT_FINE() fine()
-#else
-#define FT_FINE() ((void)0)
-#endif
     auto sync_phase = [&]() -> bool {
         stamp();
         const bool go = grid_sync(gb, nct, /*ok=*/ok);
@@ -209,73 +203,183 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
         return go;
     };
 
-    if (cta == 0) embed_rows(a.token_ids);
+    if (cta == 0) embed_row(a.token_ids);
     if (!sync_phase()) return;
 
-    // One loop over all products of a step.  Every matrix product (QKV, output projection, gate_up, logits)
-    // goes through the SAME copy of the B-fragment prologue and of the tile loop, selected by `kind`: the hot
-    // code of the kernel stays small enough to live in the instruction cache from one product to the next.
-    enum { kQkv = 0, kAttn = 1, kOproj = 2, kMlp = 3, kHead = 4 };
+    enum { kQkv = 0, kAttn = 1, kMlp = 2, kHead = 3 };
     const int L = a.n_layers;
     for (int step = 0; step < a.n_steps; ++step) {
-        build_step_tables(step);
+        // ---- this step's attention share: the rows of the head, all sequences end to end, are cut into m'
+        // equal shares, one per CTA of the group (at least 16 rows each) ----
+        if (t == 0) {
+            int R[kMaxNB];
+            long long T = 0;
+            for (int bb = 0; bb < B; ++bb) {
+                const int Ls = a.seq_lens[bb] + step, ps = a.pos[bb] + step;
+                const bool valid = !(Ls < step || Ls >= a.max_seq || ps < step || ps >= a.max_seq);
+                R[bb] = valid ? Ls + 1 : 0;
+                T += R[bb];
+            }
+            int mp = (int)(T / 16 < gm ? T / 16 : gm);
+            mp = T == 0 ? 0 : (mp < 1 ? 1 : mp);
+            s_mprime = mp;
+            const long long f0 = mp ? T * gs / mp : 0, f1 = (mp && gs < mp) ? T * (gs + 1) / mp : f0;
+            auto owner = [&](long long x) {                    // the share that holds row x of the head
+                int c = 0;
+                while (c + 1 < mp && T * (c + 1) / mp <= x) ++c;
+                return c;
+            };
+            int n = 0;
+            long long off = 0;
+            for (int bb = 0; bb < B; ++bb) {
+                const int rb = R[bb];
+                s_ncta[bb] = 0;
+                if (rb > 0) {
+                    const int first = owner(off), last = owner(off + rb - 1);
+                    s_ncta[bb] = last - first + 1;
+                    const long long lo = f0 > off ? f0 : off, hi = f1 < off + rb ? f1 : off + rb;
+                    if (in_group && lo < hi) {
+                        Segment &sg = s_segs.seg[n++];
+                        sg.b = bb; sg.h = head; sg.L = rb - 1; sg.pos = a.pos[bb] + step;
+                        sg.r0 = (int)(lo - off); sg.r1 = (int)(hi - off);
+                        sg.first_cta = head * gm + first; sg.n_cta = last - first + 1;
+                    }
+                }
+                off += rb;
+            }
+            s_segs.n = n;
+        }
         named_bar_sync(1, nct);
         if (t == 0) {
             __threadfence_block();
             atomicExch(&s_tables_ready, step + 1);              // the producer may fetch this step's K/V rows now
         }
-        for (int ph = 0; ph <= 4 * L; ++ph) {
-            const int l = ph >> 2;
-            const int kind = ph == 4 * L ? kHead : (ph & 3);
-            const LayerPtrs &lp = s_layers[l < L ? l : L - 1];
-            const int lprev = (kind == kHead ? L : l) - 1;                               // layer whose MLP sums feed x
-            const float *y_prev = lprev >= 0 ? a.acc + (size_t)(lprev & 1) * B * D : nullptr;
-            const __nv_bfloat16 *x_base = lprev >= 0 ? a.h : a.x0;                      // x = bf16(x_base + y_prev)
+        const int mprime = s_mprime;
 
-            // The gains of the norm two phases ahead are asked from L2 now (they come from HBM once per step):
-            // one CTA, one thread per 128-byte line.
-            if (cta == ncta - 1 && (kind == kAttn || kind == kMlp) && t * 64 < D) {
-                const __nv_bfloat16 *gnext = kind == kAttn ? lp.g_mlp : (l + 1 < L ? s_layers[l + 1].g_attn : a.g_final);
+        for (int ph = 0; ph <= 3 * L; ++ph) {
+            const int l = ph / 3;
+            const int kind = ph == 3 * L ? kHead : ph - 3 * l;
+            const LayerPtrs &lp = s_layers[l < L ? l : L - 1];
+
+            // The gains of the norm after next are asked from L2 now (they come from HBM once per step)
+            if (cta == ncta - 1 && (kind == kQkv || kind == kAttn) && t * 64 < D) {
+                const __nv_bfloat16 *gnext = kind == kQkv ? lp.g_mlp : (l + 1 < L ? s_layers[l + 1].g_attn : a.g_final);
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(gnext + t * 64));
             }
+
             if (kind == kAttn) {
-                // ---- attention (Algorithm 3) ----
-                const AttnArgs aa = attn_args_of(a, lp, step, ncta_attn);
-                // every CTA publishes the partial (max, sum, output) of each of its segments; nobody merges
-                // here: the output projection merges while it builds its B fragments
-                ok = attn_consume<DH, DEFER>(aa, ring, piece, cta, ListSource(&s_segs), scratch, nw) && ok;
-            } else {
-                // ---- a matrix product: B fragments, then this CTA's row tiles ----
-                const __nv_bfloat16 *src = x_base, *gain = nullptr;
-                const float *add = y_prev;
-                int tile0 = 0, ntile = 0;
-                if (kind == kQkv) { gain = lp.g_attn; tile0 = q0; ntile = qn; }
-                else if (kind == kOproj) { src = a.attn_out; add = nullptr; tile0 = o0; ntile = on; }
-                else if (kind == kMlp) { src = a.h; add = nullptr; gain = lp.g_mlp; tile0 = m0; ntile = mn; }
-                else { gain = a.g_final; tile0 = l0; ntile = ln; }
-                // residual of the output projection for the first two tiles (all there are on a full grid),
-                // fetched by the epilogue threads now instead of in the epilogue, where the tile loop would wait
-                float res[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-                const bool res_pre = kind == kOproj && nct >= 64 && t < 64 && (t & 7) < B;
-                if (res_pre) {
-                    __nv_bfloat16 xb[2][2];
-                    float ya[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        int row = (o0 + (q >> 1)) * 16 + (t >> 3) + 8 * (q & 1);
-                        if (row >= D) row = D - 1;
-                        xb[q >> 1][q & 1] = ld_cg_bf16(x_base + (size_t)(t & 7) * D + row);
-                        if (y_prev) ya[q >> 1][q & 1] = ld_cg_f32(y_prev + (size_t)(t & 7) * D + row);
+                // ---- attention (Algorithm 3) on this CTA's rows of its head; the partial is published ----
+                const AttnArgs aa = attn_args_of(a, lp, step, gm * a.n_q_heads);
+                ok = attn_consume<DH, true>(aa, ring, piece, cta, GroupSource(&s_segs), scratch, nw) && ok;
+                grp_target += (unsigned)mprime;
+                if (in_group) {
+                    // ---- the group meets: every CTA of it needs the merged output of the head ----
+                    __threadfence();
+                    named_bar_sync(1, nct);
+                    if (t == 0) {
+                        if (s_segs.n && ok) atomicAdd(grp, 1u);
+                        int met = 1;
+                        unsigned long long t0 = 0;
+                        for (unsigned it = 1; ld_acquire_u32(grp) < grp_target; ++it) {
+                            if ((it & 63u) == 0) {
+                                const unsigned long long now = global_ns();
+                                if (t0 == 0) t0 = now;
+                                else if (now - t0 > kGridWaitNanos) { met = 0; break; }
+                            }
+                        }
+                        s_go = met;
                     }
+                    named_bar_sync(1, nct);
+                    if (!s_go) ok = false;
+                    // ---- softmax merge of the head's partials: out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s ----
+                    constexpr int PS = DH + 4;
+                    for (int idx = t; idx < B * DH; idx += nct) {
+                        const int b = idx / DH, i = idx - b * DH;
+                        const int np = s_ncta[b];
+                        const float *hp = a.attn_part + ((size_t)b * a.n_q_heads + head) * kMaxSplits * PS;
+                        float M = -INFINITY, den = 0.f, o = 0.f;
+                        for (int s0 = 0; s0 < np; s0 += 4) {
+                            float ms[4], ls[4], os[4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float x = __bfloat162float(xb[q >> 1][q & 1]);
-                        res[q >> 1][q & 1] = y_prev ? bf16_round(x + ya[q >> 1][q & 1]) : x;
+                            for (int u = 0; u < 4; ++u) {
+                                const bool have = s0 + u < np;
+                                const float *p = hp + (size_t)(have ? s0 + u : 0) * PS;
+                                ms[u] = ld_cg_f32(p + DH);
+                                ls[u] = ld_cg_f32(p + DH + 1);
+                                os[u] = ld_cg_f32(p + i);
+                                if (!have) ms[u] = -INFINITY;
+                            }
+                            float Mn = M;
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) Mn = fmaxf(Mn, ms[u]);
+                            const float corr = fast_exp2(M - Mn);        // 0 in the first round (M = -inf)
+                            den *= corr; o *= corr;
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const float f = ms[u] == -INFINITY ? 0.f : fast_exp2(ms[u] - Mn);
+                                den = fmaf(f, ls[u], den);
+                                o = fmaf(f, os[u], o);
+                            }
+                            M = Mn;
+                        }
+                        s_outh[idx] = __float2bfloat16_rn(np > 0 && ok ? o / den : 0.f);
+                    }
+                    named_bar_sync(1, nct);
+                    // ---- this CTA's row tiles of the output projection, k = the head: sums go to hacc[l & 1] ----
+                    uint4 bh[KB];
+#pragma unroll
+                    for (int j = 0; j < KB; ++j)
+                        bh[j] = g < B ? *reinterpret_cast<const uint4 *>(s_outh + g * DH + 32 * j + 8 * t4) : make_uint4(0u, 0u, 0u, 0u);
+                    float *hsum = hacc + (size_t)(l & 1) * B * D;
+                    for (int p0 = 0; p0 < ont; p0 += TP, ++piece) {
+                        const int nt = ont - p0 < TP ? ont - p0 : TP;
+                        const unsigned char *slot = ring.wait(piece, ok);
+                        if (w < nt) {
+                            float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                            for (int j = 0; j < KB; ++j) {
+                                const unsigned char *blk = slot + (size_t)(w * KB + j) * kTileBytes + lane * 16;
+                                const uint4 lo = *reinterpret_cast<const uint4 *>(blk);
+                                const uint4 hi = *reinterpret_cast<const uint4 *>(blk + 512);
+                                mma_bf16_k16(c, lo.x, hi.x, lo.y, hi.y, bh[j].x, bh[j].y);
+                                mma_bf16_k16(c, lo.z, hi.z, lo.w, hi.w, bh[j].z, bh[j].w);
+                            }
+                            // accumulator fragment: rows g / g + 8 of the tile, batch rows 2 t4 / 2 t4 + 1
+                            const int row = (ot0 + p0 + w) * 16 + g, b0 = 2 * t4;
+                            if (ok && b0 < B) {
+                                if (row < D) atomicAdd(hsum + (size_t)b0 * D + row, c[0]);
+                                if (row + 8 < D) atomicAdd(hsum + (size_t)b0 * D + row + 8, c[2]);
+                            }
+                            if (ok && b0 + 1 < B) {
+                                if (row < D) atomicAdd(hsum + (size_t)(b0 + 1) * D + row, c[1]);
+                                if (row + 8 < D) atomicAdd(hsum + (size_t)(b0 + 1) * D + row + 8, c[3]);
+                            }
+                        }
+                        ring.release(piece);
                     }
                 }
-                if (DEFER && kind == kOproj) load_b_frags_attn<IPW, DH>(bf, a.attn_part, s_head_n, B, a.n_q_heads, nw);
-                else load_b_frags<IPW>(bf, src, D, B, D, nw, gain, a.eps, smem_red, add);
-                FT_FINE();
+            } else {
+                // ---- a grid-wide matrix product: B fragments, then this CTA's row tiles ----
+                const __nv_bfloat16 *src, *gain;
+                const float *add;
+                __nv_bfloat16 *store = nullptr;
+                int tile0, ntile;
+                if (kind == kQkv) {                          // x_l = h_{l-1} + y_{l-1} (layer 0: the embedding row)
+                    src = l == 0 ? a.x0 : a.h; add = l == 0 ? nullptr : a.acc + (size_t)((l - 1) & 1) * B * D;
+                    gain = lp.g_attn; store = l == 0 ? nullptr : xbuf; tile0 = q0; ntile = qn;
+                } else if (kind == kMlp) {                   // h_l = x_l + attn . W_o
+                    src = l == 0 ? a.x0 : xbuf; add = hacc + (size_t)(l & 1) * B * D;
+                    gain = lp.g_mlp; store = a.h; tile0 = m0; ntile = mn;
+                } else {                                     // x_L = h_{L-1} + y_{L-1}
+                    src = a.h; add = a.acc + (size_t)((L - 1) & 1) * B * D;
+                    gain = a.g_final; tile0 = l0; ntile = ln;
+                }
+                // the sums of the output projection of the layer before are consumed: back to zero
+                if (cta == ncta - 1 && ((kind == kQkv && l > 0) || kind == kHead)) {
+                    float *z = hacc + (size_t)((l - 1) & 1) * B * D;   // (head: l = L)
+                    for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                load_b_frags<IPW>(bf, src, D, B, D, nw, gain, a.eps, smem_red, add, store, cta, ncta);
                 if (kind == kHead) {
                     for (int u = t; u < 64; u += nct) { s_best_val[u] = -INFINITY; s_best_idx[u] = 0x7fffffff; }
                     named_bar_sync(1, nct);
@@ -295,16 +399,6 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                         const float v = hh ? v1 : v0;
                         if (kind == kQkv) {
                             if (row < nqkv) a.qkv[(size_t)b * nqkv + row] = __float2bfloat16_rn(v);
-                        } else if (kind == kOproj) {         // h = x_l + attn . W_o
-                            if (row < D) {
-                                float x;
-                                if (res_pre && tile < 2) x = tile == 0 ? res[0][hh] : res[1][hh];
-                                else {
-                                    x = __bfloat162float(ld_cg_bf16(x_base + (size_t)b * D + row));
-                                    if (y_prev) x = bf16_round(x + ld_cg_f32(y_prev + (size_t)b * D + row));
-                                }
-                                a.h[(size_t)b * D + row] = __float2bfloat16_rn(x + v);
-                            }
                         } else if (row < a.V) {              // logits and the running argmax of this thread's rows
                             const int u = cc * 8 + b;
                             if (a.logits) a.logits[(size_t)b * a.V + row] = v;
@@ -313,12 +407,11 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                     }
                 }) && ok;
                 piece += ntile * SPT;
-                FT_FINE();
 
                 if (kind == kMlp) {
                     // ---- down projection of this CTA's octets; the sums of all CTAs meet in acc[l & 1] ----
-                    if (cta == 0 && y_prev) {
-                        // layer l - 1's sums have been consumed by everyone (two barriers ago): zero them for layer l + 1
+                    if (cta == 0 && l > 0) {
+                        // layer l - 1's sums were consumed by the QKV prologue of this layer: zero them for layer l + 1
                         float *z = a.acc + (size_t)((l - 1) & 1) * B * D;
                         for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
@@ -332,7 +425,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                             for (int e = 0; e < 4; ++e) acc[i][m][e] = 0.f;
                     mlp_down_phase<IPW>(ring, piece, mn, nw, s_hi, s_lo, acc, ok);
                     piece += mn * PPO;
-                    mlp_scatter_add<IPW, !DEFER>(acc, smem_part, a.acc + (size_t)(l & 1) * B * D, B, D, nw);
+                    mlp_scatter_add<IPW, BIG>(acc, smem_part, a.acc + (size_t)(l & 1) * B * D, B, D, nw);
                 } else if (kind == kHead) {
                     named_bar_sync(1, nct);
                     if (t < 8 && t < B) {
@@ -388,7 +481,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
             if (step + 1 < a.n_steps) {
                 __threadfence();
                 named_bar_sync(1, nct);
-                embed_rows(a.tok);
+                embed_row(a.tok);
             }
         }
         if (step + 1 < a.n_steps && !sync_phase()) return;
@@ -397,11 +490,11 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
 
 }  // namespace
 
-template <int IPW, int DH, bool DEFER>
+template <int IPW, int DH, int BC>
 static int launch_step_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
 {
     const MegaLayout lay = mega_layout<DH>(a.D);
-    auto kernel = decode_step_kernel<IPW, DH, DEFER>;
+    auto kernel = decode_step_kernel<IPW, DH, BC>;
     static bool configured[16] = {};
     if (!configured[c->cfg.device & 15]) {
         FT_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemMax));
@@ -410,10 +503,10 @@ static int launch_step_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
         if (per_sm < 1) return FASTTPS_INVALID_ARG;
         configured[c->cfg.device & 15] = true;
     }
-    if ((unsigned long long)(4 * a.n_layers + 3) * (unsigned long long)a.n_steps * (unsigned long long)c->n_sm >= kBarAbort)
+    if ((unsigned long long)(3 * a.n_layers + 3) * (unsigned long long)a.n_steps * (unsigned long long)c->n_sm >= kBarAbort)
         return FASTTPS_INVALID_ARG;                      // the arrival counter must stay below the abort mark
-    // the barrier counter starts from zero every launch
-    FT_CUDA(cudaMemsetAsync(c->grid_bar, 0, 64 * sizeof(unsigned), st));
+    // the barrier counter and the group counters start from zero every launch
+    FT_CUDA(cudaMemsetAsync(c->grid_bar, 0, kGridBarWords * sizeof(unsigned), st));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c->n_sm); cfg.blockDim = dim3((lay.nw + 1) * 32); cfg.dynamicSmemBytes = lay.total; cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -435,20 +528,20 @@ bool step_kernel_supported(const Ctx *c, int batch)
     if (batch < 1 || batch > kMaxNB) return false;
     if (f.n_q_heads * f.head_dim != f.hidden) return false;      // one reduction length for every product
     if (s.nw < 1 || s.nw > 12) return false;
-    if (f.n_q_heads > kMaxStepHeads || f.n_layers > kMaxStepLayers) return false;
-    if (batch * f.n_q_heads >= kMaxSegments || c->n_sm > 255) return false;   // segment table: capacity, 8-bit CTA index
-    if (f.vocab < 1 || f.n_layers < 1) return false;
+    if (f.n_q_heads > kMaxStepHeads || f.n_q_heads > c->n_sm) return false;   // a group of at least one CTA per query head
+    if (f.n_layers > kMaxStepLayers || f.vocab < 1 || f.n_layers < 1) return false;
     return true;
 }
 
 int launch_step(Ctx *c, const StepArgs &a, cudaStream_t st)
 {
     const int ipw = warp_split(a.D).ipw;
-    const bool defer = a.batch <= 2;
-#define FT_STEP(DHV)                                                                                     \
+    const int bc = a.batch == 1 ? 0 : (a.batch == 2 ? 1 : 2);
+#define FT_STEP(DHV)                                                                                  \
     case DHV:                                                                                            \
-        if (defer) return ipw == 8 ? launch_step_inst<8, DHV, true>(c, a, st) : launch_step_inst<4, DHV, true>(c, a, st); \
-        return ipw == 8 ? launch_step_inst<8, DHV, false>(c, a, st) : launch_step_inst<4, DHV, false>(c, a, st)
+        if (bc == 2) return ipw == 8 ? launch_step_inst<8, DHV, 2>(c, a, st) : launch_step_inst<4, DHV, 2>(c, a, st); \
+        if (bc == 1) return ipw == 8 ? launch_step_inst<8, DHV, 1>(c, a, st) : launch_step_inst<4, DHV, 1>(c, a, st); \
+        return ipw == 8 ? launch_step_inst<8, DHV, 0>(c, a, st) : launch_step_inst<4, DHV, 0>(c, a, st)
     switch (a.head_dim) {
         FT_STEP(32);
         FT_STEP(64);

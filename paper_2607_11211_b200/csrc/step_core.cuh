@@ -12,7 +12,7 @@ constexpr unsigned long long kGridWaitNanos = 500ull * 1000 * 1000;   // 0.5 s p
 // registers each) hosts four warps: 128 registers per thread is the most a CTA of this size can be given.
 constexpr int kMegaThreadsMax = 416;
 constexpr int kMaxStepLayers = 48;                                     // layers the shared-memory layer table holds
-constexpr int kMaxStepHeads = 128;                                     // query heads the per-step head table holds
+constexpr int kMaxStepHeads = 128;                                     // query heads: one group counter each
 
 static __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
 {

@@ -4,7 +4,7 @@
 
 Runs a greedy multi-step decode of a Phi-3-mini-shaped stack (synthetic seeded weights and caches) in one
 launch of the step kernel and prints, for the LAST step of the launch, how long the first and the last CTA
-spent in each phase of a layer (QKV product, attention, output projection, fused MLP) and how long they then
+spent in each phase of a layer (QKV product, attention + output projection, fused MLP) and how long they then
 waited at the grid-wide barrier that closes the phase.  The stamps come from fasttps_trace_read(): the two
 CTAs read the GPU global timer immediately before and after every barrier.
 """
@@ -25,15 +25,13 @@ def main():
     ap.add_argument("--past", type=int, default=1024)
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--steps", type=int, default=4)
-    ap.add_argument("--step-kernel", type=int, default=1, help="1: step kernel with head groups; 2: general step kernel")
     args = ap.parse_args()
     dm, B, NL, NS = wl.PHI3_MINI, args.batch, args.layers, args.steps
     dev = torch.device("cuda", 0)
     max_seq = args.past + NS + 2
     ctx = fb.Context.from_dims(dm, B, max_seq, n_layers=NL)
-    ctx.set_option("step_kernel", args.step_kernel)
-    # the kernel with head groups has three phases per layer (attention and output projection are one), the general one four
-    names = ("qkv", "attn+o_proj", "mlp") if args.step_kernel == 1 else ("qkv", "attn", "o_proj", "mlp")
+    ctx.set_option("step_kernel", 1)
+    names = ("qkv", "attn+o_proj", "mlp")                  # three phases per layer: attention and output projection are one
     P = len(names)
     seed = wl.MASTER_SEED
     layers = [ctx.pack_layer(wl.layer_weights(dm, i, seed, device=dev)) for i in range(NL)]
