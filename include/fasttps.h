@@ -177,7 +177,7 @@ int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const
  *   one at the end of the step iff advance != 0;
  *   logits [B,V] float device or NULL (an internal buffer is used);
  *   next_ids [B] int32 device (may be the same buffer as token_ids).
- * For batch <= 8 (and n_q_heads * head_dim == hidden, n_q_heads <= 128, batch * n_q_heads <= 256,
+ * For batch <= 8 (and n_q_heads * head_dim == hidden, n_q_heads <= 128 and <= the number of SMs,
  * n_layers <= 48) the whole step is ONE cooperative
  * launch of a persistent kernel (one CTA per SM, grid-wide barriers between the products,
  * weights and K/V streamed ahead through shared memory across all boundaries); larger
