@@ -495,13 +495,15 @@ static int launch_step_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
 {
     const MegaLayout lay = mega_layout<DH>(a.D);
     auto kernel = decode_step_kernel<IPW, DH, BC>;
-    static bool configured[16] = {};
-    if (!configured[c->cfg.device & 15]) {
-        FT_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmemMax));
+    // the dynamic shared memory this instantiation has been allowed so far, per device (its static arrays
+    // come on top: the opt-in is for what the model shape needs, not for the maximum)
+    static size_t configured[16] = {};
+    if (configured[c->cfg.device & 15] < lay.total) {
+        FT_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lay.total));
         int per_sm = 0;
         FT_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, (lay.nw + 1) * 32, lay.total));
         if (per_sm < 1) return FASTTPS_INVALID_ARG;
-        configured[c->cfg.device & 15] = true;
+        configured[c->cfg.device & 15] = lay.total;
     }
     if ((unsigned long long)(3 * a.n_layers + 3) * (unsigned long long)a.n_steps * (unsigned long long)c->n_sm >= kBarAbort)
         return FASTTPS_INVALID_ARG;                      // the arrival counter must stay below the abort mark
