@@ -517,3 +517,53 @@ def test_model_generate_stops_at_the_end_of_the_cache(fb):
     for l in range(dims.n_layers):                       # nothing outside the rows this launch may touch has changed
         assert torch.equal(kcs[l][:, :, :12].view(torch.int16), k0[l][:, :, :12].view(torch.int16))
     ctx.close()
+
+
+# ------------------------------------------------- true Gaussian inputs (nothing depends on the generator)
+
+def gaussian_bits(rng, shape, scale=1.0, offset=0.0):
+    v = rng.standard_normal(int(np.prod(shape)), dtype=np.float32) * np.float32(scale) + np.float32(offset)
+    return orc.f32_to_bf16(v).reshape(shape)
+
+
+@pytest.mark.parametrize("dims,lens", [(wl.SMALL, [40, 7, 100]), (wl.SMALL_GQA, [33])])
+@pytest.mark.parametrize("step_kernel", [0, 1])
+def test_model_decode_with_host_generated_gaussian_inputs(fb, dims, lens, step_kernel):
+    """The seeded generator is a sum of uniforms; here every tensor comes from numpy's normal generator on the
+    host instead (unbounded tails, exact Gaussian shape) and is uploaded: same bars as everywhere else."""
+    rng = np.random.default_rng(20260711)
+    batch, max_seq = len(lens), 128
+    D, K, d, Hq, Hkv = dims.hidden, dims.inter, dims.head_dim, dims.n_q_heads, dims.n_kv_heads
+    ctx = make_ctx(fb, dims, batch, max_seq)
+    ctx.set_option("step_kernel", step_kernel)
+    ow, packed, kcs, vcs, ok, ov = [], [], [], [], [], []
+    for _ in range(dims.n_layers):
+        w = dict(g_attn=gaussian_bits(rng, (D,), 0.02, 1.0), w_qkv=gaussian_bits(rng, (D, dims.qkv_out), 0.02),
+                 w_o=gaussian_bits(rng, (Hq * d, D), 0.02), g_mlp=gaussian_bits(rng, (D,), 0.02, 1.0),
+                 w_gu=gaussian_bits(rng, (D, 2 * K), 0.02), w_down=gaussian_bits(rng, (K, D), 0.02))
+        ow.append(w)
+        packed.append(ctx.pack_layer({k: dev(v) for k, v in w.items()}))
+        kb, vb = gaussian_bits(rng, (batch, Hkv, max_seq, d)), gaussian_bits(rng, (batch, Hkv, max_seq, d))
+        ok.append(kb); ov.append(vb)
+        kcs.append(dev(kb)); vcs.append(dev(vb))
+    emb, gf, wlm = gaussian_bits(rng, (dims.vocab, D), 0.02), gaussian_bits(rng, (D,), 0.02, 1.0), gaussian_bits(rng, (dims.vocab, D), 0.02)
+    model = ctx.make_model(dev(emb), packed, dev(gf), ctx.pack_weight(fb.W_LM_HEAD, dev(wlm)), kcs, vcs)
+    ids = rng.integers(0, dims.vocab, size=batch).astype(np.int32)
+    lens = np.asarray(lens, np.int32)
+    logits = torch.zeros(batch, dims.vocab, dtype=torch.float32, device="cuda")
+    nxt = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    ctx.model_decode(model, i32(ids), i32(lens), i32(lens), logits, nxt, advance=False)
+    torch.cuda.synchronize()
+    assert ctx.get_status() == 0
+    k0 = [a.copy() for a in ok]
+    wlog, wnext = orc.model_decode(emb, ow, gf, wlm, ok, ov, ids, lens.copy(), lens.copy(), dims.rms_eps, dims.rope_theta)
+    got = logits.cpu().numpy().astype(np.float64)
+    assert (np.abs(got - wlog) <= 2e-2 + 2e-2 * np.abs(wlog)).all()
+    for l in range(dims.n_layers):
+        kg = wl.bits(kcs[l])
+        mask = np.ones(kg.shape, bool)
+        for b in range(batch):
+            mask[b, :, lens[b]] = False
+            assert_close_bits(kg[b, :, lens[b]], ok[l][b, :, lens[b]], what="k row")
+        assert (kg[mask] == k0[l][mask]).all()
+    ctx.close()
