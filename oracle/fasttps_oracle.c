@@ -31,9 +31,9 @@
  * square root of RMSNorm; pre-norm residual connections; no biases; lowest
  * index wins an argmax tie.
  *
- * Parity pins: see tests/test_oracle_*.py (closed forms, invariants, brute
- * force at tiny sizes, golden values written by an independent pure-Python
- * script).  Against the authors' own implementation the oracle is
+ * Parity pins: see tests/test_oracle_pins.py (closed forms, invariants,
+ * special cases, brute force at tiny sizes against sums expanded in plain
+ * Python floats).  Against the authors' own implementation the oracle is
  * "parity unpinned": the paper prints no numeric example of the method.
  *
  * Build: gcc -O2 -fopenmp -ffp-contract=off -shared -fPIC -o liboracle.so fasttps_oracle.c -lm
