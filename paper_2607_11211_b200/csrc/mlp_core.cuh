@@ -108,6 +108,21 @@ __device__ __forceinline__ void mlp_scatter_add_block(const float (&acc)[IPW][2]
 }
 
 
+// One round of mlp_scatter_add_warp: the warp's staged rows go to global memory.  Out of line: the caller is
+// unrolled over the chunks and would carry a copy of this loop for each of them.
+static __device__ __noinline__ void mlp_scatter_drain_warp(const float *st, float *acc_g, int i0, int nrow, int batch, int D,
+                                                           int nw)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    __syncwarp();
+    for (int idx = lane; idx < nrow * 8; idx += 32) {
+        const int row = idx >> 3, j = idx & 7;
+        const int ch = row / batch, b = row - ch * batch;
+        const float4 v = *reinterpret_cast<const float4 *>(st + row * 32 + (((j ^ row) & 7) << 2));
+        red_add_v4(acc_g + (size_t)b * D + 32 * (nw * (i0 + ch) + w) + 4 * j, v.x, v.y, v.z, v.w);
+    }
+}
+
 // The same scatter for larger batches, where the block-wide version would need two block-wide barriers per
 // value of i.  For a given i a
 // warp owns 32 contiguous output columns, 32 (nw i + w) .. + 32, so the transposition from fragment order to
@@ -136,16 +151,7 @@ __device__ __forceinline__ void mlp_scatter_add_warp(const float (&acc)[IPW][2][
                 if (b < batch) st[row * 32 + ((((n >> 2) ^ row) & 7) << 2) + (n & 3)] = acc[i][m][e];
             }
         }
-        if (ir == R - 1 || i == IPW - 1) {
-            __syncwarp();
-            const int i0 = i - ir, nrow = (ir + 1) * batch;
-            for (int idx = lane; idx < nrow * 8; idx += 32) {
-                const int row = idx >> 3, j = idx & 7;
-                const int ch = row / batch, b = row - ch * batch;
-                const float4 v = *reinterpret_cast<const float4 *>(st + row * 32 + (((j ^ row) & 7) << 2));
-                red_add_v4(acc_g + (size_t)b * D + 32 * (nw * (i0 + ch) + w) + 4 * j, v.x, v.y, v.z, v.w);
-            }
-        }
+        if (ir == R - 1 || i == IPW - 1) mlp_scatter_drain_warp(st, acc_g, i - ir, (ir + 1) * batch, batch, D, nw);
     }
 }
 
