@@ -58,6 +58,67 @@ __host__ __device__ inline WarpSplit warp_split(int n_in)
 // previous layer), the activation is bf16(x + add); if `store` is given, that activation (before the norm) is
 // also written out, one share of its 16-byte chunks per CTA.  All loads bypass L1: inside a persistent kernel
 // the activations were written by other SMs.
+// The same for ONE batch row (batch 1): the 4 * IPW chunks of 8 elements a warp needs are spread over its lanes,
+// one chunk per lane, instead of IPW chunks in each of the four lanes of row 0 -- an eighth of the loads,
+// conversions and multiplies per thread -- and the finished chunks are handed out with shuffles.  The fragment
+// words of the lanes of the unused batch columns (lane / 4 > 0) carry copies, which the products ignore.
+template <int IPW>
+__device__ __forceinline__ void load_b_frags_one_row(uint32_t (&bf)[IPW][4], const __nv_bfloat16 *x, int n_in, int nw,
+                                                     const __nv_bfloat16 *gn, float eps, float *smem_red,
+                                                     const float *add = nullptr, __nv_bfloat16 *store = nullptr,
+                                                     int store_rem = 0, int store_mod = 1)
+{
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    const int ci = lane >> 2 < IPW ? lane >> 2 : 0;            // this lane's chunk: k block ci of the warp, quarter lane % 4
+    const bool mine = (lane >> 2) < IPW;
+    const int k = 32 * (w + nw * ci) + 8 * (lane & 3);
+    uint4 gq = make_uint4(0u, 0u, 0u, 0u);
+    if (gn) gq = *reinterpret_cast<const uint4 *>(gn + k);
+    uint4 v = ld_cg_u4(x + k);
+    if (add) {
+        const float4 a0 = ld_cg_f4(add + k), a1 = ld_cg_f4(add + k + 4);
+        v.x = pack2(bf_lo(v.x) + a0.x, bf_hi(v.x) + a0.y);
+        v.y = pack2(bf_lo(v.y) + a0.z, bf_hi(v.y) + a0.w);
+        v.z = pack2(bf_lo(v.z) + a1.x, bf_hi(v.z) + a1.y);
+        v.w = pack2(bf_lo(v.w) + a1.z, bf_hi(v.w) + a1.w);
+    }
+    if (store != nullptr && mine && (k >> 3) % store_mod == store_rem) *reinterpret_cast<uint4 *>(store + k) = v;
+    uint32_t q[4] = {v.x, v.y, v.z, v.w};
+    if (gn != nullptr) {
+        float ss = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float lo = bf_lo(q[j]), hi = bf_hi(q[j]);
+            ss = fmaf(lo, lo, ss);
+            ss = fmaf(hi, hi, ss);
+        }
+        if (!mine) ss = 0.f;
+        ss = warp_sum(ss);
+        if (lane == 0) smem_red[w] = ss;                        // row 0 of the [row][warp] layout
+        named_bar_sync(1, nw * 32);
+        float tot = 0.f;
+        if ((nw & 3) == 0) {
+            for (int w4 = 0; w4 < nw; w4 += 4) {
+                const float4 p = *reinterpret_cast<const float4 *>(smem_red + w4);
+                tot += (p.x + p.y) + (p.z + p.w);
+            }
+        } else {
+            for (int w2 = 0; w2 < nw; ++w2) tot += smem_red[w2];
+        }
+        const float r = rsqrtf(tot / (float)n_in + eps);
+        const uint32_t gg[4] = {gq.x, gq.y, gq.z, gq.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) q[j] = pack2(bf_lo(q[j]) * r * bf_lo(gg[j]), bf_hi(q[j]) * r * bf_hi(gg[j]));
+        named_bar_sync(1, nw * 32);   // smem_red may be reused by the caller
+    }
+#pragma unroll
+    for (int i = 0; i < IPW; ++i) {
+        const int src = i * 4 + (lane & 3);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) bf[i][j] = __shfl_sync(kFull, q[j], src);
+    }
+}
+
 template <int IPW>
 __device__ __forceinline__ void load_b_frags(uint32_t (&bf)[IPW][4], const __nv_bfloat16 *x, int x_stride, int batch,
                                              int n_in, int nw, const __nv_bfloat16 *gn, float eps, float *smem_red,

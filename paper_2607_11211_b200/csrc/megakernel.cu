@@ -379,7 +379,8 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                     float *z = hacc + (size_t)((l - 1) & 1) * B * D;   // (head: l = L)
                     for (int idx = t; idx < B * (D >> 2); idx += nct) reinterpret_cast<float4 *>(z)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
-                load_b_frags<IPW>(bf, src, D, B, D, nw, gain, a.eps, smem_red, add, store, cta, ncta);
+                if (BC == 0) load_b_frags_one_row<IPW>(bf, src, D, nw, gain, a.eps, smem_red, add, store, cta, ncta);
+                else load_b_frags<IPW>(bf, src, D, B, D, nw, gain, a.eps, smem_red, add, store, cta, ncta);
                 if (kind == kHead) {
                     for (int u = t; u < 64; u += nct) { s_best_val[u] = -INFINITY; s_best_idx[u] = 0x7fffffff; }
                     named_bar_sync(1, nct);
