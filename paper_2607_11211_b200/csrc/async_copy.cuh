@@ -92,7 +92,7 @@ __device__ __forceinline__ bool named_bar_and(int id, int nthreads, bool pred)
 //
 // A CTA's share of a packed weight matrix is one contiguous byte range (two for the fused
 // MLP: its gate_up tiles, then its W_down octets).  A dedicated producer warp streams the
-// ranges, one after the other, in slot-sized pieces: piece g lands in slot g % nslot with
+// ranges, one after the other, in slot-sized pieces: piece g lands in slot slot_of(g) with
 // ONE bulk copy and completes on the slot's "full" mbarrier.  Each consumer warp arrives on
 // the slot's "empty" mbarrier when it has read its part, and the producer refills the slot
 // as soon as all consumer warps have.  Up to nslot pieces (about 190 KB per SM) are in
@@ -102,7 +102,7 @@ struct WeightRing {
     unsigned char *slots;        // nslot * slot_bytes, 128-byte aligned
     uint64_t *full, *empty;      // nslot mbarriers each
     volatile int *abort_flag;    // shared-memory word, set when any bounded wait ran out
-    int nslot, slot_bytes;
+    int nslot, nshift, slot_bytes;   // nslot = 1 << nshift: slot and round of a piece are a mask and a shift
     const unsigned char *base0, *base1;
     int pieces0, pieces;         // pieces of run 0, of both runs (every run is a whole number of slots)
 
@@ -113,6 +113,7 @@ struct WeightRing {
     {
         slots = slots_; full = bars; empty = bars + nslot_; abort_flag = abort_;
         nslot = nslot_; slot_bytes = slot_bytes_;
+        nshift = 31 - __clz(nslot_);
         base0 = static_cast<const unsigned char *>(b0);
         base1 = static_cast<const unsigned char *>(b1);
         pieces0 = (int)(bytes0 / slot_bytes_);
@@ -123,10 +124,12 @@ struct WeightRing {
             mbar_fence_init();
         }
     }
+    __device__ __forceinline__ int slot_of(int g) const { return g & (nslot - 1); }
+    __device__ __forceinline__ int round_of(int g) const { return g >> nshift; }
     // producer thread: wait until the slot of piece g is free again (false after a failed bounded wait)
     __device__ __forceinline__ bool acquire(int g)
     {
-        if (g >= nslot && !mbar_wait_bounded(&empty[g % nslot], (uint32_t)(g / nslot - 1) & 1u, abort_flag)) {
+        if (g >= nslot && !mbar_wait_bounded(&empty[slot_of(g)], (uint32_t)(round_of(g) - 1) & 1u, abort_flag)) {
             *abort_flag = 1;
             return false;
         }
@@ -136,7 +139,7 @@ struct WeightRing {
     __device__ __forceinline__ bool put(int g, const void *src, uint32_t bytes)
     {
         if (!acquire(g)) return false;
-        const int s = g % nslot;
+        const int s = slot_of(g);
         mbar_expect_tx(&full[s], bytes);
         bulk_g2s(slots + (size_t)s * slot_bytes, src, bytes, &full[s]);
         return true;
@@ -145,7 +148,7 @@ struct WeightRing {
     __device__ __forceinline__ bool put2(int g, const void *src0, const void *src1, uint32_t bytes, uint32_t off1)
     {
         if (!acquire(g)) return false;
-        const int s = g % nslot;
+        const int s = slot_of(g);
         mbar_expect_tx(&full[s], 2 * bytes);
         bulk_g2s(slots + (size_t)s * slot_bytes, src0, bytes, &full[s]);
         bulk_g2s(slots + (size_t)s * slot_bytes + off1, src1, bytes, &full[s]);
@@ -164,17 +167,17 @@ struct WeightRing {
     __device__ __forceinline__ const unsigned char *wait(int g, bool &ok)
     {
         bool mine = ok;
-        if (mine) mine = mbar_wait_bounded(&full[g % nslot], (uint32_t)(g / nslot) & 1u, abort_flag);
+        if (mine) mine = mbar_wait_bounded(&full[slot_of(g)], (uint32_t)(round_of(g)) & 1u, abort_flag);
         mine = __all_sync(kFull, mine);
         if (!mine && ok) *abort_flag = 1;
         ok = mine;
-        return slots + (size_t)(g % nslot) * slot_bytes;
+        return slots + (size_t)(slot_of(g)) * slot_bytes;
     }
     // consumer warp, after its last read of piece g
     __device__ __forceinline__ void release(int g)
     {
         __syncwarp();
-        if ((threadIdx.x & 31) == 0) mbar_arrive(&empty[g % nslot]);
+        if ((threadIdx.x & 31) == 0) mbar_arrive(&empty[slot_of(g)]);
     }
     // producer thread, on the way out after a failure: give the copies in flight a bounded chance to land
     __device__ __forceinline__ void drain()

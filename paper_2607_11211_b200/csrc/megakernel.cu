@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                 for (int p0 = 0; p0 < ont; p0 += TP, ++piece) {
                     const int nt = ont - p0 < TP ? ont - p0 : TP;
                     if (!ring.acquire(piece)) return;
-                    const int sl = piece % ring.nslot;
+                    const int sl = ring.slot_of(piece);
                     mbar_expect_tx(&ring.full[sl], (uint32_t)(nt * KB * kTileBytes));
                     for (int j = 0; j < nt; ++j)
                         bulk_g2s(ring.slots + (size_t)sl * ring.slot_bytes + (size_t)j * KB * kTileBytes,
@@ -334,16 +334,30 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                     for (int p0 = 0; p0 < ont; p0 += TP, ++piece) {
                         const int nt = ont - p0 < TP ? ont - p0 : TP;
                         const unsigned char *slot = ring.wait(piece, ok);
+                        float c[4] = {0.f, 0.f, 0.f, 0.f};
                         if (w < nt) {
-                            float c[4] = {0.f, 0.f, 0.f, 0.f};
+                            // independent accumulators per half k block: the products do not wait for one another
+                            float cj[2 * KB][4];
 #pragma unroll
                             for (int j = 0; j < KB; ++j) {
                                 const unsigned char *blk = slot + (size_t)(w * KB + j) * kTileBytes + lane * 16;
                                 const uint4 lo = *reinterpret_cast<const uint4 *>(blk);
                                 const uint4 hi = *reinterpret_cast<const uint4 *>(blk + 512);
-                                mma_bf16_k16(c, lo.x, hi.x, lo.y, hi.y, bh[j].x, bh[j].y);
-                                mma_bf16_k16(c, lo.z, hi.z, lo.w, hi.w, bh[j].z, bh[j].w);
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) cj[2 * j][e] = cj[2 * j + 1][e] = 0.f;
+                                mma_bf16_k16(cj[2 * j], lo.x, hi.x, lo.y, hi.y, bh[j].x, bh[j].y);
+                                mma_bf16_k16(cj[2 * j + 1], lo.z, hi.z, lo.w, hi.w, bh[j].z, bh[j].w);
                             }
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                c[e] = 0.f;
+#pragma unroll
+                                for (int j = 0; j < 2 * KB; ++j) c[e] += cj[j][e];
+                            }
+                        }
+                        // the slot goes back before the sums leave: an arrival after the reductions would wait for them
+                        ring.release(piece);
+                        if (w < nt) {
                             // accumulator fragment: rows g / g + 8 of the tile, batch rows 2 t4 / 2 t4 + 1
                             const int row = (ot0 + p0 + w) * 16 + g, b0 = 2 * t4;
                             if (ok && b0 < B) {
@@ -355,7 +369,6 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                                 if (row + 8 < D) atomicAdd(hsum + (size_t)(b0 + 1) * D + row + 8, c[3]);
                             }
                         }
-                        ring.release(piece);
                     }
                 }
             } else {

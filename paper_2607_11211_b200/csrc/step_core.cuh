@@ -81,7 +81,7 @@ __host__ __device__ inline MegaLayout mega_layout(int D)
     l.wpiece = kBlocksPerWarpPerSlot * (s.nw > 0 ? s.nw : 1) * kTileBytes;
     l.slot_stride = l.wpiece > AttnTile<DH>::kPieceBytes ? l.wpiece : AttnTile<DH>::kPieceBytes;
     l.nslot = kRingBudget / l.slot_stride;
-    if (l.nslot > 8) l.nslot = 8;
+    l.nslot = l.nslot >= 8 ? 8 : l.nslot >= 4 ? 4 : l.nslot >= 2 ? 2 : l.nslot;   // a power of two (ring indexing by mask and shift)
     l.ring_off = 0;
     l.bar_off = (size_t)l.nslot * l.slot_stride;
     l.abort_off = l.bar_off + 2 * 8 * 8;

@@ -19,7 +19,7 @@ __host__ __device__ inline StreamSmemLayout stream_smem_layout(int n_in)
     l.nw = s.nw; l.ipw = s.ipw;
     l.slot_bytes = kBlocksPerWarpPerSlot * (s.nw > 0 ? s.nw : 1) * kTileBytes;
     l.nslot = kRingBudget / l.slot_bytes;
-    if (l.nslot > 8) l.nslot = 8;
+    l.nslot = l.nslot >= 8 ? 8 : l.nslot >= 4 ? 4 : l.nslot >= 2 ? 2 : l.nslot;   // a power of two (ring indexing by mask and shift)
     l.ring_off = 0;
     l.bar_off = (size_t)l.nslot * l.slot_bytes;
     l.abort_off = l.bar_off + 2 * 8 * 8;
