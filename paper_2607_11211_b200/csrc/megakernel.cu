@@ -22,6 +22,7 @@
 // products of the 32 heads meet in an FP32 accumulator (red.add); the residual add h = x + attn W_o moves into
 // the prologue of the MLP phase, which also writes h out (one share of its chunks per CTA), as the QKV
 // prologue does for x = h + y of the layer before.
+#include <cstdlib>
 #include "step_core.cuh"
 
 namespace fasttps {
@@ -114,8 +115,15 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
         int piece = 0;
         auto weights = [&](const void *base, size_t first_byte, int npieces) -> bool {
             const unsigned char *p = static_cast<const unsigned char *>(base) + first_byte;
-            for (int i = 0; i < npieces; ++i, ++piece)
+            // the L2 runs ahead of the ring: while the consumers are held up at a phase boundary and the ring is
+            // full, HBM keeps working on the pieces that follow.  Three quarters of a ring measured best: further
+            // ahead, the prefetches of the next product get in the way of the K/V tiles of the attention phase.
+            const int ahead = ring.nslot - ring.nslot / 4;
+            for (int i = 0; i < npieces && i < ahead; ++i) bulk_prefetch_l2(p + (size_t)i * wp, wp);
+            for (int i = 0; i < npieces; ++i, ++piece) {
+                if (i + ahead < npieces) bulk_prefetch_l2(p + (size_t)(i + ahead) * wp, wp);
                 if (!ring.put(piece, p + (size_t)i * wp, wp)) return false;
+            }
             return true;
         };
         for (int step = 0; step < a.n_steps; ++step) {
@@ -134,13 +142,13 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                     __threadfence_block();
                 }
                 const AttnArgs aa = attn_args_of(a, lp, step, gm * a.n_q_heads);
+                const unsigned char *wo = reinterpret_cast<const unsigned char *>(lp.w_o);
                 const bool kv_ok = attn_for_each_tile<DH>(aa, GroupSource(&s_segs),
                                                           [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
                     return ring.put2(piece++, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
                 });
                 if (!kv_ok) return;
                 // this CTA's rows of the output projection, the head's k blocks only: KB KB per row tile
-                const unsigned char *wo = reinterpret_cast<const unsigned char *>(lp.w_o);
                 for (int p0 = 0; p0 < ont; p0 += TP, ++piece) {
                     const int nt = ont - p0 < TP ? ont - p0 : TP;
                     if (!ring.acquire(piece)) return;
