@@ -70,6 +70,18 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
+// the same with an L2 eviction policy (from l2_policy_evict_first): data that is read once
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_g2s_hint(void *dst, const void *src, uint32_t bytes, uint64_t *bar, uint64_t pol)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol) : "memory");
+}
 // asks the L2 to fetch `bytes` (a multiple of 16) at src: no completion to wait for
 __device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes)
 {
@@ -107,6 +119,7 @@ struct WeightRing {
     unsigned char *slots;        // nslot * slot_bytes, 128-byte aligned
     uint64_t *full, *empty;      // nslot mbarriers each
     volatile int *abort_flag;    // shared-memory word, set when any bounded wait ran out
+    uint64_t policy = 0;         // L2 eviction policy of the weight pieces (0: none)
     int nslot, nshift, slot_bytes;   // nslot = 1 << nshift: slot and round of a piece are a mask and a shift
     const unsigned char *base0, *base1;
     int pieces0, pieces;         // pieces of run 0, of both runs (every run is a whole number of slots)
@@ -146,7 +159,8 @@ struct WeightRing {
         if (!acquire(g)) return false;
         const int s = slot_of(g);
         mbar_expect_tx(&full[s], bytes);
-        bulk_g2s(slots + (size_t)s * slot_bytes, src, bytes, &full[s]);
+        if (policy) bulk_g2s_hint(slots + (size_t)s * slot_bytes, src, bytes, &full[s], policy);
+        else bulk_g2s(slots + (size_t)s * slot_bytes, src, bytes, &full[s]);
         return true;
     }
     // producer thread: piece g = two blocks of `bytes` each, the second landing at offset off1 of the slot

@@ -113,12 +113,17 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
         if (w > nw || lane != 0) return;
         const uint32_t wp = (uint32_t)lay.wpiece;
         int piece = 0;
-        auto weights = [&](const void *base, size_t first_byte, int npieces) -> bool {
+        // every piece is read once: its L2 lines go first, the lines prefetched for later pieces stay
+        ring.policy = l2_policy_evict_first();
+        // how far (in ring pieces) the L2 prefetch runs ahead of the ring in each product; measured on the
+        // Phi-3-mini shape with an 8-slot ring: 3 / 5 / 12 / 6.  Deeper prefetches of the QKV and gate_up pieces
+        // are issued during the phases before them and slow those down by more than they gain.
+        const int pf_qkv = (3 * ring.nslot + 7) / 8, pf_gu = (5 * ring.nslot + 7) / 8, pf_down = 3 * ring.nslot / 2,
+                  pf_lm = 3 * ring.nslot / 4;
+        auto weights = [&](const void *base, size_t first_byte, int npieces, int ahead) -> bool {
             const unsigned char *p = static_cast<const unsigned char *>(base) + first_byte;
-            // the L2 runs ahead of the ring: while the consumers are held up at a phase boundary and the ring is
-            // full, HBM keeps working on the pieces that follow.  Three quarters of a ring measured best: further
-            // ahead, the prefetches of the next product get in the way of the K/V tiles of the attention phase.
-            const int ahead = ring.nslot - ring.nslot / 4;
+            // the L2 runs `ahead` pieces ahead of the ring: while the consumers are held up at a phase boundary and
+            // the ring is full, HBM keeps working on the pieces that follow
             for (int i = 0; i < npieces && i < ahead; ++i) bulk_prefetch_l2(p + (size_t)i * wp, wp);
             for (int i = 0; i < npieces; ++i, ++piece) {
                 if (i + ahead < npieces) bulk_prefetch_l2(p + (size_t)(i + ahead) * wp, wp);
@@ -129,7 +134,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
         for (int step = 0; step < a.n_steps; ++step) {
             for (int l = 0; l < a.n_layers; ++l) {
                 const LayerPtrs &lp = s_layers[l];
-                if (!weights(lp.w_qkv, (size_t)q0 * tile_bytes, qn * SPT)) return;
+                if (!weights(lp.w_qkv, (size_t)q0 * tile_bytes, qn * SPT, pf_qkv)) return;
                 if (l == 0) {
                     // K/V tiles of this step include the row appended by the step before it, and the share is
                     // recomputed per step: both are ready once the consumers have passed the barrier that ends
@@ -159,10 +164,12 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                                  wo + ((size_t)(ot0 + p0 + j) * (nq / 32) + (size_t)head * KB) * kTileBytes,
                                  (uint32_t)(KB * kTileBytes), &ring.full[sl]);
                 }
-                if (!weights(lp.w_gu, (size_t)m0 * tile_bytes, mn * SPT)) return;
-                if (!weights(lp.w_down, (size_t)m0 * oct_bytes, mn * PPO)) return;
+                // the gate_up prefetch waits until this CTA's rows of W_o have landed
+                if (ont > 0 && !mbar_wait_bounded(&ring.full[ring.slot_of(piece - 1)], (uint32_t)ring.round_of(piece - 1) & 1u, ring.abort_flag)) return;
+                if (!weights(lp.w_gu, (size_t)m0 * tile_bytes, mn * SPT, pf_gu)) return;
+                if (!weights(lp.w_down, (size_t)m0 * oct_bytes, mn * PPO, pf_down)) return;
             }
-            if (!weights(a.w_lm, (size_t)l0 * tile_bytes, ln * SPT)) return;
+            if (!weights(a.w_lm, (size_t)l0 * tile_bytes, ln * SPT, pf_lm)) return;
         }
         return;
     }
