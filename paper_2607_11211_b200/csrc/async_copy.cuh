@@ -169,8 +169,13 @@ struct WeightRing {
         if (!acquire(g)) return false;
         const int s = slot_of(g);
         mbar_expect_tx(&full[s], 2 * bytes);
-        bulk_g2s(slots + (size_t)s * slot_bytes, src0, bytes, &full[s]);
-        bulk_g2s(slots + (size_t)s * slot_bytes + off1, src1, bytes, &full[s]);
+        if (policy) {
+            bulk_g2s_hint(slots + (size_t)s * slot_bytes, src0, bytes, &full[s], policy);
+            bulk_g2s_hint(slots + (size_t)s * slot_bytes + off1, src1, bytes, &full[s], policy);
+        } else {
+            bulk_g2s(slots + (size_t)s * slot_bytes, src0, bytes, &full[s]);
+            bulk_g2s(slots + (size_t)s * slot_bytes + off1, src1, bytes, &full[s]);
+        }
         return true;
     }
     // one thread of the producer warp: stream every piece of the two runs given to init(), then return

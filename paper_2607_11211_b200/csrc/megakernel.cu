@@ -160,9 +160,9 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                     const int sl = ring.slot_of(piece);
                     mbar_expect_tx(&ring.full[sl], (uint32_t)(nt * KB * kTileBytes));
                     for (int j = 0; j < nt; ++j)
-                        bulk_g2s(ring.slots + (size_t)sl * ring.slot_bytes + (size_t)j * KB * kTileBytes,
-                                 wo + ((size_t)(ot0 + p0 + j) * (nq / 32) + (size_t)head * KB) * kTileBytes,
-                                 (uint32_t)(KB * kTileBytes), &ring.full[sl]);
+                        bulk_g2s_hint(ring.slots + (size_t)sl * ring.slot_bytes + (size_t)j * KB * kTileBytes,
+                                      wo + ((size_t)(ot0 + p0 + j) * (nq / 32) + (size_t)head * KB) * kTileBytes,
+                                      (uint32_t)(KB * kTileBytes), &ring.full[sl], ring.policy);
                 }
                 // the gate_up prefetch waits until this CTA's rows of W_o have landed
                 if (ont > 0 && !mbar_wait_bounded(&ring.full[ring.slot_of(piece - 1)], (uint32_t)ring.round_of(piece - 1) & 1u, ring.abort_flag)) return;
