@@ -305,18 +305,30 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
 
         // ---- combine the row groups of a warp, then the warps of the CTA ----
         if (worker) {
+            // The eight row groups of a warp hold partial sums of the same EPL elements.  They are added by halving:
+            // in each of three rounds a lane keeps one half of what it holds and gets the partner's sums of that
+            // half, so the element count per lane goes EPL -> EPL/2 -> EPL/4 -> EPL/8 (7 EPL / 8 shuffles instead of
+            // 3 EPL) and every lane ends with EPL / 8 finished elements.
+            static_assert(EPL % 8 == 0, "head_dim must be a multiple of 32");
 #pragma unroll
-            for (int s = 4; s <= 16; s <<= 1) {
-                l_run += __shfl_xor_sync(kFull, l_run, s);
-#pragma unroll
-                for (int i = 0; i < EPL; ++i) acc[i] += __shfl_xor_sync(kFull, acc[i], s);
-            }
+            for (int s = 4; s <= 16; s <<= 1) l_run += __shfl_xor_sync(kFull, l_run, s);
             l_run = __shfl_sync(kFull, l_run, 0);          // the sum was kept by the sub == 0 lanes
-            if (lane < kLanesPerRow) {
+            int first = 0;                                  // index (within the lane's EPL) of the elements it still holds
 #pragma unroll
-                for (int i = 0; i < EPL; ++i) sm.wo[warp][sub * EPL + i] = acc[i];
-                if (lane == 0) { sm.wm[warp] = m_run; sm.wl[warp] = l_run; }
+            for (int r = 0; r < 3; ++r) {
+                const int half = EPL >> (r + 1);
+                const bool upper = (lane >> (4 - r)) & 1;   // rounds pair lanes 16, 8, 4 apart
+#pragma unroll
+                for (int i = 0; i < half; ++i) {
+                    const float send = upper ? acc[i] : acc[i + half];
+                    const float keep = upper ? acc[i + half] : acc[i];
+                    acc[i] = keep + __shfl_xor_sync(kFull, send, 16 >> r);
+                }
+                first += upper ? half : 0;
             }
+#pragma unroll
+            for (int i = 0; i < EPL / 8; ++i) sm.wo[warp][sub * EPL + first + i] = acc[i];
+            if (lane == 0) { sm.wm[warp] = m_run; sm.wl[warp] = l_run; }
         }
         if (!named_bar_and(1, nct, ok)) return false;
         float M = -INFINITY;
