@@ -232,7 +232,7 @@ int fasttps_profile(fasttps_ctx *ctx, int enable);
 int fasttps_profile_read(fasttps_ctx *ctx, double *ms_per_class, uint64_t *launches_per_class);
 /* Phase timeline of the last launch of the persistent step kernel, for profiling: the first and
  * the last CTA stamp the GPU global timer (ns) immediately before and after every grid-wide
- * barrier (order per step: embedding, then per layer QKV, attention, output projection, MLP,
+ * barrier (order per step: embedding, then per layer QKV, attention + output projection, MLP,
  * then logits and argmax).  Synchronises, copies up to max_per_cta stamps of each of the two CTAs
  * into stamps[0 .. max_per_cta) and stamps[max_per_cta .. 2 max_per_cta), returns the number
  * of slots copied per CTA (slots past the launch's last stamp hold older or zero values). */
@@ -241,6 +241,15 @@ int fasttps_trace_read(fasttps_ctx *ctx, uint64_t *stamps, int max_per_cta);
 uint64_t fasttps_launch_count(const fasttps_ctx *ctx);
 /* Split count the attention kernel would use for this batch (for tests/benchmarks). */
 int fasttps_attn_splits(const fasttps_ctx *ctx, int batch);
+/* Diagnostic, host only (no context, no CUDA call; no counterpart in the paper): how the persistent step kernel
+ * cuts the cached rows of one query head, all sequences of the batch end to end plus one new row each (Algorithm 3
+ * over a ragged batch), into shares for the group_size CTAs of the head in decode step `step` of a launch.
+ * seq_lens, pos: HOST arrays of `batch` (<= 8) entries, as passed to fasttps_model_decode.  For share g,
+ * nseg_out[g] segments are written to seg_out[(g * 8 + j) * 5 + 0..4] = sequence, first row, end row (exclusive; row
+ * seq_len is the new row), first share that holds rows of that sequence, number of shares that do.  Returns the
+ * number of shares in use (<= group_size; 0 if no sequence is valid), or a negative FASTTPS error code. */
+int fasttps_attention_shares(const int32_t *seq_lens, const int32_t *pos, int batch, int max_seq, int step,
+                             int group_size, int32_t *seg_out, int32_t *nseg_out);
 const char *fasttps_strerror(int code);
 /* Text of the last CUDA error seen by this thread inside the library ("" if none). */
 const char *fasttps_last_error(void);

@@ -70,11 +70,30 @@ def load_library() -> C.CDLL:
     lib.fasttps_launch_count.argtypes = [vp]
     lib.fasttps_launch_count.restype = C.c_uint64
     lib.fasttps_attn_splits.argtypes = [vp, i]
+    lib.fasttps_attention_shares.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.fasttps_strerror.argtypes = [i]
     lib.fasttps_strerror.restype = C.c_char_p
     lib.fasttps_last_error.restype = C.c_char_p
     _lib = lib
     return lib
+
+
+def attention_shares(seq_lens, pos, max_seq: int, step: int, group_size: int):
+    """How the step kernel cuts the rows of one query head (all sequences end to end, one new row each) into
+    shares for the `group_size` CTAs of the head: (shares in use, per share a list of
+    (sequence, first row, end row, first share of the sequence, number of shares of the sequence)).
+    Host only: needs the library, not a GPU."""
+    import numpy as np
+    lib = load_library()
+    sl = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    ps = np.ascontiguousarray(pos, dtype=np.int32)
+    seg = np.zeros((group_size, 8, 5), dtype=np.int32)
+    nseg = np.zeros(group_size, dtype=np.int32)
+    rc = lib.fasttps_attention_shares(sl.ctypes.data, ps.ctypes.data, len(sl), int(max_seq), int(step), int(group_size),
+                                      seg.ctypes.data, nseg.ctypes.data)
+    if rc < 0:
+        _check(rc, "fasttps_attention_shares")
+    return rc, [[tuple(int(v) for v in seg[g, j]) for j in range(nseg[g])] for g in range(group_size)]
 
 
 def _check(rc: int, what: str):

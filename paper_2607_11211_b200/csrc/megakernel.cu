@@ -55,7 +55,7 @@ struct GroupSource {
 // (RoPE of k, the append, the score from shared memory) and, in a batch, starts another segment behind it (RoPE
 // of q, combine, partial write).  Measured on the ragged batch of 8: 0 -> 2603, 64 -> 2648, 128 -> 2669,
 // 256 -> 2682 tok/s; at batch 1 the last share shrinks from 256 to about 110 of 1025 rows (+1.8 %).
-static __device__ __noinline__ void build_attention_shares(const int32_t *seq_lens, const int32_t *pos, int max_seq, int step,
+static __host__ __device__ __noinline__ void build_attention_shares(const int32_t *seq_lens, const int32_t *pos, int max_seq, int step,
                                                            int B, int gm, int gs, int head, bool in_group, GroupSegs *segs,
                                                            int *ncta_out, int *mprime_out, int *cuts)
 {
@@ -622,3 +622,29 @@ int launch_step(Ctx *c, const StepArgs &a, cudaStream_t st)
 }
 
 }  // namespace fasttps
+
+// Diagnostic entry point: the attention shares of one head group, computed on the host by the same code the
+// step kernel runs on the device.
+extern "C" int fasttps_attention_shares(const int32_t *seq_lens, const int32_t *pos, int batch, int max_seq, int step,
+                                        int group_size, int32_t *seg_out, int32_t *nseg_out)
+{
+    using namespace fasttps;
+    if (!seq_lens || !pos || !seg_out || !nseg_out || batch < 1 || batch > kMaxNB || group_size < 1 ||
+        group_size > kMaxSplits || max_seq < 1 || step < 0)
+        return FASTTPS_INVALID_ARG;
+    int mprime = 0;
+    for (int gs = 0; gs < group_size; ++gs) {
+        GroupSegs segs;
+        int ncta[kMaxNB], cuts[kMaxSplits + 1];
+        build_attention_shares(seq_lens, pos, max_seq, step, batch, group_size, gs, /*head=*/0, /*in_group=*/true, &segs, ncta,
+                               &mprime, cuts);
+        nseg_out[gs] = segs.n;
+        for (int j = 0; j < segs.n; ++j) {
+            int32_t *o = seg_out + ((size_t)gs * kMaxNB + j) * 5;
+            o[0] = segs.seg[j].b; o[1] = segs.seg[j].r0; o[2] = segs.seg[j].r1;
+            o[3] = segs.seg[j].first_cta; o[4] = segs.seg[j].n_cta;
+        }
+    }
+    return mprime;
+}
+
