@@ -192,9 +192,9 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
         // every piece is read once: its L2 lines go first, the lines prefetched for later pieces stay
         ring.policy = l2_policy_evict_first();
         // how far (in ring pieces) the L2 prefetch runs ahead of the ring in each product; measured on the
-        // Phi-3-mini shape with an 8-slot ring: 3 / 5 / 12 / 6.  Deeper prefetches of the QKV and gate_up pieces
+        // Phi-3-mini shape with an 8-slot ring: 3 / 6 / 12 / 6.  Deeper prefetches of the QKV and gate_up pieces
         // are issued during the phases before them and slow those down by more than they gain.
-        const int pf_qkv = (3 * ring.nslot + 7) / 8, pf_gu = (5 * ring.nslot + 7) / 8, pf_down = 3 * ring.nslot / 2,
+        const int pf_qkv = (3 * ring.nslot + 7) / 8, pf_gu = 3 * ring.nslot / 4, pf_down = 3 * ring.nslot / 2,
                   pf_lm = 3 * ring.nslot / 4;
         auto weights = [&](const void *base, size_t first_byte, int npieces, int ahead) -> bool {
             const unsigned char *p = static_cast<const unsigned char *>(base) + first_byte;
