@@ -178,7 +178,7 @@ __device__ __forceinline__ bool attn_produce(const AttnArgs &a, WeightRing &ring
 // Returns false (in every consumer thread alike) if a bounded wait ran out.
 // DEFER: the partial of every segment is published (even when the CTA owns the whole head) and nobody
 // merges here; the caller merges the partials of a head itself (the persistent step kernel does, per group).
-template <int DH, bool DEFER, class Src>
+template <int DH, bool DEFER, class Src, bool LATE_FENCE = false>
 __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring, int &piece, int cta, Src src,
                                              AttnScratch<DH> &sm, int nwc)
 {
@@ -196,6 +196,7 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
     const int rgrp = lane >> 2;                      // row within an 8-row group
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
     bool ok = true;
+    bool appended = false;
 
     Segment sg;
     while (src.next(sg)) {
@@ -228,8 +229,10 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
                 reinterpret_cast<uint4 *>(a.k_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(sm.knew)[i];
                 reinterpret_cast<uint4 *>(a.v_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(sm.vnew)[i];
             }
-            // later bulk copies (a later step of the same launch) must see these rows
-            asm volatile("fence.proxy.async;" ::: "memory");
+            // bulk copies of a later step of the same launch must see these rows: the stores are ordered before the
+            // asynchronous proxy, here or (LATE_FENCE) after the last segment
+            if (LATE_FENCE) appended = true;
+            else asm volatile("fence.proxy.async;" ::: "memory");
         }
 
         float qr[EPL];
@@ -391,6 +394,8 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
         }
         named_bar_sync(1, nct);                          // the scratch is reused by the next segment
     }
+    // LATE_FENCE: off the path of the rows that were still to be scored (worth it when a share holds several segments)
+    if (LATE_FENCE && appended) asm volatile("fence.proxy.async;" ::: "memory");
     return true;
 }
 

@@ -323,7 +323,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
             if (kind == kAttn) {
                 // ---- attention (Algorithm 3) on this CTA's rows of its head; the partial is published ----
                 const AttnArgs aa = attn_args_of(a, lp, step, gm * a.n_q_heads);
-                ok = attn_consume<DH, true>(aa, ring, piece, cta, GroupSource(&s_segs), scratch, nw) && ok;
+                ok = attn_consume<DH, true, GroupSource, BC != 0>(aa, ring, piece, cta, GroupSource(&s_segs), scratch, nw) && ok;
                 grp_target += (unsigned)mprime;
                 if (in_group) {
                     // ---- the group meets: every CTA of it needs the merged output of the head ----
