@@ -108,8 +108,10 @@ int fasttps_destroy(fasttps_ctx *ctx);
  *            come out of the same tile;
  *   DOWN:    for every j-octet J (8 rows of the logical [K, D] matrix) and block of 32
  *            output columns one 512-byte block holding W_down[8J..8J+7, 32c..32c+31] in
- *            the register order of an m16n8k8 A operand; blocks ordered by (J, c), so a
- *            CTA's octets are again one contiguous byte range.
+ *            the register order of two m16n8k8 A operands whose rows are assigned to the
+ *            output columns so that a thread's four results are four consecutive columns
+ *            (one 16-byte reduction); blocks ordered by (J, c), so a CTA's octets are again
+ *            one contiguous byte range.
  * Limits: D and H_q d multiples of 128 up to 3072 or multiples of 256 from 2048 to 6144;
  * K a multiple of 8. */
 size_t fasttps_packed_bytes(const fasttps_ctx *ctx, int kind);

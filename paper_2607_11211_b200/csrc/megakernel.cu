@@ -151,7 +151,6 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     AttnScratch<DH> &scratch = *reinterpret_cast<AttnScratch<DH> *>(dsm + lay.scratch_off);
 
     const int D = a.D, B = BC == 0 ? 1 : a.batch;
-    constexpr bool BIG = BC == 2;
     const int nq = a.n_q_heads * a.head_dim, nkv = a.n_kv_heads * a.head_dim, nqkv = nq + 2 * nkv;
     constexpr int SPT = IPW / kBlocksPerWarpPerSlot;      // ring pieces per 16-row tile
     constexpr int PPO = IPW / 4;                          // ring pieces per W_down octet
@@ -492,7 +491,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                             for (int e = 0; e < 4; ++e) acc[i][m][e] = 0.f;
                     mlp_down_phase<IPW>(ring, piece, mn, nw, s_hi, s_lo, acc, ok);
                     piece += mn * PPO;
-                    mlp_scatter_add<IPW, BIG>(acc, smem_part, a.acc + (size_t)(l & 1) * B * D, B, D, nw);
+                    mlp_scatter_add<IPW>(acc, a.acc + (size_t)(l & 1) * B * D, B, D, nw);
                 } else if (kind == kHead) {
                     named_bar_sync(1, nct);
                     if (t < 8 && t < B) {

@@ -87,8 +87,7 @@ __global__ void __launch_bounds__(MAXT, 1) mlp_decode_kernel(MlpArgs a)
         return;
     }
     // ---- partial y -> shared memory -> vector red.add ----
-    if (a.batch > 2) mlp_scatter_add<IPW, true>(acc, smem_part, a.acc, a.batch, a.D, nw);
-    else mlp_scatter_add<IPW, false>(acc, smem_part, a.acc, a.batch, a.D, nw);
+    mlp_scatter_add<IPW>(acc, a.acc, a.batch, a.D, nw);
     __threadfence();
     named_bar_sync(1, nct);
     if (t == 0) s_last = (atomicAdd(a.ticket, 1) == (int)gridDim.x - 1);

@@ -63,105 +63,24 @@ __device__ __forceinline__ void mlp_down_phase(WeightRing &ring, int piece0, int
     }
 }
 
-// One round of mlp_scatter_add: the staged chunks i0 .. i0 + nchunk - 1 go to global memory.  Out of line: the
-// caller is unrolled over the chunks and would carry a copy of this loop for each of them.
-static __device__ __noinline__ void mlp_scatter_drain(const float *stage, float *acc_g, int i0, int nchunk, int batch, int D,
-                                                      int cw, int nct)
-{
-    const int t = threadIdx.x, per_row = cw >> 2;
-    named_bar_sync(1, nct);
-    for (int idx = t; idx < nchunk * batch * per_row; idx += nct) {
-        const int cb = idx / per_row, j = idx - cb * per_row;      // cb = chunk * batch + b
-        const int ch = cb / batch, b = cb - ch * batch;
-        const float4 v = *reinterpret_cast<const float4 *>(stage + (size_t)cb * cw + 4 * j);
-        red_add_v4(acc_g + (size_t)b * D + (size_t)cw * (i0 + ch) + 4 * j, v.x, v.y, v.z, v.w);
-    }
-}
-
-// y^T fragments -> FP32 accumulator `acc_g` [batch][D] in global memory with vector red.add, staged
-// through shared memory in IPW chunks of 32 * nw output columns (the columns the warps own for one
-// value of i are one contiguous chunk), several chunks per round when the batch is small.  stage:
-// 8 * 32 * nw floats that are idle (the partial-tile scratch of the gate_up phase).  Consumer threads
-// only (named barrier 1).
+// y^T fragments -> FP32 accumulator `acc_g` [batch][D] in global memory.  The packed W_down orders the 32
+// output columns of a block so that the four rows a lane holds of its two MMA tiles (rows g and g + 8 of tile
+// m = 0, then of tile m = 1) are the CONSECUTIVE columns 4 g .. 4 g + 3 of the block: every lane adds its
+// accumulators with one 16-byte red.add per batch row it holds (2 t4 and 2 t4 + 1), straight from registers --
+// no staging through shared memory, no barrier.  A warp-wide instruction covers 128 contiguous bytes of each of
+// four batch rows.
 template <int IPW>
-__device__ __forceinline__ void mlp_scatter_add_block(const float (&acc)[IPW][2][4], float *stage, float *acc_g, int batch,
-                                                int D, int nw)
-{
-    const int t = threadIdx.x, lane = t & 31, w = t >> 5, g = lane >> 2, t4 = lane & 3, nct = nw * 32;
-    const int cw = 32 * nw;                                  // chunk width in columns
-    // chunks staged per round: as many as the stage holds (all 8 at batch 1: one barrier instead of fifteen)
-    const int R = batch <= 1 ? 8 : (batch <= 2 ? 4 : (batch <= 4 ? 2 : 1));
-#pragma unroll
-    for (int i = 0; i < IPW; ++i) {
-        const int ir = i % R;                                // slot of chunk i inside the round
-        if (ir == 0 && i > 0) named_bar_sync(1, nct);        // the previous round has been read
-        float *st = stage + (size_t)ir * batch * cw;
-#pragma unroll
-        for (int m = 0; m < 2; ++m) {
-            const int n = 32 * w + 16 * m + g;
-            const int b0 = 2 * t4;
-            if (b0 < batch) { st[b0 * cw + n] = acc[i][m][0]; st[b0 * cw + n + 8] = acc[i][m][2]; }
-            if (b0 + 1 < batch) { st[(b0 + 1) * cw + n] = acc[i][m][1]; st[(b0 + 1) * cw + n + 8] = acc[i][m][3]; }
-        }
-        if (ir == R - 1 || i == IPW - 1) mlp_scatter_drain(stage, acc_g, i - ir, ir + 1, batch, D, cw, nct);
-    }
-}
-
-
-// One round of mlp_scatter_add_warp: the warp's staged rows go to global memory.  Out of line: the caller is
-// unrolled over the chunks and would carry a copy of this loop for each of them.
-static __device__ __noinline__ void mlp_scatter_drain_warp(const float *st, float *acc_g, int i0, int nrow, int batch, int D,
-                                                           int nw)
-{
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    __syncwarp();
-    for (int idx = lane; idx < nrow * 8; idx += 32) {
-        const int row = idx >> 3, j = idx & 7;
-        const int ch = row / batch, b = row - ch * batch;
-        const float4 v = *reinterpret_cast<const float4 *>(st + row * 32 + (((j ^ row) & 7) << 2));
-        red_add_v4(acc_g + (size_t)b * D + 32 * (nw * (i0 + ch) + w) + 4 * j, v.x, v.y, v.z, v.w);
-    }
-}
-
-// The same scatter for larger batches, where the block-wide version would need two block-wide barriers per
-// value of i.  For a given i a
-// warp owns 32 contiguous output columns, 32 (nw i + w) .. + 32, so the transposition from fragment order to
-// rows of 4 consecutive columns is private to the warp: it goes through the warp's own 1 KB of `stage`
-// (8 * 32 * nw floats that are idle: the partial-tile scratch of the gate_up phase) with no block-wide barrier.
-// The region holds R = 8 / batch' values of i at a time as rows [chunk][batch row][32 columns]; the eight
-// 4-column groups of a row are XOR-swizzled with the row index, which makes both the fragment-order writes and
-// the 16-byte row reads free of bank conflicts.
-template <int IPW>
-__device__ __forceinline__ void mlp_scatter_add_warp(const float (&acc)[IPW][2][4], float *stage, float *acc_g, int batch,
-                                                int D, int nw)
+__device__ __forceinline__ void mlp_scatter_add(const float (&acc)[IPW][2][4], float *acc_g, int batch, int D, int nw)
 {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, g = lane >> 2, t4 = lane & 3;
-    const int R = batch <= 1 ? 8 : (batch <= 2 ? 4 : (batch <= 4 ? 2 : 1));
-    float *st = stage + w * 256;
+    const int b0 = 2 * t4;
+    float *col = acc_g + (size_t)b0 * D + 32 * w + 4 * g;    // one running address: the step per i is 32 nw columns
 #pragma unroll
     for (int i = 0; i < IPW; ++i) {
-        const int ir = i % R;                                // slot of chunk i inside the round
-        if (ir == 0 && i > 0) __syncwarp();                  // the previous round has been read
-#pragma unroll
-        for (int m = 0; m < 2; ++m) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int b = 2 * t4 + (e & 1), n = 16 * m + g + 8 * (e >> 1);
-                const int row = ir * batch + b;
-                if (b < batch) st[row * 32 + ((((n >> 2) ^ row) & 7) << 2) + (n & 3)] = acc[i][m][e];
-            }
-        }
-        if (ir == R - 1 || i == IPW - 1) mlp_scatter_drain_warp(st, acc_g, i - ir, (ir + 1) * batch, batch, D, nw);
+        if (b0 < batch) red_add_v4(col, acc[i][0][0], acc[i][0][2], acc[i][1][0], acc[i][1][2]);
+        if (b0 + 1 < batch) red_add_v4(col + D, acc[i][0][1], acc[i][0][3], acc[i][1][1], acc[i][1][3]);
+        col += 32 * nw;
     }
-}
-
-// WARP_PRIVATE: which of the two a caller wants (small batches: block-wide, one barrier in all; larger: per warp).
-template <int IPW, bool WARP_PRIVATE>
-__device__ __forceinline__ void mlp_scatter_add(const float (&acc)[IPW][2][4], float *stage, float *acc_g, int batch,
-                                                int D, int nw)
-{
-    if (WARP_PRIVATE) mlp_scatter_add_warp<IPW>(acc, stage, acc_g, batch, D, nw);
-    else mlp_scatter_add_block<IPW>(acc, stage, acc_g, batch, D, nw);
 }
 
 }  // namespace fasttps

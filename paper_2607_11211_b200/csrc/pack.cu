@@ -9,8 +9,10 @@
 //     column 8J + r for r < 8 and up column 8J + r - 8 otherwise (interlaced in blocks of 8).
 //   DOWN ("octet blocks"): for intermediate octet o and output block nb (32 columns) one
 //     512-byte block; lane (g, t4) of a warp owns 16 bytes of it: the pairs
-//     (W[8o + 2 t4][n], W[8o + 2 t4 + 1][n]) for n = 32 nb + g + {0, 8, 16, 24}, i.e. the A
-//     fragments of two m16n8k8 MMAs.  Blocks ordered by (o, nb).
+//     (W[8o + 2 t4][n], W[8o + 2 t4 + 1][n]) for n = 32 nb + 4 g + {0, 1, 2, 3}, i.e. the A
+//     fragments of two m16n8k8 MMAs whose rows g, g + 8 (first MMA) and g, g + 8 (second) are
+//     four consecutive output columns: the products leave the registers as 16-byte vectors.
+//     Blocks ordered by (o, nb).
 #include "common.cuh"
 
 namespace fasttps {
@@ -66,7 +68,7 @@ __global__ void pack_down_kernel(const __nv_bfloat16 *logical, __nv_bfloat16 *pa
     const int o = (int)(blk / NT), nb = (int)(blk % NT);
     __nv_bfloat16 *pv = packed + v * 8;
     for (int e = 0; e < 8; ++e) {
-        const int j = 8 * o + 2 * t4 + (e & 1), n = 32 * nb + g + 8 * (e >> 1);
+        const int j = 8 * o + 2 * t4 + (e & 1), n = 32 * nb + 4 * g + (e >> 1);
         const size_t li = (size_t)j * D + n;
         if (inverse) const_cast<__nv_bfloat16 *>(logical)[li] = pv[e];
         else pv[e] = logical[li];

@@ -60,7 +60,8 @@ def test_pack_unpack_round_trip_and_interlace(fb, dims):
     assert torch.equal(p.view(torch.int16), tiled(w["w_gu"].t()[col]).view(torch.int16))
     assert torch.equal(ctx.pack_weight(fb.W_QKV, w["w_qkv"]).view(torch.int16),
                        tiled(w["w_qkv"].t()).view(torch.int16))
-    # down: per (octet, 32-column block) one 512-byte block of m16n8k8 A fragments
+    # down: per (octet, 32-column block) one 512-byte block of m16n8k8 A fragments; a lane's four rows of its two
+    # MMA tiles are four consecutive output columns
     pd = ctx.pack_weight(fb.W_DOWN, w["w_down"]).view(K // 8, D // 32, 32, 4, 2)
     lane = torch.arange(32, device="cuda")
     g, t4 = lane // 4, lane % 4
@@ -68,7 +69,7 @@ def test_pack_unpack_round_trip_and_interlace(fb, dims):
     for q in range(4):
         for jj in range(2):
             want = wd[:, 2 * t4 + jj][:, :, :, :].permute(0, 2, 1, 3)      # [o, nb, lane, n32]
-            want = want[:, :, lane, g + 8 * q]
+            want = want[:, :, lane, 4 * g + q]
             assert torch.equal(pd[:, :, :, q, jj].view(torch.int16), want.contiguous().view(torch.int16))
     ctx.close()
 
