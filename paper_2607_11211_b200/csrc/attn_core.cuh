@@ -130,6 +130,14 @@ struct AttnScratch {
     int last;
 };
 
+// PRE (attn_consume): rope(q), bf16(rope(k_new)) and v_new of ALL segments of a share, prepared in one pass
+template <int DH>
+struct AttnPre {
+    alignas(16) float q[kMaxNB][DH];
+    alignas(16) __nv_bfloat16 knew[kMaxNB][DH];
+    alignas(16) __nv_bfloat16 vnew[kMaxNB][DH];
+};
+
 template <int DH> struct AttnTile {
     static constexpr int kRowBytes = DH * 2;
     static constexpr int kPieceBytes = 2 * kAttnTileRows * kRowBytes;     // K tile then V tile
@@ -178,9 +186,9 @@ __device__ __forceinline__ bool attn_produce(const AttnArgs &a, WeightRing &ring
 // Returns false (in every consumer thread alike) if a bounded wait ran out.
 // DEFER: the partial of every segment is published (even when the CTA owns the whole head) and nobody
 // merges here; the caller merges the partials of a head itself (the persistent step kernel does, per group).
-template <int DH, bool DEFER, class Src, bool LATE_FENCE = false>
+template <int DH, bool DEFER, class Src, bool LATE_FENCE = false, bool PRE = false>
 __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring, int &piece, int cta, Src src,
-                                             AttnScratch<DH> &sm, int nwc)
+                                             AttnScratch<DH> &sm, int nwc, AttnPre<DH> *pre = nullptr)
 {
     constexpr int EPL = DH / kLanesPerRow;      // elements per lane of a row
     constexpr int VPL = EPL / 8;                // 16-byte vectors per lane
@@ -198,36 +206,55 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
     bool ok = true;
     bool appended = false;
 
+    // element i (and i + HALF) of the rotated q of segment s, and of its new K/V row when the segment holds it
+    auto rope_one = [&](const Segment &s, int i, float *qv, __nv_bfloat16 *knew, __nv_bfloat16 *vnew) {
+        const int hq = s.h, hk = hq / G, b = s.b;
+        const float c = a.cos_tab[(size_t)s.pos * HALF + i], sn = a.sin_tab[(size_t)s.pos * HALF + i];
+        const __nv_bfloat16 *qg = a.q + (size_t)b * a.q_stride + (size_t)hq * DH;
+        const float x0 = __bfloat162float(ld_cg_bf16(qg + i)), x1 = __bfloat162float(ld_cg_bf16(qg + i + HALF));
+        qv[i] = __fsub_rn(__fmul_rn(x0, c), __fmul_rn(x1, sn));
+        qv[i + HALF] = __fadd_rn(__fmul_rn(x1, c), __fmul_rn(x0, sn));
+        if (s.r1 > s.L) {
+            const __nv_bfloat16 *kg = a.k_new + (size_t)b * a.kv_stride + (size_t)hk * DH;
+            const float k0 = __bfloat162float(ld_cg_bf16(kg + i)), k1 = __bfloat162float(ld_cg_bf16(kg + i + HALF));
+            knew[i] = __float2bfloat16_rn(__fsub_rn(__fmul_rn(k0, c), __fmul_rn(k1, sn)));
+            knew[i + HALF] = __float2bfloat16_rn(__fadd_rn(__fmul_rn(k1, c), __fmul_rn(k0, sn)));
+            const __nv_bfloat16 *vg = a.v_new + (size_t)b * a.kv_stride + (size_t)hk * DH;
+            vnew[i] = ld_cg_bf16(vg + i);
+            vnew[i + HALF] = ld_cg_bf16(vg + i + HALF);
+        }
+    };
+    if constexpr (PRE) {
+        // every (segment, element) pair of the share has a thread of its own: the loads of all segments go out
+        // together and cost one round trip to the L2, not one per segment
+        const int nseg = src.count();
+        for (int idx = t; idx < nseg * HALF; idx += nct) {
+            const int n = idx / HALF;
+            rope_one(src.at(n), idx - n * HALF, pre->q[n], pre->knew[n], pre->vnew[n]);
+        }
+        named_bar_sync(1, nct);
+    }
+
     Segment sg;
-    while (src.next(sg)) {
+    int segi = 0;
+    for (; src.next(sg); ++segi) {
         const int hq = sg.h, hk = hq / G, b = sg.b, L = sg.L;
         const bool has_new = sg.r1 > L;
         const int c1 = has_new ? L : sg.r1;
         const size_t slab = ((size_t)b * a.n_kv_heads + hk) * (size_t)a.max_seq * DH;
 
         // ---- joint RoPE of q and k_new with one set of cos/sin (Algorithm 3, steps 6-8) ----
-        for (int i = t; i < HALF; i += nct) {
-            const float c = a.cos_tab[(size_t)sg.pos * HALF + i], s = a.sin_tab[(size_t)sg.pos * HALF + i];
-            const __nv_bfloat16 *qg = a.q + (size_t)b * a.q_stride + (size_t)hq * DH;
-            const float x0 = __bfloat162float(ld_cg_bf16(qg + i)), x1 = __bfloat162float(ld_cg_bf16(qg + i + HALF));
-            sm.q[i] = __fsub_rn(__fmul_rn(x0, c), __fmul_rn(x1, s));
-            sm.q[i + HALF] = __fadd_rn(__fmul_rn(x1, c), __fmul_rn(x0, s));
-            if (has_new) {
-                const __nv_bfloat16 *kg = a.k_new + (size_t)b * a.kv_stride + (size_t)hk * DH;
-                const float k0 = __bfloat162float(ld_cg_bf16(kg + i)), k1 = __bfloat162float(ld_cg_bf16(kg + i + HALF));
-                sm.knew[i] = __float2bfloat16_rn(__fsub_rn(__fmul_rn(k0, c), __fmul_rn(k1, s)));
-                sm.knew[i + HALF] = __float2bfloat16_rn(__fadd_rn(__fmul_rn(k1, c), __fmul_rn(k0, s)));
-                const __nv_bfloat16 *vg = a.v_new + (size_t)b * a.kv_stride + (size_t)hk * DH;
-                sm.vnew[i] = ld_cg_bf16(vg + i);
-                sm.vnew[i + HALF] = ld_cg_bf16(vg + i + HALF);
-            }
+        float *qv = PRE ? pre->q[segi] : sm.q;
+        __nv_bfloat16 *knew = PRE ? pre->knew[segi] : sm.knew, *vnew = PRE ? pre->vnew[segi] : sm.vnew;
+        if (!PRE) {
+            for (int i = t; i < HALF; i += nct) rope_one(sg, i, qv, knew, vnew);
+            named_bar_sync(1, nct);
         }
-        named_bar_sync(1, nct);
         // ---- GKVC append (Eq. 2; Algorithm 3 steps 1 and 9): one write per row, no reload ----
         if (has_new && (hq % G) == 0) {
             for (int i = t; i < DH / 8; i += nct) {
-                reinterpret_cast<uint4 *>(a.k_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(sm.knew)[i];
-                reinterpret_cast<uint4 *>(a.v_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(sm.vnew)[i];
+                reinterpret_cast<uint4 *>(a.k_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(knew)[i];
+                reinterpret_cast<uint4 *>(a.v_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(vnew)[i];
             }
             // bulk copies of a later step of the same launch must see these rows: the stores are ordered before the
             // asynchronous proxy, here or (LATE_FENCE) after the last segment
@@ -237,7 +264,7 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
 
         float qr[EPL];
 #pragma unroll
-        for (int i = 0; i < EPL; ++i) qr[i] = sm.q[sub * EPL + i];
+        for (int i = 0; i < EPL; ++i) qr[i] = qv[sub * EPL + i];
         float m_run = -INFINITY, l_run = 0.f;
         float acc[EPL];
 #pragma unroll
@@ -302,8 +329,8 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
 
         // ---- the new row, straight from shared memory (never re-read from the cache) ----
         if (has_new && warp == 0) {
-            const float sc = dot_row(reinterpret_cast<const unsigned char *>(sm.knew));
-            update(sc, rgrp == 0, reinterpret_cast<const unsigned char *>(sm.vnew));
+            const float sc = dot_row(reinterpret_cast<const unsigned char *>(knew));
+            update(sc, rgrp == 0, reinterpret_cast<const unsigned char *>(vnew));
         }
 
         // ---- combine the row groups of a warp, then the warps of the CTA ----

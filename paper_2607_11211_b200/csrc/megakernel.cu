@@ -44,6 +44,8 @@ struct GroupSource {
         s = p->seg[i++];
         return true;
     }
+    __device__ __forceinline__ int count() const { return p->n; }
+    __device__ __forceinline__ const Segment &at(int n) const { return p->seg[n]; }
 };
 
 // BC: batch class.  0: batch 1 (the batch loops fold away at compile time), 1: batch 2, 2: batches 3 to 8 (which
@@ -136,6 +138,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
     __shared__ LayerPtrs s_layers[kMaxStepLayers];               // the layer table: no global round trip per phase
     __shared__ GroupSegs s_segs;                                 // this CTA's attention share for the current step
     __shared__ int s_cuts[kMaxSplits + 1];                       // row cuts of the shares of a head in the current step
+    __shared__ AttnPre<DH> s_pre;                                // the rotated q (and new K/V rows) of all segments of the share
     __shared__ int s_mprime;                                     // CTAs of a group that hold rows in the current step
     __shared__ int s_ncta[kMaxNB];                               // partials of (sequence b, this head) in the current step
     __shared__ __align__(16) __nv_bfloat16 s_outh[kMaxNB * DH];  // the merged outputs of this CTA's head, per sequence
@@ -322,7 +325,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
             if (kind == kAttn) {
                 // ---- attention (Algorithm 3) on this CTA's rows of its head; the partial is published ----
                 const AttnArgs aa = attn_args_of(a, lp, step, gm * a.n_q_heads);
-                ok = attn_consume<DH, true, GroupSource, BC != 0>(aa, ring, piece, cta, GroupSource(&s_segs), scratch, nw) && ok;
+                ok = attn_consume<DH, true, GroupSource, BC != 0, BC != 0>(aa, ring, piece, cta, GroupSource(&s_segs), scratch, nw, &s_pre) && ok;
                 grp_target += (unsigned)mprime;
                 if (in_group) {
                     // ---- the group meets: every CTA of it needs the merged output of the head ----
