@@ -386,6 +386,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(StepArg
                     for (int j = 0; j < KB; ++j)
                         bh[j] = g < B ? *reinterpret_cast<const uint4 *>(s_outh + g * DH + 32 * j + 8 * t4) : make_uint4(0u, 0u, 0u, 0u);
                     float *hsum = hacc + (size_t)(l & 1) * B * D;
+#pragma unroll(BC == 0 ? 1 : 2)
                     for (int p0 = 0; p0 < ont; p0 += TP, ++piece) {
                         const int nt = ont - p0 < TP ? ont - p0 : TP;
                         const unsigned char *slot = ring.wait(piece, ok);
