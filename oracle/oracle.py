@@ -240,3 +240,36 @@ def model_decode(embed, layers, g_final, w_lm, k_caches, v_caches, token_ids, po
     if want_hidden:
         return logits, next_ids, hidden
     return logits, next_ids
+
+
+def attn_float_baseline(q, k_new, v_new, k_cache, v_cache, pos, seq_lens, theta=10000.0):
+    """Decode attention with no reduced-precision step after the inputs: the "float" baseline of the
+    paper's accuracy experiment (Section 5.4, "Accuracy Stability"; Fig. 8), written out in numpy
+    float64 from the definition (half-split RoPE, scores over the cached rows and the new row,
+    softmax with the 1/sqrt(d) scale, PV).  Unlike ``attn_decode`` the rotated new K row is NOT
+    rounded to bf16 before it is scored and the output is NOT rounded; the caches are not modified.
+    Inputs are bf16 bit patterns; returns float64 [B, Hq, d].  Sequences the method would skip
+    (full cache, negative position) are not handled here."""
+    q, k_new, v_new = bf16_to_f32(_u16(q)).astype(np.float64), bf16_to_f32(_u16(k_new)).astype(np.float64), \
+        bf16_to_f32(_u16(v_new)).astype(np.float64)
+    B, Hq, d = q.shape
+    Hkv = k_new.shape[1]
+    G = Hq // Hkv
+    half = d // 2
+    freq = theta ** (-2.0 * np.arange(half) / d)
+    out = np.zeros((B, Hq, d))
+
+    def rot(v, p):
+        c, s = np.cos(p * freq), np.sin(p * freq)
+        return np.concatenate([v[:half] * c - v[half:] * s, v[half:] * c + v[:half] * s])
+
+    for b in range(B):
+        L, p = int(seq_lens[b]), int(pos[b])
+        for h in range(Hq):
+            hk = h // G
+            K = np.vstack([bf16_to_f32(k_cache[b, hk, :L]).astype(np.float64), rot(k_new[b, hk], p)[None]])
+            V = np.vstack([bf16_to_f32(v_cache[b, hk, :L]).astype(np.float64), v_new[b, hk][None]])
+            s = K @ rot(q[b, h], p) / np.sqrt(d)
+            e = np.exp(s - s.max())
+            out[b, h] = (e / e.sum()) @ V
+    return out

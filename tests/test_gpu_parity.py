@@ -10,7 +10,8 @@ import torch
 
 from oracle import oracle as orc
 from paper_2607_11211_b200 import workload as wl
-from tests.helpers import assert_close_bits, from_bf16_bits as F32, to_bf16_bits as B16, ulp_distance
+from tests.helpers import (assert_close_bits, from_bf16_bits as F32, to_bf16_bits as B16, ulp_distance, fig8_case,
+                           FIG8_BOUND, FIG8_LENGTHS)
 
 pytestmark = pytest.mark.gpu
 
@@ -184,6 +185,30 @@ def test_attn_decode_ragged_batches(fb, dims):
 @pytest.mark.parametrize("lens", [[256], [4095], [1024, 1, 2500]])
 def test_attn_decode_phi3_shape(fb, lens):
     run_attn_case(fb, wl.PHI3_MINI, lens, 4096)
+
+
+
+@pytest.mark.parametrize("n_t", FIG8_LENGTHS)
+def test_attn_decode_error_against_a_float_baseline_stays_below_the_papers_bound(fb, n_t):
+    """Section 5.4 "Accuracy Stability" / Fig. 8 on the GPU path: Phi-3 head shape, values uniform in [0, 1),
+    maximum absolute deviation from the float64 baseline < 0.22 % at every length; what is left is the rounding
+    of the output (the GPU agrees with the bf16 oracle to one ulp)."""
+    q, kn, vn, kc, vc, pos, L = fig8_case(n_t)
+    dims = wl.PHI3_MINI
+    ctx = make_ctx(fb, dims, 1, n_t)
+    kcd, vcd = dev(kc), dev(vc)
+    out = torch.zeros(1, dims.n_q_heads, dims.head_dim, dtype=torch.bfloat16, device="cuda")
+    ctx.attn_decode(dev(q), dev(kn), dev(vn), kcd, vcd, i32(pos), i32(L), out)
+    torch.cuda.synchronize()
+    assert ctx.get_status() == 0
+    got = wl.bits(out)
+    base = orc.attn_float_baseline(q, kn, vn, kc, vc, pos, L)
+    err = np.abs(F32(got).astype(np.float64) - base).max()
+    print(f"fig8 n_t={n_t} max_abs_err={err:.6f}")
+    assert err < FIG8_BOUND, (n_t, err)
+    want = orc.attn_decode(q, kn, vn, kc.copy(), vc.copy(), pos, L)
+    assert ulp_distance(got, want).max() <= 1
+    ctx.close()
 
 
 def test_attn_decode_batch_32_uses_a_single_split_path(fb):
