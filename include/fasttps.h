@@ -218,6 +218,9 @@ int fasttps_model_decode_host(fasttps_ctx *ctx, const void *embed, const fasttps
 /* Tuning switches of a context (host side, take effect at the next call):
  *   "step_kernel" 0/1  route model calls with batch <= 8 through the persistent step kernel
  *                      (default: environment variable FASTTPS_STEP_KERNEL, else 1).
+ *   "gqa_share" 0/1    fasttps_attn_decode and the per-product chain read every cached K/V row once for
+ *                      the whole group of query heads that shares it (Section 4.1; groups of 2, 4 or 8)
+ *                      instead of once per query head (default 1; 0 is the comparison point).
  * Unknown names return FASTTPS_INVALID_ARG. */
 int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value);
 

@@ -90,6 +90,7 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
         const char *e = getenv("FASTTPS_STEP_KERNEL");
         c->opt_step_kernel = (e && *e) ? atoi(e) != 0 : 1;
     }
+    c->opt_gqa_share = 1;
     {
         int rc = configure_attn_kernels();
         if (rc == FASTTPS_OK) rc = configure_linear_kernels();
@@ -348,6 +349,7 @@ int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value)
     if (!ctx || !name) return FASTTPS_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);
     if (strcmp(name, "step_kernel") == 0) c->opt_step_kernel = value != 0;
+    else if (strcmp(name, "gqa_share") == 0) c->opt_gqa_share = value != 0;
     else return FASTTPS_INVALID_ARG;
     return FASTTPS_OK;
 }

@@ -1,6 +1,7 @@
 // Stand-alone fused decode attention kernel (Algorithm 3 of the paper, "GKVC & TPSFLAT"):
 // one CTA per SM, 8 consumer warps + 1 producer warp around the shared-memory ring.
 // The algorithm lives in attn_core.cuh.
+#include <type_traits>
 #include "attn_core.cuh"
 
 namespace fasttps {
@@ -9,20 +10,37 @@ namespace {
 
 constexpr int kAttnWarps = 8;                           // consumer warps
 constexpr int kAttnThreads = (kAttnWarps + 1) * 32;     // + the producer warp
+constexpr int kMaxShareGroup = 8;                       // query heads per K/V head served by one pass over the rows
+
+// Grouped-query attention with 2, 4 or 8 query heads per K/V head streams every cached row once for the whole
+// group (the worker warps divide into the group's query heads); other ratios stream it once per query head.
+inline bool attn_shares_groups(int n_q_heads, int n_kv_heads)
+{
+    const int G = n_kv_heads > 0 ? n_q_heads / n_kv_heads : 1;
+    return G > 1 && G <= kMaxShareGroup && kAttnWarps % G == 0 && kAttnWarps <= kAttnMaxWorkers;
+}
 
 template <int DH>
 struct AttnSmem {
-    static constexpr int kSlots = (192 * 1024 / AttnTile<DH>::kPieceBytes) < 8 ? (192 * 1024 / AttnTile<DH>::kPieceBytes) : 8;
+    // a power of two (the ring finds slot and round of a piece by mask and shift): 8 pieces of up to 24 KB,
+    // 4 of the 32 KB pieces of head_dim 128
+    static constexpr int kFit = 192 * 1024 / AttnTile<DH>::kPieceBytes;
+    static constexpr int kSlots = kFit >= 8 ? 8 : kFit >= 4 ? 4 : 2;
+    static_assert((kSlots & (kSlots - 1)) == 0 && kSlots <= kFit, "ring slot count must be a power of two that fits");
     alignas(128) unsigned char slots[kSlots][AttnTile<DH>::kPieceBytes];
     alignas(16) uint64_t bars[2 * kSlots];
     AttnScratch<DH> scratch;
     int abort;
 };
-
 template <int DH>
+struct AttnSmemShare : AttnSmem<DH> {
+    alignas(16) float qgroup[kMaxShareGroup][DH];       // rope(q) of the query heads of a group
+};
+
+template <int DH, bool SHARE>
 __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a)
 {
-    using Smem = AttnSmem<DH>;
+    using Smem = typename std::conditional<SHARE, AttnSmemShare<DH>, AttnSmem<DH>>::type;
     extern __shared__ unsigned char smem_raw[];
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     const int t = threadIdx.x, warp = t >> 5;
@@ -38,7 +56,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a
 
     int piece = 0;
     if (warp == kAttnWarps) {
-        if ((t & 31) == 0) (void)attn_produce<DH>(a, ring, piece, blockIdx.x, gridDim.x);
+        if ((t & 31) == 0) (void)attn_produce<DH, SHARE>(a, ring, piece, blockIdx.x, gridDim.x);
         return;
     }
     if (blockIdx.x == 0 && t == 0) {
@@ -49,8 +67,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a
             else if (p < 0 || p >= a.max_seq) atomicOr(a.status, FASTTPS_DEV_BAD_POSITION);
         }
     }
-    if (!attn_consume<DH, false>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x), sm.scratch, kAttnWarps) && t == 0)
-        atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT);
+    bool done;
+    if constexpr (SHARE)
+        done = attn_consume<DH, false, WalkSource, false, false, true>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x, true),
+                                                                       sm.scratch, kAttnWarps, nullptr, &sm.qgroup[0][0]);
+    else
+        done = attn_consume<DH, false>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x), sm.scratch, kAttnWarps);
+    if (!done && t == 0) atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT);
 }
 
 }  // namespace
@@ -61,7 +84,8 @@ int attn_splits_for(const Ctx *c, int batch)
 {
     int n = c->n_sm;
     (void)batch;
-    const int cap = (kMaxSplits - 2) * c->cfg.n_q_heads;
+    // heads of the flattened row space: K/V heads when a group shares its rows
+    const int cap = (kMaxSplits - 2) * ((c->opt_gqa_share && attn_shares_groups(c->cfg.n_q_heads, c->cfg.n_kv_heads)) ? c->cfg.n_kv_heads : c->cfg.n_q_heads);
     if (n > cap) n = cap;
     return n < 1 ? 1 : n;
 }
@@ -69,21 +93,30 @@ int attn_splits_for(const Ctx *c, int batch)
 template <int DH>
 static int launch_attn_dh(Ctx *c, const AttnArgs &a, cudaStream_t st)
 {
-    const size_t smem = sizeof(AttnSmem<DH>) + 128;
     dim3 grid(a.n_splits);
     ProfScope prof(c, kProfAttn, st);
-    const int rc = launch_ex(attn_decode_kernel<DH>, grid, dim3(kAttnThreads), smem, st, &a);
+    const int rc = (c->opt_gqa_share && attn_shares_groups(a.n_q_heads, a.n_kv_heads))
+                       ? launch_ex(attn_decode_kernel<DH, true>, grid, dim3(kAttnThreads), sizeof(AttnSmemShare<DH>) + 128, st, &a)
+                       : launch_ex(attn_decode_kernel<DH, false>, grid, dim3(kAttnThreads), sizeof(AttnSmem<DH>) + 128, st, &a);
     c->launches++;
     return rc;
 }
 
+template <int DH>
+static int configure_attn_dh()
+{
+    FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmem<DH>) + 128));
+    FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmemShare<DH>) + 128));
+    return FASTTPS_OK;
+}
+
 int configure_attn_kernels()
 {
-    FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmem<32>) + 128));
-    FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmem<64>) + 128));
-    FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<96>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmem<96>) + 128));
-    FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmem<128>) + 128));
-    return FASTTPS_OK;
+    int rc;
+    if ((rc = configure_attn_dh<32>()) != FASTTPS_OK) return rc;
+    if ((rc = configure_attn_dh<64>()) != FASTTPS_OK) return rc;
+    if ((rc = configure_attn_dh<96>()) != FASTTPS_OK) return rc;
+    return configure_attn_dh<128>();
 }
 
 int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st)

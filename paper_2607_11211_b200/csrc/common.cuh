@@ -25,6 +25,7 @@ struct Ctx {
     LayerPtrs *d_layers, *pin_layers;
     int layers_uploaded;             // number of valid entries in pin_layers / d_layers
     int opt_step_kernel;             // 1: model calls with batch <= 8 use the persistent step kernel
+    int opt_gqa_share;               // 1: the attention kernel streams a K/V head once for its group of 2, 4 or 8 query heads
     fasttps_config cfg;
     int n_sm;
     cudaDeviceProp prop;

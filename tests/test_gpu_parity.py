@@ -211,6 +211,25 @@ def test_attn_decode_error_against_a_float_baseline_stays_below_the_papers_bound
     ctx.close()
 
 
+
+# Grouped-query shapes: Llama3-8B of Table 1 (32 query heads on 8 K/V heads, head_dim 128) and small shapes with 2
+# and 8 query heads per K/V head.  The attention kernel streams each K/V head once for its whole group.
+LLAMA3_8B_ATTN = wl.Dims(hidden=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, inter=14336, vocab=1000, n_layers=1)
+GQA_2 = wl.Dims(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, inter=384, vocab=520, n_layers=1)
+GQA_8 = wl.Dims(hidden=768, n_q_heads=8, n_kv_heads=1, head_dim=96, inter=384, vocab=520, n_layers=1)
+GQA_16 = wl.Dims(hidden=512, n_q_heads=16, n_kv_heads=1, head_dim=32, inter=384, vocab=520, n_layers=1)
+
+
+@pytest.mark.parametrize("dims,lens,max_seq", [
+    (LLAMA3_8B_ATTN, [4095], 4096), (LLAMA3_8B_ATTN, [0, 700, 3, 2047, 64], 2048), (LLAMA3_8B_ATTN, [256], 4096),
+    (GQA_2, [0, 1, 63, 64, 65, 300, 1000], 1024), (GQA_8, [5000], 5008), (GQA_8, [0, 7, 130], 256),
+    (GQA_16, [900, 2], 1024),          # 16 query heads per K/V head: not shared, one pass per query head
+])
+def test_attn_decode_grouped_query_shapes(fb, dims, lens, max_seq):
+    run_attn_case(fb, dims, lens, max_seq)
+    run_attn_case(fb, dims, lens, max_seq, pos=[max(0, l - 1) for l in lens])
+
+
 def test_attn_decode_batch_32_uses_a_single_split_path(fb):
     run_attn_case(fb, wl.SMALL, list(range(1, 330, 10))[:32], 384)
 
