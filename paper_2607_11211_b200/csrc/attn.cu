@@ -2,7 +2,7 @@
 // one CTA per SM, 8 consumer warps + 1 producer warp around the shared-memory ring.
 // The algorithm lives in attn_core.cuh.
 #include <type_traits>
-#include "attn_core.cuh"
+#include "attn_group_core.cuh"
 
 namespace fasttps {
 
@@ -10,14 +10,14 @@ namespace {
 
 constexpr int kAttnWarps = 8;                           // consumer warps
 constexpr int kAttnThreads = (kAttnWarps + 1) * 32;     // + the producer warp
-constexpr int kMaxShareGroup = 8;                       // query heads per K/V head served by one pass over the rows
+static_assert(kAttnWarps == kGroupWarps, "the grouped-query path needs one consumer warp per 8 rows of a tile");
 
-// Grouped-query attention with 2, 4 or 8 query heads per K/V head streams every cached row once for the whole
-// group (the worker warps divide into the group's query heads); other ratios stream it once per query head.
+// Grouped-query attention with 2 to 8 query heads per K/V head streams every cached row once for the whole
+// group, with the two products on the tensor cores; other ratios stream it once per query head.
 inline bool attn_shares_groups(int n_q_heads, int n_kv_heads)
 {
     const int G = n_kv_heads > 0 ? n_q_heads / n_kv_heads : 1;
-    return G > 1 && G <= kMaxShareGroup && kAttnWarps % G == 0 && kAttnWarps <= kAttnMaxWorkers;
+    return G > 1 && G <= kMaxShareGroup;
 }
 
 template <int DH>
@@ -33,8 +33,14 @@ struct AttnSmem {
     int abort;
 };
 template <int DH>
-struct AttnSmemShare : AttnSmem<DH> {
-    alignas(16) float qgroup[kMaxShareGroup][DH];       // rope(q) of the query heads of a group
+struct AttnSmemShare {
+    // the per-warp outputs of a whole group take DH KB: the ring gives up slots for them at head_dim 96
+    static constexpr int kFit = (int)(226 * 1024 - sizeof(GroupScratch<DH>)) / AttnTile<DH>::kPieceBytes;
+    static constexpr int kSlots = kFit >= 8 ? 8 : kFit >= 4 ? 4 : 2;
+    alignas(128) unsigned char slots[kSlots][AttnTile<DH>::kPieceBytes];
+    alignas(16) uint64_t bars[2 * kSlots];
+    GroupScratch<DH> scratch;
+    int abort;
 };
 
 template <int DH, bool SHARE>
@@ -69,8 +75,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a
     }
     bool done;
     if constexpr (SHARE)
-        done = attn_consume<DH, false, WalkSource, false, false, true>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x, true),
-                                                                       sm.scratch, kAttnWarps, nullptr, &sm.qgroup[0][0]);
+        done = attn_consume_group<DH>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x, true), sm.scratch);
     else
         done = attn_consume<DH, false>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x), sm.scratch, kAttnWarps);
     if (!done && t == 0) atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT);

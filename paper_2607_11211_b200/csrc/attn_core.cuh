@@ -18,11 +18,9 @@
 // round trip through global memory: it is scored from shared memory and written to the cache
 // exactly once.
 //
-// Grouped-query attention (Section 4.1: several query heads read one K/V head).  With SHARE the row
-// space is built over the K/V heads, so every cached row is fetched ONCE for its whole group: worker
-// warp w scores query head (w mod G) of the group on the row groups (w / G), (w / G) + 8 / G, ... of
-// every tile, all from the same shared-memory copy of the tile.  Without SHARE a segment is one query
-// head and a group's rows are streamed once per query head.
+// Grouped-query attention (Section 4.1: several query heads read one K/V head): here a segment is one
+// query head, and a group's rows are streamed once per query head.  attn_group_core.cuh holds the
+// variant that streams a K/V head once for its whole group.
 #pragma once
 #include "async_copy.cuh"
 
@@ -193,13 +191,10 @@ __device__ __forceinline__ bool attn_produce(const AttnArgs &a, WeightRing &ring
 // Returns false (in every consumer thread alike) if a bounded wait ran out.
 // DEFER: the partial of every segment is published (even when the CTA owns the whole head) and nobody
 // merges here; the caller merges the partials of a head itself (the persistent step kernel does, per group).
-// SHARE (grouped-query attention, G = 2, 4 or 8 dividing the worker count; not with DEFER or PRE): a segment is
-// a K/V head, `qgroup` holds G x DH floats of shared memory for the rotated queries of its group.
-template <int DH, bool DEFER, class Src, bool LATE_FENCE = false, bool PRE = false, bool SHARE = false>
+template <int DH, bool DEFER, class Src, bool LATE_FENCE = false, bool PRE = false>
 __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring, int &piece, int cta, Src src,
-                                             AttnScratch<DH> &sm, int nwc, AttnPre<DH> *pre = nullptr, float *qgroup = nullptr)
+                                             AttnScratch<DH> &sm, int nwc, AttnPre<DH> *pre = nullptr)
 {
-    static_assert(!SHARE || (!DEFER && !PRE), "the shared-group path serves the stand-alone kernel only");
     constexpr int EPL = DH / kLanesPerRow;      // elements per lane of a row
     constexpr int VPL = EPL / 8;                // 16-byte vectors per lane
     constexpr int HALF = DH / 2;
@@ -210,9 +205,6 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
     const int nwork = nwc < kAttnMaxWorkers ? nwc : kAttnMaxWorkers;
     const bool worker = warp < nwork;
     const int G = a.n_q_heads / a.n_kv_heads;
-    const int gq = SHARE ? warp % G : 0;             // SHARE: the query head of the group this warp scores ...
-    const int wrow = SHARE ? warp / G : warp;        // ... and its place among the warps of that head
-    const int wpg = SHARE ? nwork / G : nwork;
     const int sub = lane & (kLanesPerRow - 1);       // which quarter of the row
     const int rgrp = lane >> 2;                      // row within an 8-row group
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
@@ -251,30 +243,20 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
     Segment sg;
     int segi = 0;
     for (; src.next(sg); ++segi) {
-        const int hk = SHARE ? sg.h : sg.h / G, hq = SHARE ? sg.h * G + gq : sg.h, b = sg.b, L = sg.L;
+        const int hq = sg.h, hk = hq / G, b = sg.b, L = sg.L;
         const bool has_new = sg.r1 > L;
         const int c1 = has_new ? L : sg.r1;
         const size_t slab = ((size_t)b * a.n_kv_heads + hk) * (size_t)a.max_seq * DH;
 
         // ---- joint RoPE of q and k_new with one set of cos/sin (Algorithm 3, steps 6-8) ----
-        float *qv = SHARE ? qgroup + gq * DH : (PRE ? pre->q[segi] : sm.q);
+        float *qv = PRE ? pre->q[segi] : sm.q;
         __nv_bfloat16 *knew = PRE ? pre->knew[segi] : sm.knew, *vnew = PRE ? pre->vnew[segi] : sm.vnew;
-        if constexpr (SHARE) {
-            // the G queries of the group and the one new K row share the position's cos/sin
-            for (int idx = t; idx < G * HALF; idx += nct) {
-                const int g2 = idx / HALF;
-                Segment s2 = sg;
-                s2.h = sg.h * G + g2;
-                if (g2 > 0 && s2.r1 > s2.L) s2.r1 = s2.L;        // the new K/V row is prepared once, with query 0
-                rope_one(s2, idx - g2 * HALF, qgroup + g2 * DH, knew, vnew);
-            }
-            named_bar_sync(1, nct);
-        } else if (!PRE) {
+        if (!PRE) {
             for (int i = t; i < HALF; i += nct) rope_one(sg, i, qv, knew, vnew);
             named_bar_sync(1, nct);
         }
         // ---- GKVC append (Eq. 2; Algorithm 3 steps 1 and 9): one write per row, no reload ----
-        if (has_new && (SHARE || (hq % G) == 0)) {
+        if (has_new && (hq % G) == 0) {
             for (int i = t; i < DH / 8; i += nct) {
                 reinterpret_cast<uint4 *>(a.k_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(knew)[i];
                 reinterpret_cast<uint4 *>(a.v_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(vnew)[i];
@@ -339,7 +321,7 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
             const unsigned char *slot = ring.wait(piece, ok);
             if (worker) {
                 const int rows = (c1 - r) < kAttnTileRows ? (c1 - r) : kAttnTileRows;
-                for (int rg = wrow; rg < kAttnTileRows / 8; rg += wpg) {
+                for (int rg = warp; rg < kAttnTileRows / 8; rg += nwork) {
                     const int row = rg * 8 + rgrp;
                     const bool valid = ok && row < rows;
                     const unsigned char *krow = slot + row * kRowBytes;
@@ -351,7 +333,7 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
         }
 
         // ---- the new row, straight from shared memory (never re-read from the cache) ----
-        if (has_new && (SHARE ? warp < G : warp == 0)) {
+        if (has_new && warp == 0) {
             const float sc = dot_row(reinterpret_cast<const unsigned char *>(knew));
             update(sc, rgrp == 0, reinterpret_cast<const unsigned char *>(vnew));
         }
@@ -384,32 +366,12 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
             if (lane == 0) { sm.wm[warp] = m_run; sm.wl[warp] = l_run; }
         }
         if (!named_bar_and(1, nct, ok)) return false;
-        const bool whole = !DEFER && sg.n_cta == 1;      // this CTA alone finishes the head right here
-        if constexpr (SHARE) {
-            // the warps w = g2, g2 + G, ... hold query head g2 of the group
-            for (int idx = t; idx < G * DH; idx += nct) {
-                const int g2 = idx / DH, i = idx - g2 * DH, hq2 = hk * G + g2;
-                float M = -INFINITY;
-                for (int w = g2; w < nwork; w += G) M = fmaxf(M, sm.wm[w]);
-                float o = 0.f, l = 0.f;
-                for (int w = g2; w < nwork; w += G) {
-                    const float f = (sm.wm[w] == -INFINITY) ? 0.f : fast_exp2(sm.wm[w] - M);
-                    o += f * sm.wo[w][i];
-                    l += f * sm.wl[w];
-                }
-                if (whole) a.out[(size_t)b * a.out_stride + (size_t)hq2 * DH + i] = __float2bfloat16_rn(o / l);
-                else {
-                    float *part = a.part + (((size_t)b * a.n_q_heads + hq2) * kMaxSplits + (cta - sg.first_cta)) * kPartStride;
-                    part[i] = o;
-                    if (i == 0) { part[DH] = M; part[DH + 1] = l; }
-                }
-            }
-        } else {
         float M = -INFINITY;
         for (int w = 0; w < nwork; ++w) M = fmaxf(M, sm.wm[w]);
         __nv_bfloat16 *outp = a.out + (size_t)b * a.out_stride + (size_t)hq * DH;
         float *hp = a.part + ((size_t)b * a.n_q_heads + hq) * kMaxSplits * kPartStride;
         float *part = hp + (size_t)(cta - sg.first_cta) * kPartStride;
+        const bool whole = !DEFER && sg.n_cta == 1;      // this CTA alone finishes the head right here
         for (int i = t; i < DH; i += nct) {
             float o = 0.f, l = 0.f;
             for (int w = 0; w < nwork; ++w) {
@@ -423,20 +385,15 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
                 if (i == 0) { part[DH] = M; part[DH + 1] = l; }
             }
         }
-        }
         if (!DEFER && sg.n_cta > 1) {
             // ---- several CTAs share the head: the partial is published, the last one merges ----
             __threadfence();
             named_bar_sync(1, nct);
-            int *ticket = a.ticket + (size_t)b * a.n_q_heads + (SHARE ? hk * G : hq);
+            int *ticket = a.ticket + (size_t)b * a.n_q_heads + hq;
             if (t == 0) sm.last = (atomicAdd(ticket, 1) == sg.n_cta - 1);
             named_bar_sync(1, nct);
             if (sm.last) {
                 __threadfence();
-                for (int g2 = 0; g2 < (SHARE ? G : 1); ++g2) {       // SHARE: the G query heads of the group in turn
-                const int hqm = SHARE ? hk * G + g2 : hq;
-                const float *hp = a.part + ((size_t)b * a.n_q_heads + hqm) * kMaxSplits * kPartStride;
-                __nv_bfloat16 *outp = a.out + (size_t)b * a.out_stride + (size_t)hqm * DH;
                 // all loads of the merge are issued side by side: one lane per partial for (max, sum) ...
                 if (warp == 0) {
                     const bool have = lane < sg.n_cta;
@@ -463,8 +420,6 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
                         for (int u = 0; u < 8; ++u) oo = fmaf(sm.mf[(s0 + u) & (kMaxSplits - 1)], v[u], oo);
                     }
                     outp[i] = __float2bfloat16_rn(oo / sm.wl[0]);
-                }
-                if (SHARE) named_bar_sync(1, nct);                    // the merge factors are reused by the next head
                 }
                 if (t == 0) *ticket = 0;
             }

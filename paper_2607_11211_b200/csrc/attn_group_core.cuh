@@ -1,0 +1,264 @@
+// Decode attention for grouped-query models (Section 4.1 of the paper: G query heads read one K/V head;
+// Algorithm 3 is otherwise unchanged): every cached K/V row is fetched ONCE for its whole group.
+//
+// With G query vectors per row the two products of Algorithm 3 are thin matrix products, so they run on the
+// tensor cores (the FP32 dot products of attn_core.cuh already keep the ALUs as busy as HBM at G = 1; G times
+// the arithmetic per byte would make the kernel compute-bound):
+//   scores  S[head, key] = Q[head, :] . K[key, :]      mma m16n8k16, A = Q (heads 0..7 in the rows; rows 8..15
+//                                                       are padding), B = 8 keys of the tile
+//   output  O[head, col] += P[head, key] V[key, col]    mma m16n8k8,  A = P straight from the score fragment
+// A tile of the ring holds 64 rows; consumer warp w owns rows 8w .. 8w+7 of every tile and keeps its own
+// running (max, sum, output) for the G heads; the warps' states are merged per segment as in attn_core.cuh.
+// Operand order is free inside a dot product, so the head_dim index is permuted such that one 16-byte load of a
+// K row feeds two MMAs, and the output columns are permuted such that two V rows loaded as 32-bit words give
+// the B operands of two MMAs after a byte permute (no transposing load, no swizzled tile).
+// Precision: q is split into bf16 hi + lo (two score MMAs: the FP32 rotated q is kept to 2^-17), the
+// probabilities enter the second product rounded to bf16, and the row sum is taken over the rounded values.
+#pragma once
+#include "attn_core.cuh"
+#include "dot_core.cuh"
+
+namespace fasttps {
+
+constexpr int kMaxShareGroup = 8;        // query heads per K/V head this path serves (2, 4 or 8)
+constexpr int kGroupWarps = 8;           // consumer warps: one per 8 rows of a tile
+
+template <int DH>
+struct GroupScratch {
+    alignas(16) float q[kMaxShareGroup][DH];            // rope(q) of the group, FP32
+    alignas(16) __nv_bfloat16 knew[DH];                 // bf16(rope(k_new)): the row that goes into the cache
+    alignas(16) __nv_bfloat16 vnew[DH];
+    float wm[kGroupWarps][kMaxShareGroup], wl[kGroupWarps][kMaxShareGroup];   // per warp and head: max (log2 domain), sum
+    alignas(16) float wo[kGroupWarps][kMaxShareGroup][DH];
+    float mf[kMaxSplits];                               // merge factors of the partials of a shared head
+    float lsum;
+    int last;
+};
+
+
+// The MMAs of this path use rows 0..7 of the 16-row tile only (rows 8..15 of A are zero): the lower half of the
+// accumulator fragment is not kept (its inputs are constants, its outputs are dropped), which halves the
+// registers the running outputs take.
+__device__ __forceinline__ void mma_top_k16(float (&c)[2], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1)
+{
+    float d2, d3;
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%5}, {%7,%8}, {%0,%1,%9,%9};"
+                 : "+f"(c[0]), "+f"(c[1]), "=f"(d2), "=f"(d3)
+                 : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1), "f"(0.f));
+}
+__device__ __forceinline__ void mma_top_k8(float (&c)[2], uint32_t a0, uint32_t b0)
+{
+    float d2, d3;
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%7,%7};"
+                 : "+f"(c[0]), "+f"(c[1]), "=f"(d2), "=f"(d3)
+                 : "r"(a0), "r"(0u), "r"(b0), "f"(0.f));
+}
+
+// Consumer warps (kGroupWarps of them, threads 0 .. 255, synchronised by named barrier 1).  The segments of
+// `src` are K/V heads (WalkSource with share = true).  Returns false in every thread if a bounded wait ran out.
+template <int DH>
+__device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing &ring, int &piece, int cta, WalkSource src,
+                                                   GroupScratch<DH> &sm)
+{
+    constexpr int HALF = DH / 2;
+    constexpr int KB = DH / 32;                  // 32-wide blocks of head_dim in the score product
+    constexpr int JB = DH / 16;                  // 16-column blocks of the output
+    constexpr int kRowBytes = DH * 2;
+    constexpr int kPartStride = DH + 4;
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5, g = lane >> 2, t4 = lane & 3;
+    const int nct = kGroupWarps * 32;
+    const int G = a.n_q_heads / a.n_kv_heads;
+    const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
+    bool ok = true;
+
+    Segment sg;
+    while (src.next(sg)) {
+        const int hk = sg.h, b = sg.b, L = sg.L;
+        const bool has_new = sg.r1 > L;
+        const int c1 = has_new ? L : sg.r1;
+        const size_t slab = ((size_t)b * a.n_kv_heads + hk) * (size_t)a.max_seq * DH;
+
+        // ---- joint RoPE of the G queries and k_new with one set of cos/sin (Algorithm 3, steps 6-8) ----
+        for (int idx = t; idx < G * HALF; idx += nct) {
+            const int g2 = idx / HALF, i = idx - g2 * HALF;
+            const float c = a.cos_tab[(size_t)sg.pos * HALF + i], sn = a.sin_tab[(size_t)sg.pos * HALF + i];
+            const __nv_bfloat16 *qg = a.q + (size_t)b * a.q_stride + (size_t)(hk * G + g2) * DH;
+            const float x0 = __bfloat162float(ld_cg_bf16(qg + i)), x1 = __bfloat162float(ld_cg_bf16(qg + i + HALF));
+            sm.q[g2][i] = __fsub_rn(__fmul_rn(x0, c), __fmul_rn(x1, sn));
+            sm.q[g2][i + HALF] = __fadd_rn(__fmul_rn(x1, c), __fmul_rn(x0, sn));
+            if (g2 == 0 && has_new) {
+                const __nv_bfloat16 *kg = a.k_new + (size_t)b * a.kv_stride + (size_t)hk * DH;
+                const float k0 = __bfloat162float(ld_cg_bf16(kg + i)), k1 = __bfloat162float(ld_cg_bf16(kg + i + HALF));
+                sm.knew[i] = __float2bfloat16_rn(__fsub_rn(__fmul_rn(k0, c), __fmul_rn(k1, sn)));
+                sm.knew[i + HALF] = __float2bfloat16_rn(__fadd_rn(__fmul_rn(k1, c), __fmul_rn(k0, sn)));
+                const __nv_bfloat16 *vg = a.v_new + (size_t)b * a.kv_stride + (size_t)hk * DH;
+                sm.vnew[i] = ld_cg_bf16(vg + i);
+                sm.vnew[i + HALF] = ld_cg_bf16(vg + i + HALF);
+            }
+        }
+        named_bar_sync(1, nct);
+        // ---- GKVC append (Eq. 2; Algorithm 3 steps 1 and 9): one write per row, no reload ----
+        if (has_new) {
+            for (int i = t; i < DH / 8; i += nct) {
+                reinterpret_cast<uint4 *>(a.k_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(sm.knew)[i];
+                reinterpret_cast<uint4 *>(a.v_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(sm.vnew)[i];
+            }
+            asm volatile("fence.proxy.async;" ::: "memory");
+        }
+
+        // ---- A fragments of the score product: head g of the group, bf16 hi + lo of 8 consecutive elements ----
+        uint4 qhi[KB], qlo[KB];
+#pragma unroll
+        for (int kb = 0; kb < KB; ++kb) {
+            float f[8];
+            if (g < G) {
+                const float4 f0 = *reinterpret_cast<const float4 *>(&sm.q[g][kb * 32 + 8 * t4]);
+                const float4 f1 = *reinterpret_cast<const float4 *>(&sm.q[g][kb * 32 + 8 * t4 + 4]);
+                f[0] = f0.x; f[1] = f0.y; f[2] = f0.z; f[3] = f0.w; f[4] = f1.x; f[5] = f1.y; f[6] = f1.z; f[7] = f1.w;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f[i] = 0.f;
+            }
+            float r[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) r[i] = f[i] - bf16_round(f[i]);
+            qhi[kb] = make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+            qlo[kb] = make_uint4(pack2(r[0], r[1]), pack2(r[2], r[3]), pack2(r[4], r[5]), pack2(r[6], r[7]));
+        }
+        float m_run = -INFINITY, l_run = 0.f;      // of head g; the sum holds this lane's keys only until the end
+        float oa[JB][2], ob[JB][2];                // output fragments of head g: columns 16 jb + 4 t4 + {0, 2} (oa) / {1, 3} (ob)
+#pragma unroll
+        for (int jb = 0; jb < JB; ++jb)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) oa[jb][e] = ob[jb][e] = 0.f;
+
+        // One block of up to 8 keys: rows key0 .. key0 + 7 of the K tile `kt` / V tile `vt`, of which the rows below
+        // `rows` exist.  Rows that do not exist are read from the last one that does (finite data) and get weight 0.
+        auto block = [&](const unsigned char *kt, const unsigned char *vt, int key0, int rows) {
+            // ---- scores (Algorithm 3 step 10): lane (g, t4) supplies key key0 + g, receives keys key0 + 2 t4 (+1) of head g ----
+            const int kr = key0 + g < rows ? key0 + g : rows - 1;
+            float s_hi[2] = {0.f, 0.f}, s_lo[2] = {0.f, 0.f};
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb) {
+                const uint4 kv = *reinterpret_cast<const uint4 *>(kt + (size_t)kr * kRowBytes + kb * 64 + t4 * 16);
+                mma_top_k16(s_hi, qhi[kb].x, qhi[kb].y, kv.x, kv.y);
+                mma_top_k16(s_lo, qlo[kb].x, qlo[kb].y, kv.x, kv.y);
+                mma_top_k16(s_hi, qhi[kb].z, qhi[kb].w, kv.z, kv.w);
+                mma_top_k16(s_lo, qlo[kb].z, qlo[kb].w, kv.z, kv.w);
+            }
+            // ---- online softmax (step 11) ----
+            const int ka = key0 + 2 * t4;
+            const bool v0 = ka < rows, v1 = ka + 1 < rows;
+            const float s0 = v0 ? (s_hi[0] + s_lo[0]) * scale_log2 : -INFINITY;
+            const float s1 = v1 ? (s_hi[1] + s_lo[1]) * scale_log2 : -INFINITY;
+            float mt = fmaxf(s0, s1);
+            mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 1));
+            mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 2));
+            const float m_new = fmaxf(m_run, mt);                  // finite: row key0 exists
+            const float corr = fast_exp2(m_run - m_new);           // 0 while m_run = -inf
+            const float p0 = v0 ? fast_exp2(s0 - m_new) : 0.f, p1 = v1 ? fast_exp2(s1 - m_new) : 0.f;
+            const uint32_t pa = pack2(p0, p1);
+            l_run = l_run * corr + bf16_round(p0) + bf16_round(p1);
+            m_run = m_new;
+            // ---- PV (step 12): B operands from rows ka and ka + 1 of V, two column sets per 32-bit word pair ----
+            const int r0 = ka < rows ? ka : rows - 1, r1 = ka + 1 < rows ? ka + 1 : rows - 1;
+            const unsigned char *vp0 = vt + (size_t)r0 * kRowBytes + g * 4, *vp1 = vt + (size_t)r1 * kRowBytes + g * 4;
+#pragma unroll
+            for (int jb = 0; jb < JB; ++jb) {
+                const uint32_t w0 = *reinterpret_cast<const uint32_t *>(vp0 + jb * 32);
+                const uint32_t w1 = *reinterpret_cast<const uint32_t *>(vp1 + jb * 32);
+                oa[jb][0] *= corr; oa[jb][1] *= corr; ob[jb][0] *= corr; ob[jb][1] *= corr;
+                mma_top_k8(oa[jb], pa, __byte_perm(w0, w1, 0x5410));    // columns 16 jb + 2 g
+                mma_top_k8(ob[jb], pa, __byte_perm(w0, w1, 0x7632));    // columns 16 jb + 2 g + 1
+            }
+        };
+
+        // ---- stream the cached rows of the segment: warp w takes rows 8 w .. 8 w + 7 of every tile ----
+        for (int r = sg.r0; r < c1; r += kAttnTileRows, ++piece) {
+            const unsigned char *slot = ring.wait(piece, ok);
+            const int rows = (c1 - r) < kAttnTileRows ? (c1 - r) : kAttnTileRows;
+            if (ok && warp * 8 < rows) block(slot, slot + kAttnTileRows * kRowBytes, warp * 8, rows);
+            ring.release(piece);
+        }
+        // ---- the new row, straight from shared memory (never re-read from the cache) ----
+        if (has_new && warp == 0)
+            block(reinterpret_cast<const unsigned char *>(sm.knew), reinterpret_cast<const unsigned char *>(sm.vnew), 0, 1);
+
+        // ---- the warps' states meet in shared memory ----
+        l_run += __shfl_xor_sync(kFull, l_run, 1);
+        l_run += __shfl_xor_sync(kFull, l_run, 2);
+        if (g < G) {
+#pragma unroll
+            for (int jb = 0; jb < JB; ++jb)
+                *reinterpret_cast<float4 *>(&sm.wo[warp][g][16 * jb + 4 * t4]) = make_float4(oa[jb][0], ob[jb][0], oa[jb][1], ob[jb][1]);
+            if (t4 == 0) { sm.wm[warp][g] = m_run; sm.wl[warp][g] = l_run; }
+        }
+        if (!named_bar_and(1, nct, ok)) return false;
+        const bool whole = sg.n_cta == 1;                // this CTA alone finishes the group right here
+        for (int idx = t; idx < G * DH; idx += nct) {
+            const int g2 = idx / DH, i = idx - g2 * DH, hq = hk * G + g2;
+            float M = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kGroupWarps; ++w) M = fmaxf(M, sm.wm[w][g2]);
+            float o = 0.f, l = 0.f;
+#pragma unroll
+            for (int w = 0; w < kGroupWarps; ++w) {
+                const float f = (sm.wm[w][g2] == -INFINITY) ? 0.f : fast_exp2(sm.wm[w][g2] - M);
+                o += f * sm.wo[w][g2][i];
+                l += f * sm.wl[w][g2];
+            }
+            if (whole) a.out[(size_t)b * a.out_stride + (size_t)hq * DH + i] = __float2bfloat16_rn(o / l);
+            else {
+                float *part = a.part + (((size_t)b * a.n_q_heads + hq) * kMaxSplits + (cta - sg.first_cta)) * kPartStride;
+                part[i] = o;
+                if (i == 0) { part[DH] = M; part[DH + 1] = l; }
+            }
+        }
+        if (!whole) {
+            // ---- several CTAs share the K/V head: the partials are published, the last CTA merges the G heads ----
+            __threadfence();
+            named_bar_sync(1, nct);
+            int *ticket = a.ticket + (size_t)b * a.n_q_heads + hk * G;
+            if (t == 0) sm.last = (atomicAdd(ticket, 1) == sg.n_cta - 1);
+            named_bar_sync(1, nct);
+            if (sm.last) {
+                __threadfence();
+                for (int g2 = 0; g2 < G; ++g2) {
+                    const float *hp = a.part + ((size_t)b * a.n_q_heads + hk * G + g2) * kMaxSplits * kPartStride;
+                    __nv_bfloat16 *outp = a.out + (size_t)b * a.out_stride + (size_t)(hk * G + g2) * DH;
+                    if (warp == 0) {
+                        const bool have = lane < sg.n_cta;
+                        const float ms = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH) : -INFINITY;
+                        const float ls = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH + 1) : 0.f;
+                        float MM = ms;
+#pragma unroll
+                        for (int s = 16; s >= 1; s >>= 1) MM = fmaxf(MM, __shfl_xor_sync(kFull, MM, s));
+                        const float f = (ms == -INFINITY) ? 0.f : fast_exp2(ms - MM);
+                        sm.mf[lane] = f;
+                        const float ll = warp_sum(f * ls);
+                        if (lane == 0) sm.lsum = ll;
+                    }
+                    named_bar_sync(1, nct);
+                    for (int i = t; i < DH; i += nct) {
+                        float oo = 0.f;
+                        for (int s0 = 0; s0 < sg.n_cta; s0 += 8) {
+                            float v[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                v[u] = (s0 + u < sg.n_cta) ? ld_cg_f32(hp + (size_t)(s0 + u) * kPartStride + i) : 0.f;
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) oo = fmaf(sm.mf[(s0 + u) & (kMaxSplits - 1)], v[u], oo);
+                        }
+                        outp[i] = __float2bfloat16_rn(oo / sm.lsum);
+                    }
+                    named_bar_sync(1, nct);                  // the merge factors are reused by the next head
+                }
+                if (t == 0) *ticket = 0;
+            }
+        }
+        named_bar_sync(1, nct);                              // the scratch is reused by the next segment
+    }
+    return true;
+}
+
+}  // namespace fasttps
