@@ -6,9 +6,10 @@
 // the arithmetic per byte would make the kernel compute-bound):
 //   scores  S[head, key] = Q[head, :] . K[key, :]      mma m16n8k16, A = Q (heads 0..7 in the rows; rows 8..15
 //                                                       are padding), B = 8 keys of the tile
-//   output  O[head, col] += P[head, key] V[key, col]    mma m16n8k8,  A = P straight from the score fragment
-// A tile of the ring holds 64 rows; consumer warp w owns rows 8w .. 8w+7 of every tile and keeps its own
-// running (max, sum, output) for the G heads; the warps' states are merged per segment as in attn_core.cuh.
+//   output  O[head, col] += P[head, key] V[key, col]    mma m16n8k16, A = P straight from two score fragments
+// A tile of the ring holds 64 rows; consumer warps 0-3 own 16 rows each of the even pieces, warps 4-7 of the odd
+// ones, and every warp keeps its own running (max, sum, output) for the G heads; the warps' states are merged
+// per segment as in attn_core.cuh.
 // Operand order is free inside a dot product, so the head_dim index is permuted such that one 16-byte load of a
 // K row feeds two MMAs, and the output columns are permuted such that two V rows loaded as 32-bit words give
 // the B operands of two MMAs after a byte permute (no transposing load, no swizzled tile).
@@ -21,7 +22,7 @@
 namespace fasttps {
 
 constexpr int kMaxShareGroup = 8;        // query heads per K/V head this path serves (2, 4 or 8)
-constexpr int kGroupWarps = 8;           // consumer warps: one per 8 rows of a tile
+constexpr int kGroupWarps = 8;           // consumer warps: two sets of four, 16 rows of a tile each
 
 template <int DH>
 struct GroupScratch {
@@ -30,8 +31,6 @@ struct GroupScratch {
     alignas(16) __nv_bfloat16 vnew[DH];
     float wm[kGroupWarps][kMaxShareGroup], wl[kGroupWarps][kMaxShareGroup];   // per warp and head: max (log2 domain), sum
     alignas(16) float wo[kGroupWarps][kMaxShareGroup][DH];
-    float mf[kMaxSplits];                               // merge factors of the partials of a shared head
-    float lsum;
     int last;
 };
 
@@ -45,13 +44,6 @@ __device__ __forceinline__ void mma_top_k16(float (&c)[2], uint32_t a0, uint32_t
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%5}, {%7,%8}, {%0,%1,%9,%9};"
                  : "+f"(c[0]), "+f"(c[1]), "=f"(d2), "=f"(d3)
                  : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1), "f"(0.f));
-}
-__device__ __forceinline__ void mma_top_k8(float (&c)[2], uint32_t a0, uint32_t b0)
-{
-    float d2, d3;
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%7,%7};"
-                 : "+f"(c[0]), "+f"(c[1]), "=f"(d2), "=f"(d3)
-                 : "r"(a0), "r"(0u), "r"(b0), "f"(0.f));
 }
 
 // Consumer warps (kGroupWarps of them, threads 0 .. 255, synchronised by named barrier 1).  The segments of
@@ -132,52 +124,74 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
 #pragma unroll
             for (int e = 0; e < 2; ++e) oa[jb][e] = ob[jb][e] = 0.f;
 
-        // One block of up to 8 keys: rows key0 .. key0 + 7 of the K tile `kt` / V tile `vt`, of which the rows below
+        // One block of up to 16 keys: rows key0 .. key0 + 15 of the K tile `kt` / V tile `vt`, of which the rows below
         // `rows` exist.  Rows that do not exist are read from the last one that does (finite data) and get weight 0.
         auto block = [&](const unsigned char *kt, const unsigned char *vt, int key0, int rows) {
-            // ---- scores (Algorithm 3 step 10): lane (g, t4) supplies key key0 + g, receives keys key0 + 2 t4 (+1) of head g ----
-            const int kr = key0 + g < rows ? key0 + g : rows - 1;
-            float s_hi[2] = {0.f, 0.f}, s_lo[2] = {0.f, 0.f};
+            // ---- scores (Algorithm 3 step 10): two sub-blocks of 8 keys; lane (g, t4) supplies keys key0 + g and
+            //      key0 + 8 + g and receives keys key0 + 2 t4 (+1) and key0 + 8 + 2 t4 (+1) of head g.  Eight
+            //      independent accumulator chains (sub-block x hi/lo x half of the 32-wide block).
+            const int kr0 = key0 + g < rows ? key0 + g : rows - 1, kr1 = key0 + 8 + g < rows ? key0 + 8 + g : rows - 1;
+            float sc[2][4][2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) sc[u][c][0] = sc[u][c][1] = 0.f;
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
-                const uint4 kv = *reinterpret_cast<const uint4 *>(kt + (size_t)kr * kRowBytes + kb * 64 + t4 * 16);
-                mma_top_k16(s_hi, qhi[kb].x, qhi[kb].y, kv.x, kv.y);
-                mma_top_k16(s_lo, qlo[kb].x, qlo[kb].y, kv.x, kv.y);
-                mma_top_k16(s_hi, qhi[kb].z, qhi[kb].w, kv.z, kv.w);
-                mma_top_k16(s_lo, qlo[kb].z, qlo[kb].w, kv.z, kv.w);
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const uint4 kv = *reinterpret_cast<const uint4 *>(kt + (size_t)(u ? kr1 : kr0) * kRowBytes + kb * 64 + t4 * 16);
+                    mma_top_k16(sc[u][0], qhi[kb].x, qhi[kb].y, kv.x, kv.y);
+                    mma_top_k16(sc[u][1], qhi[kb].z, qhi[kb].w, kv.z, kv.w);
+                    mma_top_k16(sc[u][2], qlo[kb].x, qlo[kb].y, kv.x, kv.y);
+                    mma_top_k16(sc[u][3], qlo[kb].z, qlo[kb].w, kv.z, kv.w);
+                }
             }
             // ---- online softmax (step 11) ----
-            const int ka = key0 + 2 * t4;
-            const bool v0 = ka < rows, v1 = ka + 1 < rows;
-            const float s0 = v0 ? (s_hi[0] + s_lo[0]) * scale_log2 : -INFINITY;
-            const float s1 = v1 ? (s_hi[1] + s_lo[1]) * scale_log2 : -INFINITY;
-            float mt = fmaxf(s0, s1);
+            int ka[4];
+            float s[4];
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    ka[2 * u + e] = key0 + 8 * u + 2 * t4 + e;
+                    const float v = (sc[u][0][e] + sc[u][1][e]) + (sc[u][2][e] + sc[u][3][e]);
+                    s[2 * u + e] = ka[2 * u + e] < rows ? v * scale_log2 : -INFINITY;
+                }
+            float mt = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
             mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 1));
             mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 2));
             const float m_new = fmaxf(m_run, mt);                  // finite: row key0 exists
             const float corr = fast_exp2(m_run - m_new);           // 0 while m_run = -inf
-            const float p0 = v0 ? fast_exp2(s0 - m_new) : 0.f, p1 = v1 ? fast_exp2(s1 - m_new) : 0.f;
-            const uint32_t pa = pack2(p0, p1);
-            l_run = l_run * corr + bf16_round(p0) + bf16_round(p1);
+            float pr[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) pr[e] = ka[e] < rows ? fast_exp2(s[e] - m_new) : 0.f;
+            const uint32_t pa0 = pack2(pr[0], pr[1]), pa1 = pack2(pr[2], pr[3]);
+            l_run = l_run * corr + ((bf16_round(pr[0]) + bf16_round(pr[1])) + (bf16_round(pr[2]) + bf16_round(pr[3])));
             m_run = m_new;
-            // ---- PV (step 12): B operands from rows ka and ka + 1 of V, two column sets per 32-bit word pair ----
-            const int r0 = ka < rows ? ka : rows - 1, r1 = ka + 1 < rows ? ka + 1 : rows - 1;
-            const unsigned char *vp0 = vt + (size_t)r0 * kRowBytes + g * 4, *vp1 = vt + (size_t)r1 * kRowBytes + g * 4;
+            // ---- PV (step 12): B operands from four rows of V, two column sets per pair of 32-bit words ----
+            const unsigned char *vp[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) vp[e] = vt + (size_t)(ka[e] < rows ? ka[e] : rows - 1) * kRowBytes + g * 4;
 #pragma unroll
             for (int jb = 0; jb < JB; ++jb) {
-                const uint32_t w0 = *reinterpret_cast<const uint32_t *>(vp0 + jb * 32);
-                const uint32_t w1 = *reinterpret_cast<const uint32_t *>(vp1 + jb * 32);
+                const uint32_t w0 = *reinterpret_cast<const uint32_t *>(vp[0] + jb * 32);
+                const uint32_t w1 = *reinterpret_cast<const uint32_t *>(vp[1] + jb * 32);
+                const uint32_t w2 = *reinterpret_cast<const uint32_t *>(vp[2] + jb * 32);
+                const uint32_t w3 = *reinterpret_cast<const uint32_t *>(vp[3] + jb * 32);
                 oa[jb][0] *= corr; oa[jb][1] *= corr; ob[jb][0] *= corr; ob[jb][1] *= corr;
-                mma_top_k8(oa[jb], pa, __byte_perm(w0, w1, 0x5410));    // columns 16 jb + 2 g
-                mma_top_k8(ob[jb], pa, __byte_perm(w0, w1, 0x7632));    // columns 16 jb + 2 g + 1
+                mma_top_k16(oa[jb], pa0, pa1, __byte_perm(w0, w1, 0x5410), __byte_perm(w2, w3, 0x5410));    // columns 16 jb + 2 g
+                mma_top_k16(ob[jb], pa0, pa1, __byte_perm(w0, w1, 0x7632), __byte_perm(w2, w3, 0x7632));    // columns 16 jb + 2 g + 1
             }
         };
 
-        // ---- stream the cached rows of the segment: warp w takes rows 8 w .. 8 w + 7 of every tile ----
+        // ---- stream the cached rows of the segment: warps 0-3 take the even pieces, warps 4-7 the odd ones, 16 rows
+        //      of the tile each; every warp waits for and releases every piece (the ring protocol) ----
         for (int r = sg.r0; r < c1; r += kAttnTileRows, ++piece) {
             const unsigned char *slot = ring.wait(piece, ok);
             const int rows = (c1 - r) < kAttnTileRows ? (c1 - r) : kAttnTileRows;
-            if (ok && warp * 8 < rows) block(slot, slot + kAttnTileRows * kRowBytes, warp * 8, rows);
+            if (ok && (piece & 1) == (warp >> 2) && (warp & 3) * 16 < rows)
+                block(slot, slot + kAttnTileRows * kRowBytes, (warp & 3) * 16, rows);
             ring.release(piece);
         }
         // ---- the new row, straight from shared memory (never re-read from the cache) ----
@@ -223,35 +237,38 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             named_bar_sync(1, nct);
             if (sm.last) {
                 __threadfence();
-                for (int g2 = 0; g2 < G; ++g2) {
-                    const float *hp = a.part + ((size_t)b * a.n_q_heads + hk * G + g2) * kMaxSplits * kPartStride;
-                    __nv_bfloat16 *outp = a.out + (size_t)b * a.out_stride + (size_t)(hk * G + g2) * DH;
-                    if (warp == 0) {
-                        const bool have = lane < sg.n_cta;
-                        const float ms = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH) : -INFINITY;
-                        const float ls = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH + 1) : 0.f;
-                        float MM = ms;
+                // one warp per query head of the group, all heads at once: lane s holds (max, sum) of partial s and
+                // the merge factor that goes with it; every lane finishes DH / 32 columns
+                if (warp < G) {
+                    const float *hp = a.part + ((size_t)b * a.n_q_heads + hk * G + warp) * kMaxSplits * kPartStride;
+                    __nv_bfloat16 *outp = a.out + (size_t)b * a.out_stride + (size_t)(hk * G + warp) * DH;
+                    const bool have = lane < sg.n_cta;
+                    const float ms = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH) : -INFINITY;
+                    const float ls = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH + 1) : 0.f;
+                    float MM = ms;
 #pragma unroll
-                        for (int s = 16; s >= 1; s >>= 1) MM = fmaxf(MM, __shfl_xor_sync(kFull, MM, s));
-                        const float f = (ms == -INFINITY) ? 0.f : fast_exp2(ms - MM);
-                        sm.mf[lane] = f;
-                        const float ll = warp_sum(f * ls);
-                        if (lane == 0) sm.lsum = ll;
-                    }
-                    named_bar_sync(1, nct);
-                    for (int i = t; i < DH; i += nct) {
-                        float oo = 0.f;
-                        for (int s0 = 0; s0 < sg.n_cta; s0 += 8) {
-                            float v[8];
+                    for (int s = 16; s >= 1; s >>= 1) MM = fmaxf(MM, __shfl_xor_sync(kFull, MM, s));
+                    const float f = (ms == -INFINITY) ? 0.f : fast_exp2(ms - MM);
+                    const float ll = warp_sum(f * ls);
+                    float oo[DH / 32];
 #pragma unroll
-                            for (int u = 0; u < 8; ++u)
-                                v[u] = (s0 + u < sg.n_cta) ? ld_cg_f32(hp + (size_t)(s0 + u) * kPartStride + i) : 0.f;
+                    for (int c = 0; c < DH / 32; ++c) oo[c] = 0.f;
+                    for (int s0 = 0; s0 < sg.n_cta; s0 += 4) {
+                        float v[4][DH / 32];
 #pragma unroll
-                            for (int u = 0; u < 8; ++u) oo = fmaf(sm.mf[(s0 + u) & (kMaxSplits - 1)], v[u], oo);
+                        for (int u = 0; u < 4; ++u)
+#pragma unroll
+                            for (int c = 0; c < DH / 32; ++c)
+                                v[u][c] = (s0 + u < sg.n_cta) ? ld_cg_f32(hp + (size_t)(s0 + u) * kPartStride + lane + 32 * c) : 0.f;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const float fs = __shfl_sync(kFull, f, (s0 + u) & 31);
+#pragma unroll
+                            for (int c = 0; c < DH / 32; ++c) oo[c] = fmaf(fs, v[u][c], oo[c]);
                         }
-                        outp[i] = __float2bfloat16_rn(oo / sm.lsum);
                     }
-                    named_bar_sync(1, nct);                  // the merge factors are reused by the next head
+#pragma unroll
+                    for (int c = 0; c < DH / 32; ++c) outp[lane + 32 * c] = __float2bfloat16_rn(oo[c] / ll);
                 }
                 if (t == 0) *ticket = 0;
             }
