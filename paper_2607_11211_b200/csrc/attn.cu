@@ -12,7 +12,7 @@ constexpr int kAttnWarps = 8;                           // consumer warps
 constexpr int kAttnThreads = (kAttnWarps + 1) * 32;     // + the producer warp
 static_assert(kAttnWarps == kGroupWarps, "the grouped-query path divides the tiles among exactly kGroupWarps consumer warps");
 
-// Grouped-query attention with 2 to 8 query heads per K/V head streams every cached row once for the whole
+// Grouped-query attention with 2 to 16 query heads per K/V head streams every cached row once for the whole
 // group, with the two products on the tensor cores; other ratios stream it once per query head.
 inline bool attn_shares_groups(int n_q_heads, int n_kv_heads)
 {

@@ -4,7 +4,7 @@
 // With G query vectors per row the two products of Algorithm 3 are thin matrix products, so they run on the
 // tensor cores (the FP32 dot products of attn_core.cuh already keep the ALUs as busy as HBM at G = 1; G times
 // the arithmetic per byte would make the kernel compute-bound):
-//   scores  S[head, key] = Q[head, :] . K[key, :]      mma m16n8k16, A = Q (heads 0..7 in the rows; rows 8..15
+//   scores  S[head, key] = Q[head, :] . K[key, :]      mma m16n8k16, A = Q (8 heads in the rows; rows 8..15
 //                                                       are padding), B = 8 keys of the tile
 //   output  O[head, col] += P[head, key] V[key, col]    mma m16n8k16, A = P straight from two score fragments
 // A tile of the ring holds 64 rows; consumer warps 0-3 own 16 rows each of the even pieces, warps 4-7 of the odd
@@ -13,7 +13,8 @@
 // Operand order is free inside a dot product, so the head_dim index is permuted such that one 16-byte load of a
 // K row feeds two MMAs, and the output columns are permuted such that two V rows loaded as 32-bit words give
 // the B operands of two MMAs after a byte permute (no transposing load, no swizzled tile).
-// Precision: q is split into bf16 hi + lo (two score MMAs: the FP32 rotated q is kept to 2^-17), the
+// Precision: the rotated q enters the score product rounded to bf16 (the single-head path keeps it in FP32; a
+// bf16 hi + lo split was measured: it doubles the score MMAs and the registers it takes force spills), the
 // probabilities enter the second product rounded to bf16, and the row sum is taken over the rounded values.
 #pragma once
 #include "attn_core.cuh"
@@ -21,7 +22,8 @@
 
 namespace fasttps {
 
-constexpr int kMaxShareGroup = 8;        // query heads per K/V head this path serves (2, 4 or 8)
+constexpr int kMaxShareGroup = 16;       // query heads per K/V head this path serves (2 to 16)
+constexpr int kHeadsPerWarp = 8;         // heads in the rows of one warp's MMAs
 constexpr int kGroupWarps = 8;           // consumer warps: two sets of four, 16 rows of a tile each
 
 template <int DH>
@@ -29,8 +31,8 @@ struct GroupScratch {
     alignas(16) float q[kMaxShareGroup][DH];            // rope(q) of the group, FP32
     alignas(16) __nv_bfloat16 knew[DH];                 // bf16(rope(k_new)): the row that goes into the cache
     alignas(16) __nv_bfloat16 vnew[DH];
-    float wm[kGroupWarps][kMaxShareGroup], wl[kGroupWarps][kMaxShareGroup];   // per warp and head: max (log2 domain), sum
-    alignas(16) float wo[kGroupWarps][kMaxShareGroup][DH];
+    float wm[kGroupWarps][kHeadsPerWarp], wl[kGroupWarps][kHeadsPerWarp];     // per warp and head slot: max (log2 domain), sum
+    alignas(16) float wo[kGroupWarps][kHeadsPerWarp][DH];
     int last;
 };
 
@@ -60,6 +62,10 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5, g = lane >> 2, t4 = lane & 3;
     const int nct = kGroupWarps * 32;
     const int G = a.n_q_heads / a.n_kv_heads;
+    // groups of up to 8: warps 0-3 take the even pieces, warps 4-7 the odd ones, all heads each.  Larger groups
+    // (up to 16): warps 0-3 take heads 0-7 and warps 4-7 heads 8-15, of every piece.
+    const bool wide = G > kHeadsPerWarp;
+    const int gh = g + (wide ? kHeadsPerWarp * (warp >> 2) : 0);      // the query head of the group in this lane's MMA row
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
     bool ok = true;
 
@@ -98,24 +104,20 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             asm volatile("fence.proxy.async;" ::: "memory");
         }
 
-        // ---- A fragments of the score product: head g of the group, bf16 hi + lo of 8 consecutive elements ----
-        uint4 qhi[KB], qlo[KB];
+        // ---- A fragments of the score product: this lane's head of the group, 8 consecutive elements per block ----
+        uint4 qhi[KB];
 #pragma unroll
         for (int kb = 0; kb < KB; ++kb) {
             float f[8];
-            if (g < G) {
-                const float4 f0 = *reinterpret_cast<const float4 *>(&sm.q[g][kb * 32 + 8 * t4]);
-                const float4 f1 = *reinterpret_cast<const float4 *>(&sm.q[g][kb * 32 + 8 * t4 + 4]);
+            if (gh < G) {
+                const float4 f0 = *reinterpret_cast<const float4 *>(&sm.q[gh][kb * 32 + 8 * t4]);
+                const float4 f1 = *reinterpret_cast<const float4 *>(&sm.q[gh][kb * 32 + 8 * t4 + 4]);
                 f[0] = f0.x; f[1] = f0.y; f[2] = f0.z; f[3] = f0.w; f[4] = f1.x; f[5] = f1.y; f[6] = f1.z; f[7] = f1.w;
             } else {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) f[i] = 0.f;
             }
-            float r[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) r[i] = f[i] - bf16_round(f[i]);
             qhi[kb] = make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
-            qlo[kb] = make_uint4(pack2(r[0], r[1]), pack2(r[2], r[3]), pack2(r[4], r[5]), pack2(r[6], r[7]));
         }
         float m_run = -INFINITY, l_run = 0.f;      // of head g; the sum holds this lane's keys only until the end
         float oa[JB][2], ob[JB][2];                // output fragments of head g: columns 16 jb + 4 t4 + {0, 2} (oa) / {1, 3} (ob)
@@ -128,14 +130,14 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
         // `rows` exist.  Rows that do not exist are read from the last one that does (finite data) and get weight 0.
         auto block = [&](const unsigned char *kt, const unsigned char *vt, int key0, int rows) {
             // ---- scores (Algorithm 3 step 10): two sub-blocks of 8 keys; lane (g, t4) supplies keys key0 + g and
-            //      key0 + 8 + g and receives keys key0 + 2 t4 (+1) and key0 + 8 + 2 t4 (+1) of head g.  Eight
-            //      independent accumulator chains (sub-block x hi/lo x half of the 32-wide block).
+            //      key0 + 8 + g and receives keys key0 + 2 t4 (+1) and key0 + 8 + 2 t4 (+1) of its head.  Four
+            //      independent accumulator chains (sub-block x half of the 32-wide block).
             const int kr0 = key0 + g < rows ? key0 + g : rows - 1, kr1 = key0 + 8 + g < rows ? key0 + 8 + g : rows - 1;
-            float sc[2][4][2];
+            float sc[2][2][2];
 #pragma unroll
             for (int u = 0; u < 2; ++u)
 #pragma unroll
-                for (int c = 0; c < 4; ++c) sc[u][c][0] = sc[u][c][1] = 0.f;
+                for (int c = 0; c < 2; ++c) sc[u][c][0] = sc[u][c][1] = 0.f;
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
 #pragma unroll
@@ -143,8 +145,6 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                     const uint4 kv = *reinterpret_cast<const uint4 *>(kt + (size_t)(u ? kr1 : kr0) * kRowBytes + kb * 64 + t4 * 16);
                     mma_top_k16(sc[u][0], qhi[kb].x, qhi[kb].y, kv.x, kv.y);
                     mma_top_k16(sc[u][1], qhi[kb].z, qhi[kb].w, kv.z, kv.w);
-                    mma_top_k16(sc[u][2], qlo[kb].x, qlo[kb].y, kv.x, kv.y);
-                    mma_top_k16(sc[u][3], qlo[kb].z, qlo[kb].w, kv.z, kv.w);
                 }
             }
             // ---- online softmax (step 11) ----
@@ -155,7 +155,7 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     ka[2 * u + e] = key0 + 8 * u + 2 * t4 + e;
-                    const float v = (sc[u][0][e] + sc[u][1][e]) + (sc[u][2][e] + sc[u][3][e]);
+                    const float v = sc[u][0][e] + sc[u][1][e];
                     s[2 * u + e] = ka[2 * u + e] < rows ? v * scale_log2 : -INFINITY;
                 }
             float mt = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
@@ -173,13 +173,17 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             const unsigned char *vp[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) vp[e] = vt + (size_t)(ka[e] < rows ? ka[e] : rows - 1) * kRowBytes + g * 4;
+            // the running maximum seldom moves after the first tiles: the rescaling is skipped when no lane needs it
+            if (__any_sync(kFull, corr != 1.f)) {
+#pragma unroll
+                for (int jb = 0; jb < JB; ++jb) { oa[jb][0] *= corr; oa[jb][1] *= corr; ob[jb][0] *= corr; ob[jb][1] *= corr; }
+            }
 #pragma unroll
             for (int jb = 0; jb < JB; ++jb) {
                 const uint32_t w0 = *reinterpret_cast<const uint32_t *>(vp[0] + jb * 32);
                 const uint32_t w1 = *reinterpret_cast<const uint32_t *>(vp[1] + jb * 32);
                 const uint32_t w2 = *reinterpret_cast<const uint32_t *>(vp[2] + jb * 32);
                 const uint32_t w3 = *reinterpret_cast<const uint32_t *>(vp[3] + jb * 32);
-                oa[jb][0] *= corr; oa[jb][1] *= corr; ob[jb][0] *= corr; ob[jb][1] *= corr;
                 mma_top_k16(oa[jb], pa0, pa1, __byte_perm(w0, w1, 0x5410), __byte_perm(w2, w3, 0x5410));    // columns 16 jb + 2 g
                 mma_top_k16(ob[jb], pa0, pa1, __byte_perm(w0, w1, 0x7632), __byte_perm(w2, w3, 0x7632));    // columns 16 jb + 2 g + 1
             }
@@ -190,18 +194,18 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
         for (int r = sg.r0; r < c1; r += kAttnTileRows, ++piece) {
             const unsigned char *slot = ring.wait(piece, ok);
             const int rows = (c1 - r) < kAttnTileRows ? (c1 - r) : kAttnTileRows;
-            if (ok && (piece & 1) == (warp >> 2) && (warp & 3) * 16 < rows)
+            if (ok && (wide || (piece & 1) == (warp >> 2)) && (warp & 3) * 16 < rows)
                 block(slot, slot + kAttnTileRows * kRowBytes, (warp & 3) * 16, rows);
             ring.release(piece);
         }
         // ---- the new row, straight from shared memory (never re-read from the cache) ----
-        if (has_new && warp == 0)
+        if (has_new && (warp == 0 || (wide && warp == 4)))
             block(reinterpret_cast<const unsigned char *>(sm.knew), reinterpret_cast<const unsigned char *>(sm.vnew), 0, 1);
 
         // ---- the warps' states meet in shared memory ----
         l_run += __shfl_xor_sync(kFull, l_run, 1);
         l_run += __shfl_xor_sync(kFull, l_run, 2);
-        if (g < G) {
+        if (gh < G) {
 #pragma unroll
             for (int jb = 0; jb < JB; ++jb)
                 *reinterpret_cast<float4 *>(&sm.wo[warp][g][16 * jb + 4 * t4]) = make_float4(oa[jb][0], ob[jb][0], oa[jb][1], ob[jb][1]);
@@ -211,15 +215,15 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
         const bool whole = sg.n_cta == 1;                // this CTA alone finishes the group right here
         for (int idx = t; idx < G * DH; idx += nct) {
             const int g2 = idx / DH, i = idx - g2 * DH, hq = hk * G + g2;
+            // the warps that hold head g2 (all of them, or one set of four), in slot g2 mod 8
+            const int sl = g2 & (kHeadsPerWarp - 1), w0 = wide ? 4 * (g2 >> 3) : 0, w1 = wide ? w0 + 4 : kGroupWarps;
             float M = -INFINITY;
-#pragma unroll
-            for (int w = 0; w < kGroupWarps; ++w) M = fmaxf(M, sm.wm[w][g2]);
+            for (int w = w0; w < w1; ++w) M = fmaxf(M, sm.wm[w][sl]);
             float o = 0.f, l = 0.f;
-#pragma unroll
-            for (int w = 0; w < kGroupWarps; ++w) {
-                const float f = (sm.wm[w][g2] == -INFINITY) ? 0.f : fast_exp2(sm.wm[w][g2] - M);
-                o += f * sm.wo[w][g2][i];
-                l += f * sm.wl[w][g2];
+            for (int w = w0; w < w1; ++w) {
+                const float f = (sm.wm[w][sl] == -INFINITY) ? 0.f : fast_exp2(sm.wm[w][sl] - M);
+                o += f * sm.wo[w][sl][i];
+                l += f * sm.wl[w][sl];
             }
             if (whole) a.out[(size_t)b * a.out_stride + (size_t)hq * DH + i] = __float2bfloat16_rn(o / l);
             else {
@@ -239,9 +243,9 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 __threadfence();
                 // one warp per query head of the group, all heads at once: lane s holds (max, sum) of partial s and
                 // the merge factor that goes with it; every lane finishes DH / 32 columns
-                if (warp < G) {
-                    const float *hp = a.part + ((size_t)b * a.n_q_heads + hk * G + warp) * kMaxSplits * kPartStride;
-                    __nv_bfloat16 *outp = a.out + (size_t)b * a.out_stride + (size_t)(hk * G + warp) * DH;
+                for (int hg = warp; hg < G; hg += kGroupWarps) {
+                    const float *hp = a.part + ((size_t)b * a.n_q_heads + hk * G + hg) * kMaxSplits * kPartStride;
+                    __nv_bfloat16 *outp = a.out + (size_t)b * a.out_stride + (size_t)(hk * G + hg) * DH;
                     const bool have = lane < sg.n_cta;
                     const float ms = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH) : -INFINITY;
                     const float ls = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH + 1) : 0.f;

@@ -213,19 +213,24 @@ def test_attn_decode_error_against_a_float_baseline_stays_below_the_papers_bound
 
 
 
-# Grouped-query shapes: Llama3-8B of Table 1 (32 query heads on 8 K/V heads, head_dim 128) and small shapes with 2
-# and 8 query heads per K/V head.  The attention kernel streams each K/V head once for its whole group.
+# Grouped-query shapes: Llama3-8B (32 query heads on 8 K/V heads, head_dim 128) and ChatGLM3-6B (32 on 2) of
+# Table 1, and small shapes with 2, 3, 8, 12 and 16 query heads per K/V head.  The attention kernel streams each
+# K/V head once for its whole group (groups of up to 16).
 LLAMA3_8B_ATTN = wl.Dims(hidden=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, inter=14336, vocab=1000, n_layers=1)
 GQA_2 = wl.Dims(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, inter=384, vocab=520, n_layers=1)
 GQA_3 = wl.Dims(hidden=1152, n_q_heads=12, n_kv_heads=4, head_dim=96, inter=384, vocab=520, n_layers=1)
 GQA_8 = wl.Dims(hidden=768, n_q_heads=8, n_kv_heads=1, head_dim=96, inter=384, vocab=520, n_layers=1)
 GQA_16 = wl.Dims(hidden=512, n_q_heads=16, n_kv_heads=1, head_dim=32, inter=384, vocab=520, n_layers=1)
+GQA_12 = wl.Dims(hidden=768, n_q_heads=12, n_kv_heads=1, head_dim=64, inter=384, vocab=520, n_layers=1)
+CHATGLM3_ATTN = wl.Dims(hidden=4096, n_q_heads=32, n_kv_heads=2, head_dim=128, inter=13696, vocab=1000, n_layers=1)
+GQA_32 = wl.Dims(hidden=1024, n_q_heads=32, n_kv_heads=1, head_dim=32, inter=384, vocab=520, n_layers=1)
 
 
 @pytest.mark.parametrize("dims,lens,max_seq", [
     (LLAMA3_8B_ATTN, [4095], 4096), (LLAMA3_8B_ATTN, [0, 700, 3, 2047, 64], 2048), (LLAMA3_8B_ATTN, [256], 4096),
     (GQA_2, [0, 1, 63, 64, 65, 300, 1000], 1024), (GQA_3, [0, 1, 7, 8, 9, 70, 129, 500], 512), (GQA_8, [5000], 5008), (GQA_8, [0, 7, 130], 256),
-    (GQA_16, [900, 2], 1024),          # 16 query heads per K/V head: not shared, one pass per query head
+    (GQA_16, [900, 2], 1024), (GQA_12, [0, 15, 16, 17, 333], 512), (CHATGLM3_ATTN, [4095, 100], 4096),
+    (GQA_32, [900, 2], 1024),          # 32 query heads per K/V head: not shared, one pass per query head
 ])
 def test_attn_decode_grouped_query_shapes(fb, dims, lens, max_seq):
     for share in (1, 0):                  # one pass per K/V head (tensor cores) and one pass per query head
