@@ -128,7 +128,10 @@ int fasttps_unpack_weight(fasttps_ctx *ctx, int kind, const void *src_packed, vo
  *   pos [B] int32 device: rotary position of the new token.
  *   seq_lens [B] int32 device: rows already cached (N_p) = the row written now.
  *   out [B,H_q,d]: softmax(q' K^T / sqrt(d)) V over rows 0..seq_lens[b] inclusive.
- * Query head h uses kv head h / (H_q/H_kv).  Neither pos nor seq_lens is advanced. */
+ * Query head h uses kv head h / (H_q/H_kv) (Section 4.1).  With 2 to 16 query heads per kv head every
+ * cached row is read once for its whole group and the two products run on the tensor cores: there the
+ * rotated q and the softmax weights enter the products rounded to bf16 (FP32 accumulation); with one
+ * query head per kv head, or more than 16, both stay FP32.  Neither pos nor seq_lens is advanced. */
 int fasttps_attn_decode(fasttps_ctx *ctx, const void *q, const void *k_new, const void *v_new,
                         void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
                         void *out, int batch, void *stream);
