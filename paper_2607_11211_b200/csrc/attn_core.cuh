@@ -296,11 +296,14 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
             mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 16));
             const float m_new = fmaxf(m_run, mt);
             if (m_new == -INFINITY) return;              // nothing valid yet (warp-uniform)
-            const float corr = fast_exp2(m_run - m_new); // 0 when m_run = -inf
-            l_run *= corr;
+            // the maximum is the same in every lane of the warp and seldom moves after the first tiles
+            if (m_new != m_run) {
+                const float corr = fast_exp2(m_run - m_new); // 0 when m_run = -inf
+                l_run *= corr;
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) acc[i] *= corr;
-            m_run = m_new;
+                for (int i = 0; i < EPL; ++i) acc[i] *= corr;
+                m_run = m_new;
+            }
             if (valid) {
                 const float pj = fast_exp2(sc - m_new);
                 if (sub == 0) l_run += pj;
