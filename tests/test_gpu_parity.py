@@ -348,7 +348,7 @@ def k_rows_ok(got, want, half):
     return d1 | (np.abs(g - w) <= 2.0 ** -7 * pair)
 
 
-def run_layer_case(fb, dims, lens, max_seq, layer=0):
+def run_layer_case(fb, dims, lens, max_seq, layer=0, flips_allowed=0.0):
     batch = len(lens)
     lens = np.asarray(lens, np.int32)
     ctx = make_ctx(fb, dims, batch, max_seq)
@@ -373,12 +373,27 @@ def run_layer_case(fb, dims, lens, max_seq, layer=0):
         assert ulp_distance(vg[b, :, lens[b]], vo[b, :, lens[b]]).max() <= 1
         assert k_rows_ok(kg[b, :, lens[b]], ko[b, :, lens[b]], dims.head_dim // 2).all()
         assert (ulp_distance(kg[b, :, lens[b]], ko[b, :, lens[b]]) <= 1).mean() > 0.99
-    assert_close_bits(wl.bits(xo), want, what=f"layer out lens={lens.tolist()}")
+    def check_out(bits, what):
+        if flips_allowed == 0.0:
+            assert_close_bits(bits, want, what=what)
+            return
+        # The layer output is h + mlp(h) with h itself rounded to bf16 inside the call.  Where the two sides round h
+        # to neighbouring values, an output in which h and the MLP term cancel moves by up to one ulp of h
+        # (2^-7 |h|), which the bound on the outputs cannot absorb.  At most `flips_allowed` of the elements may
+        # leave the bound, and those by no more than one ulp at the largest magnitude in the tensor.
+        g, r = F32(bits).astype(np.float64), F32(want).astype(np.float64)
+        d = np.abs(g - r)
+        out = d > 2e-2 + 2e-2 * np.abs(r)
+        assert out.mean() <= flips_allowed, (what, int(out.sum()), out.size)
+        assert (d <= 2e-2 + 2e-2 * np.abs(r) + 2.0 ** -7 * np.abs(r).max()).all(), what
+        assert d.mean() < 1e-2, what
+
+    check_out(wl.bits(xo), f"layer out lens={lens.tolist()}")
     # in place (x_out aliases x_in)
     x2 = x.clone()
     kc2, vc2 = dev(k0), dev(v0)
     ctx.layer_decode(pw["struct"], x2, x2, kc2, vc2, i32(lens), i32(lens))
-    assert_close_bits(wl.bits(x2), want, what="layer in place")
+    check_out(wl.bits(x2), "layer in place")
     ctx.close()
 
 
@@ -392,6 +407,13 @@ def test_layer_decode_small_shapes(fb, dims, lens):
 def test_layer_decode_phi3_single_layer_configs(fb, lens):
     # the two single-layer workloads: 256 resp. 4095 past tokens, new token at that position
     run_layer_case(fb, wl.PHI3_MINI, lens, 4096)
+
+
+def test_layer_decode_llama3_8b_shape_grouped_query_layer(fb):
+    # a whole decoder layer of the Llama3-8B row of Table 1 (hidden 4096, 32 query heads on 8 K/V heads of 128,
+    # MLP 14336) through the chain: the attention inside it streams each K/V head once for its four query heads
+    dims = wl.Dims(hidden=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, inter=14336, vocab=1000, n_layers=1)
+    run_layer_case(fb, dims, [700, 64], 1024, flips_allowed=1e-3)
 
 
 # -------------------------------------------------------------------- model
