@@ -247,7 +247,8 @@ int fasttps_profile_read(fasttps_ctx *ctx, double *ms_per_class, uint64_t *launc
 int fasttps_trace_read(fasttps_ctx *ctx, uint64_t *stamps, int max_per_cta);
 /* Number of kernels this context has launched so far (host counter). */
 uint64_t fasttps_launch_count(const fasttps_ctx *ctx);
-/* Split count the attention kernel would use for this batch (for tests/benchmarks). */
+/* Number of CTAs the attention kernel is launched with for this batch (how many of them take part is decided
+ * on the device from the lengths; for tests/benchmarks). */
 int fasttps_attn_splits(const fasttps_ctx *ctx, int batch);
 /* Diagnostic, host only (no context, no CUDA call; no counterpart in the paper): how the persistent step kernel
  * cuts the cached rows of one query head, all sequences of the batch end to end plus one new row each (Algorithm 3

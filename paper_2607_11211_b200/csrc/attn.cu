@@ -83,16 +83,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a
 
 }  // namespace
 
-// Number of CTAs the attention kernel uses (one per SM, fewer for tiny head counts so that
-// no head is shared by more than kMaxSplits CTAs).
+// Number of CTAs the attention kernel is launched with: one per SM.  How many of them take part is decided on
+// the device from the lengths (the share walk): every share holds at least 16 rows, and no head is cut into
+// more shares than it has partial records.
 int attn_splits_for(const Ctx *c, int batch)
 {
-    int n = c->n_sm;
     (void)batch;
-    // heads of the flattened row space: K/V heads when a group shares its rows
-    const int cap = (kMaxSplits - 2) * ((c->opt_gqa_share && attn_shares_groups(c->cfg.n_q_heads, c->cfg.n_kv_heads)) ? c->cfg.n_kv_heads : c->cfg.n_q_heads);
-    if (n > cap) n = cap;
-    return n < 1 ? 1 : n;
+    return c->n_sm < 1 ? 1 : c->n_sm;
 }
 
 template <int DH>

@@ -66,11 +66,12 @@ struct ShareWalk {
     {
         seq_lens = sl; pos = ps; add = add_; B = B_; H = H_; max_seq = max_seq_;
         T = 0;
-        int live = 0, rows0 = 0;
+        int live = 0, rows0 = 0, rmax = 0;
         bool uniform = true;
         for (int bb = 0; bb < B; ++bb) {
             const int r = rows_of(bb);
             T += (long long)H * r;
+            rmax = r > rmax ? r : rmax;
             if (r > 0) {
                 if (live == 0) rows0 = r;
                 else if (r != rows0) uniform = false;
@@ -81,6 +82,13 @@ struct ShareWalk {
         // non-empty, so the CTAs that share a head are exactly first_cta .. first_cta + n_cta - 1
         const long long want = T / 16;
         ncta = want < 1 ? 1 : (want < ncta_ ? (int)want : ncta_);
+        // a head has kMaxSplits partial records: a share is at least 1 / (kMaxSplits - 3) of the longest head (less
+        // up to a sixteenth for the rounding of the cuts, shares being at least 16 rows), so that no head spans
+        // more than kMaxSplits shares (whole shares plus a cut one at either end)
+        if (rmax > 0) {
+            const long long cap = (long long)(kMaxSplits - 3) * T / rmax;
+            if (ncta > cap) ncta = cap < 1 ? 1 : (int)cap;
+        }
         // equal lengths and no more heads than CTAs: a whole number of CTAs per head, so that every share
         // is ONE segment and every head has the same, small number of partials
         if (uniform && live > 0 && live * H <= ncta) ncta = live * H * (ncta / (live * H));
