@@ -259,6 +259,15 @@ int fasttps_attn_splits(const fasttps_ctx *ctx, int batch);
  * number of shares in use (<= group_size; 0 if no sequence is valid), or a negative FASTTPS error code. */
 int fasttps_attention_shares(const int32_t *seq_lens, const int32_t *pos, int batch, int max_seq, int step,
                              int group_size, int32_t *seg_out, int32_t *nseg_out);
+/* Diagnostic, host only (no context, no CUDA call; no counterpart in the paper): how the stand-alone attention
+ * kernel cuts the flattened row space -- for every sequence and head (K/V heads on grouped-query shapes with up to
+ * 16 query heads per K/V head, query heads otherwise) the cached rows plus the new row -- into shares for n_cta
+ * CTAs.  seq_lens, pos: HOST arrays of `batch` entries.  Writes up to max_segs segments, in CTA order, as
+ * seg_out[7 i + 0..6] = CTA, sequence, head, first row, end row (exclusive; row seq_len is the new row), first CTA
+ * that holds rows of that head, number of CTAs that do (at most 32: a head has that many partial records).
+ * Returns the number of segments (which may exceed max_segs), or a negative FASTTPS error code. */
+int fasttps_attention_walk(const int32_t *seq_lens, const int32_t *pos, int batch, int heads, int max_seq, int n_cta,
+                           int32_t *seg_out, int max_segs);
 const char *fasttps_strerror(int code);
 /* Text of the last CUDA error seen by this thread inside the library ("" if none). */
 const char *fasttps_last_error(void);

@@ -71,6 +71,7 @@ def load_library() -> C.CDLL:
     lib.fasttps_launch_count.restype = C.c_uint64
     lib.fasttps_attn_splits.argtypes = [vp, i]
     lib.fasttps_attention_shares.argtypes = [vp, vp, i, i, i, i, vp, vp]
+    lib.fasttps_attention_walk.argtypes = [vp, vp, i, i, i, i, vp, i]
     lib.fasttps_strerror.argtypes = [i]
     lib.fasttps_strerror.restype = C.c_char_p
     lib.fasttps_last_error.restype = C.c_char_p
@@ -94,6 +95,24 @@ def attention_shares(seq_lens, pos, max_seq: int, step: int, group_size: int):
     if rc < 0:
         _check(rc, "fasttps_attention_shares")
     return rc, [[tuple(int(v) for v in seg[g, j]) for j in range(nseg[g])] for g in range(group_size)]
+
+
+def attention_walk(seq_lens, pos, heads: int, max_seq: int, n_cta: int):
+    """How the stand-alone attention kernel cuts the rows of all (sequence, head) pairs into shares for `n_cta` CTAs:
+    a list of (CTA, sequence, head, first row, end row, first CTA of the head, number of CTAs of the head).
+    Host only: needs the library, not a GPU."""
+    import numpy as np
+    lib = load_library()
+    sl = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    ps = np.ascontiguousarray(pos, dtype=np.int32)
+    cap = len(sl) * heads + n_cta + 8
+    seg = np.zeros((cap, 7), dtype=np.int32)
+    rc = lib.fasttps_attention_walk(sl.ctypes.data, ps.ctypes.data, len(sl), int(heads), int(max_seq), int(n_cta),
+                                    seg.ctypes.data, cap)
+    if rc < 0:
+        _check(rc, "fasttps_attention_walk")
+    assert rc <= cap
+    return [tuple(int(v) for v in seg[i]) for i in range(rc)]
 
 
 def _check(rc: int, what: str):

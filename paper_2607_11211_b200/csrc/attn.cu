@@ -133,3 +133,27 @@ int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st)
 }
 
 }  // namespace fasttps
+
+// Diagnostic entry point: the share walk of the stand-alone attention kernel, run on the host by the same code the
+// kernel runs on the device, for every CTA in turn; the segments go to the caller.
+extern "C" int fasttps_attention_walk(const int32_t *seq_lens, const int32_t *pos, int batch, int heads, int max_seq, int n_cta,
+                                      int32_t *seg_out, int max_segs)
+{
+    using namespace fasttps;
+    if (!seq_lens || !pos || !seg_out || batch < 1 || heads < 1 || max_seq < 1 || n_cta < 1 || max_segs < 0)
+        return FASTTPS_INVALID_ARG;
+    int n = 0;
+    for (int cta = 0; cta < n_cta; ++cta) {
+        ShareWalk w;
+        w.init(seq_lens, pos, 0, batch, heads, max_seq, cta, n_cta);
+        Segment sg;
+        while (w.next(sg)) {
+            if (n < max_segs) {
+                int32_t *o = seg_out + (size_t)n * 7;
+                o[0] = cta; o[1] = sg.b; o[2] = sg.h; o[3] = sg.r0; o[4] = sg.r1; o[5] = sg.first_cta; o[6] = sg.n_cta;
+            }
+            ++n;
+        }
+    }
+    return n;
+}

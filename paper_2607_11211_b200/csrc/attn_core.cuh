@@ -47,21 +47,21 @@ struct ShareWalk {
     long long head0;             // flattened index of row 0 of head (b, h)
     int rows_b;                  // rows per head of sequence b (L_b + 1, or 0 if the sequence is skipped)
 
-    __device__ __forceinline__ int rows_of(int bb) const
+    __host__ __device__ __forceinline__ int rows_of(int bb) const
     {
         const int L = seq_lens[bb] + add, p = pos[bb] + add;
         return (L < add || L >= max_seq || p < add || p >= max_seq) ? 0 : L + 1;
     }
-    __device__ __forceinline__ long long share_begin(int c) const { return (T * c) / ncta; }
+    __host__ __device__ __forceinline__ long long share_begin(int c) const { return (T * c) / ncta; }
     // the CTA whose share holds flattened row x
-    __device__ __forceinline__ int owner_of(long long x) const
+    __host__ __device__ __forceinline__ int owner_of(long long x) const
     {
         int c = (int)((x * ncta) / T);
         while (c + 1 < ncta && share_begin(c + 1) <= x) ++c;
         while (c > 0 && share_begin(c) > x) --c;
         return c;
     }
-    __device__ __forceinline__ void init(const int32_t *sl, const int32_t *ps, int add_, int B_, int H_, int max_seq_,
+    __host__ __device__ __forceinline__ void init(const int32_t *sl, const int32_t *ps, int add_, int B_, int H_, int max_seq_,
                                          int cta, int ncta_)
     {
         seq_lens = sl; pos = ps; add = add_; B = B_; H = H_; max_seq = max_seq_;
@@ -108,7 +108,7 @@ struct ShareWalk {
             head0 += (long long)h * rows_b;
         }
     }
-    __device__ __forceinline__ bool next(Segment &s)
+    __host__ __device__ __forceinline__ bool next(Segment &s)
     {
         while (f < f_end) {
             if (rows_b == 0 || h >= H) {          // step to the next sequence

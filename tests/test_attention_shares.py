@@ -83,3 +83,51 @@ def test_bad_arguments_are_refused():
         binding.attention_shares([1] * 9, [1] * 9, 64, 0, 4)       # more than 8 sequences
     with pytest.raises(binding.FasttpsError):
         binding.attention_shares([1], [1], 64, 0, 33)              # group larger than the partial table
+
+
+# ------------------------------------------------- the stand-alone attention kernel's share walk
+
+def _check_walk(lens, heads, max_seq, n_cta):
+    from paper_2607_11211_b200 import binding as fb
+    lens = np.asarray(lens, np.int32)
+    segs = fb.attention_walk(lens, lens, heads, max_seq, n_cta)
+    valid = [(0 <= l < max_seq) for l in lens]
+    rows = {(b, h): [] for b in range(len(lens)) if valid[b] for h in range(heads)}
+    per_cta = {}
+    for cta, b, h, r0, r1, first, n in segs:
+        assert valid[b] and 0 <= h < heads and 0 <= r0 < r1 <= lens[b] + 1
+        assert 1 <= n <= 32 and first <= cta < first + n          # 32 partial records per head, indexed cta - first
+        rows[(b, h)].append((r0, r1, cta, first, n))
+        per_cta[cta] = per_cta.get(cta, 0) + (r1 - r0)
+    for (b, h), parts in rows.items():
+        parts.sort()
+        assert parts[0][0] == 0 and parts[-1][1] == lens[b] + 1, (b, h)
+        assert all(p[1] == q[0] for p, q in zip(parts, parts[1:])), (b, h)       # the shares partition the head's rows
+        assert len({(p[3], p[4]) for p in parts}) == 1                          # and agree on the head's CTAs ...
+        assert [p[2] for p in parts] == list(range(parts[0][3], parts[0][3] + parts[0][4]))   # ... which all hold rows of it
+    total = sum((l + 1) * heads for l, v in zip(lens, valid) if v)
+    assert sum(per_cta.values()) == total
+    if per_cta:
+        assert max(per_cta.values()) - min(per_cta.values()) <= 1              # equal shares
+        assert min(per_cta.values()) >= min(16, total)
+    return max((p[0][4] for p in rows.values()), default=0), len(per_cta)
+
+
+def test_attention_walk_partitions_every_head_into_equal_shares_within_the_record_limit():
+    rng = np.random.default_rng(11)
+    worst = 0
+    for _ in range(300):
+        batch = int(rng.integers(1, 9))
+        heads = int(rng.choice([1, 2, 4, 8, 32]))
+        lens = [int(rng.integers(0, 40)) if rng.random() < 0.5 else int(rng.integers(0, 5000)) for _ in range(batch)]
+        span, _ = _check_walk(lens, heads, 5008, int(rng.choice([148, 132, 60, 16, 3])))
+        worst = max(worst, span)
+    assert worst <= 32
+    # one long sequence among short ones on few heads: the cut count is held down by the record limit
+    span, active = _check_walk([4999, 3, 0, 17], 1, 5008, 148)
+    assert span <= 32 and active < 148
+    # equal lengths and fewer heads than CTAs: a whole number of CTAs per head
+    span, active = _check_walk([4095] * 8, 8, 4096, 148)
+    assert active == 128 and span == 2
+    # sequences that cannot be served (full cache) contribute no rows
+    _check_walk([10, 4096, 7], 4, 4096, 148)
