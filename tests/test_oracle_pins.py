@@ -510,3 +510,39 @@ def test_model_embedding_logits_and_argmax_tie():
     wlm2[3] = B16(F32(nf[0])); wlm2[7] = wlm2[3]
     _, nxt = orc.model_decode(embed, [w], gf, wlm2, [kc], [vc], ids[:1], [1], [1])
     assert nxt[0] == 3
+
+
+@pytest.mark.parametrize("n_layers", [2, 3, 4])
+def test_model_layer_loop_equals_the_chain_of_single_layers(n_layers):
+    # Figure 1 repeated over the stack: the model call must be exactly the chain embedding row -> layer 0 ->
+    # layer 1 -> ... -> final norm -> logits, with layer l reading and appending to ITS weights and ITS caches.
+    # Every layer has distinct weights and distinct caches, sequences have distinct lengths and positions, and an
+    # odd and an even number of layers are run, so a wrong per-layer index or a wrong buffer after the ping-pong
+    # of the activation buffers changes the hidden state or leaves the wrong cache row written.
+    D, H, d, K, V, N = 8, 2, 4, 16, 12, 7
+    layers = [_tiny_layer(D, H, d, K) for _ in range(n_layers)]
+    embed, gf, wlm = rnd(V, D), B16(1 + 0.1 * RNG.standard_normal(D)), rnd(V, D)
+    ids = np.array([5, 2, 9], np.int32)
+    lens, pos = np.array([3, 0, 5], np.int32), np.array([4, 0, 6], np.int32)
+    caches = [_caches(3, H, N, d) for _ in range(n_layers)]
+    # the chain, one call per layer on private copies
+    ck = [c[0].copy() for c in caches]
+    cv = [c[1].copy() for c in caches]
+    x = embed[ids].copy()
+    for l in range(n_layers):
+        x = orc.layer_decode(layers[l], x, ck[l], cv[l], pos, lens)
+    want_logits = orc.gemv_t(orc.rmsnorm(x, gf, 1e-5), wlm).astype(np.float32)
+    # the model call
+    mk = [c[0].copy() for c in caches]
+    mv = [c[1].copy() for c in caches]
+    logits, nxt, hid = orc.model_decode(embed, layers, gf, wlm, mk, mv, ids, pos, lens, want_hidden=True)
+    assert (hid == x).all()
+    assert (logits == want_logits).all()
+    assert (nxt == want_logits.argmax(axis=1)).all()
+    for l in range(n_layers):
+        assert (mk[l] == ck[l]).all() and (mv[l] == cv[l]).all(), l
+        # and the appended rows of different layers really differ (the check above can tell the layers apart)
+        for b in range(3):
+            assert (mk[l][b, :, lens[b]] != caches[l][0][b, :, lens[b]]).any()
+        if l:
+            assert (mk[l][0, :, lens[0]] != mk[l - 1][0, :, lens[0]]).any()
