@@ -32,14 +32,14 @@ if str(ROOT) not in sys.path:
 METRIC = "decode_tokens_per_s"
 UNIT = "tok/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one mlp_decode_kernel launch (Phi-3 shape, batch 1) from the
-# ncu capture summarised in profiles/chain_kernels_cfg1_cfg2.md (151.09 MB read + 4.05 MB written).
+# dram__bytes_read.sum + dram__bytes_write.sum of one mlp_decode_kernel launch (Phi-3 shape, batch 1), from an
+# ncu capture of that kernel (151.09 MB read + 4.05 MB written).
 NCU_MLP_TRAFFIC_BYTES = 155.1e6
 # DRAM traffic of decode_step_kernel relative to its algorithmic bytes, from two ncu captures of one decode
-# step of the cfg3 shape cut to 4 and to 8 layers (profiles/decode_step_kernel_cfg3.md): 239.6 MB per layer
-# and 200.7 MB for the head against 239.1 MB and 197.1 MB algorithmic, i.e. 7.867 GB for a full 32-layer step
-# against 7.848 GB.  The full-size launch is too large to capture; traffic grows in proportion to the layers
-# and steps a launch processes.
+# step of the batch-1 full-stack shape cut to 4 and to 8 layers: 239.6 MB per layer and 200.7 MB for the head
+# against 239.1 MB and 197.1 MB algorithmic, i.e. 7.867 GB for a full 32-layer step against 7.848 GB.  The
+# full-size launch is too large to capture; traffic grows in proportion to the layers and steps a launch
+# processes.
 NCU_STEP_TRAFFIC_RATIO = 1.002
 
 
@@ -58,6 +58,8 @@ def parse_args():
                          "not the benchmark configuration)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-also", action="store_true",
+                    help="skip the second timed block of the default run (the ragged batch-8 stack, cfg4)")
     return ap.parse_args()
 
 
@@ -234,6 +236,50 @@ def whole_job_rate(units_per_rank: int, world: int, seconds_max: float) -> float
 
 
 # ------------------------------------------------------------------ our arm
+
+def time_ragged_batch(fb, wl, torch, dev, local, dm, layers, embed, g_final, w_lm, seed, peak, step_kernel, world, barrier,
+                      steps: int = 20, warmup: int = 5) -> dict:
+    """The full stack at batch 8 with ragged cache lengths (the cfg4 workload) on the weights already resident:
+    `steps` single decode steps, one launch each, timed with CUDA events on the launch stream after `warmup`
+    untimed ones.  Every step streams 14 GB (far beyond the L2) and appends the same rows again (the append is
+    idempotent), so all steps do the same work."""
+    W = wl.workload("cfg4")
+    B, lens0 = W.batch, np.asarray(W.past_lens, np.int32)
+    ctx = fb.Context.from_dims(dm, B, W.max_seq, device=local, n_layers=W.n_layers)
+    ctx.set_option("step_kernel", step_kernel)
+    caches = [wl.kv_cache(dm, i, B, W.max_seq, seed, device=dev) for i in range(W.n_layers)]
+    model = ctx.make_model(embed, layers, g_final, w_lm, [c[0] for c in caches], [c[1] for c in caches])
+    pos, sl = torch.tensor(lens0, device=dev), torch.tensor(lens0, device=dev)
+    tok = torch.tensor(wl.token_ids(B, dm.vocab, seed), device=dev)
+    nxt = torch.zeros(B, dtype=torch.int32, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            ctx.model_decode(model, tok, pos, sl, None, nxt, advance=False, stream=stream)
+    barrier()
+    with torch.cuda.stream(stream):
+        ev0.record(stream)
+        for _ in range(steps):
+            ctx.model_decode(model, tok, pos, sl, None, nxt, advance=False, stream=stream)
+        ev1.record(stream)
+    stream.synchronize()
+    barrier()
+    ms = max_over_ranks(ev0.elapsed_time(ev1), dev, world)
+    status = ctx.get_status()
+    nbytes = float(W.algorithmic_bytes(0))
+    gbs = nbytes / (ms / steps * 1e-3) / 1e9
+    out = {"value": whole_job_rate(B * steps, world, ms * 1e-3), "unit": UNIT, "steps": steps, "warmup": warmup,
+           "ms_per_step": ms / steps, "batch": B, "past_lens": lens0.tolist(), "max_seq": W.max_seq,
+           "algorithmic_bytes_per_step": nbytes, "device_status": status,
+           "roofline": {"bound": "hbm", "kernel": "decode_step_kernel", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                        "frac": gbs / peak, "traffic": None, "bytes_per_launch": nbytes,
+                        "avg_launch_us": ms / steps * 1e3}}
+    ctx.close()
+    del caches
+    torch.cuda.empty_cache()
+    return out
+
 
 def run_ours(args):
     import torch
@@ -417,6 +463,12 @@ def run_ours(args):
                 "kernel_avg_us": {k: round(v[0] / v[1] * 1e3, 2) for k, v in prof.items() if v[1]},
                 "how": "CUDA events around every launch on the launch stream, separate eager pass of the same steps"}
 
+    # ---- second timed block of the default run: the ragged batch of 8 on the same weights ----
+    also = None
+    if args.workload == "cfg3" and args.layers == 0 and not args.no_also:
+        also = {"cfg4": time_ragged_batch(fb, wl, torch, dev, local, dm, layers, embed, g_final, w_lm, seed, peak,
+                                          args.step_kernel, world, barrier)}
+
     # ---- end to end through the public API with host buffers ----
     e2e = None
     if not args.no_e2e:
@@ -489,6 +541,8 @@ def run_ours(args):
                 "hbm_frac_whole_step": float(step_bytes) / (ms_max / K * 1e-3) / 1e9 / peak,
                 "gpu_launches": int(launches_total),
                 "device_status": status, "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu}
+        if also is not None:
+            line["also"] = also
         print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:

@@ -97,11 +97,14 @@ int fasttps_destroy(fasttps_ctx *ctx);
  * Section 3.2 item 1 ("interlaced layout of gate-up weights").  `src` is the
  * logical row-major bf16 matrix described at fasttps_weight_kind, `dst` a
  * device buffer of fasttps_packed_bytes(kind) bytes.  Packed layouts (bf16):
- *   QKV, O, LM_HEAD: the transposed matrix W^T [out, in], with `out` padded up to a
+ *   QKV, LM_HEAD: the transposed matrix W^T [out, in], with `out` padded up to a
  *            multiple of 16 by zero rows, cut into tiles of 16 output rows x 32 inputs;
  *            a tile is stored row-major (1 KB), tiles are ordered by (row tile, input
  *            block), so that the share of a CTA -- a run of row tiles -- is one contiguous
  *            byte range and one tile is the A operand of two tensor-core instructions;
+ *   O:       the same tiling, with the 16 rows of a tile paired: row r < 8 of row tile J is output
+ *            column 16J + 2r, row r + 8 is column 16J + 2r + 1, so that the two sums a thread of the
+ *            tensor-core product holds for a batch row are neighbours (one 8-byte reduction);
  *   GATE_UP: the same tiling of a [2K, D] matrix whose rows are interlaced in blocks of
  *            8: for j-octet J the rows 16J..16J+7 are gate columns 8J..8J+7 and
  *            16J+8..16J+15 the matching up columns, so a gate value and its up value
@@ -143,7 +146,7 @@ int fasttps_attn_decode(fasttps_ctx *ctx, const void *q, const void *k_new, cons
 int fasttps_mlp_decode(fasttps_ctx *ctx, const void *x, const void *w_gate_up, const void *w_down,
                        void *out, int batch, void *stream);
 
-/* Variant of fasttps_mlp_decode that uses no workspace memory and allocates nothing.  The paper has
+/* Variant of fasttps_mlp_decode that keeps its scratch out of the workspace and allocates nothing.  The paper has
  * no counterpart: the arithmetic and the kernel are those of fasttps_mlp_decode; only the scratch of
  * the kernel (the FP32 accumulator of batch x hidden partial sums and its arrival counter) lives in a
  * fixed array in the library's own device data segment instead of the context workspace.  It is for
@@ -154,6 +157,9 @@ int fasttps_mlp_decode(fasttps_ctx *ctx, const void *x, const void *w_gate_up, c
  *   Set-up: the first call on a device looks the array's address up once (this may load the module);
  *   make it during initialisation, before capturing a stream.  No call allocates or frees.
  *   Every call clears the counter and the accumulator rows it uses, on `stream`, before the kernel.
+ *   The context still supplies the model shape and its device status word (a bounded wait that ran out is
+ *   reported there), and the call must be made with the context's device current: the array is per device,
+ *   and a call made with another device current returns FASTTPS_INVALID_ARG.
  *   The array is one per device and process: calls that overlap in time (other streams or threads)
  *   race on it; calls on one stream are ordered. */
 int fasttps_mlp_decode_static(fasttps_ctx *ctx, const void *x, const void *w_gate_up, const void *w_down,
@@ -169,7 +175,11 @@ int fasttps_linear_decode(fasttps_ctx *ctx, int kind, const void *x, const void 
 
 /* One decoder layer: RMSNorm -> QKV -> attn_decode -> o_proj (+x) -> RMSNorm -> MLP (+h).
  *   x_in [B,D], x_out [B,D] (may alias x_in); caches, pos, seq_lens as in
- *   fasttps_attn_decode (caches of THIS layer). */
+ *   fasttps_attn_decode (caches of THIS layer).
+ * For batch <= 8 (and n_q_heads * head_dim == hidden, n_q_heads <= 128 and <= the number of SMs) the layer
+ * is ONE cooperative launch of the persistent kernel described at fasttps_model_decode, restricted to one
+ * layer: the three products share one shared-memory ring and meet at grid-wide barriers; otherwise (and with
+ * option "step_kernel" 0) it is one kernel per product, chained with programmatic dependent launch. */
 int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const void *x_in, void *x_out,
                          void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
                          int batch, void *stream);
@@ -186,9 +196,10 @@ int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const
  * n_layers <= 48) the whole step is ONE cooperative
  * launch of a persistent kernel (one CTA per SM, grid-wide barriers between the products,
  * weights and K/V streamed ahead through shared memory across all boundaries); larger
- * batches run one kernel per product, chained with programmatic dependent launch.  A
- * context serves one model at a time: the layer pointers are cached on the device and
- * re-uploaded (asynchronously, on `stream`) whenever the arrays passed here change. */
+ * batches run one kernel per product, chained with programmatic dependent launch.  The
+ * layer pointers are copied into the launch parameters at the call: the host arrays may be
+ * reused or changed as soon as the call returns, and calls that pass different tables (other
+ * caches, other weights) may follow one another on the stream without synchronising. */
 int fasttps_model_decode(fasttps_ctx *ctx, const void *embed, const fasttps_layer_weights *layers,
                          const void *g_final, const void *w_lm_head,
                          void *const *k_caches, void *const *v_caches,
@@ -219,15 +230,17 @@ int fasttps_model_decode_host(fasttps_ctx *ctx, const void *embed, const fasttps
                               int32_t *host_next_ids, int batch, void *stream);
 
 /* Tuning switches of a context (host side, take effect at the next call):
- *   "step_kernel" 0/1  route model calls with batch <= 8 through the persistent step kernel
+ *   "step_kernel" 0/1  route model and layer calls with batch <= 8 through the persistent step kernel
  *                      (default: environment variable FASTTPS_STEP_KERNEL, else 1).
  *   "gqa_share" 0/1    fasttps_attn_decode and the per-product chain read every cached K/V row once for
- *                      the whole group of query heads that shares it (Section 4.1; groups of 2, 4 or 8)
+ *                      the whole group of query heads that shares it (Section 4.1; groups of 2 to 16)
  *                      instead of once per query head (default 1; 0 is the comparison point).
  * Unknown names return FASTTPS_INVALID_ARG. */
 int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value);
 
-/* Synchronises the device and returns the status word (then clears it). */
+/* Synchronises the device and returns the status word (then clears it).  If the word reports a bounded wait
+ * that ran out, the workspace's accumulators, tickets and barrier words are cleared as well: the kernels of the
+ * abandoned call left them in an unknown state, and the next call must find them at zero. */
 int fasttps_get_status(fasttps_ctx *ctx, uint32_t *host_status);
 /* Optional per-launch timing for benchmarks: while enabled, every kernel launch of this
  * context is bracketed by CUDA events on its stream (up to 8192 launches; not usable during

@@ -57,8 +57,7 @@ static void free_all(Ctx *c)
     cudaFree(c->amax_ticket); cudaFree(c->status); cudaFree(c->qkv); cudaFree(c->attn_out);
     cudaFree(c->h); cudaFree(c->xa); cudaFree(c->xb); cudaFree(c->logits); cudaFree(c->tok); cudaFree(c->tok2);
     if (c->pinned_tok) cudaFreeHost(c->pinned_tok);
-    cudaFree(c->grid_bar); cudaFree(c->hacc); cudaFree(c->d_layers); cudaFree(c->trace);
-    if (c->pin_layers) cudaFreeHost(c->pin_layers);
+    cudaFree(c->grid_bar); cudaFree(c->hacc); cudaFree(c->trace);
     if (c->prof_ev) {
         for (int i = 0; i < 2 * kProfMax; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
         delete[] c->prof_ev;
@@ -111,9 +110,6 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     A(dev_alloc(&c->grid_bar, kGridBarWords, true));
     A(dev_alloc(&c->hacc, 2 * B * D, true));
     A(dev_alloc(&c->trace, 2 * (size_t)kTraceLen, true));
-    A(dev_alloc(&c->d_layers, (size_t)(f.n_layers > 0 ? f.n_layers : 1), true));
-    if (e == cudaSuccess)
-        e = cudaMallocHost(reinterpret_cast<void **>(&c->pin_layers), sizeof(LayerPtrs) * (size_t)(f.n_layers > 0 ? f.n_layers : 1));
     A(dev_alloc(&c->mlp_ticket, 1, true));
     A(dev_alloc(&c->amax_val, (size_t)kMaxNB * 1024, true));
     A(dev_alloc(&c->amax_idx, (size_t)kMaxNB * 1024, true));
@@ -261,6 +257,7 @@ static int linear_impl(Ctx *c, int n_in, int n_out, const __nv_bfloat16 *x, int 
 {
     LinearArgs a;
     a.prof_class = prof_class;
+    a.pair_rows = prof_class == kProfOproj;      // the output projection is the one product over the packed W_o
     a.status = c->status;
     a.x = x; a.x_stride = x_stride; a.g = g; a.eps = c->cfg.rms_eps;
     a.w = static_cast<const __nv_bfloat16 *>(w);
@@ -326,6 +323,10 @@ static bool layer_ok(const fasttps_layer_weights *w)
            aligned16(w->w_gate_up) && aligned16(w->w_down);
 }
 
+static int layer_step_impl(Ctx *c, const fasttps_layer_weights &w, const __nv_bfloat16 *x_in, __nv_bfloat16 *x_out,
+                           void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens, int batch,
+                           cudaStream_t st);
+
 int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const void *x_in, void *x_out,
                          void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
                          int batch, void *stream)
@@ -335,6 +336,9 @@ int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const
     if (batch < 1 || batch > c->cfg.max_batch || !layer_ok(w)) return FASTTPS_INVALID_ARG;
     if (!aligned16(x_in) || !aligned16(x_out) || !aligned16(k_cache) || !aligned16(v_cache) || !pos || !seq_lens)
         return FASTTPS_INVALID_ARG;
+    if (c->opt_step_kernel != 0 && step_kernel_supported(c, batch, /*layer_mode=*/true))
+        return layer_step_impl(c, *w, static_cast<const __nv_bfloat16 *>(x_in), static_cast<__nv_bfloat16 *>(x_out),
+                               k_cache, v_cache, pos, seq_lens, batch, static_cast<cudaStream_t>(stream));
     return layer_impl(c, *w, static_cast<const __nv_bfloat16 *>(x_in), static_cast<__nv_bfloat16 *>(x_out), k_cache,
                       v_cache, pos, seq_lens, batch, static_cast<cudaStream_t>(stream));
 }
@@ -368,42 +372,11 @@ static int model_args_ok(const Ctx *c, const void *embed, const fasttps_layer_we
     return FASTTPS_OK;
 }
 
-// n_steps consecutive tokens in one launch of the persistent step kernel (batch <= 8)
-static int step_impl(Ctx *c, const void *embed, const fasttps_layer_weights *layers, const void *g_final,
-                     const void *w_lm_head, void *const *k_caches, void *const *v_caches, const int32_t *token_ids,
-                     int32_t *pos, int32_t *seq_lens, float *logits, int32_t *next_ids, int32_t *out_ids, int batch,
-                     int n_steps, int advance, cudaStream_t st)
+// the workspace and shape fields of a step-kernel launch
+static void step_args_common(Ctx *c, StepArgs &a, int batch)
 {
     const fasttps_config &f = c->cfg;
-    // the device table of layer pointers is refreshed only when the caller's arrays change
-    bool same = c->layers_uploaded == f.n_layers;
-    for (int l = 0; l < f.n_layers; ++l) {
-        LayerPtrs lp;
-        lp.g_attn = static_cast<const __nv_bfloat16 *>(layers[l].g_attn_norm);
-        lp.w_qkv = static_cast<const __nv_bfloat16 *>(layers[l].w_qkv);
-        lp.w_o = static_cast<const __nv_bfloat16 *>(layers[l].w_o);
-        lp.g_mlp = static_cast<const __nv_bfloat16 *>(layers[l].g_mlp_norm);
-        lp.w_gu = static_cast<const __nv_bfloat16 *>(layers[l].w_gate_up);
-        lp.w_down = static_cast<const __nv_bfloat16 *>(layers[l].w_down);
-        lp.k_cache = static_cast<__nv_bfloat16 *>(k_caches[l]);
-        lp.v_cache = static_cast<__nv_bfloat16 *>(v_caches[l]);
-        if (!same || memcmp(&c->pin_layers[l], &lp, sizeof lp) != 0) {
-            same = false;
-            c->pin_layers[l] = lp;
-        }
-    }
-    if (!same) {
-        FT_CUDA(cudaMemcpyAsync(c->d_layers, c->pin_layers, sizeof(LayerPtrs) * f.n_layers, cudaMemcpyHostToDevice, st));
-        c->layers_uploaded = f.n_layers;
-    }
-    StepArgs a;
-    a.embed = static_cast<const __nv_bfloat16 *>(embed);
-    a.layers = c->d_layers;
-    a.g_final = static_cast<const __nv_bfloat16 *>(g_final);
-    a.w_lm = static_cast<const __nv_bfloat16 *>(w_lm_head);
-    a.token_ids = token_ids; a.pos = pos; a.seq_lens = seq_lens;
-    a.logits = logits; a.next_ids = next_ids; a.out_ids = out_ids;
-    a.batch = batch; a.n_steps = n_steps; a.advance = advance; a.n_layers = f.n_layers;
+    a.batch = batch;
     a.D = f.hidden; a.n_q_heads = f.n_q_heads; a.n_kv_heads = f.n_kv_heads; a.head_dim = f.head_dim;
     a.K = f.inter; a.V = f.vocab; a.max_seq = f.max_seq; a.eps = f.rms_eps;
     a.cos_tab = c->cos_tab; a.sin_tab = c->sin_tab;
@@ -412,7 +385,58 @@ static int step_impl(Ctx *c, const void *embed, const fasttps_layer_weights *lay
     a.amax_val = c->amax_val; a.amax_idx = c->amax_idx; a.tok = c->tok2;
     a.bar = c->grid_bar; a.status = c->status;
     a.trace = c->trace; a.trace_len = kTraceLen;
+    a.x_out = nullptr;
+}
+
+static LayerPtrs layer_ptrs(const fasttps_layer_weights &w, void *k_cache, void *v_cache)
+{
+    LayerPtrs lp;
+    lp.g_attn = static_cast<const __nv_bfloat16 *>(w.g_attn_norm);
+    lp.w_qkv = static_cast<const __nv_bfloat16 *>(w.w_qkv);
+    lp.w_o = static_cast<const __nv_bfloat16 *>(w.w_o);
+    lp.g_mlp = static_cast<const __nv_bfloat16 *>(w.g_mlp_norm);
+    lp.w_gu = static_cast<const __nv_bfloat16 *>(w.w_gate_up);
+    lp.w_down = static_cast<const __nv_bfloat16 *>(w.w_down);
+    lp.k_cache = static_cast<__nv_bfloat16 *>(k_cache);
+    lp.v_cache = static_cast<__nv_bfloat16 *>(v_cache);
+    return lp;
+}
+
+// n_steps consecutive tokens in one launch of the persistent step kernel (batch <= 8)
+static int step_impl(Ctx *c, const void *embed, const fasttps_layer_weights *layers, const void *g_final,
+                     const void *w_lm_head, void *const *k_caches, void *const *v_caches, const int32_t *token_ids,
+                     int32_t *pos, int32_t *seq_lens, float *logits, int32_t *next_ids, int32_t *out_ids, int batch,
+                     int n_steps, int advance, cudaStream_t st)
+{
+    const fasttps_config &f = c->cfg;
+    StepArgs a;
+    step_args_common(c, a, batch);
+    // the layer pointers are launch parameters: a launch keeps the table it was given, whatever later calls pass
+    for (int l = 0; l < f.n_layers; ++l) a.layers[l] = layer_ptrs(layers[l], k_caches[l], v_caches[l]);
+    a.embed = static_cast<const __nv_bfloat16 *>(embed);
+    a.g_final = static_cast<const __nv_bfloat16 *>(g_final);
+    a.w_lm = static_cast<const __nv_bfloat16 *>(w_lm_head);
+    a.token_ids = token_ids; a.pos = pos; a.seq_lens = seq_lens;
+    a.logits = logits; a.next_ids = next_ids; a.out_ids = out_ids;
+    a.n_steps = n_steps; a.advance = advance; a.n_layers = f.n_layers;
     return launch_step(c, a, st);
+}
+
+// one layer on the caller's activations in one launch of the persistent step kernel (batch <= 8)
+static int layer_step_impl(Ctx *c, const fasttps_layer_weights &w, const __nv_bfloat16 *x_in, __nv_bfloat16 *x_out,
+                           void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens, int batch,
+                           cudaStream_t st)
+{
+    StepArgs a;
+    step_args_common(c, a, batch);
+    a.layers[0] = layer_ptrs(w, k_cache, v_cache);
+    a.embed = nullptr; a.g_final = nullptr; a.w_lm = nullptr; a.token_ids = nullptr;
+    a.pos = const_cast<int32_t *>(pos); a.seq_lens = const_cast<int32_t *>(seq_lens);   // read only: advance is 0
+    a.logits = nullptr; a.next_ids = nullptr; a.out_ids = nullptr;
+    a.n_steps = 1; a.advance = 0; a.n_layers = 1;
+    a.x0 = const_cast<__nv_bfloat16 *>(x_in);            // read only in layer mode
+    a.x_out = x_out;
+    return launch_layer_step(c, a, st);
 }
 
 int fasttps_model_decode(fasttps_ctx *ctx, const void *embed, const fasttps_layer_weights *layers,
@@ -497,6 +521,18 @@ int fasttps_get_status(fasttps_ctx *ctx, uint32_t *host_status)
     FT_CUDA(cudaDeviceSynchronize());
     FT_CUDA(cudaMemcpy(host_status, c->status, sizeof(uint32_t), cudaMemcpyDeviceToHost));
     FT_CUDA(cudaMemset(c->status, 0, sizeof(uint32_t)));
+    if (*host_status & FASTTPS_DEV_WAIT_TIMEOUT) {
+        // CTAs that gave up left without taking their tickets and with partial sums already added: everything the
+        // kernels expect to find at zero goes back to zero, so that the next call starts clean
+        const fasttps_config &f = c->cfg;
+        const size_t B = f.max_batch, D = f.hidden;
+        FT_CUDA(cudaMemset(c->mlp_acc, 0, 2 * B * D * sizeof(float)));
+        FT_CUDA(cudaMemset(c->hacc, 0, 2 * B * D * sizeof(float)));
+        FT_CUDA(cudaMemset(c->mlp_ticket, 0, sizeof(int)));
+        FT_CUDA(cudaMemset(c->amax_ticket, 0, sizeof(int)));
+        FT_CUDA(cudaMemset(c->attn_ticket, 0, B * f.n_q_heads * sizeof(int)));
+        FT_CUDA(cudaMemset(c->grid_bar, 0, kGridBarWords * sizeof(unsigned)));
+    }
     return FASTTPS_OK;
 }
 

@@ -184,7 +184,7 @@ struct WeightRing {
         for (int g = 0; g < pieces; ++g) {
             const unsigned char *src = g < pieces0 ? base0 + (size_t)g * slot_bytes
                                                    : base1 + (size_t)(g - pieces0) * slot_bytes;
-            if (!put(g, src, (uint32_t)slot_bytes)) return;
+            if (!put(g, src, (uint32_t)slot_bytes)) { drain(g); return; }
         }
     }
     // every lane of a consumer warp; returns the slot holding piece g (ok is cleared on a failed wait)
@@ -203,10 +203,13 @@ struct WeightRing {
         __syncwarp();
         if ((threadIdx.x & 31) == 0) mbar_arrive(&empty[slot_of(g)]);
     }
-    // producer thread, on the way out after a failure: give the copies in flight a bounded chance to land
-    __device__ __forceinline__ void drain()
+    // producer thread, on the way out after a failure with pieces [0, issued) handed to the copy engine: the
+    // copies still in flight (at most the last nslot pieces) get a bounded chance to land before the CTA's
+    // shared memory is given up
+    __device__ __forceinline__ void drain(int issued)
     {
-        for (int s = 0; s < nslot; ++s) (void)mbar_wait_bounded(&full[s], 0, nullptr);
+        for (int g = issued > nslot ? issued - nslot : 0; g < issued; ++g)
+            (void)mbar_wait_bounded(&full[slot_of(g)], (uint32_t)round_of(g) & 1u, nullptr);
     }
 };
 

@@ -189,9 +189,13 @@ __device__ __forceinline__ bool attn_for_each_tile(const AttnArgs &a, Src src, F
 template <int DH, bool SHARE = false>
 __device__ __forceinline__ bool attn_produce(const AttnArgs &a, WeightRing &ring, int &piece, int cta, int ncta)
 {
-    return attn_for_each_tile<DH, SHARE>(a, WalkSource(a, cta, ncta, SHARE), [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
-        return ring.put2(piece++, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes);
+    const bool done = attn_for_each_tile<DH, SHARE>(a, WalkSource(a, cta, ncta, SHARE), [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
+        if (!ring.put2(piece, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes)) return false;
+        ++piece;
+        return true;
     });
+    if (!done) ring.drain(piece);      // the copies in flight get a bounded chance to land before the CTA leaves
+    return done;
 }
 
 // Consumer warps (nwc of them, threads 0 .. 32 nwc - 1, synchronised by named barrier 1): the attention

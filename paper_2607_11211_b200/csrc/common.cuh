@@ -18,12 +18,10 @@ constexpr unsigned kFull = 0xffffffffu;
 struct LayerPtrs;
 
 struct Ctx {
-    // persistent step kernel: grid barrier words, device table of layer pointers and its pinned shadow
+    // persistent step kernel: grid barrier words, FP32 sums of the output projection, timeline
     unsigned *grid_bar;
     float *hacc;
     unsigned long long *trace;       // [2][kTraceLen] phase timeline of the last step-kernel launch
-    LayerPtrs *d_layers, *pin_layers;
-    int layers_uploaded;             // number of valid entries in pin_layers / d_layers
     int opt_step_kernel;             // 1: model calls with batch <= 8 use the persistent step kernel
     int opt_gqa_share;               // 1: the attention kernel streams a K/V head once for its group of 2, 4 or 8 query heads
     fasttps_config cfg;
@@ -59,6 +57,7 @@ struct Ctx {
 constexpr int kProfMax = 8192;
 constexpr int kTraceLen = 4096;             // global-timer stamps kept per traced CTA of the step kernel
 constexpr int kGridBarWords = 256;          // barrier counter + one group counter per query head (<= 128)
+constexpr int kMaxStepLayers = 48;          // layers the persistent step kernel's layer table holds
 enum ProfClass { kProfQkv = 0, kProfAttn, kProfOproj, kProfMlp, kProfLmHead, kProfEmbed, kProfStep, kProfClasses };
 
 // Brackets one kernel launch with events when profiling is on.
@@ -183,6 +182,10 @@ __device__ __forceinline__ float4 ld_cg_f4(const float *p)
     return v;
 }
 
+__device__ __forceinline__ void red_add_v2(float *p, float a, float b)
+{
+    asm volatile("red.global.add.v2.f32 [%0], {%1,%2};" ::"l"(p), "f"(a), "f"(b) : "memory");
+}
 __device__ __forceinline__ void red_add_v4(float *p, float a, float b, float c, float d)
 {
     asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
@@ -257,6 +260,7 @@ struct LinearArgs {
     int32_t *next_ids;
     int32_t *adv_pos, *adv_len;  // advanced by one by the argmax finaliser when non-null
     int prof_class;
+    int pair_rows;               // packed rows c and c + 8 of a tile are the output columns 2 c and 2 c + 1 (W_o)
     uint32_t *status;
 };
 
@@ -297,7 +301,6 @@ struct LayerPtrs {
 
 struct StepArgs {
     const __nv_bfloat16 *embed;      // [V][D]
-    const LayerPtrs *layers;         // device table [n_layers]
     const __nv_bfloat16 *g_final, *w_lm;
     const int32_t *token_ids;        // [B] tokens of the first step
     int32_t *pos, *seq_lens;         // [B]; advanced by n_steps at the end iff advance
@@ -321,11 +324,16 @@ struct StepArgs {
     uint32_t *status;
     unsigned long long *trace;       // [2][trace_len] global-timer stamps of the first and last CTA, or null
     int trace_len;
+    __nv_bfloat16 *x_out;            // layer mode: [B][D] output of the layer (x0 is then its input; may be the same buffer)
+    // the layer table travels with the launch (kernel parameter space): nothing to upload, nothing a later call
+    // could overwrite while this launch is still queued
+    LayerPtrs layers[kMaxStepLayers];
 };
 
 int launch_linear(Ctx *c, const LinearArgs &a, cudaStream_t st);
-bool step_kernel_supported(const Ctx *c, int batch);
+bool step_kernel_supported(const Ctx *c, int batch, bool layer_mode = false);
 int launch_step(Ctx *c, const StepArgs &a, cudaStream_t st);
+int launch_layer_step(Ctx *c, const StepArgs &a, cudaStream_t st);
 int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st);
 int launch_mlp(Ctx *c, const MlpArgs &a, cudaStream_t st);
 int launch_embed(Ctx *c, const __nv_bfloat16 *embed, const int32_t *ids, __nv_bfloat16 *x, int batch, cudaStream_t st);

@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(MAXT, 1) linear_kernel(LinearArgs a)
         const int u = cc * 8 + b;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const int row = (tile0 + tile) * 16 + cc + 8 * h;
+            const int row = (tile0 + tile) * 16 + (a.pair_rows ? 2 * cc + h : cc + 8 * h);
             if (row >= a.n_out) continue;
             float v = h ? v1 : v0;
             if (a.res) v += __bfloat162float(a.res[(size_t)b * a.res_stride + row]);

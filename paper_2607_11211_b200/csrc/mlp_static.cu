@@ -35,11 +35,15 @@ constexpr int kStaticMaxDevices = 64;
 std::mutex g_static_mu;
 void *g_static_addr[kStaticMaxDevices];        // per device, null until looked up
 
-// Address of the scratch array on the current device (looked up once per device).
-int static_scratch(unsigned char **out)
+// Address of the scratch array on the context's device, which must be the current one (looked up once per device).
+int static_scratch(int ctx_device, unsigned char **out)
 {
     int dev = -1;
     FT_CUDA(cudaGetDevice(&dev));
+    if (dev != ctx_device) {
+        set_last_error_text("fasttps_mlp_decode_static: the context's device is not the current device");
+        return FASTTPS_INVALID_ARG;
+    }
     if (dev < 0 || dev >= kStaticMaxDevices) {
         set_last_error_text("fasttps_mlp_decode_static: device ordinal beyond the per-device address table");
         return FASTTPS_INVALID_ARG;
@@ -79,7 +83,7 @@ extern "C" int fasttps_mlp_decode_static(fasttps_ctx *ctx, const void *x, const 
     if (((uintptr_t)x | (uintptr_t)w_gate_up | (uintptr_t)w_down | (uintptr_t)out) & 15) return FASTTPS_INVALID_ARG;
 
     unsigned char *scratch = nullptr;
-    const int rc = static_scratch(&scratch);
+    const int rc = static_scratch(c->cfg.device, &scratch);
     if (rc != FASTTPS_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 

@@ -7,6 +7,8 @@
 //     of 16 with zero rows) cut into tiles of 16 rows x 32 k, each tile row-major (1 KB),
 //     tiles ordered by (row tile, k block).  For GATE_UP packed row r of row tile J is gate
 //     column 8J + r for r < 8 and up column 8J + r - 8 otherwise (interlaced in blocks of 8).
+//     For O packed row r of row tile J is output column 16J + 2r for r < 8 and 16J + 2(r - 8) + 1
+//     otherwise: the two rows a thread of the tensor-core product holds are neighbouring columns.
 //   DOWN ("octet blocks"): for intermediate octet o and output block nb (32 columns) one
 //     512-byte block; lane (g, t4) of a warp owns 16 bytes of it: the pairs
 //     (W[8o + 2 t4][n], W[8o + 2 t4 + 1][n]) for n = 32 nb + 4 g + {0, 1, 2, 3}, i.e. the A
@@ -26,8 +28,10 @@ struct PackDesc {
     int src_is_out_in; // 1 when the logical matrix is [n_out][n_in] (LM_HEAD)
 };
 
-__device__ __forceinline__ int logical_col(int r, int interlaceK)
+__device__ __forceinline__ int logical_col(int r, int interlaceK, int kind)
 {
+    // W_o: rows g and g + 8 of a tile are the output columns 2 g and 2 g + 1 (a thread's two sums are neighbours)
+    if (kind == FASTTPS_W_O) return (r & ~15) + ((r & 8) ? 2 * (r & 7) + 1 : 2 * (r & 7));
     if (interlaceK == 0) return r;
     const int o = r >> 4, half = (r >> 3) & 1, c = r & 7;
     return half * interlaceK + o * 8 + c;
@@ -49,7 +53,7 @@ __global__ void pack_tiled_kernel(const __nv_bfloat16 *logical, __nv_bfloat16 *p
             for (int e = 0; e < 8; ++e) pv[e] = __float2bfloat16_rn(0.f);
         return;
     }
-    const int col = logical_col(row, d.interlaceK);
+    const int col = logical_col(row, d.interlaceK, d.kind);
     for (int e = 0; e < 8; ++e) {
         const size_t li = d.src_is_out_in ? (size_t)col * d.n_in + (k0 + e) : (size_t)(k0 + e) * d.n_out + col;
         if (inverse) const_cast<__nv_bfloat16 *>(logical)[li] = pv[e];

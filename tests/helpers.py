@@ -63,3 +63,79 @@ def fig8_case(n_t: int, heads: int = 32, d: int = 96, seed: int = 20260711):
     vc[:, :, n_t - 1:] = 0
     L = np.array([n_t - 1], np.int32)
     return q, k_new, v_new, kc, vc, L.copy(), L
+
+
+def shift_ulps(bits, n: int) -> np.ndarray:
+    """bf16 bit patterns moved by n units in the last place (through zero where needed)."""
+    o = ordered(bits) + n
+    return np.where(o < 0, 0x8000 | (-o), o).astype(np.uint16)
+
+
+def flip_floor(n_bits, w_bits) -> float:
+    """How far a sum n . W[:, j] computed inside the call under test can move when the two sides round ONE element of
+    the normalised activation n to neighbouring bf16 values (an FP32 and a double reciprocal root that straddle a
+    rounding boundary): one bf16 unit of the largest |n_i| times the largest |W_ij|; twice that is allowed for."""
+    n = np.abs(from_bf16_bits(n_bits).astype(np.float64)).max()
+    w = np.abs(from_bf16_bits(w_bits).astype(np.float64)).max()
+    return 2.0 * float(bf16_spacing(n)) * float(w)
+
+
+def within_one_unit_floored(got, want, floor_abs: float) -> np.ndarray:
+    """|got - want| <= one bf16 unit in the last place of `want`, the unit never taken smaller than floor_abs.  For k
+    and v that are computed INSIDE the call under test: their last places are decided by the summation order and by
+    rounding flips of the normalised input (flip_floor), not by the method, wherever the sum nearly cancels."""
+    g = from_bf16_bits(got).astype(np.float64)
+    w = from_bf16_bits(want).astype(np.float64)
+    return np.abs(g - w) <= np.maximum(bf16_spacing(w), floor_abs)
+
+
+def appended_k_rows_ok(got, want, k_before_rope, rotate, d: int, floor_abs: float) -> np.ndarray:
+    """Element-wise verdict on appended K rows when the projection that produces k runs inside the call under test.
+
+    At the attention entry point both sides rotate the same bf16 k, and the stored row must be within one bf16
+    unit in the last place of the oracle's.  When k = bf16(n . W_k) is computed inside the call, an FP32 sum and a
+    double sum that straddle a rounding boundary give k values one unit apart BEFORE the rotation; the rotation
+    x_i cos - x_{i+d/2} sin can cancel, so one unit of an input is no longer one unit of the result.  The check
+    therefore asks for what the method guarantees: every stored element is within one unit of the oracle's (the
+    unit floored as in within_one_unit_floored, twice the floor because a rotated element combines two inputs), or
+    is bit for bit the oracle's rotation (FP32, separately rounded products, one rounding to bf16) of a pair
+    (k_i, k_{i+d/2}) each within one unit of the oracle's pair.
+
+    got, want, k_before_rope: bf16 bits [..., d]; rotate(bits [..., d]) -> bf16 bits of the rotated rows."""
+    got, want = np.asarray(got, np.uint16), np.asarray(want, np.uint16)
+    ok = within_one_unit_floored(got, want, 2.0 * floor_abs)
+    if ok.all():
+        return ok
+    half = d // 2
+    for da in (-1, 0, 1):
+        for db in (-1, 0, 1):
+            cand = np.asarray(k_before_rope, np.uint16).copy()
+            cand[..., :half] = shift_ulps(cand[..., :half], da)
+            cand[..., half:] = shift_ulps(cand[..., half:], db)
+            ok |= rotate(cand) == got
+    return ok
+
+
+def bf16_spacing(x) -> np.ndarray:
+    """Distance between neighbouring bf16 values at the magnitude of x (float64 array)."""
+    a = np.maximum(np.abs(np.asarray(x, np.float64)), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(a)) - 7)
+def layer_output_ok(got_bits, want_bits, h_exact, near=0.05, atol=2e-2, rtol=2e-2) -> np.ndarray:
+    """Element-wise verdict on the output x' = bf16(h + mlp(h)) of a whole layer, where h = bf16(x + attn . W_o) is
+    rounded to bf16 INSIDE the call under test.
+
+    The output bar |gpu - oracle| <= atol + rtol |oracle| is a bar on one block given the same input.  Inside a
+    layer the residual stream passes a rounding point with weight one: where the oracle's unrounded h (h_exact,
+    float64, from the oracle's own primitives) lies within `near` of a unit in the last place of the midpoint of two
+    bf16 values, an FP32 sum and a double sum may round it to either neighbour and both are correct values of h;
+    the output then moves by that one unit of h, which a cancelling MLP term can leave larger than the bar.  So an
+    element passes if it meets the plain bar, or if h_exact is that close to a rounding boundary and the element
+    meets the bar widened by one unit in the last place of h.  Everything else must meet the plain bar."""
+    g = from_bf16_bits(got_bits).astype(np.float64)
+    w = from_bf16_bits(want_bits).astype(np.float64)
+    d = np.abs(g - w)
+    plain = d <= atol + rtol * np.abs(w)
+    u = bf16_spacing(h_exact)
+    frac = np.mod(np.asarray(h_exact, np.float64) / u, 1.0)          # position between two bf16 values, in units of u
+    boundary = np.abs(frac - 0.5) <= near
+    return plain | (boundary & (d <= atol + rtol * np.abs(w) + u))

@@ -10,8 +10,8 @@ import torch
 
 from oracle import oracle as orc
 from paper_2607_11211_b200 import workload as wl
-from tests.helpers import (assert_close_bits, from_bf16_bits as F32, to_bf16_bits as B16, ulp_distance, fig8_case,
-                           FIG8_BOUND, FIG8_LENGTHS)
+from tests.helpers import (appended_k_rows_ok, layer_output_ok, within_one_unit_floored, flip_floor, assert_close_bits, from_bf16_bits as F32, to_bf16_bits as B16,
+                           ulp_distance, fig8_case, FIG8_BOUND, FIG8_LENGTHS)
 
 pytestmark = pytest.mark.gpu
 
@@ -362,21 +362,18 @@ def test_mlp_zero_weights_and_identity_construction(fb):
 
 # -------------------------------------------------------------------- layer
 
-def k_rows_ok(got, want, half):
-    """Appended K rows when the projection that feeds them is inside the call: the two sides may
-    round k to different neighbouring bf16 values before the rotation, which moves the rotated pair
-    by up to about one ulp at the magnitude of the pair."""
-    d1 = ulp_distance(got, want) <= 1
-    g, w = F32(got).astype(np.float64), F32(want).astype(np.float64)
-    pair = np.sqrt(w[..., :half] ** 2 + w[..., half:] ** 2)
-    pair = np.concatenate([pair, pair], axis=-1)
-    return d1 | (np.abs(g - w) <= 2.0 ** -7 * pair)
+def rotate_rows(bits, pos, theta):
+    """The oracle's rotation (FP32, one rounding to bf16) of bf16 rows [H, d] at position pos."""
+    f = orc.bf16_to_f32(bits)
+    out = np.stack([orc.rope(v, pos, theta) for v in f.reshape(-1, f.shape[-1])])
+    return orc.f32_to_bf16(out).reshape(bits.shape)
 
 
-def run_layer_case(fb, dims, lens, max_seq, layer=0, flips_allowed=0.0):
+def run_layer_case(fb, dims, lens, max_seq, layer=0, step_kernel=1):
     batch = len(lens)
     lens = np.asarray(lens, np.int32)
     ctx = make_ctx(fb, dims, batch, max_seq)
+    ctx.set_option("step_kernel", step_kernel)   # 1: one launch of the persistent kernel (batch <= 8), 0: one kernel per product
     w = wl.layer_weights(dims, layer, device="cuda")
     pw = ctx.pack_layer(w)
     x = wl.activations(dims, batch, device="cuda")["x"]
@@ -394,24 +391,25 @@ def run_layer_case(fb, dims, lens, max_seq, layer=0, flips_allowed=0.0):
     for b in range(batch):
         mask[b, :, lens[b]] = False
     assert (kg[mask] == k0[mask]).all() and (vg[mask] == v0[mask]).all()
+    # the oracle's intermediate tensors, from its primitives: the k it rotates, bf16(rmsnorm(x) . W_k), and the
+    # residual stream before its rounding, h = x + attn . W_o in double
+    nq, nkv, dh = dims.n_q_heads * dims.head_dim, dims.n_kv_heads * dims.head_dim, dims.head_dim
+    n1 = orc.rmsnorm(wl.bits(x), wb["g_attn"], dims.rms_eps)
+    qkv = orc.f64_to_bf16(orc.gemv(n1, wb["w_qkv"]))
+    k_pre = qkv[:, nq:nq + nkv].reshape(batch, dims.n_kv_heads, dh)
+    a_orc = orc.attn_decode(qkv[:, :nq].reshape(batch, dims.n_q_heads, dh), k_pre, qkv[:, nq + nkv:].reshape(batch, dims.n_kv_heads, dh),
+                            k0.copy(), v0.copy(), lens, lens, dims.rope_theta)
+    h_exact = F32(wl.bits(x)).astype(np.float64) + orc.gemv(a_orc.reshape(batch, nq), wb["w_o"])
     for b in range(batch):
-        assert ulp_distance(vg[b, :, lens[b]], vo[b, :, lens[b]]).max() <= 1
-        assert k_rows_ok(kg[b, :, lens[b]], ko[b, :, lens[b]], dims.head_dim // 2).all()
-        assert (ulp_distance(kg[b, :, lens[b]], ko[b, :, lens[b]]) <= 1).mean() > 0.99
+        floor = flip_floor(n1[b], wb["w_qkv"])
+        assert within_one_unit_floored(vg[b, :, lens[b]], vo[b, :, lens[b]], floor).all()
+        assert appended_k_rows_ok(kg[b, :, lens[b]], ko[b, :, lens[b]], k_pre[b],
+                                  lambda bits: rotate_rows(bits, int(lens[b]), dims.rope_theta), dims.head_dim, floor).all()
     def check_out(bits, what):
-        if flips_allowed == 0.0:
-            assert_close_bits(bits, want, what=what)
-            return
-        # The layer output is h + mlp(h) with h itself rounded to bf16 inside the call.  Where the two sides round h
-        # to neighbouring values, an output in which h and the MLP term cancel moves by up to one ulp of h
-        # (2^-7 |h|), which the bound on the outputs cannot absorb.  At most `flips_allowed` of the elements may
-        # leave the bound, and those by no more than one ulp at the largest magnitude in the tensor.
-        g, r = F32(bits).astype(np.float64), F32(want).astype(np.float64)
-        d = np.abs(g - r)
-        out = d > 2e-2 + 2e-2 * np.abs(r)
-        assert out.mean() <= flips_allowed, (what, int(out.sum()), out.size)
-        assert (d <= 2e-2 + 2e-2 * np.abs(r) + 2.0 ** -7 * np.abs(r).max()).all(), what
-        assert d.mean() < 1e-2, what
+        # plain output bar, widened by one unit in the last place of h only where the oracle's own h sits on a
+        # rounding boundary (tests/helpers.py: layer_output_ok)
+        ok = layer_output_ok(bits, want, h_exact)
+        assert ok.all(), (what, int((~ok).sum()), ok.size)
 
     check_out(wl.bits(xo), f"layer out lens={lens.tolist()}")
     # in place (x_out aliases x_in)
@@ -424,21 +422,25 @@ def run_layer_case(fb, dims, lens, max_seq, layer=0, flips_allowed=0.0):
 
 @pytest.mark.parametrize("dims,lens", [(wl.TINY, [0]), (wl.TINY, [5, 64, 17]), (wl.SMALL, [100, 3, 250, 64, 65]),
                                        (wl.SMALL_GQA, [9, 200]), (wl.SMALL, list(range(20, 240, 20)))])
-def test_layer_decode_small_shapes(fb, dims, lens):
-    run_layer_case(fb, dims, lens, 256)
+@pytest.mark.parametrize("step_kernel", [0, 1])
+def test_layer_decode_small_shapes(fb, dims, lens, step_kernel):
+    run_layer_case(fb, dims, lens, 256, step_kernel=step_kernel)
 
 
 @pytest.mark.parametrize("lens", [[256], [4095]])
-def test_layer_decode_phi3_single_layer_configs(fb, lens):
+@pytest.mark.parametrize("step_kernel", [0, 1])
+def test_layer_decode_phi3_single_layer_configs(fb, lens, step_kernel):
     # the two single-layer workloads: 256 resp. 4095 past tokens, new token at that position
-    run_layer_case(fb, wl.PHI3_MINI, lens, 4096)
+    run_layer_case(fb, wl.PHI3_MINI, lens, 4096, step_kernel=step_kernel)
 
 
 def test_layer_decode_llama3_8b_shape_grouped_query_layer(fb):
     # a whole decoder layer of the Llama3-8B row of Table 1 (hidden 4096, 32 query heads on 8 K/V heads of 128,
     # MLP 14336) through the chain: the attention inside it streams each K/V head once for its four query heads
     dims = wl.Dims(hidden=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, inter=14336, vocab=1000, n_layers=1)
-    run_layer_case(fb, dims, [700, 64], 1024, flips_allowed=1e-3)
+    run_layer_case(fb, dims, [700, 64], 1024, step_kernel=0)
+    # the persistent kernel makes one FP32 pass per query head on this shape
+    run_layer_case(fb, dims, [700, 64], 1024, step_kernel=1)
 
 
 # -------------------------------------------------------------------- model
@@ -490,6 +492,39 @@ def test_model_decode_teacher_forced_steps(fb, dims, lens, step_kernel):
                 assert_close_bits(wl.bits(kcs[l])[b, :, r], ok[l][b, :, r], what="k row")
                 assert_close_bits(wl.bits(vcs[l])[b, :, r], ov[l][b, :, r], what="v row")
     assert ctx.get_status() == 0
+    ctx.close()
+
+
+def test_model_decode_alternating_cache_sets_without_synchronising(fb):
+    # Two conversations share one context and one stream: calls that pass different cache (and weight) tables are
+    # queued back to back with no synchronisation in between.  Every launch must use the table IT was given: the
+    # layer pointers travel as launch parameters, so a later call cannot change what a queued launch reads.
+    dims, batch, max_seq, rounds = wl.SMALL, 2, 64, 3
+    ctx = make_ctx(fb, dims, batch, max_seq)
+    mw, model_a, kca, vca = build_model(fb, ctx, dims, batch, max_seq)
+    kcb = [wl.normal_bf16(wl.MASTER_SEED + 5, wl.tid("k_cache", l), tuple(kca[l].shape), device="cuda") for l in range(dims.n_layers)]
+    vcb = [wl.normal_bf16(wl.MASTER_SEED + 5, wl.tid("v_cache", l), tuple(vca[l].shape), device="cuda") for l in range(dims.n_layers)]
+    model_b = ctx.make_model(model_a["embed"], model_a["keep"][0], model_a["g_final"], model_a["w_lm"], kcb, vcb)
+    sets = {"a": (model_a, kca, vca, np.array([20, 3], np.int32)), "b": (model_b, kcb, vcb, np.array([7, 33], np.int32))}
+    host = {k: ([wl.bits(t) for t in v[1]], [wl.bits(t) for t in v[2]]) for k, v in sets.items()}
+    ids = wl.token_ids(batch * rounds * 2, dims.vocab).reshape(rounds, 2, batch)
+    state = {k: (i32(v[3]), i32(v[3])) for k, v in sets.items()}
+    logits = {(r, k): torch.zeros(batch, dims.vocab, dtype=torch.float32, device="cuda") for r in range(rounds) for k in sets}
+    nxt = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    for r in range(rounds):                       # a, b, a, b, ... with nothing but the stream ordering them
+        for j, k in enumerate(sets):
+            ctx.model_decode(sets[k][0], i32(ids[r, j]), state[k][0], state[k][1], logits[(r, k)], nxt, advance=True)
+    torch.cuda.synchronize()
+    assert ctx.get_status() == 0
+    ow = [{kk: wl.bits(v) for kk, v in L.items()} for L in mw["layers"]]
+    for j, k in enumerate(sets):
+        cur = sets[k][3].copy()
+        for r in range(rounds):
+            wlog, _ = orc.model_decode(wl.bits(mw["embed"]), ow, wl.bits(mw["g_final"]), wl.bits(mw["w_lm"]), host[k][0], host[k][1],
+                                       ids[r, j], cur, cur, dims.rms_eps, dims.rope_theta)
+            got = logits[(r, k)].cpu().numpy().astype(np.float64)
+            assert (np.abs(got - wlog) <= 2e-2 + 2e-2 * np.abs(wlog)).all(), (k, r)
+            cur += 1
     ctx.close()
 
 
