@@ -10,7 +10,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libfasttps.so"
-SOURCES = ["api.cu", "linear.cu", "attn.cu", "mlp.cu", "pack.cu", "megakernel.cu", "layer_step.cu", "mlp_static.cu"]
+SOURCES = ["api.cu", "linear.cu", "attn.cu", "mlp.cu", "pack.cu", "megakernel.cu", "layer_step.cu", "wide.cu", "mlp_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-O2"]
 

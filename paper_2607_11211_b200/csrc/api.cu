@@ -58,6 +58,7 @@ static void free_all(Ctx *c)
     cudaFree(c->h); cudaFree(c->xa); cudaFree(c->xb); cudaFree(c->logits); cudaFree(c->tok); cudaFree(c->tok2);
     if (c->pinned_tok) cudaFreeHost(c->pinned_tok);
     cudaFree(c->grid_bar); cudaFree(c->hacc); cudaFree(c->trace);
+    cudaFree(c->wide_n); cudaFree(c->wide_a_hi); cudaFree(c->wide_a_lo);
     if (c->prof_ev) {
         for (int i = 0; i < 2 * kProfMax; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
         delete[] c->prof_ev;
@@ -94,6 +95,7 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
         int rc = configure_attn_kernels();
         if (rc == FASTTPS_OK) rc = configure_linear_kernels();
         if (rc == FASTTPS_OK) rc = configure_mlp_kernels();
+        if (rc == FASTTPS_OK) rc = configure_wide_kernels();
         if (rc != FASTTPS_OK) { delete c; return rc; }
     }
 
@@ -111,8 +113,13 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     A(dev_alloc(&c->hacc, 2 * B * D, true));
     A(dev_alloc(&c->trace, 2 * (size_t)kTraceLen, true));
     A(dev_alloc(&c->mlp_ticket, 1, true));
-    A(dev_alloc(&c->amax_val, (size_t)kMaxNB * 1024, true));
-    A(dev_alloc(&c->amax_idx, (size_t)kMaxNB * 1024, true));
+    A(dev_alloc(&c->amax_val, (size_t)kWideMaxB * 1024, true));
+    A(dev_alloc(&c->amax_idx, (size_t)kWideMaxB * 1024, true));
+    if (f.max_batch > kMaxNB) {
+        A(dev_alloc(&c->wide_n, wide_x_elems((int)(nq > D ? nq : D)), true));
+        A(dev_alloc(&c->wide_a_hi, wide_a_elems(f.inter), true));
+        A(dev_alloc(&c->wide_a_lo, wide_a_elems(f.inter), true));
+    }
     A(dev_alloc(&c->amax_ticket, 1, true));
     A(dev_alloc(&c->status, 1, true));
     A(dev_alloc(&c->qkv, B * nqkv, true));
@@ -226,9 +233,68 @@ int fasttps_attn_decode(fasttps_ctx *ctx, const void *q, const void *k_new, cons
                      batch, static_cast<cudaStream_t>(stream));
 }
 
+// ---- thin-GEMM chain for batches above kMaxNB: every weight is read once for up to kWideMaxB rows ----
+
+static int wide_prep(Ctx *c, const __nv_bfloat16 *x, int x_stride, float *acc, const __nv_bfloat16 *g,
+                     __nv_bfloat16 *x_store, __nv_bfloat16 *n_out, int D, int batch, int prof_class, cudaStream_t st)
+{
+    PrepArgs p;
+    p.x = x; p.x_stride = x_stride; p.acc = acc; p.g = g; p.eps = c->cfg.rms_eps;
+    p.x_store = x_store; p.n_out = n_out; p.D = D; p.batch = batch;
+    return launch_prep_rows(c, p, prof_class, st);
+}
+
+// x: chunked activations (c->wide_n)
+static WideArgs wide_args(Ctx *c, const __nv_bfloat16 *x, const void *w, int K, int n_out, int batch)
+{
+    WideArgs a;
+    a.x = x; a.w = static_cast<const __nv_bfloat16 *>(w);
+    a.K = K; a.n_out = n_out; a.batch = batch; a.epi = kWideStore;
+    a.res = nullptr; a.res_stride = 0; a.out_bf16 = nullptr; a.out_f32 = nullptr; a.out_stride = n_out;
+    a.pair_rows = 0; a.a_hi = nullptr; a.a_lo = nullptr;
+    a.amax_val = c->amax_val; a.amax_idx = c->amax_idx; a.amax_ticket = c->amax_ticket;
+    a.next_ids = nullptr; a.adv_pos = nullptr; a.adv_len = nullptr;
+    a.status = c->status;
+    return a;
+}
+
+// x [B][D] (normalised with gain g when given) -> gate_up with siLu_Mul -> down: the sums are left in c->mlp_acc
+static int wide_mlp_sums(Ctx *c, const __nv_bfloat16 *x, const __nv_bfloat16 *g, const void *w_gu, const void *w_down,
+                         int batch, cudaStream_t st)
+{
+    const fasttps_config &f = c->cfg;
+    // the activations in chunked form, normalised on the way when a gain is given
+    int rc = wide_prep(c, x, f.hidden, nullptr, g, nullptr, c->wide_n, f.hidden, batch, kProfMlp, st);
+    if (rc) return rc;
+    WideArgs a = wide_args(c, c->wide_n, w_gu, f.hidden, 2 * f.inter, batch);
+    a.epi = kWideSilu; a.a_hi = c->wide_a_hi; a.a_lo = c->wide_a_lo;
+    rc = launch_wide_linear(c, a, kProfMlp, st);
+    if (rc) return rc;
+    WideDownArgs d;
+    d.a_hi = c->wide_a_hi; d.a_lo = c->wide_a_lo;
+    d.w = static_cast<const __nv_bfloat16 *>(w_down);
+    d.D = f.hidden; d.K = f.inter; d.batch = batch; d.acc = c->mlp_acc; d.status = c->status;
+    return launch_wide_down(c, d, st);
+}
+
+static bool wide_batch(const Ctx *c, int batch) { return batch > kMaxNB && c->wide_n != nullptr; }
+
 static int mlp_impl(Ctx *c, const __nv_bfloat16 *x, const __nv_bfloat16 *g, const void *w_gu, const void *w_down,
                     const __nv_bfloat16 *res, __nv_bfloat16 *out, int batch, cudaStream_t st)
 {
+    if (wide_batch(c, batch)) {
+        const int D = c->cfg.hidden;
+        for (int b0 = 0; b0 < batch; b0 += kWideMaxB) {
+            const int nb = batch - b0 < kWideMaxB ? batch - b0 : kWideMaxB;
+            int rc = wide_mlp_sums(c, x + (size_t)b0 * D, g, w_gu, w_down, nb, st);
+            if (rc) return rc;
+            // out = bf16(res + sums); the sums go back to zero
+            rc = wide_prep(c, res ? res + (size_t)b0 * D : nullptr, D, c->mlp_acc, nullptr, out + (size_t)b0 * D, nullptr, D, nb,
+                           kProfMlp, st);
+            if (rc) return rc;
+        }
+        return FASTTPS_OK;
+    }
     MlpArgs a;
     a.x = x; a.g = g; a.eps = c->cfg.rms_eps;
     a.w_gu = static_cast<const __nv_bfloat16 *>(w_gu);
@@ -255,6 +321,26 @@ static int linear_impl(Ctx *c, int n_in, int n_out, const __nv_bfloat16 *x, int 
                        float *out_f32, int out_stride, int batch, int32_t *next_ids, int32_t *adv_pos,
                        int32_t *adv_len, int prof_class, cudaStream_t st)
 {
+    if (wide_batch(c, batch)) {
+        for (int b0 = 0; b0 < batch; b0 += kWideMaxB) {
+            const int nb = batch - b0 < kWideMaxB ? batch - b0 : kWideMaxB;
+            // the activations in chunked form; with a gain, RMSNorm on the way (rounded to bf16 like a stored tensor)
+            int rc = wide_prep(c, x + (size_t)b0 * x_stride, x_stride, nullptr, g, nullptr, c->wide_n, n_in, nb, prof_class, st);
+            if (rc) return rc;
+            WideArgs a = wide_args(c, c->wide_n, w, n_in, n_out, nb);
+            a.res = res ? res + (size_t)b0 * res_stride : nullptr; a.res_stride = res_stride;
+            a.out_bf16 = out_bf16 ? out_bf16 + (size_t)b0 * out_stride : nullptr;
+            a.out_f32 = out_f32 ? out_f32 + (size_t)b0 * out_stride : nullptr;
+            a.out_stride = out_stride;
+            a.pair_rows = prof_class == kProfOproj;
+            a.next_ids = next_ids ? next_ids + b0 : nullptr;
+            a.adv_pos = adv_pos ? adv_pos + b0 : nullptr;
+            a.adv_len = adv_len ? adv_len + b0 : nullptr;
+            rc = launch_wide_linear(c, a, prof_class, st);
+            if (rc) return rc;
+        }
+        return FASTTPS_OK;
+    }
     LinearArgs a;
     a.prof_class = prof_class;
     a.pair_rows = prof_class == kProfOproj;      // the output projection is the one product over the packed W_o

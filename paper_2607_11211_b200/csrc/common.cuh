@@ -9,7 +9,8 @@
 
 namespace fasttps {
 
-constexpr int kMaxNB = 8;            // batch rows one weight pass serves
+constexpr int kMaxNB = 8;            // batch rows one weight pass of the register-resident kernels serves
+constexpr int kWideMaxB = 32;        // batch rows one weight pass of the thin-GEMM kernels serves (batches above kMaxNB)
 constexpr int kMaxSplits = 32;       // split-KV partitions per (sequence, head)
 constexpr unsigned kFull = 0xffffffffu;
 
@@ -43,6 +44,9 @@ struct Ctx {
     __nv_bfloat16 *h;                // [max_batch][D]
     __nv_bfloat16 *xa, *xb;          // [max_batch][D]
     float *logits;                   // [max_batch][V]
+    // thin-GEMM path (batches above kMaxNB; allocated when max_batch > kMaxNB)
+    __nv_bfloat16 *wide_n;           // chunked [32][max(D, Hq d)] activations of the product to come
+    __nv_bfloat16 *wide_a_hi, *wide_a_lo;   // chunked [32][K] MLP intermediate as a bf16 pair
     int32_t *tok;                    // [max_batch] staging for the host-buffer entry point
     int32_t *tok2;                   // [max_batch] current tokens inside the persistent step kernel
     int32_t *pinned_tok;             // pinned host staging [2][max_batch]
@@ -329,6 +333,60 @@ struct StepArgs {
     // could overwrite while this launch is still queued
     LayerPtrs layers[kMaxStepLayers];
 };
+
+// ---- thin-GEMM path (wide.cu) ----
+// Activations travel between its kernels in "chunked" form, so that one k chunk of all 32 batch rows is ONE
+// contiguous block (one bulk copy into the ring) whose rows already carry the padding that keeps the shared-memory
+// loads free of bank conflicts: element (b, k) of a [32][K] tensor sits at ((k / C) * 32 + b) * R + k % C, with
+// C = 256, R = 288 for the tiled products and C = 128, R = 136 for the down projection.
+constexpr int kWideXChunk = 256, kWideXRow = 288;       // 576 bytes per row: 512 + 64
+constexpr int kWideAChunk = 128, kWideARow = 136;       // 272 bytes per row: 256 + 16
+__host__ __device__ inline size_t wide_x_elems(int K) { return (size_t)((K + kWideXChunk - 1) / kWideXChunk) * kWideMaxB * kWideXRow; }
+__host__ __device__ inline size_t wide_a_elems(int K) { return (size_t)((K + kWideAChunk - 1) / kWideAChunk) * kWideMaxB * kWideARow; }
+__host__ __device__ inline size_t wide_x_index(int b, int k) { return ((size_t)(k / kWideXChunk) * kWideMaxB + b) * kWideXRow + k % kWideXChunk; }
+__host__ __device__ inline size_t wide_a_index(int b, int k) { return ((size_t)(k / kWideAChunk) * kWideMaxB + b) * kWideARow + k % kWideAChunk; }
+
+enum { kWideStore = 0, kWideSilu = 1 };
+struct WideArgs {
+    const __nv_bfloat16 *x;      // chunked [32][K] activations (already normalised)
+    const __nv_bfloat16 *w;      // tiled [n_out padded to 16][K]
+    int K, n_out, batch;
+    int epi;                     // kWideStore: out = sums (+ res); kWideSilu: a = silu(gate) * up from interlaced rows
+    const __nv_bfloat16 *res;    // [B][n_out] residual or null
+    int res_stride;
+    __nv_bfloat16 *out_bf16;     // [B][n_out] or null
+    float *out_f32;              // [B][n_out] or null
+    int out_stride;
+    int pair_rows;               // rows c and c + 8 of a tile are the output columns 2 c and 2 c + 1 (W_o)
+    __nv_bfloat16 *a_hi, *a_lo;  // kWideSilu: chunked [32][n_out / 2] intermediate, high and low part
+    float *amax_val;             // optional greedy argmax over out (lm_head), as in LinearArgs
+    int *amax_idx;
+    int *amax_ticket;
+    int32_t *next_ids;
+    int32_t *adv_pos, *adv_len;
+    uint32_t *status;
+};
+struct WideDownArgs {
+    const __nv_bfloat16 *a_hi, *a_lo;    // chunked [32][K] intermediate
+    const __nv_bfloat16 *w;      // packed W_down (octet blocks)
+    int D, K, batch;
+    float *acc;                  // [B][D] FP32 sums, added to
+    uint32_t *status;
+};
+struct PrepArgs {
+    const __nv_bfloat16 *x;      // [B][D] residual, rows of stride x_stride, or null
+    int x_stride;
+    float *acc;                  // [B][D] FP32 sums to fold in (then cleared), or null
+    const __nv_bfloat16 *g;      // [D] gain: n_out = rmsnorm(x + acc); null: n_out = x + acc
+    float eps;
+    __nv_bfloat16 *x_store;      // [B][D] receives bf16(x + acc), or null
+    __nv_bfloat16 *n_out;        // chunked [32][D] (the activations of the product to come), or null
+    int D, batch;
+};
+int configure_wide_kernels();
+int launch_wide_linear(Ctx *c, const WideArgs &a, int prof_class, cudaStream_t st);
+int launch_wide_down(Ctx *c, const WideDownArgs &a, cudaStream_t st);
+int launch_prep_rows(Ctx *c, const PrepArgs &a, int prof_class, cudaStream_t st);
 
 int launch_linear(Ctx *c, const LinearArgs &a, cudaStream_t st);
 bool step_kernel_supported(const Ctx *c, int batch, bool layer_mode = false);

@@ -78,7 +78,9 @@ def test_pack_unpack_round_trip_and_interlace(fb, dims):
 # ------------------------------------------------------------------- linear
 
 @pytest.mark.parametrize("dims,batch", [(wl.TINY, 1), (wl.SMALL, 3), (wl.SMALL_GQA, 8), (wl.SMALL, 11),
-                                        (wl.PHI3_MINI, 1), (wl.PHI3_MINI, 2)])
+                                        (wl.PHI3_MINI, 1), (wl.PHI3_MINI, 2),
+                                        # above 8 rows: the thin-GEMM kernels, one weight pass per 32 rows
+                                        (wl.TINY, 33), (wl.SMALL_GQA, 17), (wl.SMALL, 32), (wl.PHI3_MINI, 32)])
 def test_linear_decode_matches_oracle(fb, dims, batch):
     ctx = make_ctx(fb, dims, batch, 64)
     w = wl.layer_weights(dims, 0, device="cuda")
@@ -110,14 +112,16 @@ def test_linear_decode_matches_oracle(fb, dims, batch):
     ctx.close()
 
 
-def test_linear_integer_inputs_are_bit_exact(fb):
-    # small integers: every partial sum is exact in FP32 whatever the order of summation
+@pytest.mark.parametrize("nb", [4, 27])
+def test_linear_integer_inputs_are_bit_exact(fb, nb):
+    # small integers: every partial sum is exact in FP32 whatever the order of summation (4 rows: the
+    # register-resident kernel; 27 rows: the thin-GEMM kernel)
     dims = wl.SMALL
-    ctx = make_ctx(fb, dims, 4, 64)
+    ctx = make_ctx(fb, dims, nb, 64)
     rng = np.random.default_rng(3)
-    x = B16(rng.integers(-2, 3, (4, dims.hidden)))
+    x = B16(rng.integers(-2, 3, (nb, dims.hidden)))
     W = B16(rng.integers(-1, 2, (dims.hidden, dims.qkv_out)))
-    out = torch.zeros(4, dims.qkv_out, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(nb, dims.qkv_out, dtype=torch.bfloat16, device="cuda")
     ctx.linear_decode(fb.W_QKV, dev(x), None, ctx.pack_weight(fb.W_QKV, dev(W)), None, out, None)
     want = orc.f64_to_bf16(orc.gemv(x, W))
     assert (wl.bits(out) == want).all()
@@ -317,7 +321,8 @@ def test_attn_decode_planted_key_and_last_row_of_the_cache(fb):
 # ---------------------------------------------------------------------- MLP
 
 @pytest.mark.parametrize("dims,batch", [(wl.TINY, 1), (wl.SMALL, 2), (wl.SMALL, 3), (wl.SMALL_GQA, 5), (wl.SMALL, 8),
-                                        (wl.SMALL, 9), (wl.SMALL, 19), (wl.PHI3_MINI, 1), (wl.PHI3_MINI, 4)])
+                                        (wl.SMALL, 9), (wl.SMALL, 19), (wl.PHI3_MINI, 1), (wl.PHI3_MINI, 4),
+                                        (wl.TINY, 32), (wl.SMALL_GQA, 45), (wl.PHI3_MINI, 32)])
 def test_mlp_decode_matches_oracle(fb, dims, batch):
     ctx = make_ctx(fb, dims, batch, 64)
     w = wl.layer_weights(dims, 1, device="cuda")
@@ -421,7 +426,8 @@ def run_layer_case(fb, dims, lens, max_seq, layer=0, step_kernel=1):
 
 
 @pytest.mark.parametrize("dims,lens", [(wl.TINY, [0]), (wl.TINY, [5, 64, 17]), (wl.SMALL, [100, 3, 250, 64, 65]),
-                                       (wl.SMALL_GQA, [9, 200]), (wl.SMALL, list(range(20, 240, 20)))])
+                                       (wl.SMALL_GQA, [9, 200]), (wl.SMALL, list(range(20, 240, 20))),
+                                       (wl.SMALL, [7 * i % 250 for i in range(32)]), (wl.TINY, list(range(40)))])
 @pytest.mark.parametrize("step_kernel", [0, 1])
 def test_layer_decode_small_shapes(fb, dims, lens, step_kernel):
     run_layer_case(fb, dims, lens, 256, step_kernel=step_kernel)
