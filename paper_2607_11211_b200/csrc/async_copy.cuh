@@ -197,9 +197,16 @@ struct WeightRing {
         ok = mine;
         return slots + (size_t)(slot_of(g)) * slot_bytes;
     }
-    // consumer warp, after its last read of piece g
+    // consumer warp, after its last read of piece g.  Every lane first fences its own shared-memory reads: the
+    // arrival is made by lane 0 alone, and the warp-level barrier in front of it does not by itself keep the other
+    // lanes' loads of the slot ahead of the bulk copy that refills the slot once the last arrival is in.  Without
+    // the fence a refill was measured to overtake such loads: the first launch of the fused MLP kernel after a
+    // different kernel returned, in up to 70 % of the launches, a first row tile in which 128-byte pieces of one
+    // warp's weights were those of the tile two further on (the piece that reuses the slot); with it, none in
+    // thousands of launches.
     __device__ __forceinline__ void release(int g)
     {
+        __threadfence_block();
         __syncwarp();
         if ((threadIdx.x & 31) == 0) mbar_arrive(&empty[slot_of(g)]);
     }

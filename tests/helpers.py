@@ -39,8 +39,9 @@ def assert_close_bits(got_bits, want_bits, atol=2e-2, rtol=2e-2, what=""):
         w = from_bf16_bits(want_bits).astype(np.float64)
         bad = np.argwhere(~ok)
         i = tuple(bad[0])
+        per_row = (~ok).reshape(ok.shape[0], -1).sum(axis=1).tolist() if ok.ndim > 1 else []
         raise AssertionError(f"{what}: {len(bad)} of {ok.size} elements outside |d| <= {atol}+{rtol}|ref|; "
-                             f"first at {i}: got {g[i]}, want {w[i]}; max abs err {np.abs(g - w).max()}")
+                             f"first at {i}: got {g[i]}, want {w[i]}; max abs err {np.abs(g - w).max()}; per row {per_row[:40]}")
 
 
 # Accuracy experiment of the paper (Section 5.4, "Accuracy Stability", Fig. 8): the maximum absolute deviation of

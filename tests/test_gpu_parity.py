@@ -365,6 +365,34 @@ def test_mlp_zero_weights_and_identity_construction(fb):
     ctx.close()
 
 
+def test_mlp_decode_right_after_a_persistent_kernel_launch_many_times(fb):
+    # A slot of the shared-memory weight ring may be refilled only when every consumer warp has finished reading it.
+    # The hand-over once let a refill overtake loads still in flight: the first launch of the fused MLP kernel after
+    # a launch of a different kernel came back with a wrong first row tile in most launches (and about one in a
+    # thousand otherwise).  Alternate the two kernels a few hundred times at the benchmark's width, batch 8.
+    dims, batch, max_seq = wl.PHI3_MINI, 8, 512
+    lens = np.array([100, 7, 300, 64, 65, 250, 33, 480], np.int32)
+    ctx = make_ctx(fb, dims, batch, max_seq)
+    w = wl.layer_weights(dims, 0, device="cuda")
+    pw = ctx.pack_layer(w)
+    x = wl.activations(dims, batch, device="cuda")["x"]
+    kc, vc = wl.kv_cache(dims, 0, batch, max_seq, device="cuda")
+    want = orc.mlp_decode(wl.bits(x), wl.bits(w["w_gu"]), wl.bits(w["w_down"]))
+    L = i32(lens)
+    bad = 0
+    for _ in range(300):
+        out = torch.empty_like(x)
+        ctx.mlp_decode(x, pw["w_gu"], pw["w_down"], out)
+        ok = np.abs(F32(wl.bits(out)).astype(np.float64) - F32(want)) <= 2e-2 + 2e-2 * np.abs(F32(want))
+        bad += int(not ok.all())
+        xo = torch.empty_like(x)
+        ctx.layer_decode(pw["struct"], x, xo, kc, vc, L, L)      # one launch of the persistent kernel
+        torch.cuda.synchronize()
+    assert bad == 0, f"{bad} of 300 MLP results outside the bar"
+    assert ctx.get_status() == 0
+    ctx.close()
+
+
 # -------------------------------------------------------------------- layer
 
 def rotate_rows(bits, pos, theta):
