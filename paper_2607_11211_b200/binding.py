@@ -34,6 +34,19 @@ class LayerWeights(C.Structure):
                 ("g_mlp_norm", C.c_void_p), ("w_gate_up", C.c_void_p), ("w_down", C.c_void_p)]
 
 
+class BaselineAttnShape(C.Structure):
+    _fields_ = [("batch", C.c_int), ("n_q_heads", C.c_int), ("n_kv_heads", C.c_int), ("head_dim", C.c_int),
+                ("max_seq", C.c_int), ("cat_seq", C.c_int), ("rope_theta", C.c_float)]
+
+
+class BaselineAttnBuffers(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("q_rope", "k_rope", "q_trans", "k_trans", "v_trans", "k_cat", "v_cat", "s", "p")]
+
+
+class BaselineMlpBuffers(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("h_g", "h_s", "h_u", "h_m")]
+
+
 _lib = None
 
 
@@ -72,6 +85,9 @@ def load_library() -> C.CDLL:
     lib.fasttps_attn_splits.argtypes = [vp, i]
     lib.fasttps_attention_shares.argtypes = [vp, vp, i, i, i, i, vp, vp]
     lib.fasttps_attention_walk.argtypes = [vp, vp, i, i, i, i, vp, i]
+    lib.fasttps_baseline_attn.argtypes = [C.POINTER(BaselineAttnShape), C.POINTER(BaselineAttnBuffers), vp, vp, vp, vp, vp,
+                                          ip, ip, vp, vp, vp]
+    lib.fasttps_baseline_mlp.argtypes = [i, i, i, C.POINTER(BaselineMlpBuffers), vp, vp, vp, vp, vp, vp, vp]
     lib.fasttps_strerror.argtypes = [i]
     lib.fasttps_strerror.restype = C.c_char_p
     lib.fasttps_last_error.restype = C.c_char_p
@@ -292,3 +308,39 @@ class Context:
 
     def attn_splits(self, batch: int) -> int:
         return int(self.lib.fasttps_attn_splits(self.handle, batch))
+
+
+# ---------------------------------------------------------------------------------------------------------
+# The non-fused comparison arm (include/fasttps_baseline.h): argument marshalling only, as above.
+
+def baseline_attn(q, k_new, v_new, k_cache, v_cache, pos, seq_lens, out, cat_seq, rope_theta=10000.0, timed=False, stream=None):
+    """fasttps_baseline_attn: Algorithm 1 as ten separate launches.  Allocates the scratch tensors with torch and
+    returns (k_cat, v_cat, launch_us or None); the caller's caches are not modified."""
+    lib = load_library()
+    B, Hq, d = q.shape
+    Hkv, max_seq = k_cache.shape[1], k_cache.shape[2]
+    dev = q.device
+    e = lambda *shape, dt=torch.bfloat16: torch.empty(*shape, dtype=dt, device=dev)
+    keep = dict(q_rope=e(B, Hq, d), k_rope=e(B, Hkv, d), q_trans=e(B, Hq, d), k_trans=e(B, Hkv, d), v_trans=e(B, Hkv, d),
+                k_cat=e(B, Hkv, cat_seq, d), v_cat=e(B, Hkv, cat_seq, d), s=e(B, Hq, cat_seq, dt=torch.float32),
+                p=e(B, Hq, cat_seq, dt=torch.float32))
+    bufs = BaselineAttnBuffers(*[_ptr(keep[n]) for n, _ in BaselineAttnBuffers._fields_])
+    shape = BaselineAttnShape(B, Hq, Hkv, d, max_seq, cat_seq, rope_theta)
+    us = (C.c_float * 10)() if timed else None
+    _check(lib.fasttps_baseline_attn(C.byref(shape), C.byref(bufs), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache),
+                                     _ptr(v_cache), _ptr(pos), _ptr(seq_lens), _ptr(out), us, _stream(stream)),
+           "fasttps_baseline_attn")
+    return keep["k_cat"], keep["v_cat"], (list(us) if timed else None)
+
+
+def baseline_mlp(x, wt_gate, wt_up, wt_down, out, timed=False, stream=None):
+    """fasttps_baseline_mlp: Algorithm 2 as five separate launches on the transposed row-major matrices."""
+    lib = load_library()
+    B, D = x.shape
+    K = wt_gate.shape[0]
+    keep = [torch.empty(B, K, dtype=torch.bfloat16, device=x.device) for _ in range(4)]
+    bufs = BaselineMlpBuffers(*[_ptr(t) for t in keep])
+    us = (C.c_float * 5)() if timed else None
+    _check(lib.fasttps_baseline_mlp(B, D, K, C.byref(bufs), _ptr(x), _ptr(wt_gate), _ptr(wt_up), _ptr(wt_down), _ptr(out), us,
+                                    _stream(stream)), "fasttps_baseline_mlp")
+    return list(us) if timed else None

@@ -10,7 +10,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libfasttps.so"
-SOURCES = ["api.cu", "linear.cu", "attn.cu", "mlp.cu", "pack.cu", "megakernel.cu", "layer_step.cu", "wide.cu", "mlp_static.cu"]
+SOURCES = ["api.cu", "linear.cu", "attn.cu", "mlp.cu", "pack.cu", "megakernel.cu", "layer_step.cu", "wide.cu", "baseline.cu", "mlp_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-O2"]
 
@@ -30,7 +30,7 @@ def _stale(target: Path, deps) -> bool:
 
 
 def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) -> Path:
-    headers = list(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "fasttps.h"]
+    headers = list(CSRC.glob("*.cuh")) + list((PKG.parent / "include").glob("*.h"))
     objdir = PKG / "build"
     objdir.mkdir(exist_ok=True)
     nvcc = _nvcc()
