@@ -258,6 +258,68 @@ void orc_attn_decode(const uint16_t *q, const uint16_t *k_new, const uint16_t *v
     }
 }
 
+/* Algorithm 3 for N new tokens per sequence (the algorithm is written for Q, K, V in R^{B x N x H x d}; the token
+ * phase proper is N = 1).  Token j of sequence b has rotary position pos[b] + j and goes into cache row
+ * seq_lens[b] + j; it attends rows 0 .. seq_lens[b] + j: everything cached before the step and the new tokens up to
+ * and including itself (causal mask inside the chunk).  Written as the masked definition: all N rows are appended
+ * first, then every (token, head) takes its softmax over its own prefix of the rows.
+ *   q [B,N,Hq,d], k_new, v_new [B,N,Hkv,d], out [B,N,Hq,d]; caches, pos, seq_lens as in orc_attn_decode.
+ * A sequence is skipped unless all N rows fit: seq_lens[b] >= 0, seq_lens[b] + N <= max_seq, pos[b] >= 0. */
+void orc_attn_decode_multi(const uint16_t *q, const uint16_t *k_new, const uint16_t *v_new,
+                           uint16_t *k_cache, uint16_t *v_cache,
+                           const int32_t *pos, const int32_t *seq_lens, uint16_t *out,
+                           int B, int N, int Hq, int Hkv, int d, int max_seq, double theta)
+{
+    int G = Hq / Hkv;
+    for (int b = 0; b < B; ++b) {
+        int L = seq_lens[b];
+        if (L < 0 || L + N > max_seq || pos[b] < 0) continue;
+        for (int j = 0; j < N; ++j) {
+            for (int h = 0; h < Hkv; ++h) {
+                float kr[1024];
+                size_t src = (((size_t)b * N + j) * Hkv + h) * d;
+                for (int c = 0; c < d; ++c) kr[c] = orc_bf16_to_f32(k_new[src + c]);
+                orc_rope(kr, d, pos[b] + j, theta);
+                size_t row = (((size_t)b * Hkv + h) * max_seq + L + j) * d;
+                for (int c = 0; c < d; ++c) {
+                    k_cache[row + c] = orc_f32_to_bf16(kr[c]);
+                    v_cache[row + c] = v_new[src + c];
+                }
+            }
+        }
+    }
+    #pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        for (int jh = 0; jh < N * Hq; ++jh) {
+            int L = seq_lens[b];
+            if (L < 0 || L + N > max_seq || pos[b] < 0) continue;
+            int j = jh / Hq, h = jh % Hq, hk = h / G;
+            int Nt = L + j + 1;                              /* rows this token may see */
+            float qr[1024];
+            size_t qo = (((size_t)b * N + j) * Hq + h) * d;
+            for (int c = 0; c < d; ++c) qr[c] = orc_bf16_to_f32(q[qo + c]);
+            orc_rope(qr, d, pos[b] + j, theta);
+            const uint16_t *Kh = k_cache + ((size_t)b * Hkv + hk) * max_seq * d;
+            const uint16_t *Vh = v_cache + ((size_t)b * Hkv + hk) * max_seq * d;
+            double *s = (double *)malloc(sizeof(double) * (size_t)Nt);
+            double scale = 1.0 / sqrt((double)d), m = -INFINITY, denom = 0.0;
+            for (int r = 0; r < Nt; ++r) {
+                double acc = 0.0;
+                for (int c = 0; c < d; ++c) acc += (double)qr[c] * (double)orc_bf16_to_f32(Kh[(size_t)r * d + c]);
+                s[r] = acc * scale;
+                if (s[r] > m) m = s[r];
+            }
+            for (int r = 0; r < Nt; ++r) { s[r] = exp(s[r] - m); denom += s[r]; }
+            for (int c = 0; c < d; ++c) {
+                double o = 0.0;
+                for (int r = 0; r < Nt; ++r) o += (s[r] / denom) * (double)orc_bf16_to_f32(Vh[(size_t)r * d + c]);
+                out[qo + c] = orc_f64_to_bf16(o);
+            }
+            free(s);
+        }
+    }
+}
+
 /* Softmax probabilities of one (b, query head) after the append has been
  * done, for tests of the row-sum invariant.  p [seq_lens[b]+1] double. */
 void orc_attn_probs(const uint16_t *q, const uint16_t *k_cache, int pos, int L,
@@ -330,14 +392,16 @@ void orc_mlp_decode(const uint16_t *x, const uint16_t *w_gu, const uint16_t *w_d
  *   n2 = bf16(rmsnorm(h, g_mlp))
  *   x' = bf16(h + mlp(n2))
  */
-void orc_layer_decode(const uint16_t *g_attn, const uint16_t *w_qkv, const uint16_t *w_o,
-                      const uint16_t *g_mlp, const uint16_t *w_gu, const uint16_t *w_down,
-                      const uint16_t *x_in, uint16_t *x_out,
-                      uint16_t *k_cache, uint16_t *v_cache,
-                      const int32_t *pos, const int32_t *seq_lens,
-                      int B, int D, int Hq, int Hkv, int d, int K, int max_seq,
-                      double eps, double theta)
+static void layer_decode_n(const uint16_t *g_attn, const uint16_t *w_qkv, const uint16_t *w_o,
+                           const uint16_t *g_mlp, const uint16_t *w_gu, const uint16_t *w_down,
+                           const uint16_t *x_in, uint16_t *x_out,
+                           uint16_t *k_cache, uint16_t *v_cache,
+                           const int32_t *pos, const int32_t *seq_lens,
+                           int n_seq, int n_new, int D, int Hq, int Hkv, int d, int K, int max_seq,
+                           double eps, double theta)
 {
+    /* B: token rows of the step = sequences x new tokens per sequence; only the attention tells them apart */
+    int B = n_seq * n_new;
     int nq = Hq * d, nkv = Hkv * d, nqkv = nq + 2 * nkv;
     uint16_t *n1 = (uint16_t *)malloc(2 * (size_t)B * D);
     double *qkv = (double *)malloc(sizeof(double) * (size_t)B * nqkv);
@@ -359,7 +423,8 @@ void orc_layer_decode(const uint16_t *g_attn, const uint16_t *w_qkv, const uint1
     }
     /* a skipped sequence (bad length) leaves its attention output at zero */
     memset(ab, 0, 2 * (size_t)B * nq);
-    orc_attn_decode(qb, kb, vb, k_cache, v_cache, pos, seq_lens, ab, B, Hq, Hkv, d, max_seq, theta);
+    if (n_new == 1) orc_attn_decode(qb, kb, vb, k_cache, v_cache, pos, seq_lens, ab, B, Hq, Hkv, d, max_seq, theta);
+    else orc_attn_decode_multi(qb, kb, vb, k_cache, v_cache, pos, seq_lens, ab, n_seq, n_new, Hq, Hkv, d, max_seq, theta);
     orc_gemv(ab, w_o, proj, B, nq, D);
     for (size_t i = 0; i < (size_t)B * D; ++i)
         h[i] = orc_f64_to_bf16((double)orc_bf16_to_f32(x_in[i]) + proj[i]);
@@ -369,6 +434,32 @@ void orc_layer_decode(const uint16_t *g_attn, const uint16_t *w_qkv, const uint1
         x_out[i] = orc_f64_to_bf16((double)orc_bf16_to_f32(h[i]) + y[i]);
 
     free(n1); free(qkv); free(qb); free(kb); free(vb); free(ab); free(proj); free(h); free(n2); free(y);
+}
+
+void orc_layer_decode(const uint16_t *g_attn, const uint16_t *w_qkv, const uint16_t *w_o,
+                      const uint16_t *g_mlp, const uint16_t *w_gu, const uint16_t *w_down,
+                      const uint16_t *x_in, uint16_t *x_out,
+                      uint16_t *k_cache, uint16_t *v_cache,
+                      const int32_t *pos, const int32_t *seq_lens,
+                      int B, int D, int Hq, int Hkv, int d, int K, int max_seq,
+                      double eps, double theta)
+{
+    layer_decode_n(g_attn, w_qkv, w_o, g_mlp, w_gu, w_down, x_in, x_out, k_cache, v_cache, pos, seq_lens,
+                   B, 1, D, Hq, Hkv, d, K, max_seq, eps, theta);
+}
+
+/* The same layer for N new tokens per sequence: x_in, x_out [B*N, D] (token j of sequence b in row b*N + j);
+ * every block but the attention treats the rows alike (Algorithm 4 is written for h_t in R^{N x D}). */
+void orc_layer_decode_multi(const uint16_t *g_attn, const uint16_t *w_qkv, const uint16_t *w_o,
+                            const uint16_t *g_mlp, const uint16_t *w_gu, const uint16_t *w_down,
+                            const uint16_t *x_in, uint16_t *x_out,
+                            uint16_t *k_cache, uint16_t *v_cache,
+                            const int32_t *pos, const int32_t *seq_lens,
+                            int B, int N, int D, int Hq, int Hkv, int d, int K, int max_seq,
+                            double eps, double theta)
+{
+    layer_decode_n(g_attn, w_qkv, w_o, g_mlp, w_gu, w_down, x_in, x_out, k_cache, v_cache, pos, seq_lens,
+                   B, N, D, Hq, Hkv, d, K, max_seq, eps, theta);
 }
 
 /* ------------------------------------------------------------ model decode */

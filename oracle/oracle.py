@@ -151,6 +151,24 @@ def attn_decode(q, k_new, v_new, k_cache, v_cache, pos, seq_lens, theta=10000.0)
     return out
 
 
+def attn_decode_multi(q, k_new, v_new, k_cache, v_cache, pos, seq_lens, theta=10000.0):
+    """N new tokens per sequence: q [B,N,Hq,d], k_new / v_new [B,N,Hkv,d]; token j goes into row seq_lens[b] + j at
+    rotary position pos[b] + j and attends rows 0 .. seq_lens[b] + j.  Appends in place; returns out [B,N,Hq,d]."""
+    q, k_new, v_new = _u16(q), _u16(k_new), _u16(v_new)
+    assert k_cache.dtype == np.uint16 and k_cache.flags.c_contiguous and k_cache.flags.writeable
+    assert v_cache.dtype == np.uint16 and v_cache.flags.c_contiguous and v_cache.flags.writeable
+    B, N, Hq, d = q.shape
+    Hkv = k_new.shape[2]
+    max_seq = k_cache.shape[2]
+    assert k_new.shape == (B, N, Hkv, d) and k_cache.shape == (B, Hkv, max_seq, d) and v_cache.shape == k_cache.shape
+    pos, seq_lens = _i32(pos), _i32(seq_lens)
+    out = np.zeros((B, N, Hq, d), dtype=np.uint16)
+    lib().orc_attn_decode_multi(_p(q, _u16p), _p(k_new, _u16p), _p(v_new, _u16p), _p(k_cache, _u16p), _p(v_cache, _u16p),
+                                _p(pos, _i32p), _p(seq_lens, _i32p), _p(out, _u16p), C.c_int(B), C.c_int(N), C.c_int(Hq),
+                                C.c_int(Hkv), C.c_int(d), C.c_int(max_seq), C.c_double(theta))
+    return out
+
+
 def attn_probs(q, k_cache, pos, L, b, h, theta=10000.0):
     q = _u16(q)
     B, Hq, d = q.shape
@@ -201,6 +219,27 @@ def layer_decode(w: dict, x_in, k_cache, v_cache, pos, seq_lens, eps=1e-5, theta
                            _p(pos, _i32p), _p(seq_lens, _i32p),
                            C.c_int(B), C.c_int(D), C.c_int(Hq), C.c_int(Hkv), C.c_int(d), C.c_int(K),
                            C.c_int(max_seq), C.c_double(eps), C.c_double(theta))
+    return x_out
+
+
+def layer_decode_multi(w: dict, x_in, n_new, k_cache, v_cache, pos, seq_lens, eps=1e-5, theta=10000.0):
+    """layer_decode for n_new tokens per sequence: x_in [B*n_new, D] (token j of sequence b in row b*n_new + j),
+    pos / seq_lens [B].  Returns x_out [B*n_new, D]; caches appended in place (n_new rows per head and sequence)."""
+    x_in = _u16(x_in)
+    rows, D = x_in.shape
+    B = rows // n_new
+    assert B * n_new == rows
+    _, Hkv, max_seq, d = k_cache.shape
+    Hq = w["w_o"].shape[0] // d
+    K = w["w_down"].shape[0]
+    pos, seq_lens = _i32(pos), _i32(seq_lens)
+    assert pos.size == B and seq_lens.size == B
+    x_out = np.empty_like(x_in)
+    lib().orc_layer_decode_multi(_p(_u16(w["g_attn"]), _u16p), _p(_u16(w["w_qkv"]), _u16p), _p(_u16(w["w_o"]), _u16p),
+                                 _p(_u16(w["g_mlp"]), _u16p), _p(_u16(w["w_gu"]), _u16p), _p(_u16(w["w_down"]), _u16p),
+                                 _p(x_in, _u16p), _p(x_out, _u16p), _p(k_cache, _u16p), _p(v_cache, _u16p),
+                                 _p(pos, _i32p), _p(seq_lens, _i32p), C.c_int(B), C.c_int(n_new), C.c_int(D), C.c_int(Hq),
+                                 C.c_int(Hkv), C.c_int(d), C.c_int(K), C.c_int(max_seq), C.c_double(eps), C.c_double(theta))
     return x_out
 
 

@@ -546,3 +546,88 @@ def test_model_layer_loop_equals_the_chain_of_single_layers(n_layers):
             assert (mk[l][b, :, lens[b]] != caches[l][0][b, :, lens[b]]).any()
         if l:
             assert (mk[l][0, :, lens[0]] != mk[l - 1][0, :, lens[0]]).any()
+
+
+# ------------------------------------------------- several new tokens per step (Algorithm 3 for general N)
+
+def _multi_case(Bn=2, N=3, Hq=4, Hkv=2, d=8, max_seq=12):
+    q, kn, vn = rnd(Bn, N, Hq, d), rnd(Bn, N, Hkv, d), rnd(Bn, N, Hkv, d)
+    kc, vc = _caches(Bn, Hkv, max_seq, d)
+    lens, pos = np.array([4, 0][:Bn], np.int32), np.array([6, 0][:Bn], np.int32)
+    return q, kn, vn, kc, vc, pos, lens
+
+
+def test_multi_token_step_equals_single_token_steps_in_sequence():
+    # The chunk with its causal mask IS N decode steps taken one after the other: same rows written, same outputs,
+    # bit for bit (the masked form appends all rows first and masks; the sequential form never has the later rows).
+    q, kn, vn, kc, vc, pos, lens = _multi_case()
+    k1, v1 = kc.copy(), vc.copy()
+    want = np.zeros_like(q)
+    for j in range(q.shape[1]):
+        want[:, j] = orc.attn_decode(q[:, j].copy(), kn[:, j].copy(), vn[:, j].copy(), k1, v1, pos + j, lens + j)
+    k2, v2 = kc.copy(), vc.copy()
+    got = orc.attn_decode_multi(q, kn, vn, k2, v2, pos, lens)
+    assert (got == want).all()
+    assert (k2 == k1).all() and (v2 == v1).all()
+    # one new token per sequence is the decode step itself
+    g1 = orc.attn_decode_multi(q[:, :1].copy(), kn[:, :1].copy(), vn[:, :1].copy(), kc.copy(), vc.copy(), pos, lens)
+    assert (g1[:, 0] == orc.attn_decode(q[:, 0].copy(), kn[:, 0].copy(), vn[:, 0].copy(), kc.copy(), vc.copy(), pos, lens)).all()
+
+
+def test_multi_token_step_is_causal_inside_the_chunk_and_matches_the_masked_matrix_form():
+    q, kn, vn, kc, vc, pos, lens = _multi_case(Bn=1, N=4)
+    base = orc.attn_decode_multi(q, kn, vn, kc.copy(), vc.copy(), pos, lens)
+    # changing token 2 (its q, k and v) leaves tokens 0 and 1 untouched and changes tokens 2 and 3
+    q2, k2n, v2n = q.copy(), kn.copy(), vn.copy()
+    q2[:, 2], k2n[:, 2], v2n[:, 2] = rnd(1, 4, 8), rnd(1, 2, 8), rnd(1, 2, 8)
+    pert = orc.attn_decode_multi(q2, k2n, v2n, kc.copy(), vc.copy(), pos, lens)
+    assert (pert[:, :2] == base[:, :2]).all()
+    assert (pert[:, 2] != base[:, 2]).any() and (pert[:, 3] != base[:, 3]).any()
+    # numpy float64, written as ONE masked score matrix per head: rows = new tokens, columns = cache rows
+    Bn, N, Hq, d = q.shape
+    Hkv, L, p0, G = kn.shape[2], int(lens[0]), int(pos[0]), q.shape[2] // kn.shape[2]
+    K = F32(kc[0]).astype(np.float64)[:, :L + N].copy()
+    V = F32(vc[0]).astype(np.float64)[:, :L + N].copy()
+    for j in range(N):
+        for h in range(Hkv):
+            K[h, L + j] = F32(B16(orc.rope(F32(kn[0, j, h]), p0 + j)))
+            V[h, L + j] = F32(vn[0, j, h])
+    for h in range(Hq):
+        Q = np.stack([orc.rope(F32(q[0, j, h]), p0 + j) for j in range(N)]).astype(np.float64)
+        S = Q @ K[h // G].T / math.sqrt(d)
+        mask = np.arange(L + N)[None, :] > (L + np.arange(N))[:, None]
+        S[mask] = -np.inf
+        P = np.exp(S - S.max(axis=1, keepdims=True))
+        P /= P.sum(axis=1, keepdims=True)
+        assert ulp_distance(base[0, :, h], B16((P @ V[h // G]).astype(np.float32))).max() <= 1, h
+
+
+def test_multi_token_step_skips_a_sequence_whose_rows_do_not_all_fit():
+    q, kn, vn, kc, vc, pos, lens = _multi_case(Bn=2, N=3, max_seq=6)      # sequence 0: rows 4, 5, 6 -> row 6 does not exist
+    k2, v2 = kc.copy(), vc.copy()
+    out = orc.attn_decode_multi(q, kn, vn, k2, v2, pos, lens)
+    assert (k2[0] == kc[0]).all() and (v2[0] == vc[0]).all() and (out[0] == 0).all()
+    assert (k2[1, :, :3] != kc[1, :, :3]).any() and (out[1] != 0).any()
+
+
+def test_layer_with_several_new_tokens_equals_the_blocks_chained_by_hand():
+    # every block but the attention treats the B*N token rows alike: the multi-token layer must be
+    # norm -> QKV on all rows -> multi-token attention -> output projection + residual -> norm -> MLP + residual
+    D, H, d, K, N, Bn, max_seq = 8, 2, 4, 16, 3, 2, 10
+    w = _tiny_layer(D, H, d, K)
+    x = rnd(Bn * N, D)
+    kc, vc = _caches(Bn, H, max_seq, d)
+    lens, pos = np.array([3, 0], np.int32), np.array([3, 1], np.int32)
+    k1, v1 = kc.copy(), vc.copy()
+    got = orc.layer_decode_multi(w, x, N, k1, v1, pos, lens)
+    qkv = orc.f64_to_bf16(orc.gemv(orc.rmsnorm(x, w["g_attn"], 1e-5), w["w_qkv"]))
+    nq = H * d
+    sp = lambda t: t.reshape(Bn, N, H, d)
+    k2, v2 = kc.copy(), vc.copy()
+    a = orc.attn_decode_multi(sp(qkv[:, :nq]), sp(qkv[:, nq:2 * nq]), sp(qkv[:, 2 * nq:]), k2, v2, pos, lens)
+    h = orc.f64_to_bf16(F32(x).astype(np.float64) + orc.gemv(a.reshape(Bn * N, nq), w["w_o"]))
+    want = orc.f64_to_bf16(F32(h).astype(np.float64) + orc.mlp_f64(orc.rmsnorm(h, w["g_mlp"], 1e-5), w["w_gu"], w["w_down"]))
+    assert (got == want).all() and (k1 == k2).all() and (v1 == v2).all()
+    # and one new token per sequence is the decode layer itself
+    x1 = x[::N].copy()
+    assert (orc.layer_decode_multi(w, x1, 1, kc.copy(), vc.copy(), pos, lens) == orc.layer_decode(w, x1, kc.copy(), vc.copy(), pos, lens)).all()
