@@ -139,6 +139,18 @@ int fasttps_attn_decode(fasttps_ctx *ctx, const void *q, const void *k_new, cons
                         void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
                         void *out, int batch, void *stream);
 
+/* Algorithm 3 with N = n_new new tokens per sequence (the algorithm takes Q, K, V in R^{B x N x H x d}; speculative
+ * verification, chunked decode), 1 <= n_new <= 8, batch * n_new <= max_batch:
+ *   q [B,N,H_q,d], k_new, v_new [B,N,H_kv,d], out [B,N,H_q,d]; caches, pos, seq_lens [B] as above.
+ * Token j of sequence b is rotated at position pos[b] + j, goes into row seq_lens[b] + j of every head (B*N*H_kv
+ * runs of d elements are written, nothing else) and attends rows 0 .. seq_lens[b] + j: the cached rows and the new
+ * tokens up to and including itself (causal inside the chunk).  The cached rows are streamed once per new token
+ * and query head, in FP32 (the one-pass-per-query-head kernel); the new rows are scored from shared memory.  A
+ * sequence whose n_new rows do not all fit (seq_lens[b] + n_new > max_seq) is skipped and reported. */
+int fasttps_attn_decode_multi(fasttps_ctx *ctx, const void *q, const void *k_new, const void *v_new,
+                              void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
+                              void *out, int batch, int n_new, void *stream);
+
 /* Algorithm 4 steps 2-15 / Eq. 1: out = (silu(x W_gate) * (x W_up)) W_down.
  *   x [B,D]; w_gate_up, w_down packed; out [B,D].  The gate_up products, the
  *   SiLU*mul result and the down-projection partial sums stay on chip; partial
@@ -183,6 +195,14 @@ int fasttps_linear_decode(fasttps_ctx *ctx, int kind, const void *x, const void 
 int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const void *x_in, void *x_out,
                          void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
                          int batch, void *stream);
+
+/* The same layer for n_new tokens per sequence (Algorithm 3 and Algorithm 4 for general N): x_in, x_out
+ * [B * n_new, D], token j of sequence b in row b * n_new + j; pos, seq_lens [B]; 1 <= n_new <= 8 and
+ * batch * n_new <= max_batch.  The projections and the MLP treat the token rows alike; the attention is
+ * fasttps_attn_decode_multi.  Runs one kernel per product. */
+int fasttps_layer_decode_multi(fasttps_ctx *ctx, const fasttps_layer_weights *w, const void *x_in, void *x_out,
+                               void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
+                               int batch, int n_new, void *stream);
 
 /* Whole stack, one token per sequence: embedding gather -> n_layers layers ->
  * final RMSNorm -> logits -> greedy argmax (lowest index on ties).

@@ -67,6 +67,8 @@ def load_library() -> C.CDLL:
     lib.fasttps_pack_weight.argtypes = [vp, i, vp, vp, vp]
     lib.fasttps_unpack_weight.argtypes = [vp, i, vp, vp, vp]
     lib.fasttps_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, vp, i, vp]
+    lib.fasttps_attn_decode_multi.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, vp, i, i, vp]
+    lib.fasttps_layer_decode_multi.argtypes = [vp, C.POINTER(LayerWeights), vp, vp, vp, vp, ip, ip, i, i, vp]
     lib.fasttps_mlp_decode.argtypes = [vp, vp, vp, vp, vp, i, vp]
     lib.fasttps_mlp_decode_static.argtypes = [vp, vp, vp, vp, vp, i, vp]
     lib.fasttps_linear_decode.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, i, vp]
@@ -216,6 +218,21 @@ class Context:
                                             _ptr(v_cache), _ptr(pos), _ptr(seq_lens), _ptr(out), batch,
                                             _stream(stream)), "fasttps_attn_decode")
         return out
+
+    def attn_decode_multi(self, q, k_new, v_new, k_cache, v_cache, pos, seq_lens, out, stream=None):
+        """q [B,N,Hq,d]: N new tokens per sequence."""
+        batch, n_new = q.shape[0], q.shape[1]
+        _check(self.lib.fasttps_attn_decode_multi(self.handle, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache),
+                                                  _ptr(v_cache), _ptr(pos), _ptr(seq_lens), _ptr(out), batch, n_new,
+                                                  _stream(stream)), "fasttps_attn_decode_multi")
+        return out
+
+    def layer_decode_multi(self, lw: LayerWeights, x_in, x_out, n_new, k_cache, v_cache, pos, seq_lens, stream=None):
+        """x_in [B * n_new, D]: token j of sequence b in row b * n_new + j."""
+        _check(self.lib.fasttps_layer_decode_multi(self.handle, C.byref(lw), _ptr(x_in), _ptr(x_out), _ptr(k_cache),
+                                                   _ptr(v_cache), _ptr(pos), _ptr(seq_lens), x_in.shape[0] // n_new, n_new,
+                                                   _stream(stream)), "fasttps_layer_decode_multi")
+        return x_out
 
     def mlp_decode(self, x, w_gate_up, w_down, out, stream=None):
         _check(self.lib.fasttps_mlp_decode(self.handle, _ptr(x), _ptr(w_gate_up), _ptr(w_down), _ptr(out),

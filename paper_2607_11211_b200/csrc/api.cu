@@ -195,9 +195,10 @@ int fasttps_attn_splits(const fasttps_ctx *ctx, int batch)
     return attn_splits_for(reinterpret_cast<const Ctx *>(ctx), batch);
 }
 
+// batch: token rows (sequences x n_new); pos / seq_lens and the caches are per sequence
 static int attn_impl(Ctx *c, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                      int q_stride, int kv_stride, void *k_cache, void *v_cache, const int32_t *pos,
-                     const int32_t *seq_lens, __nv_bfloat16 *out, int out_stride, int batch, cudaStream_t st)
+                     const int32_t *seq_lens, __nv_bfloat16 *out, int out_stride, int batch, cudaStream_t st, int n_new = 1)
 {
     const fasttps_config &f = c->cfg;
     AttnArgs a;
@@ -210,7 +211,7 @@ static int attn_impl(Ctx *c, const __nv_bfloat16 *q, const __nv_bfloat16 *k, con
     a.batch = batch; a.n_q_heads = f.n_q_heads; a.n_kv_heads = f.n_kv_heads;
     a.head_dim = f.head_dim; a.max_seq = f.max_seq;
     a.n_splits = attn_splits_for(c, batch);
-    a.len_add = 0;
+    a.len_add = 0; a.n_new = n_new;
     a.cos_tab = c->cos_tab; a.sin_tab = c->sin_tab;
     a.part = c->attn_part; a.ticket = c->attn_ticket; a.status = c->status;
     return launch_attn(c, a, st);
@@ -278,6 +279,23 @@ static int wide_mlp_sums(Ctx *c, const __nv_bfloat16 *x, const __nv_bfloat16 *g,
 }
 
 static bool wide_batch(const Ctx *c, int batch) { return batch > kMaxNB && c->wide_n != nullptr; }
+
+int fasttps_attn_decode_multi(fasttps_ctx *ctx, const void *q, const void *k_new, const void *v_new,
+                              void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
+                              void *out, int batch, int n_new, void *stream)
+{
+    if (!ctx) return FASTTPS_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (batch < 1 || n_new < 1 || n_new > kMaxNB || (long long)batch * n_new > c->cfg.max_batch) return FASTTPS_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache) ||
+        !aligned16(out) || !pos || !seq_lens)
+        return FASTTPS_INVALID_ARG;
+    const fasttps_config &f = c->cfg;
+    return attn_impl(c, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_new),
+                     static_cast<const __nv_bfloat16 *>(v_new), f.n_q_heads * f.head_dim, f.n_kv_heads * f.head_dim,
+                     k_cache, v_cache, pos, seq_lens, static_cast<__nv_bfloat16 *>(out), f.n_q_heads * f.head_dim,
+                     batch * n_new, static_cast<cudaStream_t>(stream), n_new);
+}
 
 static int mlp_impl(Ctx *c, const __nv_bfloat16 *x, const __nv_bfloat16 *g, const void *w_gu, const void *w_down,
                     const __nv_bfloat16 *res, __nv_bfloat16 *out, int batch, cudaStream_t st)
@@ -380,9 +398,10 @@ int fasttps_linear_decode(fasttps_ctx *ctx, int kind, const void *x, const void 
                        static_cast<cudaStream_t>(stream));
 }
 
+// batch: token rows (sequences x n_new)
 static int layer_impl(Ctx *c, const fasttps_layer_weights &w, const __nv_bfloat16 *x_in, __nv_bfloat16 *x_out,
                       void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens, int batch,
-                      cudaStream_t st)
+                      cudaStream_t st, int n_new = 1)
 {
     const fasttps_config &f = c->cfg;
     const int D = f.hidden, nq = f.n_q_heads * f.head_dim, nkv = f.n_kv_heads * f.head_dim, nqkv = nq + 2 * nkv;
@@ -392,7 +411,7 @@ static int layer_impl(Ctx *c, const fasttps_layer_weights &w, const __nv_bfloat1
                      c->qkv, nullptr, nqkv, batch, nullptr, nullptr, nullptr, kProfQkv, st);
     if (rc) return rc;
     rc = attn_impl(c, c->qkv, c->qkv + nq, c->qkv + nq + nkv, nqkv, nqkv, k_cache, v_cache, pos, seq_lens,
-                   c->attn_out, nq, batch, st);
+                   c->attn_out, nq, batch, st, n_new);
     if (rc) return rc;
     // h = x + attn . W_o
     rc = linear_impl(c, nq, D, c->attn_out, nq, nullptr, w.w_o, x_in, D, c->h, nullptr, D, batch, nullptr, nullptr,
@@ -427,6 +446,22 @@ int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const
                                k_cache, v_cache, pos, seq_lens, batch, static_cast<cudaStream_t>(stream));
     return layer_impl(c, *w, static_cast<const __nv_bfloat16 *>(x_in), static_cast<__nv_bfloat16 *>(x_out), k_cache,
                       v_cache, pos, seq_lens, batch, static_cast<cudaStream_t>(stream));
+}
+
+int fasttps_layer_decode_multi(fasttps_ctx *ctx, const fasttps_layer_weights *w, const void *x_in, void *x_out,
+                               void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
+                               int batch, int n_new, void *stream)
+{
+    if (!ctx) return FASTTPS_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (batch < 1 || n_new < 1 || n_new > kMaxNB || (long long)batch * n_new > c->cfg.max_batch || !layer_ok(w))
+        return FASTTPS_INVALID_ARG;
+    if (!aligned16(x_in) || !aligned16(x_out) || !aligned16(k_cache) || !aligned16(v_cache) || !pos || !seq_lens)
+        return FASTTPS_INVALID_ARG;
+    if (n_new == 1) return fasttps_layer_decode(ctx, w, x_in, x_out, k_cache, v_cache, pos, seq_lens, batch, stream);
+    // the projections and the MLP see batch * n_new token rows; only the attention tells the tokens of a sequence apart
+    return layer_impl(c, *w, static_cast<const __nv_bfloat16 *>(x_in), static_cast<__nv_bfloat16 *>(x_out), k_cache,
+                      v_cache, pos, seq_lens, batch * n_new, static_cast<cudaStream_t>(stream), n_new);
 }
 
 static bool use_step_kernel(const Ctx *c, int batch)

@@ -30,6 +30,7 @@ struct AttnSmem {
     alignas(128) unsigned char slots[kSlots][AttnTile<DH>::kPieceBytes];
     alignas(16) uint64_t bars[2 * kSlots];
     AttnScratch<DH> scratch;
+    AttnMulti<DH> multi;             // rows of the new tokens of a chunk (several new tokens per sequence)
     int abort;
 };
 template <int DH>
@@ -43,9 +44,11 @@ struct AttnSmemShare {
     int abort;
 };
 
-template <int DH, bool SHARE>
+// SHARE: one pass per K/V head for its group of query heads (tensor cores).  MULTI: several new tokens per sequence.
+template <int DH, bool SHARE, bool MULTI = false>
 __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a)
 {
+    static_assert(!(SHARE && MULTI), "the multi-token path is the one-pass-per-query-head kernel");
     using Smem = typename std::conditional<SHARE, AttnSmemShare<DH>, AttnSmem<DH>>::type;
     extern __shared__ unsigned char smem_raw[];
     Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -67,15 +70,18 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a
     }
     if (blockIdx.x == 0 && t == 0) {
         // sequences that cannot be served are reported once and contribute no rows
-        for (int bb = 0; bb < a.batch; ++bb) {
+        for (int bb = 0; bb < a.batch / a.n_new; ++bb) {
             const int L = a.seq_lens[bb], p = a.pos[bb];
-            if (L < 0 || L >= a.max_seq) atomicOr(a.status, FASTTPS_DEV_CACHE_FULL);
-            else if (p < 0 || p >= a.max_seq) atomicOr(a.status, FASTTPS_DEV_BAD_POSITION);
+            if (L < 0 || L + a.n_new > a.max_seq) atomicOr(a.status, FASTTPS_DEV_CACHE_FULL);
+            else if (p < 0 || p + a.n_new > a.max_seq) atomicOr(a.status, FASTTPS_DEV_BAD_POSITION);
         }
     }
     bool done;
     if constexpr (SHARE)
         done = attn_consume_group<DH>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x, true), sm.scratch);
+    else if constexpr (MULTI)
+        done = attn_consume<DH, false, WalkSource, false, false, true>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x),
+                                                                       sm.scratch, kAttnWarps, nullptr, &sm.multi);
     else
         done = attn_consume<DH, false>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x), sm.scratch, kAttnWarps);
     if (!done && t == 0) atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT);
@@ -97,7 +103,9 @@ static int launch_attn_dh(Ctx *c, const AttnArgs &a, cudaStream_t st)
 {
     dim3 grid(a.n_splits);
     ProfScope prof(c, kProfAttn, st);
-    const int rc = (c->opt_gqa_share && attn_shares_groups(a.n_q_heads, a.n_kv_heads))
+    const int rc = a.n_new > 1
+                       ? launch_ex(attn_decode_kernel<DH, false, true>, grid, dim3(kAttnThreads), sizeof(AttnSmem<DH>) + 128, st, &a)
+                   : (c->opt_gqa_share && attn_shares_groups(a.n_q_heads, a.n_kv_heads))
                        ? launch_ex(attn_decode_kernel<DH, true>, grid, dim3(kAttnThreads), sizeof(AttnSmemShare<DH>) + 128, st, &a)
                        : launch_ex(attn_decode_kernel<DH, false>, grid, dim3(kAttnThreads), sizeof(AttnSmem<DH>) + 128, st, &a);
     c->launches++;
@@ -109,6 +117,7 @@ static int configure_attn_dh()
 {
     FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmem<DH>) + 128));
     FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmemShare<DH>) + 128));
+    FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmem<DH>) + 128));
     return FASTTPS_OK;
 }
 

@@ -42,15 +42,18 @@ struct Segment {
 struct ShareWalk {
     const int32_t *seq_lens, *pos;
     int B, H, max_seq, ncta, add;
+    int N = 1;                   // new tokens per sequence: row bb of the walk is token bb % N of sequence bb / N
     long long T, f, f_end;       // total rows, cursor, end of this CTA's share
     int b, h;
     long long head0;             // flattened index of row 0 of head (b, h)
     int rows_b;                  // rows per head of sequence b (L_b + 1, or 0 if the sequence is skipped)
 
+    // rows of one head of walk row bb: the cached rows plus ONE for the new rows (with N new tokens per sequence
+    // the last "row" of token j stands for the new rows 0 .. j, which never come from the cache)
     __host__ __device__ __forceinline__ int rows_of(int bb) const
     {
-        const int L = seq_lens[bb] + add, p = pos[bb] + add;
-        return (L < add || L >= max_seq || p < add || p >= max_seq) ? 0 : L + 1;
+        const int L = seq_lens[bb / N] + add, p = pos[bb / N] + add;
+        return (L < add || L + N > max_seq || p < add || p + N > max_seq) ? 0 : L + 1;
     }
     __host__ __device__ __forceinline__ long long share_begin(int c) const { return (T * c) / ncta; }
     // the CTA whose share holds flattened row x
@@ -119,7 +122,7 @@ struct ShareWalk {
             }
             const long long head1 = head0 + rows_b;
             const long long e = head1 < f_end ? head1 : f_end;
-            s.b = b; s.h = h; s.L = rows_b - 1; s.pos = pos[b] + add;
+            s.b = b; s.h = h; s.L = rows_b - 1; s.pos = pos[b / N] + add + b % N;
             s.r0 = (int)(f - head0); s.r1 = (int)(e - head0);
             s.first_cta = owner_of(head0);
             s.n_cta = owner_of(head1 - 1) - s.first_cta + 1;
@@ -150,6 +153,13 @@ struct AttnPre {
     alignas(16) __nv_bfloat16 vnew[kMaxNB][DH];
 };
 
+// MULTI (attn_consume): the rotated K rows and the V rows of the new tokens 0 .. j of the sequence a segment belongs to
+template <int DH>
+struct AttnMulti {
+    alignas(16) __nv_bfloat16 knew[kMaxNB][DH];
+    alignas(16) __nv_bfloat16 vnew[kMaxNB][DH];
+};
+
 template <int DH> struct AttnTile {
     static constexpr int kRowBytes = DH * 2;
     static constexpr int kPieceBytes = 2 * kAttnTileRows * kRowBytes;     // K tile then V tile
@@ -161,6 +171,7 @@ struct WalkSource {
     // share: the flattened row space runs over the K/V heads (segment.h is then a K/V head)
     __device__ __forceinline__ WalkSource(const AttnArgs &a, int cta, int ncta, bool share = false)
     {
+        walk.N = a.n_new;
         walk.init(a.seq_lens, a.pos, a.len_add, a.batch, share ? a.n_kv_heads : a.n_q_heads, a.max_seq, cta, ncta);
     }
     __device__ __forceinline__ bool next(Segment &s) { return walk.next(s); }
@@ -174,7 +185,7 @@ __device__ __forceinline__ bool attn_for_each_tile(const AttnArgs &a, Src src, F
     Segment sg;
     while (src.next(sg)) {
         const int c1 = sg.r1 < sg.L ? sg.r1 : sg.L;              // cached rows of the segment: [r0, c1)
-        const size_t slab = ((size_t)sg.b * a.n_kv_heads + sg.h / G) * (size_t)a.max_seq * DH;
+        const size_t slab = ((size_t)(sg.b / a.n_new) * a.n_kv_heads + sg.h / G) * (size_t)a.max_seq * DH;
         for (int r = sg.r0; r < c1; r += kAttnTileRows) {
             const int rows = (c1 - r) < kAttnTileRows ? (c1 - r) : kAttnTileRows;
             if (!f(a.k_cache + slab + (size_t)r * DH, a.v_cache + slab + (size_t)r * DH,
@@ -203,10 +214,14 @@ __device__ __forceinline__ bool attn_produce(const AttnArgs &a, WeightRing &ring
 // Returns false (in every consumer thread alike) if a bounded wait ran out.
 // DEFER: the partial of every segment is published (even when the CTA owns the whole head) and nobody
 // merges here; the caller merges the partials of a head itself (the persistent step kernel does, per group).
-template <int DH, bool DEFER, class Src, bool LATE_FENCE = false, bool PRE = false>
+// MULTI: several new tokens per sequence (a.n_new <= 8): the segment of token j scores the cached rows and then the
+// new rows 0 .. j of its sequence from shared memory (causal inside the chunk), and appends row j.
+template <int DH, bool DEFER, class Src, bool LATE_FENCE = false, bool PRE = false, bool MULTI = false>
 __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring, int &piece, int cta, Src src,
-                                             AttnScratch<DH> &sm, int nwc, AttnPre<DH> *pre = nullptr)
+                                             AttnScratch<DH> &sm, int nwc, AttnPre<DH> *pre = nullptr,
+                                             AttnMulti<DH> *mt = nullptr)
 {
+    static_assert(!(MULTI && PRE), "the multi-token path prepares its rows per segment");
     constexpr int EPL = DH / kLanesPerRow;      // elements per lane of a row
     constexpr int VPL = EPL / 8;                // 16-byte vectors per lane
     constexpr int HALF = DH / 2;
@@ -258,20 +273,47 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
         const int hq = sg.h, hk = hq / G, b = sg.b, L = sg.L;
         const bool has_new = sg.r1 > L;
         const int c1 = has_new ? L : sg.r1;
-        const size_t slab = ((size_t)b * a.n_kv_heads + hk) * (size_t)a.max_seq * DH;
+        const int tok = MULTI ? b % a.n_new : 0;                  // this token's index among its sequence's new tokens
+        const size_t slab = ((size_t)(MULTI ? b / a.n_new : b) * a.n_kv_heads + hk) * (size_t)a.max_seq * DH;
 
         // ---- joint RoPE of q and k_new with one set of cos/sin (Algorithm 3, steps 6-8) ----
         float *qv = PRE ? pre->q[segi] : sm.q;
         __nv_bfloat16 *knew = PRE ? pre->knew[segi] : sm.knew, *vnew = PRE ? pre->vnew[segi] : sm.vnew;
-        if (!PRE) {
+        if constexpr (MULTI) {
+            // q of this token at its own position; K / V rows of the new tokens 0 .. tok at theirs
+            const int n_rows = has_new ? tok + 1 : 0;
+            for (int idx = t; idx < (1 + n_rows) * HALF; idx += nct) {
+                const int which = idx / HALF, i = idx - which * HALF;
+                if (which == 0) {
+                    const float c = a.cos_tab[(size_t)sg.pos * HALF + i], sn = a.sin_tab[(size_t)sg.pos * HALF + i];
+                    const __nv_bfloat16 *qg = a.q + (size_t)b * a.q_stride + (size_t)hq * DH;
+                    const float x0 = __bfloat162float(ld_cg_bf16(qg + i)), x1 = __bfloat162float(ld_cg_bf16(qg + i + HALF));
+                    qv[i] = __fsub_rn(__fmul_rn(x0, c), __fmul_rn(x1, sn));
+                    qv[i + HALF] = __fadd_rn(__fmul_rn(x1, c), __fmul_rn(x0, sn));
+                } else {
+                    const int r = which - 1, row = b - tok + r, p = sg.pos - tok + r;     // token r of the same sequence
+                    const float c = a.cos_tab[(size_t)p * HALF + i], sn = a.sin_tab[(size_t)p * HALF + i];
+                    const __nv_bfloat16 *kg = a.k_new + (size_t)row * a.kv_stride + (size_t)hk * DH;
+                    const float k0 = __bfloat162float(ld_cg_bf16(kg + i)), k1 = __bfloat162float(ld_cg_bf16(kg + i + HALF));
+                    mt->knew[r][i] = __float2bfloat16_rn(__fsub_rn(__fmul_rn(k0, c), __fmul_rn(k1, sn)));
+                    mt->knew[r][i + HALF] = __float2bfloat16_rn(__fadd_rn(__fmul_rn(k1, c), __fmul_rn(k0, sn)));
+                    const __nv_bfloat16 *vg = a.v_new + (size_t)row * a.kv_stride + (size_t)hk * DH;
+                    mt->vnew[r][i] = ld_cg_bf16(vg + i);
+                    mt->vnew[r][i + HALF] = ld_cg_bf16(vg + i + HALF);
+                }
+            }
+            named_bar_sync(1, nct);
+            knew = mt->knew[tok]; vnew = mt->vnew[tok];          // the row this token appends
+        } else if (!PRE) {
             for (int i = t; i < HALF; i += nct) rope_one(sg, i, qv, knew, vnew);
             named_bar_sync(1, nct);
         }
         // ---- GKVC append (Eq. 2; Algorithm 3 steps 1 and 9): one write per row, no reload ----
         if (has_new && (hq % G) == 0) {
+            const size_t arow = (size_t)(L + tok) * DH;           // token j of the chunk goes into row L + j
             for (int i = t; i < DH / 8; i += nct) {
-                reinterpret_cast<uint4 *>(a.k_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(knew)[i];
-                reinterpret_cast<uint4 *>(a.v_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(vnew)[i];
+                reinterpret_cast<uint4 *>(a.k_cache + slab + arow)[i] = reinterpret_cast<const uint4 *>(knew)[i];
+                reinterpret_cast<uint4 *>(a.v_cache + slab + arow)[i] = reinterpret_cast<const uint4 *>(vnew)[i];
             }
             // bulk copies of a later step of the same launch must see these rows: the stores are ordered before the
             // asynchronous proxy, here or (LATE_FENCE) after the last segment
@@ -349,8 +391,15 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
 
         // ---- the new row, straight from shared memory (never re-read from the cache) ----
         if (has_new && warp == 0) {
-            const float sc = dot_row(reinterpret_cast<const unsigned char *>(knew));
-            update(sc, rgrp == 0, reinterpret_cast<const unsigned char *>(vnew));
+            if constexpr (MULTI) {
+                // one new row per lane group: rows 0 .. tok of the chunk are visible to this token, the later ones are not
+                const int r = rgrp <= tok ? rgrp : 0;
+                const float sc = dot_row(reinterpret_cast<const unsigned char *>(mt->knew[r]));
+                update(sc, rgrp <= tok, reinterpret_cast<const unsigned char *>(mt->vnew[r]));
+            } else {
+                const float sc = dot_row(reinterpret_cast<const unsigned char *>(knew));
+                update(sc, rgrp == 0, reinterpret_cast<const unsigned char *>(vnew));
+            }
         }
 
         // ---- combine the row groups of a warp, then the warps of the CTA ----

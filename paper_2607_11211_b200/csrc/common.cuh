@@ -277,6 +277,9 @@ struct AttnArgs {
     int out_stride;
     int batch, n_q_heads, n_kv_heads, head_dim, max_seq, n_splits;
     int len_add;                      // added to every seq_lens / pos entry (step index of a multi-step launch)
+    int n_new;                        // new tokens per sequence (1: the decode step).  With n_new > 1 `batch` counts token
+                                      // rows (sequence b, token j -> row b * n_new + j of q / k_new / v_new / out) while
+                                      // the caches, pos and seq_lens stay per sequence
     const float *cos_tab, *sin_tab;
     float *part;
     int *ticket;
