@@ -28,10 +28,11 @@ namespace fasttps {
 
 namespace {
 
-constexpr int kWideWarps = 8;                                   // consumer warps
+constexpr int kWideWarps = 16;                                  // consumer warps: two per k block of a piece, two tiles each
 constexpr int kWideThreads = (kWideWarps + 1) * 32;             // + the producer warp
 constexpr int kWideTiles = 4;                                   // 16-row weight tiles per pass
-constexpr int kWideChunk = 8;                                   // k blocks (32 k each) per ring piece: one per consumer warp
+constexpr int kWideTilesPerWarp = 2;
+constexpr int kWideChunk = 8;                                   // k blocks (32 k each) per ring piece
 constexpr int kWideXStride = kWideXRow * 2;                     // bytes between batch rows of an activation chunk: 512 + 64,
                                                                 // so that the 16-byte loads of two neighbouring rows
                                                                 // fall on different banks
@@ -122,15 +123,16 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
     pdl_launch_dependents();
     bool ok = true;
     int piece = 0;
-    // running argmax of the (at most two) batch rows this thread finishes in the epilogue
-    const int r = t & 15;
-    float bv[2] = {-INFINITY, -INFINITY};
-    int bi[2] = {0x7fffffff, 0x7fffffff};
+    // running argmax of the batch row this thread finishes in the epilogue
+    const int r = t & 15, eb = t >> 4;                       // epilogue: row r of a tile, batch row eb
+    const int kb = w & (kWideChunk - 1), th = w >> 3;        // main loop: k block kb of every piece, tiles 2 th and 2 th + 1
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
     for (int p0 = 0; p0 < ntile; p0 += kWideTiles) {
         const int nt = ntile - p0 < kWideTiles ? ntile - p0 : kWideTiles;
-        float acc[kWideTiles][4][4];
+        float acc[kWideTilesPerWarp][4][4];
 #pragma unroll
-        for (int i = 0; i < kWideTiles; ++i)
+        for (int i = 0; i < kWideTilesPerWarp; ++i)
 #pragma unroll
             for (int j = 0; j < 4; ++j)
 #pragma unroll
@@ -138,36 +140,38 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
         for (int c = 0; c < nchunk; ++c, ++piece) {
             const int kbs = nkb - c * kWideChunk < kWideChunk ? nkb - c * kWideChunk : kWideChunk;
             const unsigned char *slot = ring.wait(piece, ok);
-            if (ok && w < kbs) {
-                // B fragments of k block w for the four batch tiles: rows 8 j + g, 8 consecutive k from 8 t4
+            if (ok && kb < kbs && kWideTilesPerWarp * th < nt) {
+                // B fragments of k block kb for the four batch tiles: rows 8 j + g, 8 consecutive k from 8 t4
                 uint4 bq[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    bq[j] = *reinterpret_cast<const uint4 *>(slot + (8 * j + g) * kWideXStride + w * 64 + t4 * 16);
+                    bq[j] = *reinterpret_cast<const uint4 *>(slot + (8 * j + g) * kWideXStride + kb * 64 + t4 * 16);
 #pragma unroll
-                for (int i = 0; i < kWideTiles; ++i) {
-                    if (i < nt) {
-                        const unsigned char *blk = slot + kWideXBytes + (i * kWideChunk + w) * kTileBytes + lane * 16;
+                for (int i = 0; i < kWideTilesPerWarp; ++i) {
+                    const int tile = kWideTilesPerWarp * th + i;
+                    if (tile < nt) {
+                        const unsigned char *blk = slot + kWideXBytes + (tile * kWideChunk + kb) * kTileBytes + lane * 16;
                         const uint4 lo = *reinterpret_cast<const uint4 *>(blk);          // row g,     k 8 t4 ..
                         const uint4 hi = *reinterpret_cast<const uint4 *>(blk + 512);    // row g + 8, k 8 t4 ..
+                        // the two products into one accumulator are four instructions apart, not back to back
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            mma_bf16_k16(acc[i][j], lo.x, hi.x, lo.y, hi.y, bq[j].x, bq[j].y);
-                            mma_bf16_k16(acc[i][j], lo.z, hi.z, lo.w, hi.w, bq[j].z, bq[j].w);
-                        }
+                        for (int j = 0; j < 4; ++j) mma_bf16_k16(acc[i][j], lo.x, hi.x, lo.y, hi.y, bq[j].x, bq[j].y);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) mma_bf16_k16(acc[i][j], lo.z, hi.z, lo.w, hi.w, bq[j].z, bq[j].w);
                     }
                 }
             }
             ring.release(piece);
         }
-        // ---- the k blocks of the eight warps meet in shared memory ----
+        // ---- the k blocks of the warps meet in shared memory ----
 #pragma unroll
-        for (int i = 0; i < kWideTiles; ++i) {
-            if (i < nt) {
+        for (int i = 0; i < kWideTilesPerWarp; ++i) {
+            const int tile = kWideTilesPerWarp * th + i;
+            if (tile < nt) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     // fragment: rows g / g + 8 of the tile, batch rows 8 j + 2 t4 / + 1
-                    float *p = sm.sums + (size_t)(i * kWideMaxB + 8 * j + 2 * t4) * kWideAccStride + g;
+                    float *p = sm.sums + (size_t)(tile * kWideMaxB + 8 * j + 2 * t4) * kWideAccStride + g;
                     atomicAdd(p, acc[i][j][0]);
                     atomicAdd(p + kWideAccStride, acc[i][j][1]);
                     atomicAdd(p + 8, acc[i][j][2]);
@@ -179,10 +183,9 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
             if (t == 0) atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT);
             return;
         }
-        // ---- epilogue: thread (r = t % 16, b = t / 16 and b + 16) finishes row r of every tile of the pass ----
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int b = (t >> 4) + 16 * half;
+        // ---- epilogue: thread (r = t % 16, b = t / 16) finishes row r of every tile of the pass for batch row b ----
+        {
+            const int b = eb;
             for (int i = 0; i < nt; ++i) {
                 float *p = sm.sums + (size_t)(i * kWideMaxB + b) * kWideAccStride;
                 const int tile = tile0 + p0 + i;
@@ -207,7 +210,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
                         if (a.res) v += __bfloat162float(a.res[(size_t)b * a.res_stride + col]);
                         if (a.out_bf16) a.out_bf16[(size_t)b * a.out_stride + col] = __float2bfloat16_rn(v);
                         if (a.out_f32) a.out_f32[(size_t)b * a.out_stride + col] = v;
-                        if (v > bv[half] || (v == bv[half] && col < bi[half])) { bv[half] = v; bi[half] = col; }
+                        if (v > bv || (v == bv && col < bi)) { bv = v; bi = col; }
                     }
                 }
             }
@@ -218,18 +221,14 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
 
     // ---- greedy argmax: 16 threads per batch row -> CTA candidates -> the last CTA finishes (lowest index on ties) ----
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-#pragma unroll
-        for (int s = 8; s >= 1; s >>= 1) {
-            const float ov = __shfl_xor_sync(kFull, bv[half], s);
-            const int oi = __shfl_xor_sync(kFull, bi[half], s);
-            if (ov > bv[half] || (ov == bv[half] && oi < bi[half])) { bv[half] = ov; bi[half] = oi; }
-        }
-        const int b = (t >> 4) + 16 * half;
-        if (r == 0 && b < a.batch) {
-            a.amax_val[(size_t)b * gridDim.x + cta] = bv[half];
-            a.amax_idx[(size_t)b * gridDim.x + cta] = bi[half];
-        }
+    for (int s = 8; s >= 1; s >>= 1) {
+        const float ov = __shfl_xor_sync(kFull, bv, s);
+        const int oi = __shfl_xor_sync(kFull, bi, s);
+        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    if (r == 0 && eb < a.batch) {
+        a.amax_val[(size_t)eb * gridDim.x + cta] = bv;
+        a.amax_idx[(size_t)eb * gridDim.x + cta] = bi;
     }
     __threadfence();
     named_bar_sync(1, nct);
@@ -325,7 +324,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_down_kernel(WideDownArgs
 
     pdl_wait();
     pdl_launch_dependents();
-    const int nb = w & 3, par = w >> 2;                        // this warp: column block nb of the group, octets of parity par
+    const int nb = w & 3, par = w >> 2;                        // this warp: column block nb of the group, octets par, par + 4, ...
     float acc[2][4][4];
     auto clear = [&]() {
 #pragma unroll
@@ -355,7 +354,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_down_kernel(WideDownArgs
         if (cg != cur_cg) { if (ok) flush(cur_cg); clear(); cur_cg = cg; }
         const unsigned char *slot = ring.wait(i, ok);
         if (ok) {
-            for (int o = par; o < octs; o += 2) {
+            for (int o = par; o < octs; o += kWideWarps / 4) {
                 const uint4 av = *reinterpret_cast<const uint4 *>(slot + 2 * kDownXBytes + o * kDownRun + nb * 512 + lane * 16);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
