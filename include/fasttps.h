@@ -271,13 +271,6 @@ int fasttps_get_status(fasttps_ctx *ctx, uint32_t *host_status);
 #define FASTTPS_PROFILE_CLASSES 7
 int fasttps_profile(fasttps_ctx *ctx, int enable);
 int fasttps_profile_read(fasttps_ctx *ctx, double *ms_per_class, uint64_t *launches_per_class);
-/* Phase timeline of the last launch of the persistent step kernel, for profiling: the first and
- * the last CTA stamp the GPU global timer (ns) immediately before and after every grid-wide
- * barrier (order per step: embedding, then per layer QKV, attention + output projection, MLP,
- * then logits and argmax).  Synchronises, copies up to max_per_cta stamps of each of the two CTAs
- * into stamps[0 .. max_per_cta) and stamps[max_per_cta .. 2 max_per_cta), returns the number
- * of slots copied per CTA (slots past the launch's last stamp hold older or zero values). */
-int fasttps_trace_read(fasttps_ctx *ctx, uint64_t *stamps, int max_per_cta);
 /* Number of kernels this context has launched so far (host counter). */
 uint64_t fasttps_launch_count(const fasttps_ctx *ctx);
 /* Number of CTAs the attention kernel is launched with for this batch (how many of them take part is decided

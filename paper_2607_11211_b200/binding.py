@@ -310,16 +310,6 @@ class Context:
         self.lib.fasttps_set_option.argtypes = [C.c_void_p, C.c_char_p, C.c_int]
         _check(self.lib.fasttps_set_option(self.handle, name.encode(), int(value)), "fasttps_set_option")
 
-    def trace_read(self, n: int = 4096):
-        """(first_cta, last_cta) numpy uint64 arrays of global-timer stamps around the grid barriers."""
-        import numpy as np
-        buf = np.zeros(2 * n, dtype=np.uint64)
-        self.lib.fasttps_trace_read.argtypes = [C.c_void_p, C.c_void_p, C.c_int]
-        got = self.lib.fasttps_trace_read(self.handle, buf.ctypes.data, n)
-        if got < 0:
-            _check(got, "fasttps_trace_read")
-        return buf[:got], buf[n:n + got]
-
     def launch_count(self) -> int:
         return int(self.lib.fasttps_launch_count(self.handle))
 

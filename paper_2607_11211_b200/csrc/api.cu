@@ -57,7 +57,7 @@ static void free_all(Ctx *c)
     cudaFree(c->amax_ticket); cudaFree(c->status); cudaFree(c->qkv); cudaFree(c->attn_out);
     cudaFree(c->h); cudaFree(c->xa); cudaFree(c->xb); cudaFree(c->logits); cudaFree(c->tok); cudaFree(c->tok2);
     if (c->pinned_tok) cudaFreeHost(c->pinned_tok);
-    cudaFree(c->grid_bar); cudaFree(c->hacc); cudaFree(c->trace);
+    cudaFree(c->grid_bar); cudaFree(c->hacc);
     cudaFree(c->wide_n); cudaFree(c->wide_a_hi); cudaFree(c->wide_a_lo);
     if (c->prof_ev) {
         for (int i = 0; i < 2 * kProfMax; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
@@ -111,7 +111,6 @@ int fasttps_create(fasttps_ctx **out, const fasttps_config *cfg)
     A(dev_alloc(&c->mlp_acc, 2 * B * D, true));
     A(dev_alloc(&c->grid_bar, kGridBarWords, true));
     A(dev_alloc(&c->hacc, 2 * B * D, true));
-    A(dev_alloc(&c->trace, 2 * (size_t)kTraceLen, true));
     A(dev_alloc(&c->mlp_ticket, 1, true));
     A(dev_alloc(&c->amax_val, (size_t)kWideMaxB * 1024, true));
     A(dev_alloc(&c->amax_idx, (size_t)kWideMaxB * 1024, true));
@@ -505,7 +504,6 @@ static void step_args_common(Ctx *c, StepArgs &a, int batch)
     a.acc = c->mlp_acc; a.hacc = c->hacc; a.attn_part = c->attn_part; a.attn_ticket = c->attn_ticket;
     a.amax_val = c->amax_val; a.amax_idx = c->amax_idx; a.tok = c->tok2;
     a.bar = c->grid_bar; a.status = c->status;
-    a.trace = c->trace; a.trace_len = kTraceLen;
     a.x_out = nullptr;
 }
 
@@ -686,18 +684,6 @@ int fasttps_profile_read(fasttps_ctx *ctx, double *ms_per_class, uint64_t *launc
         launches_per_class[c->prof_cls[i]] += 1;
     }
     return FASTTPS_OK;
-}
-
-int fasttps_trace_read(fasttps_ctx *ctx, uint64_t *stamps, int max_per_cta)
-{
-    if (!ctx || !stamps || max_per_cta < 1) return FASTTPS_INVALID_ARG;
-    Ctx *c = reinterpret_cast<Ctx *>(ctx);
-    const int n = max_per_cta < kTraceLen ? max_per_cta : kTraceLen;
-    FT_CUDA(cudaDeviceSynchronize());
-    for (int k = 0; k < 2; ++k)
-        FT_CUDA(cudaMemcpy(stamps + (size_t)k * max_per_cta, c->trace + (size_t)k * kTraceLen, sizeof(uint64_t) * n,
-                           cudaMemcpyDeviceToHost));
-    return n;
 }
 
 uint64_t fasttps_launch_count(const fasttps_ctx *ctx)

@@ -19,10 +19,9 @@ constexpr unsigned kFull = 0xffffffffu;
 struct LayerPtrs;
 
 struct Ctx {
-    // persistent step kernel: grid barrier words, FP32 sums of the output projection, timeline
+    // persistent step kernel: grid barrier words, FP32 sums of the output projection
     unsigned *grid_bar;
     float *hacc;
-    unsigned long long *trace;       // [2][kTraceLen] phase timeline of the last step-kernel launch
     int opt_step_kernel;             // 1: model calls with batch <= 8 use the persistent step kernel
     int opt_gqa_share;               // 1: the attention kernel streams a K/V head once for its group of 2, 4 or 8 query heads
     fasttps_config cfg;
@@ -59,8 +58,8 @@ struct Ctx {
 };
 
 constexpr int kProfMax = 8192;
-constexpr int kTraceLen = 4096;             // global-timer stamps kept per traced CTA of the step kernel
-constexpr int kGridBarWords = 256;          // barrier counter + one group counter per query head (<= 128)
+constexpr int kGridBarWords = 256;          // barrier counter, sign-off counter, one group counter per query head (<= 128)
+constexpr int kGridBarDoneWord = 32;        // CTAs that have left the launch (on a cache line of its own)
 constexpr int kMaxStepLayers = 48;          // layers the persistent step kernel's layer table holds
 enum ProfClass { kProfQkv = 0, kProfAttn, kProfOproj, kProfMlp, kProfLmHead, kProfEmbed, kProfStep, kProfClasses };
 
@@ -327,10 +326,8 @@ struct StepArgs {
     float *amax_val;
     int *amax_idx;
     int32_t *tok;                    // [B] current tokens
-    unsigned *bar;                   // [kGridBarWords], zeroed by the host per launch: [0] grid barrier arrivals, [64 + h] group arrivals of head h
+    unsigned *bar;                   // [kGridBarWords], zeroed by the host per launch: [0] grid barrier arrivals, [32] CTAs signed off, [64 + h] group arrivals of head h; zero between launches
     uint32_t *status;
-    unsigned long long *trace;       // [2][trace_len] global-timer stamps of the first and last CTA, or null
-    int trace_len;
     __nv_bfloat16 *x_out;            // layer mode: [B][D] output of the layer (x0 is then its input; may be the same buffer)
     // the layer table travels with the launch (kernel parameter space): nothing to upload, nothing a later call
     // could overwrite while this launch is still queued

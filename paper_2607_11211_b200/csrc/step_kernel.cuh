@@ -291,19 +291,16 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(const _
     int piece = 0;
     bool ok = true;
 
-    // optional timeline for profiling: the first and the last CTA stamp the global timer before and
-    // after every grid barrier
-    int n_stamp = 0;
-    auto stamp = [&]() {
-        if (a.trace && t == 0 && (cta == 0 || cta == ncta - 1) && n_stamp < a.trace_len)
-            a.trace[(size_t)(cta ? 1 : 0) * a.trace_len + n_stamp] = global_ns();
-        ++n_stamp;
-    };
-    auto sync_phase = [&]() -> bool {
-        stamp();
-        const bool go = grid_sync(gb, nct, /*ok=*/ok);
-        stamp();
-        return go;
+    auto sync_phase = [&]() -> bool { return grid_sync(gb, nct, /*ok=*/ok); };
+    // On the way out of a launch that ran to its end every CTA signs off; the last one puts the barrier words back
+    // to zero (nobody polls them any more), so the next launch needs no clearing pass in front of it.  A launch that
+    // was abandoned leaves them as they are: fasttps_get_status clears them when it reports the timeout.
+    auto sign_off = [&]() {
+        if (t == 0 && atomicAdd(a.bar + kGridBarDoneWord, 1u) == (unsigned)ncta - 1u) {
+            a.bar[0] = 0u;
+            for (int hh = 0; hh < a.n_q_heads; ++hh) a.bar[64 + hh] = 0u;
+            a.bar[kGridBarDoneWord] = 0u;
+        }
     };
 
     if constexpr (!LAYER) {
@@ -539,6 +536,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(const _
                 *reinterpret_cast<float4 *>(hs + (size_t)idx * 8) = z;
                 *reinterpret_cast<float4 *>(hs + (size_t)idx * 8 + 4) = z;
             }
+            sign_off();
             return;
         }
 
@@ -586,6 +584,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(const _
         }
         if (step + 1 < a.n_steps && !sync_phase()) return;
     }
+    sign_off();
 }
 
 }  // namespace
@@ -607,8 +606,8 @@ static int launch_step_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
     }
     if ((unsigned long long)(3 * a.n_layers + 3) * (unsigned long long)a.n_steps * (unsigned long long)c->n_sm >= kBarAbort)
         return FASTTPS_INVALID_ARG;                      // the arrival counter must stay below the abort mark
-    // the barrier counter and the group counters start from zero every launch
-    FT_CUDA(cudaMemsetAsync(c->grid_bar, 0, kGridBarWords * sizeof(unsigned), st));
+    // the barrier counter and the group counters are zero here: the workspace starts out cleared, every launch that
+    // runs to its end clears them on its way out, and fasttps_get_status clears them after an abandoned one
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c->n_sm); cfg.blockDim = dim3((lay.nw + 1) * 32); cfg.dynamicSmemBytes = lay.total; cfg.stream = st;
     cudaLaunchAttribute attr[1];
