@@ -48,7 +48,10 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=128)
     ap.add_argument("--warmup", type=int, default=8)
-    ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg3",
+                    choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "llama3-8b", "chatglm3-6b", "llama2-7b", "llama3.2-1b"],
+                    help="cfg1..cfg5: the five Phi-3-mini workloads; a model name: that shape of the paper's Table 1 as a "
+                         "full stack at batch 8 with 4095 cached tokens per sequence")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--graph", type=int, default=1, help="replay the step as a CUDA graph (1) or launch eagerly (0)")
     ap.add_argument("--step-kernel", type=int, default=1,
@@ -450,9 +453,16 @@ def run_ours(args):
         dom_bytes = float(sum(W.algorithmic_bytes(s if advance else 0) for s in range(steps_per_launch)))
         dom_name = "decode_step_kernel"
         ncu_traffic = dom_bytes * NCU_STEP_TRAFFIC_RATIO if (dm is wl.PHI3_MINI and B == 1) else None
+    elif dom == "attn":                                       # one launch = the attention of one layer
+        kv = dm.kv_bytes_per_token_per_layer * float(sum(int(l) + 1 for l in lens0))
+        dom_bytes = kv + 2 * B * dm.n_q_heads * dm.head_dim * 2 + 2 * B * dm.n_kv_heads * dm.head_dim * 2
+        dom_name, ncu_traffic = "attn_decode_kernel", None
     else:
         dom, (dom_ms, dom_n) = "mlp", prof["mlp"]
-        dom_bytes, dom_name, ncu_traffic = float(mlp_bytes), "mlp_decode_kernel", NCU_MLP_TRAFFIC_BYTES
+        dom_bytes, dom_name = float(mlp_bytes), "mlp_decode_kernel"
+        ncu_traffic = NCU_MLP_TRAFFIC_BYTES if (dm is wl.PHI3_MINI and B == 1) else None
+        if B > 8:                                             # thin-GEMM path: prep, gate_up, down, prep per layer
+            dom_name, dom_n = "prep_rows + wide_linear (gate_up) + wide_down + prep_rows kernels, per layer", max(dom_n // 4, 1)
     peak, peak_kind = measured_peaks()
     achieved = dom_bytes / (dom_ms / dom_n * 1e-3) / 1e9 if dom_n else None
     roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak,

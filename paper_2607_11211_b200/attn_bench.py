@@ -1,6 +1,6 @@
 """Times ``fasttps_attn_decode`` alone on one of the attention shapes the paper evaluates (its Table 1).
 
-    python -m paper_2607_11211_b200.attn_bench --model llama3-8b --batch 8 --past 4095 [--gqa-share 0]
+    python -m paper_2607_11211_b200.attn_bench --model llama3-8b --batch 8 --past 4095 [--gqa-share 0|1|2]
 
 The call is enqueued ``--iters`` times on one stream between two CUDA events, rotating over enough cache sets
 that no K/V row is still in the L2 when it is read again.  Algorithmic bytes per call: every cached row of every

@@ -473,7 +473,7 @@ int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value)
     if (!ctx || !name) return FASTTPS_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);
     if (strcmp(name, "step_kernel") == 0) c->opt_step_kernel = value != 0;
-    else if (strcmp(name, "gqa_share") == 0) c->opt_gqa_share = value != 0;
+    else if (strcmp(name, "gqa_share") == 0) c->opt_gqa_share = value < 0 ? 0 : (value > 2 ? 2 : value);
     else return FASTTPS_INVALID_ARG;
     return FASTTPS_OK;
 }

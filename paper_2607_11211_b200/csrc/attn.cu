@@ -44,8 +44,9 @@ struct AttnSmemShare {
     int abort;
 };
 
-// SHARE: one pass per K/V head for its group of query heads (tensor cores).  MULTI: several new tokens per sequence.
-template <int DH, bool SHARE, bool MULTI = false>
+// SHARE: one pass per K/V head for its group of query heads (tensor cores; PRECISE: q and the softmax weights as bf16
+// hi + lo pairs).  MULTI: several new tokens per sequence.
+template <int DH, bool SHARE, bool MULTI = false, bool PRECISE = false>
 __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a)
 {
     static_assert(!(SHARE && MULTI), "the multi-token path is the one-pass-per-query-head kernel");
@@ -78,7 +79,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a
     }
     bool done;
     if constexpr (SHARE)
-        done = attn_consume_group<DH>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x, true), sm.scratch);
+        done = attn_consume_group<DH, PRECISE>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x, true), sm.scratch);
     else if constexpr (MULTI)
         done = attn_consume<DH, false, WalkSource, false, false, true>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x),
                                                                        sm.scratch, kAttnWarps, nullptr, &sm.multi);
@@ -105,6 +106,8 @@ static int launch_attn_dh(Ctx *c, const AttnArgs &a, cudaStream_t st)
     ProfScope prof(c, kProfAttn, st);
     const int rc = a.n_new > 1
                        ? launch_ex(attn_decode_kernel<DH, false, true>, grid, dim3(kAttnThreads), sizeof(AttnSmem<DH>) + 128, st, &a)
+                   : (c->opt_gqa_share == 1 && attn_shares_groups(a.n_q_heads, a.n_kv_heads))
+                       ? launch_ex(attn_decode_kernel<DH, true, false, true>, grid, dim3(kAttnThreads), sizeof(AttnSmemShare<DH>) + 128, st, &a)
                    : (c->opt_gqa_share && attn_shares_groups(a.n_q_heads, a.n_kv_heads))
                        ? launch_ex(attn_decode_kernel<DH, true>, grid, dim3(kAttnThreads), sizeof(AttnSmemShare<DH>) + 128, st, &a)
                        : launch_ex(attn_decode_kernel<DH, false>, grid, dim3(kAttnThreads), sizeof(AttnSmem<DH>) + 128, st, &a);
@@ -117,6 +120,7 @@ static int configure_attn_dh()
 {
     FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmem<DH>) + 128));
     FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmemShare<DH>) + 128));
+    FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmemShare<DH>) + 128));
     FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmem<DH>) + 128));
     return FASTTPS_OK;
 }

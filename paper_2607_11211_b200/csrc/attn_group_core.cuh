@@ -13,9 +13,11 @@
 // Operand order is free inside a dot product, so the head_dim index is permuted such that one 16-byte load of a
 // K row feeds two MMAs, and the output columns are permuted such that two V rows loaded as 32-bit words give
 // the B operands of two MMAs after a byte permute (no transposing load, no swizzled tile).
-// Precision: the rotated q enters the score product rounded to bf16 (the single-head path keeps it in FP32; a
-// bf16 hi + lo split was measured: it doubles the score MMAs and the registers it takes force spills), the
-// probabilities enter the second product rounded to bf16, and the row sum is taken over the rounded values.
+// Precision.  The tensor cores take bf16 operands; K and V ARE bf16, but the rotated q and the softmax weights are
+// FP32 values.  PRECISE (the default): both enter their product as a bf16 hi + lo pair (two MMAs each, about 16
+// mantissa bits), so the result matches the FP32 path of attn_core.cuh to rounding and a layer built on it meets the
+// same bars.  Without it (option "gqa_share" 2) they are rounded to bf16 once: faster, but the deviation of a layer
+// output from the oracle was measured 4.5 times larger (rms 0.015 against 0.0034 on a Llama3-8B-shaped layer).
 #pragma once
 #include "attn_core.cuh"
 #include "dot_core.cuh"
@@ -50,7 +52,7 @@ __device__ __forceinline__ void mma_top_k16(float (&c)[2], uint32_t a0, uint32_t
 
 // Consumer warps (kGroupWarps of them, threads 0 .. 255, synchronised by named barrier 1).  The segments of
 // `src` are K/V heads (WalkSource with share = true).  Returns false in every thread if a bounded wait ran out.
-template <int DH>
+template <int DH, bool PRECISE>
 __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing &ring, int &piece, int cta, WalkSource src,
                                                    GroupScratch<DH> &sm)
 {
@@ -105,7 +107,7 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
         }
 
         // ---- A fragments of the score product: this lane's head of the group, 8 consecutive elements per block ----
-        uint4 qhi[KB];
+        uint4 qhi[KB], qlo[PRECISE ? KB : 1];
 #pragma unroll
         for (int kb = 0; kb < KB; ++kb) {
             float f[8];
@@ -118,6 +120,11 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 for (int i = 0; i < 8; ++i) f[i] = 0.f;
             }
             qhi[kb] = make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+            if constexpr (PRECISE) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f[i] -= bf16_round(f[i]);          // what the rounding left out
+                qlo[kb] = make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+            }
         }
         float m_run = -INFINITY, l_run = 0.f;      // of head g; the sum holds this lane's keys only until the end
         float oa[JB][2], ob[JB][2];                // output fragments of head g: columns 16 jb + 4 t4 + {0, 2} (oa) / {1, 3} (ob)
@@ -145,6 +152,10 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                     const uint4 kv = *reinterpret_cast<const uint4 *>(kt + (size_t)(u ? kr1 : kr0) * kRowBytes + kb * 64 + t4 * 16);
                     mma_top_k16(sc[u][0], qhi[kb].x, qhi[kb].y, kv.x, kv.y);
                     mma_top_k16(sc[u][1], qhi[kb].z, qhi[kb].w, kv.z, kv.w);
+                    if constexpr (PRECISE) {
+                        mma_top_k16(sc[u][0], qlo[kb].x, qlo[kb].y, kv.x, kv.y);
+                        mma_top_k16(sc[u][1], qlo[kb].z, qlo[kb].w, kv.z, kv.w);
+                    }
                 }
             }
             // ---- online softmax (step 11) ----
@@ -167,7 +178,15 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
 #pragma unroll
             for (int e = 0; e < 4; ++e) pr[e] = ka[e] < rows ? fast_exp2(s[e] - m_new) : 0.f;
             const uint32_t pa0 = pack2(pr[0], pr[1]), pa1 = pack2(pr[2], pr[3]);
-            l_run = l_run * corr + ((bf16_round(pr[0]) + bf16_round(pr[1])) + (bf16_round(pr[2]) + bf16_round(pr[3])));
+            uint32_t pl0 = 0u, pl1 = 0u;
+            if constexpr (PRECISE) {
+                // the weights go in as hi + lo: the row sum is the sum of the weights themselves
+                l_run = l_run * corr + ((pr[0] + pr[1]) + (pr[2] + pr[3]));
+                pl0 = pack2(pr[0] - bf16_round(pr[0]), pr[1] - bf16_round(pr[1]));
+                pl1 = pack2(pr[2] - bf16_round(pr[2]), pr[3] - bf16_round(pr[3]));
+            } else {
+                l_run = l_run * corr + ((bf16_round(pr[0]) + bf16_round(pr[1])) + (bf16_round(pr[2]) + bf16_round(pr[3])));
+            }
             m_run = m_new;
             // ---- PV (step 12): B operands from four rows of V, two column sets per pair of 32-bit words ----
             const unsigned char *vp[4];
@@ -184,8 +203,14 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 const uint32_t w1 = *reinterpret_cast<const uint32_t *>(vp[1] + jb * 32);
                 const uint32_t w2 = *reinterpret_cast<const uint32_t *>(vp[2] + jb * 32);
                 const uint32_t w3 = *reinterpret_cast<const uint32_t *>(vp[3] + jb * 32);
-                mma_top_k16(oa[jb], pa0, pa1, __byte_perm(w0, w1, 0x5410), __byte_perm(w2, w3, 0x5410));    // columns 16 jb + 2 g
-                mma_top_k16(ob[jb], pa0, pa1, __byte_perm(w0, w1, 0x7632), __byte_perm(w2, w3, 0x7632));    // columns 16 jb + 2 g + 1
+                const uint32_t be0 = __byte_perm(w0, w1, 0x5410), be1 = __byte_perm(w2, w3, 0x5410);
+                const uint32_t bo0 = __byte_perm(w0, w1, 0x7632), bo1 = __byte_perm(w2, w3, 0x7632);
+                mma_top_k16(oa[jb], pa0, pa1, be0, be1);    // columns 16 jb + 2 g
+                mma_top_k16(ob[jb], pa0, pa1, bo0, bo1);    // columns 16 jb + 2 g + 1
+                if constexpr (PRECISE) {
+                    mma_top_k16(oa[jb], pl0, pl1, be0, be1);
+                    mma_top_k16(ob[jb], pl0, pl1, bo0, bo1);
+                }
             }
         };
 

@@ -125,6 +125,17 @@ TINY = Dims(hidden=128, n_q_heads=4, n_kv_heads=4, head_dim=32, inter=128, vocab
 SMALL = Dims(hidden=256, n_q_heads=4, n_kv_heads=4, head_dim=64, inter=640, vocab=1000, n_layers=3)
 SMALL_GQA = Dims(hidden=256, n_q_heads=8, n_kv_heads=2, head_dim=32, inter=384, vocab=520, n_layers=2)
 
+# The other model shapes of the paper's Table 1 (query heads, K/V heads, head_dim and MLP width as printed there;
+# hidden = query heads x head_dim; layer counts and vocabulary sizes of the public model cards, which only scale the
+# work).  Synthetic weights of these shapes stand in for the checkpoints.
+TABLE1 = {
+    "llama3-8b": Dims(hidden=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, inter=14336, vocab=128256, n_layers=32),
+    "chatglm3-6b": Dims(hidden=4096, n_q_heads=32, n_kv_heads=2, head_dim=128, inter=13696, vocab=65024, n_layers=28),
+    "llama2-7b": Dims(hidden=4096, n_q_heads=32, n_kv_heads=32, head_dim=128, inter=11008, vocab=32000, n_layers=32),
+    "phi3-mini": PHI3_MINI,
+    "llama3.2-1b": Dims(hidden=2048, n_q_heads=32, n_kv_heads=32, head_dim=64, inter=8192, vocab=128256, n_layers=16),
+}
+
 # tensor-id scheme: 1000*layer + kind; layer = 999 for model-level tensors
 _KIND = dict(g_attn=1, w_qkv=2, w_o=3, g_mlp=4, w_gu=5, w_down=6, k_cache=7, v_cache=8,
              embed=11, g_final=12, w_lm=13, x=21, q=22, k_new=23, v_new=24)
@@ -224,4 +235,7 @@ def workload(name: str) -> Workload:
         return Workload(name, P, 32, True, 8, tuple(int(v) for v in ragged_lengths(8, 512, 4096)), 4224, 1)
     if name == "cfg5":
         return Workload(name, P, 32, True, 32, (4095,) * 32, 4096, 1)
+    if name in TABLE1:          # a Table-1 shape as a full stack: batch 8, every sequence at 4095 cached tokens, one step
+        dm = TABLE1[name]
+        return Workload(name, dm, dm.n_layers, True, 8, (4095,) * 8, 4096, 1)
     raise KeyError(name)

@@ -56,9 +56,17 @@ def rotate_rows(bits, pos, theta):
     return orc.f32_to_bf16(out).reshape(bits.shape)
 
 
-@pytest.mark.parametrize("name,n_layers", [("cfg3", 32), ("cfg4", 32), ("cfg5", 32)])
+def table1_case(model):
+    """A Table-1 shape as a small stack: 2 layers, 3 sequences of unequal length, a 2048-entry vocabulary."""
+    import dataclasses
+    dm = dataclasses.replace(wl.TABLE1[model], vocab=2048, n_layers=2)
+    return wl.Workload(model, dm, 2, True, 3, (700, 64, 301), 1024, 1)
+
+
+@pytest.mark.parametrize("name,n_layers", [("cfg3", 32), ("cfg4", 32), ("cfg5", 32), ("llama3-8b", 2), ("chatglm3-6b", 2),
+                                           ("llama2-7b", 2), ("llama3.2-1b", 2)])
 def test_every_layer_on_the_oracles_input(fb, name, n_layers):
-    W = wl.workload(name)
+    W = table1_case(name) if name in wl.TABLE1 else wl.workload(name)
     dims, B, max_seq = W.dims, W.batch, W.max_seq
     D, d, Hq, Hkv = dims.hidden, dims.head_dim, dims.n_q_heads, dims.n_kv_heads
     nq, nkv = Hq * d, Hkv * d
