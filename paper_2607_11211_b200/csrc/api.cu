@@ -197,7 +197,8 @@ int fasttps_attn_splits(const fasttps_ctx *ctx, int batch)
 // batch: token rows (sequences x n_new); pos / seq_lens and the caches are per sequence
 static int attn_impl(Ctx *c, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                      int q_stride, int kv_stride, void *k_cache, void *v_cache, const int32_t *pos,
-                     const int32_t *seq_lens, __nv_bfloat16 *out, int out_stride, int batch, cudaStream_t st, int n_new = 1)
+                     const int32_t *seq_lens, __nv_bfloat16 *out, int out_stride, int batch, cudaStream_t st, int n_new = 1,
+                     int out_chunked = 0)
 {
     const fasttps_config &f = c->cfg;
     AttnArgs a;
@@ -206,7 +207,7 @@ static int attn_impl(Ctx *c, const __nv_bfloat16 *q, const __nv_bfloat16 *k, con
     a.k_cache = static_cast<__nv_bfloat16 *>(k_cache);
     a.v_cache = static_cast<__nv_bfloat16 *>(v_cache);
     a.pos = pos; a.seq_lens = seq_lens;
-    a.out = out; a.out_stride = out_stride;
+    a.out = out; a.out_stride = out_stride; a.out_chunked = out_chunked;
     a.batch = batch; a.n_q_heads = f.n_q_heads; a.n_kv_heads = f.n_kv_heads;
     a.head_dim = f.head_dim; a.max_seq = f.max_seq;
     a.n_splits = attn_splits_for(c, batch);
@@ -397,11 +398,46 @@ int fasttps_linear_decode(fasttps_ctx *ctx, int kind, const void *x, const void 
                        static_cast<cudaStream_t>(stream));
 }
 
+// One layer of the thin-GEMM chain for up to kWideMaxB token rows.  The layer input is x_res (+ the FP32 sums `pend`
+// still to be folded in, which are cleared); it is materialised in x_store when given (it is the residual of the
+// output projection: with pend it must be).  Leaves h in c->h and the MLP sums in c->mlp_acc: the caller's next
+// prep folds them in (the input of the next layer, or the layer output).
+static int layer_body_wide(Ctx *c, const fasttps_layer_weights &w, const __nv_bfloat16 *x_res, float *pend,
+                           __nv_bfloat16 *x_store, void *k_cache, void *v_cache, const int32_t *pos,
+                           const int32_t *seq_lens, int batch, int n_new, cudaStream_t st)
+{
+    const fasttps_config &f = c->cfg;
+    const int D = f.hidden, nq = f.n_q_heads * f.head_dim, nkv = f.n_kv_heads * f.head_dim, nqkv = nq + 2 * nkv;
+    const __nv_bfloat16 *resid = x_store ? x_store : x_res;
+    // x = x_res + pend (stored), n1 = rmsnorm(x) in chunked form
+    int rc = wide_prep(c, x_res, D, pend, static_cast<const __nv_bfloat16 *>(w.g_attn_norm), x_store, c->wide_n, D, batch, kProfQkv, st);
+    if (rc) return rc;
+    WideArgs a = wide_args(c, c->wide_n, w.w_qkv, D, nqkv, batch);
+    a.out_bf16 = c->qkv; a.out_stride = nqkv;
+    rc = launch_wide_linear(c, a, kProfQkv, st);
+    if (rc) return rc;
+    // the attention writes its output straight into the chunked activations of the output projection
+    rc = attn_impl(c, c->qkv, c->qkv + nq, c->qkv + nq + nkv, nqkv, nqkv, k_cache, v_cache, pos, seq_lens, c->wide_n, nq,
+                   batch, st, n_new, /*out_chunked=*/1);
+    if (rc) return rc;
+    a = wide_args(c, c->wide_n, w.w_o, nq, D, batch);            // h = x + attn . W_o
+    a.res = resid; a.res_stride = D; a.out_bf16 = c->h; a.out_stride = D; a.pair_rows = 1;
+    rc = launch_wide_linear(c, a, kProfOproj, st);
+    if (rc) return rc;
+    return wide_mlp_sums(c, c->h, static_cast<const __nv_bfloat16 *>(w.g_mlp_norm), w.w_gate_up, w.w_down, batch, st);
+}
+
 // batch: token rows (sequences x n_new)
 static int layer_impl(Ctx *c, const fasttps_layer_weights &w, const __nv_bfloat16 *x_in, __nv_bfloat16 *x_out,
                       void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens, int batch,
                       cudaStream_t st, int n_new = 1)
 {
+    if (wide_batch(c, batch) && batch <= kWideMaxB) {
+        int rc = layer_body_wide(c, w, x_in, nullptr, nullptr, k_cache, v_cache, pos, seq_lens, batch, n_new, st);
+        if (rc) return rc;
+        // x' = h + MLP sums
+        return wide_prep(c, c->h, c->cfg.hidden, c->mlp_acc, nullptr, x_out, nullptr, c->cfg.hidden, batch, kProfMlp, st);
+    }
     const fasttps_config &f = c->cfg;
     const int D = f.hidden, nq = f.n_q_heads * f.head_dim, nkv = f.n_kv_heads * f.head_dim, nqkv = nq + 2 * nkv;
     int rc;
@@ -576,6 +612,22 @@ int fasttps_model_decode(fasttps_ctx *ctx, const void *embed, const fasttps_laye
     // larger batches: one kernel per product, chained with programmatic dependent launch
     rc = launch_embed(c, static_cast<const __nv_bfloat16 *>(embed), token_ids, c->xa, batch, st);
     if (rc) return rc;
+    if (wide_batch(c, batch) && batch <= kWideMaxB) {
+        // thin-GEMM chain: the sums of a layer's MLP are folded into the next layer's input by its first kernel
+        for (int l = 0; l < f.n_layers; ++l) {
+            rc = layer_body_wide(c, layers[l], l == 0 ? c->xa : c->h, l == 0 ? nullptr : c->mlp_acc, l == 0 ? nullptr : c->xb,
+                                 k_caches[l], v_caches[l], pos, seq_lens, batch, 1, st);
+            if (rc) return rc;
+        }
+        // x_L = h + sums, final RMSNorm, logits from the chunked activations
+        rc = wide_prep(c, c->h, f.hidden, c->mlp_acc, static_cast<const __nv_bfloat16 *>(g_final), nullptr, c->wide_n, f.hidden,
+                       batch, kProfLmHead, st);
+        if (rc) return rc;
+        WideArgs a = wide_args(c, c->wide_n, w_lm_head, f.hidden, f.vocab, batch);
+        a.out_f32 = logits ? logits : c->logits; a.out_stride = f.vocab;
+        a.next_ids = next_ids; a.adv_pos = advance ? pos : nullptr; a.adv_len = advance ? seq_lens : nullptr;
+        return launch_wide_linear(c, a, kProfLmHead, st);
+    }
     __nv_bfloat16 *cur = c->xa, *nxt = c->xb;
     for (int l = 0; l < f.n_layers; ++l) {
         rc = layer_impl(c, layers[l], cur, nxt, k_caches[l], v_caches[l], pos, seq_lens, batch, st);

@@ -134,6 +134,12 @@ struct ShareWalk {
     }
 };
 
+// where element `col` of the attention output of sequence (token row) b goes
+__device__ __forceinline__ __nv_bfloat16 *attn_out_at(const AttnArgs &a, int b, int col)
+{
+    return a.out + (a.out_chunked ? wide_x_index(b, col) : (size_t)b * a.out_stride + col);
+}
+
 template <int DH>
 struct AttnScratch {
     alignas(16) float q[DH];                 // rope(q), FP32
@@ -432,7 +438,6 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
         if (!named_bar_and(1, nct, ok)) return false;
         float M = -INFINITY;
         for (int w = 0; w < nwork; ++w) M = fmaxf(M, sm.wm[w]);
-        __nv_bfloat16 *outp = a.out + (size_t)b * a.out_stride + (size_t)hq * DH;
         float *hp = a.part + ((size_t)b * a.n_q_heads + hq) * kMaxSplits * kPartStride;
         float *part = hp + (size_t)(cta - sg.first_cta) * kPartStride;
         const bool whole = !DEFER && sg.n_cta == 1;      // this CTA alone finishes the head right here
@@ -443,7 +448,7 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
                 o += f * sm.wo[w][i];
                 l += f * sm.wl[w];
             }
-            if (whole) outp[i] = __float2bfloat16_rn(o / l);
+            if (whole) *attn_out_at(a, b, hq * DH + i) = __float2bfloat16_rn(o / l);
             else {
                 part[i] = o;
                 if (i == 0) { part[DH] = M; part[DH + 1] = l; }
@@ -483,7 +488,7 @@ __device__ __forceinline__ bool attn_consume(const AttnArgs &a, WeightRing &ring
 #pragma unroll
                         for (int u = 0; u < 8; ++u) oo = fmaf(sm.mf[(s0 + u) & (kMaxSplits - 1)], v[u], oo);
                     }
-                    outp[i] = __float2bfloat16_rn(oo / sm.wl[0]);
+                    *attn_out_at(a, b, hq * DH + i) = __float2bfloat16_rn(oo / sm.wl[0]);
                 }
                 if (t == 0) *ticket = 0;
             }

@@ -250,7 +250,7 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 o += f * sm.wo[w][sl][i];
                 l += f * sm.wl[w][sl];
             }
-            if (whole) a.out[(size_t)b * a.out_stride + (size_t)hq * DH + i] = __float2bfloat16_rn(o / l);
+            if (whole) *attn_out_at(a, b, hq * DH + i) = __float2bfloat16_rn(o / l);
             else {
                 float *part = a.part + (((size_t)b * a.n_q_heads + hq) * kMaxSplits + (cta - sg.first_cta)) * kPartStride;
                 part[i] = o;
@@ -270,7 +270,6 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 // the merge factor that goes with it; every lane finishes DH / 32 columns
                 for (int hg = warp; hg < G; hg += kGroupWarps) {
                     const float *hp = a.part + ((size_t)b * a.n_q_heads + hk * G + hg) * kMaxSplits * kPartStride;
-                    __nv_bfloat16 *outp = a.out + (size_t)b * a.out_stride + (size_t)(hk * G + hg) * DH;
                     const bool have = lane < sg.n_cta;
                     const float ms = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH) : -INFINITY;
                     const float ls = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH + 1) : 0.f;
@@ -297,7 +296,7 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                         }
                     }
 #pragma unroll
-                    for (int c = 0; c < DH / 32; ++c) outp[lane + 32 * c] = __float2bfloat16_rn(oo[c] / ll);
+                    for (int c = 0; c < DH / 32; ++c) *attn_out_at(a, b, (hk * G + hg) * DH + lane + 32 * c) = __float2bfloat16_rn(oo[c] / ll);
                 }
                 if (t == 0) *ticket = 0;
             }

@@ -274,6 +274,7 @@ struct AttnArgs {
     const int32_t *pos, *seq_lens;
     __nv_bfloat16 *out;
     int out_stride;
+    int out_chunked;                  // 1: `out` is the chunked [32][H_q d] layout of the thin-GEMM path (wide_x_index)
     int batch, n_q_heads, n_kv_heads, head_dim, max_seq, n_splits;
     int len_add;                      // added to every seq_lens / pos entry (step index of a multi-step launch)
     int n_new;                        // new tokens per sequence (1: the decode step).  With n_new > 1 `batch` counts token

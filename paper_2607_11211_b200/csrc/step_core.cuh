@@ -102,7 +102,7 @@ static __device__ __forceinline__ AttnArgs attn_args_of(const StepArgs &a, const
     aa.q_stride = nq + 2 * nkv; aa.kv_stride = nq + 2 * nkv;
     aa.k_cache = lp.k_cache; aa.v_cache = lp.v_cache;
     aa.pos = a.pos; aa.seq_lens = a.seq_lens;
-    aa.out = a.attn_out; aa.out_stride = nq;
+    aa.out = a.attn_out; aa.out_stride = nq; aa.out_chunked = 0;
     aa.batch = a.batch; aa.n_q_heads = a.n_q_heads; aa.n_kv_heads = a.n_kv_heads;
     aa.head_dim = a.head_dim; aa.max_seq = a.max_seq; aa.n_splits = ncta_attn; aa.len_add = step; aa.n_new = 1;
     aa.cos_tab = a.cos_tab; aa.sin_tab = a.sin_tab;
