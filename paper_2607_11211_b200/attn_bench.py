@@ -28,28 +28,36 @@ def main():
     ap.add_argument("--past", type=int, default=4095, help="cached rows per sequence before the step")
     ap.add_argument("--iters", type=int, default=200)
     ap.add_argument("--gqa-share", type=int, default=1)
+    ap.add_argument("--n-new", type=int, default=1,
+                    help="new tokens per sequence and step (> 1: fasttps_attn_decode_multi, causal inside the chunk)")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device: there is no CPU path")
     build.build()
     hq, hkv, d = SHAPES[args.model]
     dims = wl.Dims(hidden=hq * d, n_q_heads=hq, n_kv_heads=hkv, head_dim=d, inter=1024, vocab=1024, n_layers=1)
-    B, L = args.batch, args.past
-    max_seq = L + 1
-    ctx = fb.Context.from_dims(dims, B, max_seq)
+    B, L, N = args.batch, args.past, args.n_new
+    max_seq = L + N
+    ctx = fb.Context.from_dims(dims, B * N, max_seq)
     ctx.set_option("gqa_share", args.gqa_share)
     cache_bytes = 2 * B * hkv * max_seq * d * 2
     n_sets = max(2, -(-(400 << 20) // cache_bytes))                  # > 3 x the 126 MB L2 between two visits
     sets = [wl.kv_cache(dims, i, B, max_seq, wl.MASTER_SEED, device="cuda") for i in range(n_sets)]
-    act = wl.activations(dims, B, wl.MASTER_SEED, device="cuda")
+    act = wl.activations(dims, B * N, wl.MASTER_SEED, device="cuda")
+    if N > 1:
+        act = {k: v.view(B, N, *v.shape[1:]) for k, v in act.items()}
     lens = torch.full((B,), L, dtype=torch.int32, device="cuda")
-    out = torch.zeros(B, hq, d, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(B * N, hq, d, dtype=torch.bfloat16, device="cuda").view(*act["q"].shape)
+    torch.cuda.synchronize()
     st = torch.cuda.Stream()
 
     def run(n):
         for i in range(n):
             kc, vc = sets[i % n_sets]
-            ctx.attn_decode(act["q"], act["k_new"], act["v_new"], kc, vc, lens, lens, out, stream=st)
+            if N > 1:
+                ctx.attn_decode_multi(act["q"], act["k_new"], act["v_new"], kc, vc, lens, lens, out, stream=st)
+            else:
+                ctx.attn_decode(act["q"], act["k_new"], act["v_new"], kc, vc, lens, lens, out, stream=st)
 
     with torch.cuda.stream(st):
         run(2 * n_sets)
@@ -61,12 +69,13 @@ def main():
         st.synchronize()
     us = e0.elapsed_time(e1) / args.iters * 1e3
     status = ctx.get_status()
-    alg = 2 * B * hkv * (L + 1) * d * 2 + 2 * B * hq * d * 2
+    # every cached row once (whatever the number of new tokens), the new rows written, q in, the output out
+    alg = 2 * B * hkv * (L + N) * d * 2 + 2 * B * N * hq * d * 2
     peaks = Path(__file__).resolve().parent.parent / "MEASURED_PEAKS.json"
     peak = float(json.loads(peaks.read_text())["hbm_gbs"]) if peaks.exists() else 6650.0
     gbs = alg / (us * 1e-6) / 1e9
     print(json.dumps({"kernel": "attn_decode_kernel", "model": args.model, "q_heads": hq, "kv_heads": hkv, "head_dim": d,
-                      "batch": B, "past": L, "gqa_share": args.gqa_share, "cache_sets": n_sets, "iters": args.iters,
+                      "batch": B, "past": L, "n_new": N, "gqa_share": args.gqa_share, "cache_sets": n_sets, "iters": args.iters,
                       "us_per_call": us, "algorithmic_bytes": alg, "achieved_gbs": gbs, "peak_gbs": peak,
                       "frac": gbs / peak, "peak_source": "of measured" if peaks.exists() else "of fallback",
                       "device_status": status}))

@@ -14,9 +14,10 @@ static_assert(kAttnWarps == kGroupWarps, "the grouped-query path divides the til
 
 // Grouped-query attention with 2 to 16 query heads per K/V head streams every cached row once for the whole
 // group, with the two products on the tensor cores; other ratios stream it once per query head.
-inline bool attn_shares_groups(int n_q_heads, int n_kv_heads)
+// The members of a group are its query heads times the new tokens of the sequence (n_new > 1: a chunk).
+inline bool attn_shares_groups(int n_q_heads, int n_kv_heads, int n_new = 1)
 {
-    const int G = n_kv_heads > 0 ? n_q_heads / n_kv_heads : 1;
+    const int G = (n_kv_heads > 0 ? n_q_heads / n_kv_heads : 1) * n_new;
     return G > 1 && G <= kMaxShareGroup;
 }
 
@@ -104,12 +105,13 @@ static int launch_attn_dh(Ctx *c, const AttnArgs &a, cudaStream_t st)
 {
     dim3 grid(a.n_splits);
     ProfScope prof(c, kProfAttn, st);
-    const int rc = a.n_new > 1
-                       ? launch_ex(attn_decode_kernel<DH, false, true>, grid, dim3(kAttnThreads), sizeof(AttnSmem<DH>) + 128, st, &a)
-                   : (c->opt_gqa_share == 1 && attn_shares_groups(a.n_q_heads, a.n_kv_heads))
+    const bool share = attn_shares_groups(a.n_q_heads, a.n_kv_heads, a.n_new);
+    const int rc = (c->opt_gqa_share == 1 && share)
                        ? launch_ex(attn_decode_kernel<DH, true, false, true>, grid, dim3(kAttnThreads), sizeof(AttnSmemShare<DH>) + 128, st, &a)
-                   : (c->opt_gqa_share && attn_shares_groups(a.n_q_heads, a.n_kv_heads))
+                   : (c->opt_gqa_share && share)
                        ? launch_ex(attn_decode_kernel<DH, true>, grid, dim3(kAttnThreads), sizeof(AttnSmemShare<DH>) + 128, st, &a)
+                   : a.n_new > 1
+                       ? launch_ex(attn_decode_kernel<DH, false, true>, grid, dim3(kAttnThreads), sizeof(AttnSmem<DH>) + 128, st, &a)
                        : launch_ex(attn_decode_kernel<DH, false>, grid, dim3(kAttnThreads), sizeof(AttnSmem<DH>) + 128, st, &a);
     c->launches++;
     return rc;

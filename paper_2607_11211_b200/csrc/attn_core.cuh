@@ -43,6 +43,8 @@ struct ShareWalk {
     const int32_t *seq_lens, *pos;
     int B, H, max_seq, ncta, add;
     int N = 1;                   // new tokens per sequence: row bb of the walk is token bb % N of sequence bb / N
+    int need = 1;                // new rows per sequence that must fit into its cache (N, or the chunk length when the
+                                 // walk runs over sequences and the chunk's tokens share the pass)
     long long T, f, f_end;       // total rows, cursor, end of this CTA's share
     int b, h;
     long long head0;             // flattened index of row 0 of head (b, h)
@@ -53,7 +55,7 @@ struct ShareWalk {
     __host__ __device__ __forceinline__ int rows_of(int bb) const
     {
         const int L = seq_lens[bb / N] + add, p = pos[bb / N] + add;
-        return (L < add || L + N > max_seq || p < add || p + N > max_seq) ? 0 : L + 1;
+        return (L < add || L + need > max_seq || p < add || p + need > max_seq) ? 0 : L + 1;
     }
     __host__ __device__ __forceinline__ long long share_begin(int c) const { return (T * c) / ncta; }
     // the CTA whose share holds flattened row x
@@ -174,11 +176,14 @@ template <int DH> struct AttnTile {
 // Segment sources: `bool next(Segment &)`.
 struct WalkSource {
     ShareWalk walk;
-    // share: the flattened row space runs over the K/V heads (segment.h is then a K/V head)
+    // share: the flattened row space runs over the K/V heads (segment.h is then a K/V head) of the SEQUENCES: the new
+    // tokens of a sequence and the query heads of a K/V head all share one pass
     __device__ __forceinline__ WalkSource(const AttnArgs &a, int cta, int ncta, bool share = false)
     {
-        walk.N = a.n_new;
-        walk.init(a.seq_lens, a.pos, a.len_add, a.batch, share ? a.n_kv_heads : a.n_q_heads, a.max_seq, cta, ncta);
+        walk.N = share ? 1 : a.n_new;
+        walk.need = a.n_new;
+        walk.init(a.seq_lens, a.pos, a.len_add, share ? a.batch / a.n_new : a.batch, share ? a.n_kv_heads : a.n_q_heads,
+                  a.max_seq, cta, ncta);
     }
     __device__ __forceinline__ bool next(Segment &s) { return walk.next(s); }
 };
@@ -191,7 +196,7 @@ __device__ __forceinline__ bool attn_for_each_tile(const AttnArgs &a, Src src, F
     Segment sg;
     while (src.next(sg)) {
         const int c1 = sg.r1 < sg.L ? sg.r1 : sg.L;              // cached rows of the segment: [r0, c1)
-        const size_t slab = ((size_t)(sg.b / a.n_new) * a.n_kv_heads + sg.h / G) * (size_t)a.max_seq * DH;
+        const size_t slab = ((size_t)(SHARE ? sg.b : sg.b / a.n_new) * a.n_kv_heads + sg.h / G) * (size_t)a.max_seq * DH;
         for (int r = sg.r0; r < c1; r += kAttnTileRows) {
             const int rows = (c1 - r) < kAttnTileRows ? (c1 - r) : kAttnTileRows;
             if (!f(a.k_cache + slab + (size_t)r * DH, a.v_cache + slab + (size_t)r * DH,

@@ -31,8 +31,8 @@ constexpr int kGroupWarps = 8;           // consumer warps: two sets of four, 16
 template <int DH>
 struct GroupScratch {
     alignas(16) float q[kMaxShareGroup][DH];            // rope(q) of the group, FP32
-    alignas(16) __nv_bfloat16 knew[DH];                 // bf16(rope(k_new)): the row that goes into the cache
-    alignas(16) __nv_bfloat16 vnew[DH];
+    alignas(16) __nv_bfloat16 knew[kMaxNB][DH];         // bf16(rope(k_new)): the rows that go into the cache (one per new token)
+    alignas(16) __nv_bfloat16 vnew[kMaxNB][DH];
     float wm[kGroupWarps][kHeadsPerWarp], wl[kGroupWarps][kHeadsPerWarp];     // per warp and head slot: max (log2 domain), sum
     alignas(16) float wo[kGroupWarps][kHeadsPerWarp][DH];
     int last;
@@ -63,11 +63,15 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
     constexpr int kPartStride = DH + 4;
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5, g = lane >> 2, t4 = lane & 3;
     const int nct = kGroupWarps * 32;
-    const int G = a.n_q_heads / a.n_kv_heads;
-    // groups of up to 8: warps 0-3 take the even pieces, warps 4-7 the odd ones, all heads each.  Larger groups
-    // (up to 16): warps 0-3 take heads 0-7 and warps 4-7 heads 8-15, of every piece.
+    const int Gh = a.n_q_heads / a.n_kv_heads, N = a.n_new;
+    // The members of a group are the query heads of the K/V head, for every new token of the sequence: member
+    // m = j * Gh + g2 is head g2 of the group for token j (N = 1: the decode step, members = query heads).
+    const int G = Gh * N;
+    // groups of up to 8: warps 0-3 take the even pieces, warps 4-7 the odd ones, all members each.  Larger groups
+    // (up to 16): warps 0-3 take members 0-7 and warps 4-7 members 8-15, of every piece.
     const bool wide = G > kHeadsPerWarp;
-    const int gh = g + (wide ? kHeadsPerWarp * (warp >> 2) : 0);      // the query head of the group in this lane's MMA row
+    const int gh = g + (wide ? kHeadsPerWarp * (warp >> 2) : 0);      // the member of the group in this lane's MMA row
+    const int my_tok = gh / Gh;                                       // its token: it sees the new rows 0 .. my_tok
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
     bool ok = true;
 
@@ -80,28 +84,30 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
 
         // ---- joint RoPE of the G queries and k_new with one set of cos/sin (Algorithm 3, steps 6-8) ----
         for (int idx = t; idx < G * HALF; idx += nct) {
-            const int g2 = idx / HALF, i = idx - g2 * HALF;
-            const float c = a.cos_tab[(size_t)sg.pos * HALF + i], sn = a.sin_tab[(size_t)sg.pos * HALF + i];
-            const __nv_bfloat16 *qg = a.q + (size_t)b * a.q_stride + (size_t)(hk * G + g2) * DH;
+            const int m = idx / HALF, i = idx - m * HALF, j = m / Gh, g2 = m - j * Gh;
+            const size_t row = (size_t)b * N + j;                          // token j of sequence b
+            const float c = a.cos_tab[(size_t)(sg.pos + j) * HALF + i], sn = a.sin_tab[(size_t)(sg.pos + j) * HALF + i];
+            const __nv_bfloat16 *qg = a.q + row * a.q_stride + (size_t)(hk * Gh + g2) * DH;
             const float x0 = __bfloat162float(ld_cg_bf16(qg + i)), x1 = __bfloat162float(ld_cg_bf16(qg + i + HALF));
-            sm.q[g2][i] = __fsub_rn(__fmul_rn(x0, c), __fmul_rn(x1, sn));
-            sm.q[g2][i + HALF] = __fadd_rn(__fmul_rn(x1, c), __fmul_rn(x0, sn));
+            sm.q[m][i] = __fsub_rn(__fmul_rn(x0, c), __fmul_rn(x1, sn));
+            sm.q[m][i + HALF] = __fadd_rn(__fmul_rn(x1, c), __fmul_rn(x0, sn));
             if (g2 == 0 && has_new) {
-                const __nv_bfloat16 *kg = a.k_new + (size_t)b * a.kv_stride + (size_t)hk * DH;
+                const __nv_bfloat16 *kg = a.k_new + row * a.kv_stride + (size_t)hk * DH;
                 const float k0 = __bfloat162float(ld_cg_bf16(kg + i)), k1 = __bfloat162float(ld_cg_bf16(kg + i + HALF));
-                sm.knew[i] = __float2bfloat16_rn(__fsub_rn(__fmul_rn(k0, c), __fmul_rn(k1, sn)));
-                sm.knew[i + HALF] = __float2bfloat16_rn(__fadd_rn(__fmul_rn(k1, c), __fmul_rn(k0, sn)));
-                const __nv_bfloat16 *vg = a.v_new + (size_t)b * a.kv_stride + (size_t)hk * DH;
-                sm.vnew[i] = ld_cg_bf16(vg + i);
-                sm.vnew[i + HALF] = ld_cg_bf16(vg + i + HALF);
+                sm.knew[j][i] = __float2bfloat16_rn(__fsub_rn(__fmul_rn(k0, c), __fmul_rn(k1, sn)));
+                sm.knew[j][i + HALF] = __float2bfloat16_rn(__fadd_rn(__fmul_rn(k1, c), __fmul_rn(k0, sn)));
+                const __nv_bfloat16 *vg = a.v_new + row * a.kv_stride + (size_t)hk * DH;
+                sm.vnew[j][i] = ld_cg_bf16(vg + i);
+                sm.vnew[j][i + HALF] = ld_cg_bf16(vg + i + HALF);
             }
         }
         named_bar_sync(1, nct);
         // ---- GKVC append (Eq. 2; Algorithm 3 steps 1 and 9): one write per row, no reload ----
         if (has_new) {
-            for (int i = t; i < DH / 8; i += nct) {
-                reinterpret_cast<uint4 *>(a.k_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(sm.knew)[i];
-                reinterpret_cast<uint4 *>(a.v_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(sm.vnew)[i];
+            // the N new rows are consecutive in the cache (rows L .. L + N - 1) and in shared memory
+            for (int i = t; i < N * (DH / 8); i += nct) {
+                reinterpret_cast<uint4 *>(a.k_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(&sm.knew[0][0])[i];
+                reinterpret_cast<uint4 *>(a.v_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(&sm.vnew[0][0])[i];
             }
             asm volatile("fence.proxy.async;" ::: "memory");
         }
@@ -135,7 +141,8 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
 
         // One block of up to 16 keys: rows key0 .. key0 + 15 of the K tile `kt` / V tile `vt`, of which the rows below
         // `rows` exist.  Rows that do not exist are read from the last one that does (finite data) and get weight 0.
-        auto block = [&](const unsigned char *kt, const unsigned char *vt, int key0, int rows) {
+        // `causal`: the rows are the new tokens of the chunk: key i is visible to this lane's member only if i <= its token
+        auto block = [&](const unsigned char *kt, const unsigned char *vt, int key0, int rows, bool causal = false) {
             // ---- scores (Algorithm 3 step 10): two sub-blocks of 8 keys; lane (g, t4) supplies keys key0 + g and
             //      key0 + 8 + g and receives keys key0 + 2 t4 (+1) and key0 + 8 + 2 t4 (+1) of its head.  Four
             //      independent accumulator chains (sub-block x half of the 32-wide block).
@@ -160,6 +167,7 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             }
             // ---- online softmax (step 11) ----
             int ka[4];
+            bool see[4];
             float s[4];
 #pragma unroll
             for (int u = 0; u < 2; ++u)
@@ -167,16 +175,18 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 for (int e = 0; e < 2; ++e) {
                     ka[2 * u + e] = key0 + 8 * u + 2 * t4 + e;
                     const float v = sc[u][0][e] + sc[u][1][e];
-                    s[2 * u + e] = ka[2 * u + e] < rows ? v * scale_log2 : -INFINITY;
+                    // a masked key gets weight 0 for this lane's member; the V row of the key still feeds the other members
+                    see[2 * u + e] = ka[2 * u + e] < rows && !(causal && ka[2 * u + e] > my_tok);
+                    s[2 * u + e] = see[2 * u + e] ? v * scale_log2 : -INFINITY;
                 }
             float mt = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
             mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 1));
             mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 2));
-            const float m_new = fmaxf(m_run, mt);                  // finite: row key0 exists
+            const float m_new = fmaxf(m_run, mt);                  // finite: row key0 exists and is visible to every member
             const float corr = fast_exp2(m_run - m_new);           // 0 while m_run = -inf
             float pr[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) pr[e] = ka[e] < rows ? fast_exp2(s[e] - m_new) : 0.f;
+            for (int e = 0; e < 4; ++e) pr[e] = see[e] ? fast_exp2(s[e] - m_new) : 0.f;
             const uint32_t pa0 = pack2(pr[0], pr[1]), pa1 = pack2(pr[2], pr[3]);
             uint32_t pl0 = 0u, pl1 = 0u;
             if constexpr (PRECISE) {
@@ -225,7 +235,7 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
         }
         // ---- the new row, straight from shared memory (never re-read from the cache) ----
         if (has_new && (warp == 0 || (wide && warp == 4)))
-            block(reinterpret_cast<const unsigned char *>(sm.knew), reinterpret_cast<const unsigned char *>(sm.vnew), 0, 1);
+            block(reinterpret_cast<const unsigned char *>(&sm.knew[0][0]), reinterpret_cast<const unsigned char *>(&sm.vnew[0][0]), 0, N, N > 1);
 
         // ---- the warps' states meet in shared memory ----
         l_run += __shfl_xor_sync(kFull, l_run, 1);
@@ -239,9 +249,10 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
         if (!named_bar_and(1, nct, ok)) return false;
         const bool whole = sg.n_cta == 1;                // this CTA alone finishes the group right here
         for (int idx = t; idx < G * DH; idx += nct) {
-            const int g2 = idx / DH, i = idx - g2 * DH, hq = hk * G + g2;
-            // the warps that hold head g2 (all of them, or one set of four), in slot g2 mod 8
-            const int sl = g2 & (kHeadsPerWarp - 1), w0 = wide ? 4 * (g2 >> 3) : 0, w1 = wide ? w0 + 4 : kGroupWarps;
+            const int m = idx / DH, i = idx - m * DH, j = m / Gh, hq = hk * Gh + (m - j * Gh);
+            const int ob = b * N + j;                        // output / partial row of member m: token j of sequence b
+            // the warps that hold member m (all of them, or one set of four), in slot m mod 8
+            const int sl = m & (kHeadsPerWarp - 1), w0 = wide ? 4 * (m >> 3) : 0, w1 = wide ? w0 + 4 : kGroupWarps;
             float M = -INFINITY;
             for (int w = w0; w < w1; ++w) M = fmaxf(M, sm.wm[w][sl]);
             float o = 0.f, l = 0.f;
@@ -250,9 +261,9 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 o += f * sm.wo[w][sl][i];
                 l += f * sm.wl[w][sl];
             }
-            if (whole) *attn_out_at(a, b, hq * DH + i) = __float2bfloat16_rn(o / l);
+            if (whole) *attn_out_at(a, ob, hq * DH + i) = __float2bfloat16_rn(o / l);
             else {
-                float *part = a.part + (((size_t)b * a.n_q_heads + hq) * kMaxSplits + (cta - sg.first_cta)) * kPartStride;
+                float *part = a.part + (((size_t)ob * a.n_q_heads + hq) * kMaxSplits + (cta - sg.first_cta)) * kPartStride;
                 part[i] = o;
                 if (i == 0) { part[DH] = M; part[DH + 1] = l; }
             }
@@ -261,7 +272,7 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             // ---- several CTAs share the K/V head: the partials are published, the last CTA merges the G heads ----
             __threadfence();
             named_bar_sync(1, nct);
-            int *ticket = a.ticket + (size_t)b * a.n_q_heads + hk * G;
+            int *ticket = a.ticket + (size_t)b * N * a.n_q_heads + hk * Gh;
             if (t == 0) sm.last = (atomicAdd(ticket, 1) == sg.n_cta - 1);
             named_bar_sync(1, nct);
             if (sm.last) {
@@ -269,7 +280,8 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 // one warp per query head of the group, all heads at once: lane s holds (max, sum) of partial s and
                 // the merge factor that goes with it; every lane finishes DH / 32 columns
                 for (int hg = warp; hg < G; hg += kGroupWarps) {
-                    const float *hp = a.part + ((size_t)b * a.n_q_heads + hk * G + hg) * kMaxSplits * kPartStride;
+                    const int mj = hg / Gh, mh = hk * Gh + (hg - mj * Gh), ob = b * N + mj;     // member hg: token mj, head mh
+                    const float *hp = a.part + ((size_t)ob * a.n_q_heads + mh) * kMaxSplits * kPartStride;
                     const bool have = lane < sg.n_cta;
                     const float ms = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH) : -INFINITY;
                     const float ls = have ? ld_cg_f32(hp + (size_t)lane * kPartStride + DH + 1) : 0.f;
@@ -296,7 +308,7 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                         }
                     }
 #pragma unroll
-                    for (int c = 0; c < DH / 32; ++c) *attn_out_at(a, b, (hk * G + hg) * DH + lane + 32 * c) = __float2bfloat16_rn(oo[c] / ll);
+                    for (int c = 0; c < DH / 32; ++c) *attn_out_at(a, ob, mh * DH + lane + 32 * c) = __float2bfloat16_rn(oo[c] / ll);
                 }
                 if (t == 0) *ticket = 0;
             }

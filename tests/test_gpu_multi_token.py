@@ -27,14 +27,19 @@ def dev(bits):
     return wl.from_bits(bits, "cuda")
 
 
-@pytest.mark.parametrize("dims,lens,n_new", [(wl.TINY, [0], 2), (wl.TINY, [5, 64, 17], 3), (wl.SMALL, [100, 3], 8),
-                                             (wl.SMALL_GQA, [9, 200, 31], 4), (wl.PHI3_MINI, [1000, 17], 4),
-                                             (wl.PHI3_MINI, [4088], 8), (wl.SMALL, [40, 7, 100], 1)])
-def test_attn_decode_multi_matches_oracle(fb, dims, lens, n_new):
+# share 1: the tokens of a chunk (times the query heads of a K/V head) go through one pass over the cache on the tensor
+# cores while there are at most 16 of them, one pass per token and query head otherwise; share 0: always the latter.
+@pytest.mark.parametrize("dims,lens,n_new,share", [
+    (wl.TINY, [0], 2, 1), (wl.TINY, [5, 64, 17], 3, 1), (wl.SMALL, [100, 3], 8, 1), (wl.SMALL_GQA, [9, 200, 31], 4, 1),
+    (wl.SMALL_GQA, [9, 200, 31], 3, 1), (wl.SMALL_GQA, [50, 6], 8, 1), (wl.PHI3_MINI, [1000, 17], 4, 1),
+    (wl.PHI3_MINI, [4088], 8, 1), (wl.SMALL, [40, 7, 100], 1, 1), (wl.TINY, [5, 64, 17], 3, 0),
+    (wl.SMALL_GQA, [9, 200, 31], 5, 0), (wl.PHI3_MINI, [1000, 17], 4, 0), (wl.PHI3_MINI, [4088], 7, 2)])
+def test_attn_decode_multi_matches_oracle(fb, dims, lens, n_new, share):
     B, max_seq = len(lens), 4096 if dims is wl.PHI3_MINI else 256
     lens = np.asarray(lens, np.int32)
     pos = lens + 3 if dims is not wl.PHI3_MINI else lens          # the rotary position need not be the cache row
     ctx = fb.Context.from_dims(dims, B * n_new, max_seq)
+    ctx.set_option("gqa_share", share)
     d, Hq, Hkv = dims.head_dim, dims.n_q_heads, dims.n_kv_heads
     rng = np.random.default_rng(11)
     mk = lambda *s: orc.f32_to_bf16(rng.standard_normal(s).astype(np.float32))
