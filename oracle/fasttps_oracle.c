@@ -15,6 +15,7 @@
  *   - MLP step order                   Algorithm 4 (RMSNorm, gate_up, siLu_Mul, down)
  *   - block structure (norm, QKV, attention, output projection, norm, MLP)
  *                                      Figure 1 caption, Section 2.2, Section 2.3
+ *   - the same attention step over a cache of 8-bit (E4M3) codes   Section 6.2 (compatibility with quantisation)
  *
  * Precision model.  Every tensor that crosses one of the three block
  * functions (attention, MLP, layer) is bf16, rounded to nearest even.  Inside
@@ -339,6 +340,99 @@ void orc_attn_probs(const uint16_t *q, const uint16_t *k_cache, int pos, int L,
     }
     for (int j = 0; j < Nt; ++j) { p[j] = exp(p[j] - m); denom += p[j]; }
     for (int j = 0; j < Nt; ++j) p[j] /= denom;
+}
+
+/* ---------------------------------------------- attention decode, FP8 KV cache */
+
+/* The 8-bit floating-point format E4M3 (the "fn" variant: no infinities) by its definition: bit 7 sign, bits 6..3
+ * exponent e (bias 7), bits 2..0 mantissa m.  e = 0: subnormal, m/8 * 2^-6; otherwise (1 + m/8) * 2^(e-7); the
+ * pattern e = 15, m = 7 is NaN, so the largest finite value is 1.75 * 2^8 = 448. */
+float orc_e4m3_to_f32(uint8_t c)
+{
+    int e = (c >> 3) & 15, m = c & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    v = e == 0 ? ldexp((double)m / 8.0, -6) : ldexp(1.0 + (double)m / 8.0, e - 7);
+    return (float)((c & 0x80) ? -v : v);
+}
+
+/* FP32 -> E4M3: the finite code nearest to x, ties to the code with an even mantissa, magnitudes beyond 448
+ * saturate to 448 (no code for infinity), NaN gives the NaN code.  Found by looking at all 127 finite magnitudes. */
+uint8_t orc_f32_to_e4m3(float x)
+{
+    uint8_t sign = signbit(x) ? 0x80 : 0x00;
+    double a = fabs((double)x), best_d = INFINITY;
+    int best = 0;
+    if (isnan(x)) return 0x7f;
+    for (int c = 0; c <= 0x7e; ++c) {
+        double dd = fabs((double)orc_e4m3_to_f32((uint8_t)c) - a);
+        if (dd < best_d || (dd == best_d && (c & 1) == 0)) { best_d = dd; best = c; }
+    }
+    return (uint8_t)(sign | best);
+}
+
+/* Algorithm 3 with the cache held in E4M3 (Section 6.2 states that the method composes with quantisation; the
+ * paper gives no scheme, so the reading is the plainest one: one FP32 scale per tensor, given by the caller).
+ *   stored code = e4m3(value / scale)  (FP32 division, then the rounding above); value read back = code * scale.
+ *   k_cache, v_cache [B,Hkv,max_seq,d] uint8 codes, modified in place: row seq_lens[b] of every head receives the
+ *   codes of rope(k_new) / k_scale resp. v_new / v_scale.  The new token attends to its own row AS STORED (the
+ *   dequantised codes), so that this step and every later step see the same key and value for it.
+ * Everything else (shapes, RoPE in FP32, skipping rules, double accumulation, bf16 output) as orc_attn_decode. */
+void orc_attn_decode_fp8(const uint16_t *q, const uint16_t *k_new, const uint16_t *v_new,
+                         uint8_t *k_cache, uint8_t *v_cache, float k_scale, float v_scale,
+                         const int32_t *pos, const int32_t *seq_lens, uint16_t *out,
+                         int B, int Hq, int Hkv, int d, int max_seq, double theta)
+{
+    int G = Hq / Hkv;
+    for (int b = 0; b < B; ++b) {
+        int L = seq_lens[b];
+        if (L < 0 || L >= max_seq || pos[b] < 0) continue;
+        for (int h = 0; h < Hkv; ++h) {
+            float kr[1024];
+            for (int c = 0; c < d; ++c) kr[c] = orc_bf16_to_f32(k_new[((size_t)b * Hkv + h) * d + c]);
+            orc_rope(kr, d, pos[b], theta);
+            size_t row = (((size_t)b * Hkv + h) * max_seq + L) * d;
+            for (int c = 0; c < d; ++c) {
+                volatile float ks = kr[c] / k_scale;
+                volatile float vs = orc_bf16_to_f32(v_new[((size_t)b * Hkv + h) * d + c]) / v_scale;
+                k_cache[row + c] = orc_f32_to_e4m3(ks);
+                v_cache[row + c] = orc_f32_to_e4m3(vs);
+            }
+        }
+    }
+    #pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        for (int h = 0; h < Hq; ++h) {
+            int L = seq_lens[b];
+            if (L < 0 || L >= max_seq || pos[b] < 0) continue;
+            int Nt = L + 1;
+            int hk = h / G;
+            float qr[1024];
+            for (int c = 0; c < d; ++c) qr[c] = orc_bf16_to_f32(q[((size_t)b * Hq + h) * d + c]);
+            orc_rope(qr, d, pos[b], theta);
+            const uint8_t *Kh = k_cache + ((size_t)b * Hkv + hk) * max_seq * d;
+            const uint8_t *Vh = v_cache + ((size_t)b * Hkv + hk) * max_seq * d;
+            double *s = (double *)malloc(sizeof(double) * (size_t)Nt);
+            double scale = 1.0 / sqrt((double)d);
+            double m = -INFINITY;
+            for (int j = 0; j < Nt; ++j) {
+                double acc = 0.0;
+                for (int c = 0; c < d; ++c)
+                    acc += (double)qr[c] * ((double)orc_e4m3_to_f32(Kh[(size_t)j * d + c]) * (double)k_scale);
+                s[j] = acc * scale;
+                if (s[j] > m) m = s[j];
+            }
+            double denom = 0.0;
+            for (int j = 0; j < Nt; ++j) { s[j] = exp(s[j] - m); denom += s[j]; }
+            for (int c = 0; c < d; ++c) {
+                double o = 0.0;
+                for (int j = 0; j < Nt; ++j)
+                    o += (s[j] / denom) * ((double)orc_e4m3_to_f32(Vh[(size_t)j * d + c]) * (double)v_scale);
+                out[((size_t)b * Hq + h) * d + c] = orc_f64_to_bf16(o);
+            }
+            free(s);
+        }
+    }
 }
 
 /* ------------------------------------------------------------- MLP decode */

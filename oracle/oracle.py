@@ -169,6 +169,42 @@ def attn_decode_multi(q, k_new, v_new, k_cache, v_cache, pos, seq_lens, theta=10
     return out
 
 
+def e4m3_to_f32(codes) -> np.ndarray:
+    """uint8 E4M3 codes -> float32 values (NaN for the two NaN codes)."""
+    c = np.ascontiguousarray(np.asarray(codes, dtype=np.uint8))
+    f = lib().orc_e4m3_to_f32
+    f.restype, f.argtypes = C.c_float, [C.c_uint8]
+    return np.array([f(int(v)) for v in c.ravel()], dtype=np.float32).reshape(c.shape)
+
+
+def f32_to_e4m3(x) -> np.ndarray:
+    """float32 values -> uint8 E4M3 codes: nearest, ties to even, saturating at 448."""
+    v = np.ascontiguousarray(np.asarray(x, dtype=np.float32))
+    f = lib().orc_f32_to_e4m3
+    f.restype, f.argtypes = C.c_uint8, [C.c_float]
+    return np.array([f(float(t)) for t in v.ravel()], dtype=np.uint8).reshape(v.shape)
+
+
+def attn_decode_fp8(q, k_new, v_new, k_cache, v_cache, k_scale, v_scale, pos, seq_lens, theta=10000.0):
+    """Algorithm 3 over a cache of E4M3 codes (uint8 [B,Hkv,max_seq,d], appended in place) with one scale per tensor;
+    returns out [B,Hq,d] bf16 bits."""
+    q, k_new, v_new = _u16(q), _u16(k_new), _u16(v_new)
+    assert k_cache.dtype == np.uint8 and k_cache.flags.c_contiguous and k_cache.flags.writeable
+    assert v_cache.dtype == np.uint8 and v_cache.flags.c_contiguous and v_cache.flags.writeable
+    B, Hq, d = q.shape
+    Hkv = k_new.shape[1]
+    max_seq = k_cache.shape[2]
+    assert k_cache.shape == (B, Hkv, max_seq, d) and v_cache.shape == k_cache.shape
+    pos, seq_lens = _i32(pos), _i32(seq_lens)
+    out = np.zeros((B, Hq, d), dtype=np.uint16)
+    u8p = C.POINTER(C.c_uint8)
+    lib().orc_attn_decode_fp8(_p(q, _u16p), _p(k_new, _u16p), _p(v_new, _u16p), _p(k_cache, u8p), _p(v_cache, u8p),
+                              C.c_float(k_scale), C.c_float(v_scale), _p(pos, _i32p), _p(seq_lens, _i32p),
+                              _p(out, _u16p), C.c_int(B), C.c_int(Hq), C.c_int(Hkv), C.c_int(d), C.c_int(max_seq),
+                              C.c_double(theta))
+    return out
+
+
 def attn_probs(q, k_cache, pos, L, b, h, theta=10000.0):
     q = _u16(q)
     B, Hq, d = q.shape

@@ -631,3 +631,111 @@ def test_layer_with_several_new_tokens_equals_the_blocks_chained_by_hand():
     # and one new token per sequence is the decode layer itself
     x1 = x[::N].copy()
     assert (orc.layer_decode_multi(w, x1, 1, kc.copy(), vc.copy(), pos, lens) == orc.layer_decode(w, x1, kc.copy(), vc.copy(), pos, lens)).all()
+
+
+# ------------------------------------------- attention over a cache of 8-bit (E4M3) codes (Section 6.2)
+
+def _torch_e4m3_values():
+    import torch
+    return torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).float().numpy()
+
+
+def test_e4m3_decode_is_the_format():
+    allc = np.arange(256, dtype=np.uint8)
+    f = orc.e4m3_to_f32(allc)
+    # facts of the format: 1.0, the largest finite value 448, the smallest subnormal 2^-9 and normal 2^-6, two zeros,
+    # NaN at 0x7f / 0xff and nowhere else, no infinities, 8 values per binade, magnitudes strictly increasing with the code
+    assert f[0x38] == 1.0 and f[0x7e] == 448.0 and f[0x01] == 2.0 ** -9 and f[0x08] == 2.0 ** -6
+    assert f[0] == 0 and f[0x80] == 0 and np.signbit(f[0x80]) and not np.signbit(f[0])
+    assert np.isnan(f[[0x7f, 0xff]]).all() and np.isfinite(np.delete(f, [0x7f, 0xff])).all()
+    assert (np.diff(f[:0x7f]) > 0).all() and (f[0x80:0xff] == -f[:0x7f]).all()
+    assert (f[0x40:0x48] == 2.0 * f[0x38:0x40]).all()
+    # and a library's table of the same format
+    t = _torch_e4m3_values()
+    assert ((f == t) | (np.isnan(f) & np.isnan(t))).all()
+
+
+def test_e4m3_encode_rounds_to_nearest_even_and_saturates():
+    import torch
+    vals = orc.e4m3_to_f32(np.arange(0x7f, dtype=np.uint8)).astype(np.float64)
+    allc = np.delete(np.arange(256, dtype=np.uint8), [0x7f, 0xff])
+    assert (orc.f32_to_e4m3(orc.e4m3_to_f32(allc)) == allc).all()                     # every code is its own nearest
+    mid = ((vals[:-1] + vals[1:]) / 2).astype(np.float32)                            # exact in FP32
+    want_even = np.where(np.arange(0x7e) % 2 == 0, np.arange(0x7e), np.arange(0x7e) + 1)
+    assert (orc.f32_to_e4m3(mid) == want_even).all() and (orc.f32_to_e4m3(-mid) == (want_even | 0x80)).all()
+    assert (orc.f32_to_e4m3(np.nextafter(mid, np.float32(0))) == np.arange(0x7e)).all()      # just below a midpoint
+    assert (orc.f32_to_e4m3(np.nextafter(mid, np.float32(1e9))) == np.arange(0x7e) + 1).all()
+    assert (orc.f32_to_e4m3([449.0, 1e9, np.inf, -np.inf, -500.0]) == [0x7e, 0x7e, 0x7e, 0xfe, 0xfe]).all()
+    assert orc.f32_to_e4m3([np.nan])[0] & 0x7f == 0x7f
+    x = (RNG.standard_normal(4000) * np.exp(RNG.uniform(-8, 5, 4000))).astype(np.float32)
+    x = x[np.abs(x) <= 448]
+    lib_codes = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert (orc.f32_to_e4m3(x) == lib_codes).all()
+
+
+def _fp8_case(Bn=2, Hq=4, Hkv=2, d=8, max_seq=12, lens=(5, 0), on_grid=False):
+    codes = lambda *s: RNG.choice(np.delete(np.arange(256), [0x7f, 0xff]), size=s).astype(np.uint8)
+    kc, vc = codes(Bn, Hkv, max_seq, d), codes(Bn, Hkv, max_seq, d)
+    # keep the codes moderate so that scores stay in a range where the softmax is not one-hot
+    kc, vc = (kc & 0x80) | (0x20 + (kc & 0x1f)), (vc & 0x80) | (0x20 + (vc & 0x1f))
+    q = rnd(Bn, Hq, d)
+    if on_grid:       # new rows that ARE E4M3 values: quantising them changes nothing
+        kn = B16(orc.e4m3_to_f32((codes(Bn, Hkv, d) & 0x9f) | 0x20))
+        vn = B16(orc.e4m3_to_f32((codes(Bn, Hkv, d) & 0x9f) | 0x20))
+    else:
+        kn, vn = rnd(Bn, Hkv, d), rnd(Bn, Hkv, d)
+    return q, kn, vn, kc.astype(np.uint8), vc.astype(np.uint8), np.asarray(lens, np.int32)
+
+
+def test_fp8_attention_on_exactly_representable_data_is_the_bf16_attention():
+    # power-of-two scales and position 0 (no rotation): every dequantised value is a bf16 number and the new rows
+    # survive quantisation unchanged, so the step must equal the bf16 step on the dequantised cache, bit for bit
+    q, kn, vn, kc, vc, lens = _fp8_case(on_grid=True)
+    ks, vs = 0.25, 2.0
+    pos = np.zeros_like(lens)
+    kb = B16(orc.e4m3_to_f32(kc) * np.float32(ks))
+    vb = B16(orc.e4m3_to_f32(vc) * np.float32(vs))
+    knb, vnb = B16(F32(kn) * np.float32(ks)), B16(F32(vn) * np.float32(vs))
+    out8 = orc.attn_decode_fp8(q, knb, vnb, kc, vc, ks, vs, pos, lens)
+    out16 = orc.attn_decode(q, knb, vnb, kb, vb, pos, lens)
+    assert (out8 == out16).all()
+    assert (B16(orc.e4m3_to_f32(kc) * np.float32(ks)) == kb).all() and (B16(orc.e4m3_to_f32(vc) * np.float32(vs)) == vb).all()
+
+
+def test_fp8_attention_against_the_definition_written_out():
+    q, kn, vn, kc, vc, lens = _fp8_case()
+    Bn, Hq, d = q.shape
+    Hkv, max_seq = kn.shape[1], kc.shape[2]
+    ks, vs = 0.37, 1.6                                     # scales that are not powers of two
+    pos = lens + 2
+    k0, v0 = kc.copy(), vc.copy()
+    out = orc.attn_decode_fp8(q, kn, vn, kc, vc, ks, vs, pos, lens)
+    for b in range(Bn):
+        L = int(lens[b])
+        for hk in range(Hkv):
+            # the appended codes: FP32 rotation, FP32 division by the scale, nearest code; nothing else changes
+            kr = orc.rope(F32(kn[b, hk]), pos[b]) / np.float32(ks)
+            assert (kc[b, hk, L] == orc.f32_to_e4m3(kr)).all()
+            assert (vc[b, hk, L] == orc.f32_to_e4m3(F32(vn[b, hk]) / np.float32(vs))).all()
+            keep = np.arange(max_seq) != L
+            assert (kc[b, hk, keep] == k0[b, hk, keep]).all() and (vc[b, hk, keep] == v0[b, hk, keep]).all()
+        for h in range(Hq):
+            hk = h // (Hq // Hkv)
+            K = orc.e4m3_to_f32(kc[b, hk, :L + 1]).astype(np.float64) * np.float64(np.float32(ks))
+            V = orc.e4m3_to_f32(vc[b, hk, :L + 1]).astype(np.float64) * np.float64(np.float32(vs))
+            s = K @ orc.rope(F32(q[b, h]), pos[b]).astype(np.float64) / math.sqrt(d)
+            p = np.exp(s - s.max())
+            want = (p / p.sum()) @ V
+            assert ulp_distance(out[b, h], orc.f64_to_bf16(want)).max() <= 1
+
+
+def test_fp8_attention_skips_a_full_cache_and_saturates_large_rows():
+    q, kn, vn, kc, vc, _ = _fp8_case(max_seq=6)
+    lens = np.array([6, 2], np.int32)
+    k0, v0 = kc.copy(), vc.copy()
+    out = orc.attn_decode_fp8(q, kn, vn, kc, vc, 1.0, 1.0, lens, lens)
+    assert (kc[0] == k0[0]).all() and (vc[0] == v0[0]).all() and (out[0] == 0).all() and (out[1] != 0).any()
+    # a scale far too small: the stored magnitudes stop at 448
+    vbig = B16(np.full(vn.shape, 3.0, np.float32))
+    orc.attn_decode_fp8(q, kn, vbig, kc, vc, 1.0, 1e-3, lens, lens)
+    assert (vc[1, :, 2] == 0x7e).all()
