@@ -132,9 +132,10 @@ int fasttps_unpack_weight(fasttps_ctx *ctx, int kind, const void *src_packed, vo
  *   seq_lens [B] int32 device: rows already cached (N_p) = the row written now.
  *   out [B,H_q,d]: softmax(q' K^T / sqrt(d)) V over rows 0..seq_lens[b] inclusive.
  * Query head h uses kv head h / (H_q/H_kv) (Section 4.1).  With 2 to 16 query heads per kv head every
- * cached row is read once for its whole group and the two products run on the tensor cores: there the
- * rotated q and the softmax weights enter the products rounded to bf16 (FP32 accumulation); with one
- * query head per kv head, or more than 16, both stay FP32.  Neither pos nor seq_lens is advanced. */
+ * cached row is read once for its whole group and the two products run on the tensor cores (FP32
+ * accumulation): there the rotated q and the softmax weights enter the products as pairs of bf16 numbers
+ * (value = hi + lo), or rounded to bf16 once with option "gqa_share" 2; with one query head per kv head, more
+ * than 16, or option "gqa_share" 0, both stay FP32.  Neither pos nor seq_lens is advanced. */
 int fasttps_attn_decode(fasttps_ctx *ctx, const void *q, const void *k_new, const void *v_new,
                         void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
                         void *out, int batch, void *stream);
@@ -144,9 +145,11 @@ int fasttps_attn_decode(fasttps_ctx *ctx, const void *q, const void *k_new, cons
  *   q [B,N,H_q,d], k_new, v_new [B,N,H_kv,d], out [B,N,H_q,d]; caches, pos, seq_lens [B] as above.
  * Token j of sequence b is rotated at position pos[b] + j, goes into row seq_lens[b] + j of every head (B*N*H_kv
  * runs of d elements are written, nothing else) and attends rows 0 .. seq_lens[b] + j: the cached rows and the new
- * tokens up to and including itself (causal inside the chunk).  The cached rows are streamed once per new token
- * and query head, in FP32 (the one-pass-per-query-head kernel); the new rows are scored from shared memory.  A
- * sequence whose n_new rows do not all fit (seq_lens[b] + n_new > max_seq) is skipped and reported. */
+ * tokens up to and including itself (causal inside the chunk).  While n_new * (H_q / H_kv) <= 16 the new tokens of a
+ * sequence (times the query heads of a kv head) share ONE pass over the cached rows, on the tensor cores as described
+ * above; otherwise, and with option "gqa_share" 0, the cached rows are streamed once per new token and query head in
+ * FP32.  The new rows are scored from shared memory either way.  A sequence whose n_new rows do not all fit
+ * (seq_lens[b] + n_new > max_seq) is skipped and reported. */
 int fasttps_attn_decode_multi(fasttps_ctx *ctx, const void *q, const void *k_new, const void *v_new,
                               void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
                               void *out, int batch, int n_new, void *stream);
@@ -176,6 +179,21 @@ int fasttps_mlp_decode(fasttps_ctx *ctx, const void *x, const void *w_gate_up, c
  *   race on it; calls on one stream are ordered. */
 int fasttps_mlp_decode_static(fasttps_ctx *ctx, const void *x, const void *w_gate_up, const void *w_down,
                               void *out, int batch, void *stream);
+
+/* Algorithm 3 over a KV cache of 8-bit floating-point codes (E4M3: 4 exponent bits, bias 7, 3 mantissa bits, no
+ * infinities, largest value 448), the quantised cache the paper names as compatible (Section 6.2); one FP32 scale per
+ * tensor, given by the caller:
+ *   k_cache, v_cache [B,H_kv,max_seq,d] uint8 device, updated in place: row seq_lens[b] of every head receives the
+ *       codes of rope(k_new) / k_scale resp. v_new / v_scale (FP32 division, round to nearest even, magnitudes
+ *       beyond 448 saturate): B*H_kv runs of d BYTES, nothing else is written.  A stored code c stands for c * scale.
+ *   q, k_new, v_new, pos, seq_lens, out as in fasttps_attn_decode (bf16).  The new token attends its own row as
+ *       stored (the dequantised codes).  k_scale, v_scale > 0 and finite, else FASTTPS_INVALID_ARG.
+ * Every cached row is read once for all query heads of its kv head (1 to 16 of them, else FASTTPS_INVALID_ARG); the
+ * codes are widened to fp16 in registers (exact) and the two products run on the tensor cores with the rotated q and
+ * the softmax weights as fp16 hi + lo pairs, FP32 accumulation. */
+int fasttps_attn_decode_fp8(fasttps_ctx *ctx, const void *q, const void *k_new, const void *v_new,
+                            void *k_cache, void *v_cache, float k_scale, float v_scale, const int32_t *pos,
+                            const int32_t *seq_lens, void *out, int batch, void *stream);
 
 /* Building block of the chain (QKV, output projection, lm_head; Figure 1):
  *   out[b,n] = (g_norm ? rmsnorm(x[b], g_norm) : x[b]) . W[n,:] (+ residual[b,n])

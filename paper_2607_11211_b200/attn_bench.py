@@ -1,11 +1,12 @@
 """Times ``fasttps_attn_decode`` alone on one of the attention shapes the paper evaluates (its Table 1).
 
-    python -m paper_2607_11211_b200.attn_bench --model llama3-8b --batch 8 --past 4095 [--gqa-share 0|1|2]
+    python -m paper_2607_11211_b200.attn_bench --model llama3-8b --batch 8 --past 4095 [--gqa-share 0|1|2] [--n-new N] [--fp8]
 
 The call is enqueued ``--iters`` times on one stream between two CUDA events, rotating over enough cache sets
 that no K/V row is still in the L2 when it is read again.  Algorithmic bytes per call: every cached row of every
 K/V head read once (K and V), the new rows written once, q and the output; with ``--gqa-share 0`` the kernel
-reads a K/V head once per query head, and the same algorithmic bytes are charged.  Prints one JSON line.
+reads a K/V head once per query head, and the same algorithmic bytes are charged.  ``--fp8``: the caches hold 8-bit
+E4M3 codes (``fasttps_attn_decode_fp8``), one byte per cached element.  Prints one JSON line.
 """
 import argparse
 import json
@@ -30,7 +31,10 @@ def main():
     ap.add_argument("--gqa-share", type=int, default=1)
     ap.add_argument("--n-new", type=int, default=1,
                     help="new tokens per sequence and step (> 1: fasttps_attn_decode_multi, causal inside the chunk)")
+    ap.add_argument("--fp8", action="store_true", help="KV cache of 8-bit E4M3 codes (fasttps_attn_decode_fp8)")
     args = ap.parse_args()
+    if args.fp8 and args.n_new != 1:
+        raise SystemExit("--fp8 times the one-token step")
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device: there is no CPU path")
     build.build()
@@ -40,9 +44,14 @@ def main():
     max_seq = L + N
     ctx = fb.Context.from_dims(dims, B * N, max_seq)
     ctx.set_option("gqa_share", args.gqa_share)
-    cache_bytes = 2 * B * hkv * max_seq * d * 2
+    eb = 1 if args.fp8 else 2                                        # bytes per cached element
+    k_scale, v_scale = 1.0 / 16, 1.0 / 16
+    cache_bytes = 2 * B * hkv * max_seq * d * eb
     n_sets = max(2, -(-(400 << 20) // cache_bytes))                  # > 3 x the 126 MB L2 between two visits
-    sets = [wl.kv_cache(dims, i, B, max_seq, wl.MASTER_SEED, device="cuda") for i in range(n_sets)]
+    if args.fp8:
+        sets = [wl.kv_cache_e4m3(dims, i, B, max_seq, k_scale, v_scale, wl.MASTER_SEED, device="cuda") for i in range(n_sets)]
+    else:
+        sets = [wl.kv_cache(dims, i, B, max_seq, wl.MASTER_SEED, device="cuda") for i in range(n_sets)]
     act = wl.activations(dims, B * N, wl.MASTER_SEED, device="cuda")
     if N > 1:
         act = {k: v.view(B, N, *v.shape[1:]) for k, v in act.items()}
@@ -54,7 +63,9 @@ def main():
     def run(n):
         for i in range(n):
             kc, vc = sets[i % n_sets]
-            if N > 1:
+            if args.fp8:
+                ctx.attn_decode_fp8(act["q"], act["k_new"], act["v_new"], kc, vc, k_scale, v_scale, lens, lens, out, stream=st)
+            elif N > 1:
                 ctx.attn_decode_multi(act["q"], act["k_new"], act["v_new"], kc, vc, lens, lens, out, stream=st)
             else:
                 ctx.attn_decode(act["q"], act["k_new"], act["v_new"], kc, vc, lens, lens, out, stream=st)
@@ -70,12 +81,12 @@ def main():
     us = e0.elapsed_time(e1) / args.iters * 1e3
     status = ctx.get_status()
     # every cached row once (whatever the number of new tokens), the new rows written, q in, the output out
-    alg = 2 * B * hkv * (L + N) * d * 2 + 2 * B * N * hq * d * 2
+    alg = 2 * B * hkv * (L + N) * d * eb + 2 * B * N * hq * d * 2
     peaks = Path(__file__).resolve().parent.parent / "MEASURED_PEAKS.json"
     peak = float(json.loads(peaks.read_text())["hbm_gbs"]) if peaks.exists() else 6650.0
     gbs = alg / (us * 1e-6) / 1e9
     print(json.dumps({"kernel": "attn_decode_kernel", "model": args.model, "q_heads": hq, "kv_heads": hkv, "head_dim": d,
-                      "batch": B, "past": L, "n_new": N, "gqa_share": args.gqa_share, "cache_sets": n_sets, "iters": args.iters,
+                      "batch": B, "past": L, "n_new": N, "kv_dtype": "e4m3" if args.fp8 else "bf16", "gqa_share": args.gqa_share, "cache_sets": n_sets, "iters": args.iters,
                       "us_per_call": us, "algorithmic_bytes": alg, "achieved_gbs": gbs, "peak_gbs": peak,
                       "frac": gbs / peak, "peak_source": "of measured" if peaks.exists() else "of fallback",
                       "device_status": status}))

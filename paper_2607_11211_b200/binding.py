@@ -68,6 +68,7 @@ def load_library() -> C.CDLL:
     lib.fasttps_unpack_weight.argtypes = [vp, i, vp, vp, vp]
     lib.fasttps_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, vp, i, vp]
     lib.fasttps_attn_decode_multi.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, vp, i, i, vp]
+    lib.fasttps_attn_decode_fp8.argtypes = [vp, vp, vp, vp, vp, vp, C.c_float, C.c_float, ip, ip, vp, i, vp]
     lib.fasttps_layer_decode_multi.argtypes = [vp, C.POINTER(LayerWeights), vp, vp, vp, vp, ip, ip, i, i, vp]
     lib.fasttps_mlp_decode.argtypes = [vp, vp, vp, vp, vp, i, vp]
     lib.fasttps_mlp_decode_static.argtypes = [vp, vp, vp, vp, vp, i, vp]
@@ -217,6 +218,14 @@ class Context:
         _check(self.lib.fasttps_attn_decode(self.handle, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache),
                                             _ptr(v_cache), _ptr(pos), _ptr(seq_lens), _ptr(out), batch,
                                             _stream(stream)), "fasttps_attn_decode")
+        return out
+
+    def attn_decode_fp8(self, q, k_new, v_new, k_cache, v_cache, k_scale, v_scale, pos, seq_lens, out, stream=None):
+        """k_cache / v_cache: uint8 tensors of E4M3 codes [B,Hkv,max_seq,d]; a code c stands for c * scale."""
+        batch = q.shape[0]
+        _check(self.lib.fasttps_attn_decode_fp8(self.handle, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache),
+                                                _ptr(v_cache), float(k_scale), float(v_scale), _ptr(pos), _ptr(seq_lens),
+                                                _ptr(out), batch, _stream(stream)), "fasttps_attn_decode_fp8")
         return out
 
     def attn_decode_multi(self, q, k_new, v_new, k_cache, v_cache, pos, seq_lens, out, stream=None):

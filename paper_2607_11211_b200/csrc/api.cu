@@ -198,7 +198,7 @@ int fasttps_attn_splits(const fasttps_ctx *ctx, int batch)
 static int attn_impl(Ctx *c, const __nv_bfloat16 *q, const __nv_bfloat16 *k, const __nv_bfloat16 *v,
                      int q_stride, int kv_stride, void *k_cache, void *v_cache, const int32_t *pos,
                      const int32_t *seq_lens, __nv_bfloat16 *out, int out_stride, int batch, cudaStream_t st, int n_new = 1,
-                     int out_chunked = 0)
+                     int out_chunked = 0, bool fp8 = false, float k_scale = 1.f, float v_scale = 1.f)
 {
     const fasttps_config &f = c->cfg;
     AttnArgs a;
@@ -214,7 +214,8 @@ static int attn_impl(Ctx *c, const __nv_bfloat16 *q, const __nv_bfloat16 *k, con
     a.len_add = 0; a.n_new = n_new;
     a.cos_tab = c->cos_tab; a.sin_tab = c->sin_tab;
     a.part = c->attn_part; a.ticket = c->attn_ticket; a.status = c->status;
-    return launch_attn(c, a, st);
+    a.k_scale = k_scale; a.v_scale = v_scale;
+    return launch_attn(c, a, st, fp8);
 }
 
 int fasttps_attn_decode(fasttps_ctx *ctx, const void *q, const void *k_new, const void *v_new,
@@ -232,6 +233,24 @@ int fasttps_attn_decode(fasttps_ctx *ctx, const void *q, const void *k_new, cons
                      static_cast<const __nv_bfloat16 *>(v_new), f.n_q_heads * f.head_dim, f.n_kv_heads * f.head_dim,
                      k_cache, v_cache, pos, seq_lens, static_cast<__nv_bfloat16 *>(out), f.n_q_heads * f.head_dim,
                      batch, static_cast<cudaStream_t>(stream));
+}
+
+int fasttps_attn_decode_fp8(fasttps_ctx *ctx, const void *q, const void *k_new, const void *v_new,
+                            void *k_cache, void *v_cache, float k_scale, float v_scale, const int32_t *pos,
+                            const int32_t *seq_lens, void *out, int batch, void *stream)
+{
+    if (!ctx) return FASTTPS_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (batch < 1 || batch > c->cfg.max_batch) return FASTTPS_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache) ||
+        !aligned16(out) || !pos || !seq_lens)
+        return FASTTPS_INVALID_ARG;
+    if (!(k_scale > 0.f) || !(v_scale > 0.f) || std::isinf(k_scale) || std::isinf(v_scale)) return FASTTPS_INVALID_ARG;
+    const fasttps_config &f = c->cfg;
+    return attn_impl(c, static_cast<const __nv_bfloat16 *>(q), static_cast<const __nv_bfloat16 *>(k_new),
+                     static_cast<const __nv_bfloat16 *>(v_new), f.n_q_heads * f.head_dim, f.n_kv_heads * f.head_dim,
+                     k_cache, v_cache, pos, seq_lens, static_cast<__nv_bfloat16 *>(out), f.n_q_heads * f.head_dim,
+                     batch, static_cast<cudaStream_t>(stream), 1, 0, /*fp8=*/true, k_scale, v_scale);
 }
 
 // ---- thin-GEMM chain for batches above kMaxNB: every weight is read once for up to kWideMaxB rows ----

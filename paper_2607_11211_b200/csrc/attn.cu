@@ -46,10 +46,11 @@ struct AttnSmemShare {
 };
 
 // SHARE: one pass per K/V head for its group of query heads (tensor cores; PRECISE: q and the softmax weights as bf16
-// hi + lo pairs).  MULTI: several new tokens per sequence.
-template <int DH, bool SHARE, bool MULTI = false, bool PRECISE = false>
+// hi + lo pairs).  MULTI: several new tokens per sequence.  FP8: the cache holds E4M3 codes (SHARE and PRECISE).
+template <int DH, bool SHARE, bool MULTI = false, bool PRECISE = false, bool FP8 = false>
 __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a)
 {
+    static_assert(!FP8 || (SHARE && PRECISE), "the E4M3 cache is served by the one-pass-per-K/V-head kernel");
     static_assert(!(SHARE && MULTI), "the multi-token path is the one-pass-per-query-head kernel");
     using Smem = typename std::conditional<SHARE, AttnSmemShare<DH>, AttnSmem<DH>>::type;
     extern __shared__ unsigned char smem_raw[];
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a
 
     int piece = 0;
     if (warp == kAttnWarps) {
-        if ((t & 31) == 0) (void)attn_produce<DH, SHARE>(a, ring, piece, blockIdx.x, gridDim.x);
+        if ((t & 31) == 0) (void)attn_produce<DH, SHARE, FP8 ? 1 : 2, FP8 ? 2 * kAttnTileRows : kAttnTileRows>(a, ring, piece, blockIdx.x, gridDim.x);
         return;
     }
     if (blockIdx.x == 0 && t == 0) {
@@ -80,7 +81,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attn_decode_kernel(AttnArgs a
     }
     bool done;
     if constexpr (SHARE)
-        done = attn_consume_group<DH, PRECISE>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x, true), sm.scratch);
+        done = attn_consume_group<DH, PRECISE, FP8>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x, true), sm.scratch);
     else if constexpr (MULTI)
         done = attn_consume<DH, false, WalkSource, false, false, true>(a, ring, piece, blockIdx.x, WalkSource(a, blockIdx.x, gridDim.x),
                                                                        sm.scratch, kAttnWarps, nullptr, &sm.multi);
@@ -101,12 +102,13 @@ int attn_splits_for(const Ctx *c, int batch)
 }
 
 template <int DH>
-static int launch_attn_dh(Ctx *c, const AttnArgs &a, cudaStream_t st)
+static int launch_attn_dh(Ctx *c, const AttnArgs &a, cudaStream_t st, bool fp8)
 {
     dim3 grid(a.n_splits);
     ProfScope prof(c, kProfAttn, st);
     const bool share = attn_shares_groups(a.n_q_heads, a.n_kv_heads, a.n_new);
-    const int rc = (c->opt_gqa_share == 1 && share)
+    const int rc = fp8 ? launch_ex(attn_decode_kernel<DH, true, false, true, true>, grid, dim3(kAttnThreads), sizeof(AttnSmemShare<DH>) + 128, st, &a)
+                   : (c->opt_gqa_share == 1 && share)
                        ? launch_ex(attn_decode_kernel<DH, true, false, true>, grid, dim3(kAttnThreads), sizeof(AttnSmemShare<DH>) + 128, st, &a)
                    : (c->opt_gqa_share && share)
                        ? launch_ex(attn_decode_kernel<DH, true>, grid, dim3(kAttnThreads), sizeof(AttnSmemShare<DH>) + 128, st, &a)
@@ -124,6 +126,7 @@ static int configure_attn_dh()
     FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmemShare<DH>) + 128));
     FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmemShare<DH>) + 128));
     FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmem<DH>) + 128));
+    FT_CUDA(cudaFuncSetAttribute(attn_decode_kernel<DH, true, false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(AttnSmemShare<DH>) + 128));
     return FASTTPS_OK;
 }
 
@@ -136,13 +139,18 @@ int configure_attn_kernels()
     return configure_attn_dh<128>();
 }
 
-int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st)
+// fp8: the caches hold E4M3 codes (a.k_scale / a.v_scale set); the group (query heads x new tokens) is 1 to 16 members
+int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st, bool fp8)
 {
+    if (fp8) {
+        const int G = (a.n_kv_heads > 0 ? a.n_q_heads / a.n_kv_heads : 0) * a.n_new;
+        if (G < 1 || G > kMaxShareGroup) return FASTTPS_INVALID_ARG;
+    }
     switch (a.head_dim) {
-    case 32: return launch_attn_dh<32>(c, a, st);
-    case 64: return launch_attn_dh<64>(c, a, st);
-    case 96: return launch_attn_dh<96>(c, a, st);
-    case 128: return launch_attn_dh<128>(c, a, st);
+    case 32: return launch_attn_dh<32>(c, a, st, fp8);
+    case 64: return launch_attn_dh<64>(c, a, st, fp8);
+    case 96: return launch_attn_dh<96>(c, a, st, fp8);
+    case 128: return launch_attn_dh<128>(c, a, st, fp8);
     default: return FASTTPS_INVALID_ARG;
     }
 }

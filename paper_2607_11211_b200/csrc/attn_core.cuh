@@ -188,19 +188,19 @@ struct WalkSource {
     __device__ __forceinline__ bool next(Segment &s) { return walk.next(s); }
 };
 // Calls f(k_tile, v_tile, bytes_each) for every K/V tile of this CTA's share, in walk order; stops and
-// returns false as soon as f does.
-template <int DH, bool SHARE = false, class Src, class F>
+// returns false as soon as f does.  EB: bytes per cache element (2: bf16, 1: E4M3 codes); TR: rows per tile.
+template <int DH, bool SHARE = false, int EB = 2, int TR = kAttnTileRows, class Src, class F>
 __device__ __forceinline__ bool attn_for_each_tile(const AttnArgs &a, Src src, F f)
 {
     const int G = SHARE ? 1 : a.n_q_heads / a.n_kv_heads;
+    const unsigned char *kc = reinterpret_cast<const unsigned char *>(a.k_cache), *vc = reinterpret_cast<const unsigned char *>(a.v_cache);
     Segment sg;
     while (src.next(sg)) {
         const int c1 = sg.r1 < sg.L ? sg.r1 : sg.L;              // cached rows of the segment: [r0, c1)
         const size_t slab = ((size_t)(SHARE ? sg.b : sg.b / a.n_new) * a.n_kv_heads + sg.h / G) * (size_t)a.max_seq * DH;
-        for (int r = sg.r0; r < c1; r += kAttnTileRows) {
-            const int rows = (c1 - r) < kAttnTileRows ? (c1 - r) : kAttnTileRows;
-            if (!f(a.k_cache + slab + (size_t)r * DH, a.v_cache + slab + (size_t)r * DH,
-                   (uint32_t)rows * AttnTile<DH>::kRowBytes))
+        for (int r = sg.r0; r < c1; r += TR) {
+            const int rows = (c1 - r) < TR ? (c1 - r) : TR;
+            if (!f(kc + (slab + (size_t)r * DH) * EB, vc + (slab + (size_t)r * DH) * EB, (uint32_t)rows * DH * EB))
                 return false;
         }
     }
@@ -208,11 +208,11 @@ __device__ __forceinline__ bool attn_for_each_tile(const AttnArgs &a, Src src, F
 }
 
 // Producer thread: issues the K/V tiles of this CTA's share, in walk order, as ring pieces starting at `piece`.
-template <int DH, bool SHARE = false>
+template <int DH, bool SHARE = false, int EB = 2, int TR = kAttnTileRows>
 __device__ __forceinline__ bool attn_produce(const AttnArgs &a, WeightRing &ring, int &piece, int cta, int ncta)
 {
-    const bool done = attn_for_each_tile<DH, SHARE>(a, WalkSource(a, cta, ncta, SHARE), [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
-        if (!ring.put2(piece, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes)) return false;
+    const bool done = attn_for_each_tile<DH, SHARE, EB, TR>(a, WalkSource(a, cta, ncta, SHARE), [&](const unsigned char *k, const unsigned char *v, uint32_t bytes) {
+        if (!ring.put2(piece, k, v, bytes, TR * DH * EB)) return false;
         ++piece;
         return true;
     });

@@ -18,7 +18,13 @@
 // mantissa bits), so the result matches the FP32 path of attn_core.cuh to rounding and a layer built on it meets the
 // same bars.  Without it (option "gqa_share" 2) they are rounded to bf16 once: faster, but the deviation of a layer
 // output from the oracle was measured 4.5 times larger (rms 0.015 against 0.0034 on a Llama3-8B-shaped layer).
+// FP8: the cache holds E4M3 codes (one byte per element, value = code * scale with one scale per tensor).  A tile of
+// the ring then holds 128 rows (the same bytes as 64 bf16 rows); the codes are widened to fp16 in registers (exact:
+// every E4M3 value, subnormals included, is a normal fp16 number), the MMAs take fp16 operands, q and the softmax
+// weights go in as fp16 hi + lo pairs, and the two scales are applied to the scores and to the outputs once.
 #pragma once
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include "attn_core.cuh"
 #include "dot_core.cuh"
 
@@ -42,25 +48,60 @@ struct GroupScratch {
 // The MMAs of this path use rows 0..7 of the 16-row tile only (rows 8..15 of A are zero): the lower half of the
 // accumulator fragment is not kept (its inputs are constants, its outputs are dropped), which halves the
 // registers the running outputs take.
+template <bool F16 = false>
 __device__ __forceinline__ void mma_top_k16(float (&c)[2], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1)
 {
     float d2, d3;
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%5}, {%7,%8}, {%0,%1,%9,%9};"
-                 : "+f"(c[0]), "+f"(c[1]), "=f"(d2), "=f"(d3)
-                 : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1), "f"(0.f));
+    if constexpr (F16)
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%5}, {%7,%8}, {%0,%1,%9,%9};"
+                     : "+f"(c[0]), "+f"(c[1]), "=f"(d2), "=f"(d3)
+                     : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1), "f"(0.f));
+    else
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%5}, {%7,%8}, {%0,%1,%9,%9};"
+                     : "+f"(c[0]), "+f"(c[1]), "=f"(d2), "=f"(d3)
+                     : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1), "f"(0.f));
+}
+
+// two FP32 values as one register of two 16-bit floats (x in the low half), and what that rounding keeps of a value
+template <bool F16>
+__device__ __forceinline__ uint32_t pack2t(float x, float y)
+{
+    if constexpr (F16) {
+        const __half2 h = __floats2half2_rn(x, y);
+        return *reinterpret_cast<const uint32_t *>(&h);
+    } else {
+        return pack2(x, y);
+    }
+}
+template <bool F16>
+__device__ __forceinline__ float round16(float x)
+{
+    if constexpr (F16) return __half2float(__float2half_rn(x));
+    else return bf16_round(x);
+}
+// two E4M3 codes (the low 16 bits of c) as two fp16 numbers
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t c)
+{
+    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(c & 0xffffu), __NV_E4M3);
+    return (uint32_t)h.x | ((uint32_t)h.y << 16);
 }
 
 // Consumer warps (kGroupWarps of them, threads 0 .. 255, synchronised by named barrier 1).  The segments of
 // `src` are K/V heads (WalkSource with share = true).  Returns false in every thread if a bounded wait ran out.
-template <int DH, bool PRECISE>
+template <int DH, bool PRECISE, bool FP8 = false>
 __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing &ring, int &piece, int cta, WalkSource src,
                                                    GroupScratch<DH> &sm)
 {
+    static_assert(PRECISE || !FP8, "the E4M3 path always takes q and the weights as hi + lo pairs");
     constexpr int HALF = DH / 2;
     constexpr int KB = DH / 32;                  // 32-wide blocks of head_dim in the score product
     constexpr int JB = DH / 16;                  // 16-column blocks of the output
-    constexpr int kRowBytes = DH * 2;
+    constexpr int EB = FP8 ? 1 : 2;              // bytes per cache element
+    constexpr int TR = FP8 ? 2 * kAttnTileRows : kAttnTileRows;      // rows per tile of the ring
+    constexpr int kRowBytes = DH * EB;
     constexpr int kPartStride = DH + 4;
+    unsigned char *const kc8 = reinterpret_cast<unsigned char *>(a.k_cache), *const vc8 = reinterpret_cast<unsigned char *>(a.v_cache);
+    unsigned char *const knew8 = reinterpret_cast<unsigned char *>(&sm.knew[0][0]), *const vnew8 = reinterpret_cast<unsigned char *>(&sm.vnew[0][0]);
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5, g = lane >> 2, t4 = lane & 3;
     const int nct = kGroupWarps * 32;
     const int Gh = a.n_q_heads / a.n_kv_heads, N = a.n_new;
@@ -72,7 +113,9 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
     const bool wide = G > kHeadsPerWarp;
     const int gh = g + (wide ? kHeadsPerWarp * (warp >> 2) : 0);      // the member of the group in this lane's MMA row
     const int my_tok = gh / Gh;                                       // its token: it sees the new rows 0 .. my_tok
-    const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
+    // scores in the log2 domain; with E4M3 codes the products are in units of the scales
+    const float scale_log2 = (FP8 ? a.k_scale : 1.f) * (1.4426950408889634f / sqrtf((float)DH));
+    const float out_scale = FP8 ? a.v_scale : 1.f;
     bool ok = true;
 
     Segment sg;
@@ -94,20 +137,29 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             if (g2 == 0 && has_new) {
                 const __nv_bfloat16 *kg = a.k_new + row * a.kv_stride + (size_t)hk * DH;
                 const float k0 = __bfloat162float(ld_cg_bf16(kg + i)), k1 = __bfloat162float(ld_cg_bf16(kg + i + HALF));
-                sm.knew[j][i] = __float2bfloat16_rn(__fsub_rn(__fmul_rn(k0, c), __fmul_rn(k1, sn)));
-                sm.knew[j][i + HALF] = __float2bfloat16_rn(__fadd_rn(__fmul_rn(k1, c), __fmul_rn(k0, sn)));
+                const float r0 = __fsub_rn(__fmul_rn(k0, c), __fmul_rn(k1, sn)), r1 = __fadd_rn(__fmul_rn(k1, c), __fmul_rn(k0, sn));
                 const __nv_bfloat16 *vg = a.v_new + row * a.kv_stride + (size_t)hk * DH;
-                sm.vnew[j][i] = ld_cg_bf16(vg + i);
-                sm.vnew[j][i + HALF] = ld_cg_bf16(vg + i + HALF);
+                if constexpr (FP8) {
+                    // the codes that go into the cache: value / scale, nearest code (ties to even), saturating at 448
+                    knew8[j * DH + i] = __nv_cvt_float_to_fp8(__fdiv_rn(r0, a.k_scale), __NV_SATFINITE, __NV_E4M3);
+                    knew8[j * DH + i + HALF] = __nv_cvt_float_to_fp8(__fdiv_rn(r1, a.k_scale), __NV_SATFINITE, __NV_E4M3);
+                    vnew8[j * DH + i] = __nv_cvt_float_to_fp8(__fdiv_rn(__bfloat162float(ld_cg_bf16(vg + i)), a.v_scale), __NV_SATFINITE, __NV_E4M3);
+                    vnew8[j * DH + i + HALF] = __nv_cvt_float_to_fp8(__fdiv_rn(__bfloat162float(ld_cg_bf16(vg + i + HALF)), a.v_scale), __NV_SATFINITE, __NV_E4M3);
+                } else {
+                    sm.knew[j][i] = __float2bfloat16_rn(r0);
+                    sm.knew[j][i + HALF] = __float2bfloat16_rn(r1);
+                    sm.vnew[j][i] = ld_cg_bf16(vg + i);
+                    sm.vnew[j][i + HALF] = ld_cg_bf16(vg + i + HALF);
+                }
             }
         }
         named_bar_sync(1, nct);
         // ---- GKVC append (Eq. 2; Algorithm 3 steps 1 and 9): one write per row, no reload ----
         if (has_new) {
             // the N new rows are consecutive in the cache (rows L .. L + N - 1) and in shared memory
-            for (int i = t; i < N * (DH / 8); i += nct) {
-                reinterpret_cast<uint4 *>(a.k_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(&sm.knew[0][0])[i];
-                reinterpret_cast<uint4 *>(a.v_cache + slab + (size_t)L * DH)[i] = reinterpret_cast<const uint4 *>(&sm.vnew[0][0])[i];
+            for (int i = t; i < N * (kRowBytes / 16); i += nct) {
+                reinterpret_cast<uint4 *>(kc8 + (slab + (size_t)L * DH) * EB)[i] = reinterpret_cast<const uint4 *>(knew8)[i];
+                reinterpret_cast<uint4 *>(vc8 + (slab + (size_t)L * DH) * EB)[i] = reinterpret_cast<const uint4 *>(vnew8)[i];
             }
             asm volatile("fence.proxy.async;" ::: "memory");
         }
@@ -125,11 +177,11 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
 #pragma unroll
                 for (int i = 0; i < 8; ++i) f[i] = 0.f;
             }
-            qhi[kb] = make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+            qhi[kb] = make_uint4(pack2t<FP8>(f[0], f[1]), pack2t<FP8>(f[2], f[3]), pack2t<FP8>(f[4], f[5]), pack2t<FP8>(f[6], f[7]));
             if constexpr (PRECISE) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) f[i] -= bf16_round(f[i]);          // what the rounding left out
-                qlo[kb] = make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+                for (int i = 0; i < 8; ++i) f[i] -= round16<FP8>(f[i]);          // what the rounding left out
+                qlo[kb] = make_uint4(pack2t<FP8>(f[0], f[1]), pack2t<FP8>(f[2], f[3]), pack2t<FP8>(f[4], f[5]), pack2t<FP8>(f[6], f[7]));
             }
         }
         float m_run = -INFINITY, l_run = 0.f;      // of head g; the sum holds this lane's keys only until the end
@@ -156,12 +208,18 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             for (int kb = 0; kb < KB; ++kb) {
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    const uint4 kv = *reinterpret_cast<const uint4 *>(kt + (size_t)(u ? kr1 : kr0) * kRowBytes + kb * 64 + t4 * 16);
-                    mma_top_k16(sc[u][0], qhi[kb].x, qhi[kb].y, kv.x, kv.y);
-                    mma_top_k16(sc[u][1], qhi[kb].z, qhi[kb].w, kv.z, kv.w);
+                    uint4 kv;
+                    if constexpr (FP8) {
+                        const uint2 c8 = *reinterpret_cast<const uint2 *>(kt + (size_t)(u ? kr1 : kr0) * kRowBytes + kb * 32 + t4 * 8);
+                        kv = make_uint4(e4m3x2_to_f16x2(c8.x), e4m3x2_to_f16x2(c8.x >> 16), e4m3x2_to_f16x2(c8.y), e4m3x2_to_f16x2(c8.y >> 16));
+                    } else {
+                        kv = *reinterpret_cast<const uint4 *>(kt + (size_t)(u ? kr1 : kr0) * kRowBytes + kb * 64 + t4 * 16);
+                    }
+                    mma_top_k16<FP8>(sc[u][0], qhi[kb].x, qhi[kb].y, kv.x, kv.y);
+                    mma_top_k16<FP8>(sc[u][1], qhi[kb].z, qhi[kb].w, kv.z, kv.w);
                     if constexpr (PRECISE) {
-                        mma_top_k16(sc[u][0], qlo[kb].x, qlo[kb].y, kv.x, kv.y);
-                        mma_top_k16(sc[u][1], qlo[kb].z, qlo[kb].w, kv.z, kv.w);
+                        mma_top_k16<FP8>(sc[u][0], qlo[kb].x, qlo[kb].y, kv.x, kv.y);
+                        mma_top_k16<FP8>(sc[u][1], qlo[kb].z, qlo[kb].w, kv.z, kv.w);
                     }
                 }
             }
@@ -187,13 +245,13 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             float pr[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) pr[e] = see[e] ? fast_exp2(s[e] - m_new) : 0.f;
-            const uint32_t pa0 = pack2(pr[0], pr[1]), pa1 = pack2(pr[2], pr[3]);
+            const uint32_t pa0 = pack2t<FP8>(pr[0], pr[1]), pa1 = pack2t<FP8>(pr[2], pr[3]);
             uint32_t pl0 = 0u, pl1 = 0u;
             if constexpr (PRECISE) {
                 // the weights go in as hi + lo: the row sum is the sum of the weights themselves
                 l_run = l_run * corr + ((pr[0] + pr[1]) + (pr[2] + pr[3]));
-                pl0 = pack2(pr[0] - bf16_round(pr[0]), pr[1] - bf16_round(pr[1]));
-                pl1 = pack2(pr[2] - bf16_round(pr[2]), pr[3] - bf16_round(pr[3]));
+                pl0 = pack2t<FP8>(pr[0] - round16<FP8>(pr[0]), pr[1] - round16<FP8>(pr[1]));
+                pl1 = pack2t<FP8>(pr[2] - round16<FP8>(pr[2]), pr[3] - round16<FP8>(pr[3]));
             } else {
                 l_run = l_run * corr + ((bf16_round(pr[0]) + bf16_round(pr[1])) + (bf16_round(pr[2]) + bf16_round(pr[3])));
             }
@@ -201,7 +259,7 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             // ---- PV (step 12): B operands from four rows of V, two column sets per pair of 32-bit words ----
             const unsigned char *vp[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) vp[e] = vt + (size_t)(ka[e] < rows ? ka[e] : rows - 1) * kRowBytes + g * 4;
+            for (int e = 0; e < 4; ++e) vp[e] = vt + (size_t)(ka[e] < rows ? ka[e] : rows - 1) * kRowBytes + g * 2 * EB;
             // the running maximum seldom moves after the first tiles: the rescaling is skipped when no lane needs it
             if (__any_sync(kFull, corr != 1.f)) {
 #pragma unroll
@@ -209,33 +267,50 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             }
 #pragma unroll
             for (int jb = 0; jb < JB; ++jb) {
-                const uint32_t w0 = *reinterpret_cast<const uint32_t *>(vp[0] + jb * 32);
-                const uint32_t w1 = *reinterpret_cast<const uint32_t *>(vp[1] + jb * 32);
-                const uint32_t w2 = *reinterpret_cast<const uint32_t *>(vp[2] + jb * 32);
-                const uint32_t w3 = *reinterpret_cast<const uint32_t *>(vp[3] + jb * 32);
+                uint32_t w0, w1, w2, w3;            // columns 16 jb + 2 g (+1) of the four rows, as 16-bit floats
+                if constexpr (FP8) {
+                    w0 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[0] + jb * 16));
+                    w1 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[1] + jb * 16));
+                    w2 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[2] + jb * 16));
+                    w3 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[3] + jb * 16));
+                } else {
+                    w0 = *reinterpret_cast<const uint32_t *>(vp[0] + jb * 32);
+                    w1 = *reinterpret_cast<const uint32_t *>(vp[1] + jb * 32);
+                    w2 = *reinterpret_cast<const uint32_t *>(vp[2] + jb * 32);
+                    w3 = *reinterpret_cast<const uint32_t *>(vp[3] + jb * 32);
+                }
                 const uint32_t be0 = __byte_perm(w0, w1, 0x5410), be1 = __byte_perm(w2, w3, 0x5410);
                 const uint32_t bo0 = __byte_perm(w0, w1, 0x7632), bo1 = __byte_perm(w2, w3, 0x7632);
-                mma_top_k16(oa[jb], pa0, pa1, be0, be1);    // columns 16 jb + 2 g
-                mma_top_k16(ob[jb], pa0, pa1, bo0, bo1);    // columns 16 jb + 2 g + 1
+                mma_top_k16<FP8>(oa[jb], pa0, pa1, be0, be1);    // columns 16 jb + 2 g
+                mma_top_k16<FP8>(ob[jb], pa0, pa1, bo0, bo1);    // columns 16 jb + 2 g + 1
                 if constexpr (PRECISE) {
-                    mma_top_k16(oa[jb], pl0, pl1, be0, be1);
-                    mma_top_k16(ob[jb], pl0, pl1, bo0, bo1);
+                    mma_top_k16<FP8>(oa[jb], pl0, pl1, be0, be1);
+                    mma_top_k16<FP8>(ob[jb], pl0, pl1, bo0, bo1);
                 }
             }
         };
 
         // ---- stream the cached rows of the segment: warps 0-3 take the even pieces, warps 4-7 the odd ones, 16 rows
         //      of the tile each; every warp waits for and releases every piece (the ring protocol) ----
-        for (int r = sg.r0; r < c1; r += kAttnTileRows, ++piece) {
+        for (int r = sg.r0; r < c1; r += TR, ++piece) {
             const unsigned char *slot = ring.wait(piece, ok);
-            const int rows = (c1 - r) < kAttnTileRows ? (c1 - r) : kAttnTileRows;
-            if (ok && (wide || (piece & 1) == (warp >> 2)) && (warp & 3) * 16 < rows)
-                block(slot, slot + kAttnTileRows * kRowBytes, (warp & 3) * 16, rows);
+            const int rows = (c1 - r) < TR ? (c1 - r) : TR;
+            if constexpr (FP8) {
+                // 128 rows per piece: every warp 16 of them (small groups), or 32 per warp of either set (large groups)
+                if (ok && !wide && warp * 16 < rows) block(slot, slot + TR * kRowBytes, warp * 16, rows);
+                if (ok && wide) {
+                    if ((warp & 3) * 16 < rows) block(slot, slot + TR * kRowBytes, (warp & 3) * 16, rows);
+                    if (64 + (warp & 3) * 16 < rows) block(slot, slot + TR * kRowBytes, 64 + (warp & 3) * 16, rows);
+                }
+            } else {
+                if (ok && (wide || (piece & 1) == (warp >> 2)) && (warp & 3) * 16 < rows)
+                    block(slot, slot + TR * kRowBytes, (warp & 3) * 16, rows);
+            }
             ring.release(piece);
         }
         // ---- the new row, straight from shared memory (never re-read from the cache) ----
         if (has_new && (warp == 0 || (wide && warp == 4)))
-            block(reinterpret_cast<const unsigned char *>(&sm.knew[0][0]), reinterpret_cast<const unsigned char *>(&sm.vnew[0][0]), 0, N, N > 1);
+            block(knew8, vnew8, 0, N, N > 1);
 
         // ---- the warps' states meet in shared memory ----
         l_run += __shfl_xor_sync(kFull, l_run, 1);
@@ -243,7 +318,8 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
         if (gh < G) {
 #pragma unroll
             for (int jb = 0; jb < JB; ++jb)
-                *reinterpret_cast<float4 *>(&sm.wo[warp][g][16 * jb + 4 * t4]) = make_float4(oa[jb][0], ob[jb][0], oa[jb][1], ob[jb][1]);
+                *reinterpret_cast<float4 *>(&sm.wo[warp][g][16 * jb + 4 * t4]) =
+                    make_float4(oa[jb][0] * out_scale, ob[jb][0] * out_scale, oa[jb][1] * out_scale, ob[jb][1] * out_scale);
             if (t4 == 0) { sm.wm[warp][g] = m_run; sm.wl[warp][g] = l_run; }
         }
         if (!named_bar_and(1, nct, ok)) return false;

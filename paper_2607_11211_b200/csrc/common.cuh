@@ -284,6 +284,7 @@ struct AttnArgs {
     float *part;
     int *ticket;
     uint32_t *status;
+    float k_scale, v_scale;           // E4M3 caches only (k_cache / v_cache then point at bytes): value = code * scale
 };
 
 struct MlpArgs {
@@ -393,7 +394,7 @@ int launch_linear(Ctx *c, const LinearArgs &a, cudaStream_t st);
 bool step_kernel_supported(const Ctx *c, int batch, bool layer_mode = false);
 int launch_step(Ctx *c, const StepArgs &a, cudaStream_t st);
 int launch_layer_step(Ctx *c, const StepArgs &a, cudaStream_t st);
-int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st);
+int launch_attn(Ctx *c, const AttnArgs &a, cudaStream_t st, bool fp8 = false);
 int launch_mlp(Ctx *c, const MlpArgs &a, cudaStream_t st);
 int launch_embed(Ctx *c, const __nv_bfloat16 *embed, const int32_t *ids, __nv_bfloat16 *x, int batch, cudaStream_t st);
 int launch_pack(Ctx *c, int kind, const void *src, void *dst, bool inverse, cudaStream_t st);

@@ -104,7 +104,7 @@ static __device__ __forceinline__ AttnArgs attn_args_of(const StepArgs &a, const
     aa.pos = a.pos; aa.seq_lens = a.seq_lens;
     aa.out = a.attn_out; aa.out_stride = nq; aa.out_chunked = 0;
     aa.batch = a.batch; aa.n_q_heads = a.n_q_heads; aa.n_kv_heads = a.n_kv_heads;
-    aa.head_dim = a.head_dim; aa.max_seq = a.max_seq; aa.n_splits = ncta_attn; aa.len_add = step; aa.n_new = 1;
+    aa.head_dim = a.head_dim; aa.max_seq = a.max_seq; aa.n_splits = ncta_attn; aa.len_add = step; aa.n_new = 1; aa.k_scale = aa.v_scale = 1.f;
     aa.cos_tab = a.cos_tab; aa.sin_tab = a.sin_tab;
     aa.part = a.attn_part; aa.ticket = a.attn_ticket; aa.status = a.status;
     return aa;

@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(const _
                     const AttnArgs aa = attn_args_of(a, lp, step, gm * a.n_q_heads);
                     const unsigned char *wo = reinterpret_cast<const unsigned char *>(lp.w_o);
                     const bool kv_ok = attn_for_each_tile<DH>(aa, GroupSource(&s_segs),
-                                                              [&](const __nv_bfloat16 *k, const __nv_bfloat16 *v, uint32_t bytes) {
+                                                              [&](const unsigned char *k, const unsigned char *v, uint32_t bytes) {
                         if (!ring.put2(piece, k, v, bytes, kAttnTileRows * AttnTile<DH>::kRowBytes)) return false;
                         ++piece;
                         return true;

@@ -176,6 +176,16 @@ def kv_cache(dims: Dims, layer: int, batch: int, max_seq: int, seed: int = MASTE
             normal_bf16(seed, tid("v_cache", layer), shp, 1.0, 0.0, device))
 
 
+def kv_cache_e4m3(dims: Dims, layer: int, batch: int, max_seq: int, k_scale: float, v_scale: float,
+                  seed: int = MASTER_SEED, device="cpu"):
+    """The same N(0,1) caches stored as 8-bit E4M3 codes (uint8 tensors [B,Hkv,max_seq,d]) of value / scale; the
+    conversion is the library's (round to nearest even; the values are clamped to the format's range first)."""
+    out = []
+    for t, s in zip(kv_cache(dims, layer, batch, max_seq, seed, device), (k_scale, v_scale)):
+        out.append((t.float() / s).clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8))
+    return tuple(out)
+
+
 def activations(dims: Dims, batch: int, seed: int = MASTER_SEED, device="cpu") -> dict:
     """Block-level inputs: x [B,D], q [B,Hq,d], k_new/v_new [B,Hkv,d] ~ N(0,1)."""
     d = dims.head_dim

@@ -1,0 +1,82 @@
+"""Algorithm 3 over a KV cache of 8-bit E4M3 codes (the quantised cache of Section 6.2): the CUDA path against the
+oracle.  The appended codes are an integer decision taken in FP32 on both sides (rotation, division by the scale,
+nearest code): they are compared bit for bit, like every byte the step must not touch."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2607_11211_b200 import workload as wl
+from tests.helpers import assert_close_bits
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fb():
+    from paper_2607_11211_b200 import binding, build
+    build.build()
+    return binding
+
+
+def i32(a):
+    return torch.tensor(np.asarray(a, dtype=np.int32), device="cuda")
+
+
+def run_case(fb, dims, lens, max_seq, k_scale, v_scale, pos=None, seed=5):
+    B = len(lens)
+    lens = np.asarray(lens, np.int32)
+    pos = lens if pos is None else np.asarray(pos, np.int32)
+    ctx = fb.Context.from_dims(dims, B, max_seq)
+    act = wl.activations(dims, B, seed=seed, device="cuda")
+    kc, vc = wl.kv_cache_e4m3(dims, 0, B, max_seq, k_scale, v_scale, seed=seed, device="cuda")
+    k0, v0 = kc.cpu().numpy().copy(), vc.cpu().numpy().copy()
+    out = torch.zeros(B, dims.n_q_heads, dims.head_dim, dtype=torch.bfloat16, device="cuda")
+    ctx.attn_decode_fp8(act["q"], act["k_new"], act["v_new"], kc, vc, k_scale, v_scale, i32(pos), i32(lens), out)
+    torch.cuda.synchronize()
+    status = ctx.get_status()
+    ko, vo = k0.copy(), v0.copy()
+    want = orc.attn_decode_fp8(wl.bits(act["q"]), wl.bits(act["k_new"]), wl.bits(act["v_new"]), ko, vo, k_scale, v_scale,
+                               pos, lens, dims.rope_theta)
+    ctx.close()
+    return wl.bits(out), want, kc.cpu().numpy(), vc.cpu().numpy(), ko, vo, k0, v0, status
+
+
+@pytest.mark.parametrize("dims,lens,max_seq", [
+    (wl.TINY, [0], 64), (wl.TINY, [5, 64, 17, 129], 256), (wl.SMALL, [100, 3, 255], 256), (wl.SMALL_GQA, [9, 200, 31], 256),
+    (wl.PHI3_MINI, [1000, 17], 1024), (wl.PHI3_MINI, [4095], 4096), (wl.TABLE1["llama3-8b"], [777, 128, 2047], 2048),
+    (wl.TABLE1["chatglm3-6b"], [300, 1500], 2048), (wl.TABLE1["llama3.2-1b"], [127, 128, 129, 1], 512)])
+def test_attn_decode_fp8_matches_oracle(fb, dims, lens, max_seq):
+    k_scale, v_scale = 0.0625 * 1.3, 0.05
+    got, want, kg, vg, ko, vo, k0, v0, status = run_case(fb, dims, lens, max_seq, k_scale, v_scale)
+    assert status == 0
+    assert_close_bits(got, want, what="attention over an E4M3 cache")
+    # the whole cache, byte for byte: the appended codes and every byte that must stay as it was
+    assert (kg == ko).all() and (vg == vo).all()
+    changed = (kg != k0) | (vg != v0)
+    for b, L in enumerate(lens):
+        changed[b, :, L] = False
+    assert not changed.any()
+
+
+def test_attn_decode_fp8_saturates_and_reports_a_full_cache(fb):
+    dims, max_seq = wl.SMALL, 64
+    lens = [64, 10]                                             # sequence 0 has no room
+    got, want, kg, vg, ko, vo, k0, v0, status = run_case(fb, dims, lens, max_seq, 1e-4, 2e-4, pos=[3, 10])
+    assert status & fb.DEV_CACHE_FULL
+    assert (kg == ko).all() and (vg == vo).all() and (kg[0] == k0[0]).all()
+    new = kg[1, :, 10] & 0x7f
+    assert (new == 0x7e).mean() > 0.9                           # scales far too small: nearly every new code is +-448
+    assert_close_bits(got[1:], want[1:], what="attention over a saturated E4M3 cache")
+
+
+def test_attn_decode_fp8_rejects_bad_scales_and_groups(fb):
+    dims = wl.SMALL
+    ctx = fb.Context.from_dims(dims, 1, 64)
+    act = wl.activations(dims, 1, device="cuda")
+    kc, vc = wl.kv_cache_e4m3(dims, 0, 1, 64, 1.0, 1.0, device="cuda")
+    out = torch.zeros(1, dims.n_q_heads, dims.head_dim, dtype=torch.bfloat16, device="cuda")
+    for ks, vs in ((0.0, 1.0), (1.0, -2.0), (float("nan"), 1.0), (1.0, float("inf"))):
+        with pytest.raises(fb.FasttpsError):
+            ctx.attn_decode_fp8(act["q"], act["k_new"], act["v_new"], kc, vc, ks, vs, i32([0]), i32([0]), out)
+    ctx.close()
