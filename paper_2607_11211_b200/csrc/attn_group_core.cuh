@@ -206,20 +206,27 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 for (int c = 0; c < 2; ++c) sc[u][c][0] = sc[u][c][1] = 0.f;
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
+                uint4 kv[2];
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    uint4 kv;
                     if constexpr (FP8) {
                         const uint2 c8 = *reinterpret_cast<const uint2 *>(kt + (size_t)(u ? kr1 : kr0) * kRowBytes + kb * 32 + t4 * 8);
-                        kv = make_uint4(e4m3x2_to_f16x2(c8.x), e4m3x2_to_f16x2(c8.x >> 16), e4m3x2_to_f16x2(c8.y), e4m3x2_to_f16x2(c8.y >> 16));
+                        kv[u] = make_uint4(e4m3x2_to_f16x2(c8.x), e4m3x2_to_f16x2(c8.x >> 16), e4m3x2_to_f16x2(c8.y), e4m3x2_to_f16x2(c8.y >> 16));
                     } else {
-                        kv = *reinterpret_cast<const uint4 *>(kt + (size_t)(u ? kr1 : kr0) * kRowBytes + kb * 64 + t4 * 16);
+                        kv[u] = *reinterpret_cast<const uint4 *>(kt + (size_t)(u ? kr1 : kr0) * kRowBytes + kb * 64 + t4 * 16);
                     }
-                    mma_top_k16<FP8>(sc[u][0], qhi[kb].x, qhi[kb].y, kv.x, kv.y);
-                    mma_top_k16<FP8>(sc[u][1], qhi[kb].z, qhi[kb].w, kv.z, kv.w);
-                    if constexpr (PRECISE) {
-                        mma_top_k16<FP8>(sc[u][0], qlo[kb].x, qlo[kb].y, kv.x, kv.y);
-                        mma_top_k16<FP8>(sc[u][1], qlo[kb].z, qlo[kb].w, kv.z, kv.w);
+                }
+                // four accumulators: a product never follows the one it depends on by less than four instructions
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    mma_top_k16<FP8>(sc[u][0], qhi[kb].x, qhi[kb].y, kv[u].x, kv[u].y);
+                    mma_top_k16<FP8>(sc[u][1], qhi[kb].z, qhi[kb].w, kv[u].z, kv[u].w);
+                }
+                if constexpr (PRECISE) {
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        mma_top_k16<FP8>(sc[u][0], qlo[kb].x, qlo[kb].y, kv[u].x, kv[u].y);
+                        mma_top_k16<FP8>(sc[u][1], qlo[kb].z, qlo[kb].w, kv[u].z, kv[u].w);
                     }
                 }
             }
@@ -265,27 +272,39 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
 #pragma unroll
                 for (int jb = 0; jb < JB; ++jb) { oa[jb][0] *= corr; oa[jb][1] *= corr; ob[jb][0] *= corr; ob[jb][1] *= corr; }
             }
+            // two column blocks at a time: their loads go first, and the hi and lo products of an accumulator are
+            // four instructions apart
 #pragma unroll
-            for (int jb = 0; jb < JB; ++jb) {
-                uint32_t w0, w1, w2, w3;            // columns 16 jb + 2 g (+1) of the four rows, as 16-bit floats
-                if constexpr (FP8) {
-                    w0 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[0] + jb * 16));
-                    w1 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[1] + jb * 16));
-                    w2 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[2] + jb * 16));
-                    w3 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[3] + jb * 16));
-                } else {
-                    w0 = *reinterpret_cast<const uint32_t *>(vp[0] + jb * 32);
-                    w1 = *reinterpret_cast<const uint32_t *>(vp[1] + jb * 32);
-                    w2 = *reinterpret_cast<const uint32_t *>(vp[2] + jb * 32);
-                    w3 = *reinterpret_cast<const uint32_t *>(vp[3] + jb * 32);
+            for (int jb = 0; jb < JB; jb += 2) {
+                uint32_t be0[2], be1[2], bo0[2], bo1[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t w0, w1, w2, w3;            // columns 16 (jb + h) + 2 g (+1) of the four rows, as 16-bit floats
+                    if constexpr (FP8) {
+                        w0 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[0] + (jb + h) * 16));
+                        w1 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[1] + (jb + h) * 16));
+                        w2 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[2] + (jb + h) * 16));
+                        w3 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[3] + (jb + h) * 16));
+                    } else {
+                        w0 = *reinterpret_cast<const uint32_t *>(vp[0] + (jb + h) * 32);
+                        w1 = *reinterpret_cast<const uint32_t *>(vp[1] + (jb + h) * 32);
+                        w2 = *reinterpret_cast<const uint32_t *>(vp[2] + (jb + h) * 32);
+                        w3 = *reinterpret_cast<const uint32_t *>(vp[3] + (jb + h) * 32);
+                    }
+                    be0[h] = __byte_perm(w0, w1, 0x5410); be1[h] = __byte_perm(w2, w3, 0x5410);
+                    bo0[h] = __byte_perm(w0, w1, 0x7632); bo1[h] = __byte_perm(w2, w3, 0x7632);
                 }
-                const uint32_t be0 = __byte_perm(w0, w1, 0x5410), be1 = __byte_perm(w2, w3, 0x5410);
-                const uint32_t bo0 = __byte_perm(w0, w1, 0x7632), bo1 = __byte_perm(w2, w3, 0x7632);
-                mma_top_k16<FP8>(oa[jb], pa0, pa1, be0, be1);    // columns 16 jb + 2 g
-                mma_top_k16<FP8>(ob[jb], pa0, pa1, bo0, bo1);    // columns 16 jb + 2 g + 1
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    mma_top_k16<FP8>(oa[jb + h], pa0, pa1, be0[h], be1[h]);    // columns 16 jb + 2 g
+                    mma_top_k16<FP8>(ob[jb + h], pa0, pa1, bo0[h], bo1[h]);    // columns 16 jb + 2 g + 1
+                }
                 if constexpr (PRECISE) {
-                    mma_top_k16<FP8>(oa[jb], pl0, pl1, be0, be1);
-                    mma_top_k16<FP8>(ob[jb], pl0, pl1, bo0, bo1);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        mma_top_k16<FP8>(oa[jb + h], pl0, pl1, be0[h], be1[h]);
+                        mma_top_k16<FP8>(ob[jb + h], pl0, pl1, bo0[h], bo1[h]);
+                    }
                 }
             }
         };
