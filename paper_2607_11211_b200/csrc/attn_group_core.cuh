@@ -62,6 +62,18 @@ __device__ __forceinline__ void mma_top_k16(float (&c)[2], uint32_t a0, uint32_t
                      : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1), "f"(0.f));
 }
 
+// the whole 16-row product (the output product: rows = 16 output columns, n = 8 members, k = 16 keys)
+template <bool F16 = false>
+__device__ __forceinline__ void mma_k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    if constexpr (F16)
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 // two FP32 values as one register of two 16-bit floats (x in the low half), and what that rounding keeps of a value
 template <bool F16>
 __device__ __forceinline__ uint32_t pack2t(float x, float y)
@@ -95,7 +107,7 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
     static_assert(PRECISE || !FP8, "the E4M3 path always takes q and the weights as hi + lo pairs");
     constexpr int HALF = DH / 2;
     constexpr int KB = DH / 32;                  // 32-wide blocks of head_dim in the score product
-    constexpr int JB = DH / 16;                  // 16-column blocks of the output
+    constexpr int CB = DH / 32;                  // 32-column blocks of the output
     constexpr int EB = FP8 ? 1 : 2;              // bytes per cache element
     constexpr int TR = FP8 ? 2 * kAttnTileRows : kAttnTileRows;      // rows per tile of the ring
     constexpr int kRowBytes = DH * EB;
@@ -185,11 +197,15 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             }
         }
         float m_run = -INFINITY, l_run = 0.f;      // of head g; the sum holds this lane's keys only until the end
-        float oa[JB][2], ob[JB][2];                // output fragments of head g: columns 16 jb + 4 t4 + {0, 2} (oa) / {1, 3} (ob)
+        // output fragments, TRANSPOSED (rows of the product = output columns, n = members): acc[cb][m][i] belongs to
+        // column 32 cb + 4 g + 2 m + (i >> 1) and member 2 t4 + (i & 1)
+        float acc[CB][2][4];
 #pragma unroll
-        for (int jb = 0; jb < JB; ++jb)
+        for (int cb = 0; cb < CB; ++cb)
 #pragma unroll
-            for (int e = 0; e < 2; ++e) oa[jb][e] = ob[jb][e] = 0.f;
+            for (int m = 0; m < 2; ++m)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[cb][m][i] = 0.f;
 
         // One block of up to 16 keys: rows key0 .. key0 + 15 of the K tile `kt` / V tile `vt`, of which the rows below
         // `rows` exist.  Rows that do not exist are read from the last one that does (finite data) and get weight 0.
@@ -263,48 +279,68 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 l_run = l_run * corr + ((bf16_round(pr[0]) + bf16_round(pr[1])) + (bf16_round(pr[2]) + bf16_round(pr[3])));
             }
             m_run = m_new;
-            // ---- PV (step 12): B operands from four rows of V, two column sets per pair of 32-bit words ----
+            // ---- PV (step 12), transposed: O^T[column, member] += V^T[column, key] P^T[key, member].  The weights are
+            //      the B operand exactly as the score fragments hold them (keys 2 t4 (+1) and 8 + 2 t4 (+1) of member g);
+            //      V^T comes from four rows of V: four consecutive columns per lane and row, the same column of two
+            //      keys paired by a byte permute.  All 16 rows of the product carry output columns. ----
             const unsigned char *vp[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) vp[e] = vt + (size_t)(ka[e] < rows ? ka[e] : rows - 1) * kRowBytes + g * 2 * EB;
+            for (int e = 0; e < 4; ++e) vp[e] = vt + (size_t)(ka[e] < rows ? ka[e] : rows - 1) * kRowBytes + g * 4 * EB;
             // the running maximum seldom moves after the first tiles: the rescaling is skipped when no lane needs it
             if (__any_sync(kFull, corr != 1.f)) {
+                const float c0 = __shfl_sync(kFull, corr, 8 * t4), c1 = __shfl_sync(kFull, corr, 8 * t4 + 4);     // members 2 t4, 2 t4 + 1
 #pragma unroll
-                for (int jb = 0; jb < JB; ++jb) { oa[jb][0] *= corr; oa[jb][1] *= corr; ob[jb][0] *= corr; ob[jb][1] *= corr; }
+                for (int cb = 0; cb < CB; ++cb)
+#pragma unroll
+                    for (int m = 0; m < 2; ++m) { acc[cb][m][0] *= c0; acc[cb][m][1] *= c1; acc[cb][m][2] *= c0; acc[cb][m][3] *= c1; }
             }
-            // two column blocks at a time: their loads go first, and the hi and lo products of an accumulator are
-            // four instructions apart
+            // two column blocks at a time: loads first, then the products; the hi and lo product of an accumulator
+            // are at least two (mostly four) instructions apart
 #pragma unroll
-            for (int jb = 0; jb < JB; jb += 2) {
-                uint32_t be0[2], be1[2], bo0[2], bo1[2];
+            for (int cb0 = 0; cb0 < CB; cb0 += 2) {
+                constexpr int kPair = 2;
+                uint32_t av[kPair][2][4];          // [block][column pair m][a0..a3]
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t w0, w1, w2, w3;            // columns 16 (jb + h) + 2 g (+1) of the four rows, as 16-bit floats
-                    if constexpr (FP8) {
-                        w0 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[0] + (jb + h) * 16));
-                        w1 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[1] + (jb + h) * 16));
-                        w2 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[2] + (jb + h) * 16));
-                        w3 = e4m3x2_to_f16x2(*reinterpret_cast<const uint16_t *>(vp[3] + (jb + h) * 16));
-                    } else {
-                        w0 = *reinterpret_cast<const uint32_t *>(vp[0] + (jb + h) * 32);
-                        w1 = *reinterpret_cast<const uint32_t *>(vp[1] + (jb + h) * 32);
-                        w2 = *reinterpret_cast<const uint32_t *>(vp[2] + (jb + h) * 32);
-                        w3 = *reinterpret_cast<const uint32_t *>(vp[3] + (jb + h) * 32);
+                for (int h = 0; h < kPair; ++h) {
+                    if (cb0 + h < CB) {
+                        const int cb = cb0 + h;
+                        if constexpr (FP8) {
+                            uint32_t x[4];             // codes of columns 32 cb + 4 g .. + 3 of the four rows
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) x[e] = *reinterpret_cast<const uint32_t *>(vp[e] + cb * 32);
+#pragma unroll
+                            for (int m = 0; m < 2; ++m) {
+                                av[h][m][0] = e4m3x2_to_f16x2(__byte_perm(x[0], x[1], m ? 0x0062 : 0x0040));
+                                av[h][m][1] = e4m3x2_to_f16x2(__byte_perm(x[0], x[1], m ? 0x0073 : 0x0051));
+                                av[h][m][2] = e4m3x2_to_f16x2(__byte_perm(x[2], x[3], m ? 0x0062 : 0x0040));
+                                av[h][m][3] = e4m3x2_to_f16x2(__byte_perm(x[2], x[3], m ? 0x0073 : 0x0051));
+                            }
+                        } else {
+                            uint2 x[4];                // columns 32 cb + 4 g .. + 3 of the four rows
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) x[e] = *reinterpret_cast<const uint2 *>(vp[e] + cb * 64);
+                            av[h][0][0] = __byte_perm(x[0].x, x[1].x, 0x5410); av[h][0][1] = __byte_perm(x[0].x, x[1].x, 0x7632);
+                            av[h][0][2] = __byte_perm(x[2].x, x[3].x, 0x5410); av[h][0][3] = __byte_perm(x[2].x, x[3].x, 0x7632);
+                            av[h][1][0] = __byte_perm(x[0].y, x[1].y, 0x5410); av[h][1][1] = __byte_perm(x[0].y, x[1].y, 0x7632);
+                            av[h][1][2] = __byte_perm(x[2].y, x[3].y, 0x5410); av[h][1][3] = __byte_perm(x[2].y, x[3].y, 0x7632);
+                        }
                     }
-                    be0[h] = __byte_perm(w0, w1, 0x5410); be1[h] = __byte_perm(w2, w3, 0x5410);
-                    bo0[h] = __byte_perm(w0, w1, 0x7632); bo1[h] = __byte_perm(w2, w3, 0x7632);
                 }
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    mma_top_k16<FP8>(oa[jb + h], pa0, pa1, be0[h], be1[h]);    // columns 16 jb + 2 g
-                    mma_top_k16<FP8>(ob[jb + h], pa0, pa1, bo0[h], bo1[h]);    // columns 16 jb + 2 g + 1
-                }
+                for (int h = 0; h < kPair; ++h)
+                    if (cb0 + h < CB) {
+#pragma unroll
+                        for (int m = 0; m < 2; ++m)
+                            mma_k16<FP8>(acc[cb0 + h][m], av[h][m][0], av[h][m][1], av[h][m][2], av[h][m][3], pa0, pa1);
+                    }
                 if constexpr (PRECISE) {
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        mma_top_k16<FP8>(oa[jb + h], pl0, pl1, be0[h], be1[h]);
-                        mma_top_k16<FP8>(ob[jb + h], pl0, pl1, bo0[h], bo1[h]);
-                    }
+                    for (int h = 0; h < kPair; ++h)
+                        if (cb0 + h < CB) {
+#pragma unroll
+                            for (int m = 0; m < 2; ++m)
+                                mma_k16<FP8>(acc[cb0 + h][m], av[h][m][0], av[h][m][1], av[h][m][2], av[h][m][3], pl0, pl1);
+                        }
                 }
             }
         };
@@ -334,13 +370,15 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
         // ---- the warps' states meet in shared memory ----
         l_run += __shfl_xor_sync(kFull, l_run, 1);
         l_run += __shfl_xor_sync(kFull, l_run, 2);
-        if (gh < G) {
+        // this lane's outputs: members 2 t4 (+1) in the warp's slots, two pairs of neighbouring columns per 32-column block
 #pragma unroll
-            for (int jb = 0; jb < JB; ++jb)
-                *reinterpret_cast<float4 *>(&sm.wo[warp][g][16 * jb + 4 * t4]) =
-                    make_float4(oa[jb][0] * out_scale, ob[jb][0] * out_scale, oa[jb][1] * out_scale, ob[jb][1] * out_scale);
-            if (t4 == 0) { sm.wm[warp][g] = m_run; sm.wl[warp][g] = l_run; }
-        }
+        for (int cb = 0; cb < CB; ++cb)
+#pragma unroll
+            for (int m = 0; m < 2; ++m) {
+                *reinterpret_cast<float2 *>(&sm.wo[warp][2 * t4][32 * cb + 4 * g + 2 * m]) = make_float2(acc[cb][m][0] * out_scale, acc[cb][m][2] * out_scale);
+                *reinterpret_cast<float2 *>(&sm.wo[warp][2 * t4 + 1][32 * cb + 4 * g + 2 * m]) = make_float2(acc[cb][m][1] * out_scale, acc[cb][m][3] * out_scale);
+            }
+        if (gh < G && t4 == 0) { sm.wm[warp][g] = m_run; sm.wl[warp][g] = l_run; }
         if (!named_bar_and(1, nct, ok)) return false;
         const bool whole = sg.n_cta == 1;                // this CTA alone finishes the group right here
         for (int idx = t; idx < G * DH; idx += nct) {
