@@ -215,11 +215,16 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
             //      key0 + 8 + g and receives keys key0 + 2 t4 (+1) and key0 + 8 + 2 t4 (+1) of its head.  Four
             //      independent accumulator chains (sub-block x half of the 32-wide block).
             const int kr0 = key0 + g < rows ? key0 + g : rows - 1, kr1 = key0 + 8 + g < rows ? key0 + 8 + g : rows - 1;
-            float sc[2][2][2];
+            // PRECISE: rows 8..15 of A carry the lo parts of the same members, so one product gives q_hi . k (elements 0, 1)
+            // and q_lo . k (elements 2, 3)
+            constexpr int SE = PRECISE ? 4 : 2;
+            float sc[2][2][SE];
 #pragma unroll
             for (int u = 0; u < 2; ++u)
 #pragma unroll
-                for (int c = 0; c < 2; ++c) sc[u][c][0] = sc[u][c][1] = 0.f;
+                for (int c = 0; c < 2; ++c)
+#pragma unroll
+                    for (int e = 0; e < SE; ++e) sc[u][c][e] = 0.f;
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
                 uint4 kv[2];
@@ -235,14 +240,12 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
                 // four accumulators: a product never follows the one it depends on by less than four instructions
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    mma_top_k16<FP8>(sc[u][0], qhi[kb].x, qhi[kb].y, kv[u].x, kv[u].y);
-                    mma_top_k16<FP8>(sc[u][1], qhi[kb].z, qhi[kb].w, kv[u].z, kv[u].w);
-                }
-                if constexpr (PRECISE) {
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        mma_top_k16<FP8>(sc[u][0], qlo[kb].x, qlo[kb].y, kv[u].x, kv[u].y);
-                        mma_top_k16<FP8>(sc[u][1], qlo[kb].z, qlo[kb].w, kv[u].z, kv[u].w);
+                    if constexpr (PRECISE) {
+                        mma_k16<FP8>(sc[u][0], qhi[kb].x, qlo[kb].x, qhi[kb].y, qlo[kb].y, kv[u].x, kv[u].y);
+                        mma_k16<FP8>(sc[u][1], qhi[kb].z, qlo[kb].z, qhi[kb].w, qlo[kb].w, kv[u].z, kv[u].w);
+                    } else {
+                        mma_top_k16<FP8>(sc[u][0], qhi[kb].x, qhi[kb].y, kv[u].x, kv[u].y);
+                        mma_top_k16<FP8>(sc[u][1], qhi[kb].z, qhi[kb].w, kv[u].z, kv[u].w);
                     }
                 }
             }
@@ -255,7 +258,8 @@ __device__ __forceinline__ bool attn_consume_group(const AttnArgs &a, WeightRing
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     ka[2 * u + e] = key0 + 8 * u + 2 * t4 + e;
-                    const float v = sc[u][0][e] + sc[u][1][e];
+                    float v = sc[u][0][e] + sc[u][1][e];
+                    if constexpr (PRECISE) v += sc[u][0][2 + e] + sc[u][1][2 + e];
                     // a masked key gets weight 0 for this lane's member; the V row of the key still feeds the other members
                     see[2 * u + e] = ka[2 * u + e] < rows && !(causal && ka[2 * u + e] > my_tok);
                     s[2 * u + e] = see[2 * u + e] ? v * scale_log2 : -INFINITY;
