@@ -19,15 +19,6 @@ void set_last_error(cudaError_t e, const char *where)
 
 void set_last_error_text(const char *msg) { snprintf(g_last_error, sizeof g_last_error, "%s", msg); }
 
-bool step_pdl_enabled()
-{
-    static const bool on = [] {
-        const char *e = getenv("FASTTPS_STEP_PDL");
-        return e && e[0] == '1';
-    }();
-    return on;
-}
-
 bool pdl_enabled()
 {
     static const bool on = [] {

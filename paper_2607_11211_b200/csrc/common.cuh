@@ -94,7 +94,6 @@ void set_last_error_text(const char *msg);
 // prefetch weights, which no kernel writes) while its predecessor in the stream drains, and
 // orders everything else behind `griddepcontrol.wait`.
 bool pdl_enabled();
-bool step_pdl_enabled();       // the persistent step kernel as a programmatic dependent of its predecessor
 
 template <class Args>
 static int launch_ex(void (*kernel)(Args), dim3 grid, dim3 block, size_t smem, cudaStream_t st, const Args *a)

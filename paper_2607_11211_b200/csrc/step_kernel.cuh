@@ -263,12 +263,6 @@ __global__ void __launch_bounds__(kMegaThreadsMax, 1) decode_step_kernel(const _
     }
 
     // =========================================================================== consumer warps
-    // Launched as a programmatic dependent of its predecessor in the stream, this kernel's CTAs take over an SM as
-    // soon as the predecessor's CTA there has left: the producer warp above already streams the first weights (no
-    // kernel writes weights); everything else (lengths, activations, caches, the barrier words) is read only after
-    // the predecessor has completed.  The successor may be set up right away: it cannot start before this CTA exits.
-    pdl_wait();
-    pdl_launch_dependents();
     GridBarrier gb;
     gb.count = a.bar; gb.status = a.status;
     gb.ncta = ncta; gb.s_go = &s_go;
@@ -616,12 +610,12 @@ static int launch_step_inst(Ctx *c, const StepArgs &a, cudaStream_t st)
     // runs to its end clears them on its way out, and fasttps_get_status clears them after an abandoned one
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(c->n_sm); cfg.blockDim = dim3((lay.nw + 1) * 32); cfg.dynamicSmemBytes = lay.total; cfg.stream = st;
-    cudaLaunchAttribute attr[2];
+    // (launching it as a programmatic dependent of its predecessor as well, so that the producer warps stream the
+    // first weights while the predecessor's last CTAs finish, was measured on the one-layer workloads: no change)
+    cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = step_pdl_enabled() ? 2 : 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
     void *params[] = {const_cast<StepArgs *>(&a)};
     ProfScope prof(c, kProfStep, st);
     FT_CUDA(cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(kernel), params));
