@@ -90,7 +90,6 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
 
     WeightRing ring;
     ring.init(&sm.slots[0][0], sm.bars, &sm.abort, kWideSlots, kWidePiece, kWideWarps, nullptr, 0, nullptr, 0);
-    for (int i = t; i < kWideTiles * kWideMaxB * kWideAccStride; i += blockDim.x) sm.sums[i] = 0.f;
     if (t < kWideMaxB) { sm.best_val[t] = -INFINITY; sm.best_idx[t] = 0x7fffffff; }
     __syncthreads();
 
@@ -137,9 +136,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
             for (int j = 0; j < 4; ++j)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
+        const unsigned char *slot = nullptr;
         for (int c = 0; c < nchunk; ++c, ++piece) {
             const int kbs = nkb - c * kWideChunk < kWideChunk ? nkb - c * kWideChunk : kWideChunk;
-            const unsigned char *slot = ring.wait(piece, ok);
+            slot = ring.wait(piece, ok);
             if (ok && kb < kbs && kWideTilesPerWarp * th < nt) {
                 // B fragments of k block kb for the four batch tiles: rows 8 j + g, 8 consecutive k from 8 t4
                 uint4 bq[4];
@@ -161,27 +161,58 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
                     }
                 }
             }
-            ring.release(piece);
+            if (c + 1 < nchunk) ring.release(piece);          // the slot of the pass's last piece is kept: see below
         }
-        // ---- the k blocks of the warps meet in shared memory ----
-#pragma unroll
-        for (int i = 0; i < kWideTilesPerWarp; ++i) {
-            const int tile = kWideTilesPerWarp * th + i;
-            if (tile < nt) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    // fragment: rows g / g + 8 of the tile, batch rows 8 j + 2 t4 / + 1
-                    float *p = sm.sums + (size_t)(tile * kWideMaxB + 8 * j + 2 * t4) * kWideAccStride + g;
-                    atomicAdd(p, acc[i][j][0]);
-                    atomicAdd(p + kWideAccStride, acc[i][j][1]);
-                    atomicAdd(p + 8, acc[i][j][2]);
-                    atomicAdd(p + kWideAccStride + 8, acc[i][j][3]);
-                }
-            }
-        }
-        if (!named_bar_and(1, nct, ok)) {
+        if (!named_bar_and(1, nct, ok)) {                     // every warp has read the last piece
             if (t == 0) atomicOr(a.status, FASTTPS_DEV_WAIT_TIMEOUT);
             return;
+        }
+        // ---- the sums of the eight k blocks of a tile pair meet: a merge tree over the eight warps (three levels, one
+        //      block-wide barrier each), a warp's 32 sums travelling lane to lane through the slot of the pass's last
+        //      piece, which is handed back to the producer afterwards.  (Shared-memory atomics straight into `sums`, eight
+        //      warps on the same addresses, cost about 2 us per pass.)  A sender writes the region that only itself has
+        //      read before, so one barrier per level is enough. ----
+        {
+            float *xb = reinterpret_cast<float *>(const_cast<unsigned char *>(slot)) + (size_t)th * 4 * 1024 + lane;
+            for (int s = 4; s >= 1; s >>= 1) {
+                if (kb >= s && kb < 2 * s) {
+                    float *x = xb + (kb & 3) * 1024;
+#pragma unroll
+                    for (int i = 0; i < kWideTilesPerWarp; ++i)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) x[((i * 4 + j) * 4 + e) * 32] = acc[i][j][e];
+                }
+                named_bar_sync(1, nct);
+                if (kb < s) {
+                    const float *x = xb + ((kb + s) & 3) * 1024;
+#pragma unroll
+                    for (int i = 0; i < kWideTilesPerWarp; ++i)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) acc[i][j][e] += x[((i * 4 + j) * 4 + e) * 32];
+                }
+            }
+            if (kb == 0) {
+#pragma unroll
+                for (int i = 0; i < kWideTilesPerWarp; ++i) {
+                    const int tile = kWideTilesPerWarp * th + i;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // fragment: rows g / g + 8 of the tile, batch rows 8 j + 2 t4 / + 1
+                        float *p = sm.sums + (size_t)(tile * kWideMaxB + 8 * j + 2 * t4) * kWideAccStride + g;
+                        p[0] = acc[i][j][0];
+                        p[kWideAccStride] = acc[i][j][1];
+                        p[8] = acc[i][j][2];
+                        p[kWideAccStride + 8] = acc[i][j][3];
+                    }
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the slot goes back to the copy engine
+            ring.release(piece - 1);
+            named_bar_sync(1, nct);
         }
         // ---- epilogue: thread (r = t % 16, b = t / 16) finishes row r of every tile of the pass for batch row b ----
         {
@@ -193,7 +224,6 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
                     // rows c and c + 8 of a gate_up tile are a gate column and ITS up column (interlaced in blocks of 8)
                     if (r < 8) {
                         const float gate = p[r], up = p[r + 8];
-                        p[r] = 0.f; p[r + 8] = 0.f;
                         if (b < a.batch) {
                             const float act = gate / (1.f + __expf(-gate)) * up;
                             const __nv_bfloat16 hi = __float2bfloat16_rn(act);
@@ -204,7 +234,6 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
                     }
                 } else {
                     float v = p[r];
-                    p[r] = 0.f;
                     const int col = tile * 16 + (a.pair_rows ? ((r & 7) * 2 + (r >> 3)) : r);
                     if (b < a.batch && col < a.n_out) {
                         if (a.res) v += __bfloat162float(a.res[(size_t)b * a.res_stride + col]);
@@ -215,7 +244,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
                 }
             }
         }
-        named_bar_sync(1, nct);                          // the sums are zero again before the next pass adds to them
+        named_bar_sync(1, nct);                          // the sums have been read before the next pass writes them
     }
     if (a.next_ids == nullptr) return;
 
