@@ -290,14 +290,15 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_linear_kernel(WideArgs a
 
 // ------------------------------------------------------------------------------------------- down projection
 
-constexpr int kDownOct = 16;                                    // intermediate octets per ring piece
-constexpr int kDownCols = 128;                                  // output columns per unit (four 32-column blocks)
+constexpr int kDownQuad = 4;                                    // intermediate octets per ring piece
+constexpr int kDownBlocks = kWideWarps;                         // 32-column blocks per unit: one per consumer warp (512 columns)
+constexpr int kDownChunkOct = kWideAChunk / 8;                  // octets per chunk of the chunked intermediate (16)
 constexpr int kDownXStride = kWideARow * 2;                     // 272 bytes between batch rows: conflict-free 4-byte loads
 constexpr int kDownXBytes = kWideMaxB * kDownXStride;           // one of hi / lo: one contiguous block of the chunked layout
-static_assert(kDownOct * 8 == kWideAChunk, "a ring piece holds one chunk of the intermediate");
-constexpr int kDownRun = (kDownCols / 32) * 512;                // bytes of one octet's blocks of a column group: 2 KB
-constexpr int kDownPiece = 2 * kDownXBytes + kDownOct * kDownRun;    // 49 KB
+constexpr int kDownRun = kDownBlocks * 512;                     // bytes of one octet's blocks of a column group: 8 KB
+constexpr int kDownPiece = 2 * kDownXBytes + kDownQuad * kDownRun;   // 49 KB
 constexpr int kDownSlots = 4;
+static_assert(kDownChunkOct % kDownQuad == 0, "a piece lies inside one chunk of the intermediate");
 
 __device__ __forceinline__ unsigned char *slot_of_piece(WeightRing &ring, int s) { return ring.slots + (size_t)s * ring.slot_bytes; }
 
@@ -307,6 +308,11 @@ struct DownSmem {
     int abort;
 };
 
+// A unit = four octets of the intermediate x sixteen 32-column blocks of the output (512 columns): in the packed
+// W_down the sixteen blocks of an octet are 8 KB contiguous, so a ring piece is four weight copies plus the chunk of
+// the intermediate (hi and lo) the octets belong to.  (Units of 16 octets x 4 blocks, sixteen 2 KB copies per piece,
+// were bound by the rate at which one thread can issue bulk copies: 2.4 us per piece.)  Consumer warp w owns column
+// block w of the unit; its sums stay in registers while the CTA's units stay in one column group.
 __global__ void __launch_bounds__(kWideThreads, 1) wide_down_kernel(WideDownArgs a)
 {
     extern __shared__ unsigned char smem_raw[];
@@ -315,8 +321,8 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_down_kernel(WideDownArgs
     constexpr int nct = kWideWarps * 32;
 
     const int NT = a.D >> 5;                                   // 32-column blocks of an octet
-    const int n_oct = a.K >> 3, noc = (n_oct + kDownOct - 1) / kDownOct, ncg = a.D / kDownCols;
-    const int n_units = ncg * noc;                             // ordered by (column group, octet chunk)
+    const int n_oct = a.K >> 3, noq = (n_oct + kDownQuad - 1) / kDownQuad, ncg = (NT + kDownBlocks - 1) / kDownBlocks;
+    const int n_units = ncg * noq;                             // ordered by (column group, octet quad)
     const int base = n_units / gridDim.x, rem = n_units % gridDim.x, cta = blockIdx.x;
     const int u0 = cta * base + (cta < rem ? cta : rem), nu = base + (cta < rem ? 1 : 0);
 
@@ -328,16 +334,18 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_down_kernel(WideDownArgs
         pdl_wait();                                            // the intermediate was written by the previous kernel
         ring.policy = l2_policy_evict_first();
         for (int i = 0; i < nu; ++i) {
-            const int u = u0 + i, cg = u / noc, oc = u - cg * noc;
-            const int o0 = oc * kDownOct, octs = n_oct - o0 < kDownOct ? n_oct - o0 : kDownOct;
+            const int u = u0 + i, cg = u / noq, oq = u - cg * noq;
+            const int o0 = oq * kDownQuad, octs = n_oct - o0 < kDownQuad ? n_oct - o0 : kDownQuad;
+            const int nbu = NT - cg * kDownBlocks < kDownBlocks ? NT - cg * kDownBlocks : kDownBlocks;
+            const int chunk = o0 / kDownChunkOct;
             const int s = ring.slot_of(i);
             int okv = 1;
             if (lane == 0) {
                 okv = ring.acquire(i) ? 1 : 0;
                 if (okv) {
-                    mbar_expect_tx(&ring.full[s], (uint32_t)(2 * kDownXBytes + octs * kDownRun));
-                    bulk_g2s(slot_of_piece(ring, s), reinterpret_cast<const unsigned char *>(a.a_hi) + (size_t)oc * kDownXBytes, (uint32_t)kDownXBytes, &ring.full[s]);
-                    bulk_g2s(slot_of_piece(ring, s) + kDownXBytes, reinterpret_cast<const unsigned char *>(a.a_lo) + (size_t)oc * kDownXBytes, (uint32_t)kDownXBytes, &ring.full[s]);
+                    mbar_expect_tx(&ring.full[s], (uint32_t)(2 * kDownXBytes + octs * nbu * 512));
+                    bulk_g2s(slot_of_piece(ring, s), reinterpret_cast<const unsigned char *>(a.a_hi) + (size_t)chunk * kDownXBytes, (uint32_t)kDownXBytes, &ring.full[s]);
+                    bulk_g2s(slot_of_piece(ring, s) + kDownXBytes, reinterpret_cast<const unsigned char *>(a.a_lo) + (size_t)chunk * kDownXBytes, (uint32_t)kDownXBytes, &ring.full[s]);
                 }
             }
             okv = __shfl_sync(kFull, okv, 0);
@@ -345,15 +353,14 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_down_kernel(WideDownArgs
             unsigned char *slot = slot_of_piece(ring, s);
             if (lane < octs)
                 bulk_g2s_hint(slot + 2 * kDownXBytes + lane * kDownRun,
-                              reinterpret_cast<const unsigned char *>(a.w) + ((size_t)(o0 + lane) * NT + (size_t)cg * (kDownCols / 32)) * 512,
-                              (uint32_t)kDownRun, &ring.full[s], ring.policy);
+                              reinterpret_cast<const unsigned char *>(a.w) + ((size_t)(o0 + lane) * NT + (size_t)cg * kDownBlocks) * 512,
+                              (uint32_t)(nbu * 512), &ring.full[s], ring.policy);
         }
         return;
     }
 
     pdl_wait();
     pdl_launch_dependents();
-    const int nb = w & 3, par = w >> 2;                        // this warp: column block nb of the group, octets par, par + 4, ...
     float acc[2][4][4];
     auto clear = [&]() {
 #pragma unroll
@@ -366,7 +373,8 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_down_kernel(WideDownArgs
     // the four sums a lane holds of its two MMA tiles are four CONSECUTIVE columns (the order of the packed W_down):
     // one 16-byte reduction per batch row
     auto flush = [&](int cg) {
-        float *colp = a.acc + (size_t)(cg * kDownCols + 32 * nb + 4 * g);
+        if (cg * kDownBlocks + w >= NT) return;
+        float *colp = a.acc + (size_t)((cg * kDownBlocks + w) * 32 + 4 * g);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int b0 = 8 * j + 2 * t4;
@@ -376,24 +384,54 @@ __global__ void __launch_bounds__(kWideThreads, 1) wide_down_kernel(WideDownArgs
     };
     clear();
     bool ok = true;
-    int cur_cg = nu > 0 ? u0 / noc : 0;
+    int cur_cg = nu > 0 ? u0 / noq : 0;
     for (int i = 0; i < nu; ++i) {
-        const int u = u0 + i, cg = u / noc, oc = u - cg * noc;
-        const int octs = n_oct - oc * kDownOct < kDownOct ? n_oct - oc * kDownOct : kDownOct;
+        const int u = u0 + i, cg = u / noq, oq = u - cg * noq;
+        const int o0 = oq * kDownQuad, octs = n_oct - o0 < kDownQuad ? n_oct - o0 : kDownQuad;
         if (cg != cur_cg) { if (ok) flush(cur_cg); clear(); cur_cg = cg; }
         const unsigned char *slot = ring.wait(i, ok);
-        if (ok) {
-            for (int o = par; o < octs; o += kWideWarps / 4) {
-                const uint4 av = *reinterpret_cast<const uint4 *>(slot + 2 * kDownXBytes + o * kDownRun + nb * 512 + lane * 16);
+        if (ok && cg * kDownBlocks + w < NT) {
+            const unsigned char *wb = slot + 2 * kDownXBytes + w * 512 + lane * 16;
+            const int xo = (o0 % kDownChunkOct) * 16 + t4 * 4;        // the piece's first octet inside its chunk of the intermediate
+            // two octets at a time as ONE k = 16 product (the A fragments of two octet blocks are the two k halves of an
+            // m16n8k16 fragment); all hi products first, then the lo ones: the two products into an accumulator are
+            // eight instructions apart
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const unsigned char *xp = slot + (8 * j + g) * kDownXStride + o * 16 + t4 * 4;
-                    const uint32_t bh = *reinterpret_cast<const uint32_t *>(xp);
-                    const uint32_t bl = *reinterpret_cast<const uint32_t *>(xp + kDownXBytes);
-                    mma_bf16_k8(acc[0][j], av.x, av.y, bh);
-                    mma_bf16_k8(acc[0][j], av.x, av.y, bl);
-                    mma_bf16_k8(acc[1][j], av.z, av.w, bh);
-                    mma_bf16_k8(acc[1][j], av.z, av.w, bl);
+            for (int o = 0; o < kDownQuad; o += 2) {
+                if (o + 1 < octs) {
+                    const uint4 av = *reinterpret_cast<const uint4 *>(wb + o * kDownRun);
+                    const uint4 aw = *reinterpret_cast<const uint4 *>(wb + (o + 1) * kDownRun);
+                    uint32_t bh[4][2], bl[4][2];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const unsigned char *xp = slot + (8 * j + g) * kDownXStride + xo + o * 16;
+                        bh[j][0] = *reinterpret_cast<const uint32_t *>(xp);
+                        bh[j][1] = *reinterpret_cast<const uint32_t *>(xp + 16);
+                        bl[j][0] = *reinterpret_cast<const uint32_t *>(xp + kDownXBytes);
+                        bl[j][1] = *reinterpret_cast<const uint32_t *>(xp + kDownXBytes + 16);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        mma_bf16_k16(acc[0][j], av.x, av.y, aw.x, aw.y, bh[j][0], bh[j][1]);
+                        mma_bf16_k16(acc[1][j], av.z, av.w, aw.z, aw.w, bh[j][0], bh[j][1]);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        mma_bf16_k16(acc[0][j], av.x, av.y, aw.x, aw.y, bl[j][0], bl[j][1]);
+                        mma_bf16_k16(acc[1][j], av.z, av.w, aw.z, aw.w, bl[j][0], bl[j][1]);
+                    }
+                } else if (o < octs) {                            // an octet without a partner (a ragged last piece)
+                    const uint4 av = *reinterpret_cast<const uint4 *>(wb + o * kDownRun);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const unsigned char *xp = slot + (8 * j + g) * kDownXStride + xo + o * 16;
+                        const uint32_t bh = *reinterpret_cast<const uint32_t *>(xp);
+                        const uint32_t bl = *reinterpret_cast<const uint32_t *>(xp + kDownXBytes);
+                        mma_bf16_k8(acc[0][j], av.x, av.y, bh);
+                        mma_bf16_k8(acc[1][j], av.z, av.w, bh);
+                        mma_bf16_k8(acc[0][j], av.x, av.y, bl);
+                        mma_bf16_k8(acc[1][j], av.z, av.w, bl);
+                    }
                 }
             }
         }
@@ -498,8 +536,8 @@ int launch_wide_linear(Ctx *c, const WideArgs &a, int prof_class, cudaStream_t s
 
 int launch_wide_down(Ctx *c, const WideDownArgs &a, cudaStream_t st)
 {
-    if (a.batch < 1 || a.batch > kWideMaxB || a.D % kDownCols || a.K < 8 || (a.K & 7)) return FASTTPS_INVALID_ARG;
-    const int units = (a.D / kDownCols) * ((a.K / 8 + kDownOct - 1) / kDownOct);
+    if (a.batch < 1 || a.batch > kWideMaxB || (a.D & 31) || a.K < 8 || (a.K & 7)) return FASTTPS_INVALID_ARG;
+    const int units = ((a.D / 32 + kDownBlocks - 1) / kDownBlocks) * ((a.K / 8 + kDownQuad - 1) / kDownQuad);
     int grid = c->n_sm < units ? c->n_sm : units;
     ProfScope prof(c, kProfMlp, st);
     const int rc = launch_ex(wide_down_kernel, dim3(grid), dim3(kWideThreads), sizeof(DownSmem) + 128, st, &a);
