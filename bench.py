@@ -35,12 +35,16 @@ UNIT = "tok/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one mlp_decode_kernel launch (Phi-3 shape, batch 1), from an
 # ncu capture of that kernel (151.09 MB read + 4.05 MB written).
 NCU_MLP_TRAFFIC_BYTES = 155.1e6
-# DRAM traffic of decode_step_kernel relative to its algorithmic bytes, from two ncu captures of one decode
-# step of the batch-1 full-stack shape cut to 4 and to 8 layers: 239.6 MB per layer and 200.7 MB for the head
-# against 239.1 MB and 197.1 MB algorithmic, i.e. 7.867 GB for a full 32-layer step against 7.848 GB.  The
-# full-size launch is too large to capture; traffic grows in proportion to the layers and steps a launch
-# processes.
-NCU_STEP_TRAFFIC_RATIO = 1.002
+# DRAM traffic of decode_step_kernel relative to its algorithmic bytes, from ncu captures
+# (dram__bytes_read.sum + dram__bytes_write.sum) of small cases of the same kernel.  Batch-1 full stack cut to 4 and
+# to 8 layers, one step: 239.8 MB per layer and 198.6 MB for the head against 239.1 MB and 197.1 MB algorithmic,
+# i.e. 7.872 GB for a full 32-layer step against 7.848 GB.  The full-size launch is too large to capture; traffic
+# grows in proportion to the layers and steps a launch processes.  One layer per launch (the single-layer
+# workloads): 233.5 MB against 229.7 MB and 281.5 MB against 276.8 MB (the FP32 sums of the two reductions are
+# written and read once more per launch).  Ragged batch of 8, stack cut to 2 layers: 1081.4 MB against 1075.9 MB.
+NCU_STEP_TRAFFIC_RATIO = 1.003
+NCU_LAYER_TRAFFIC_RATIO = 1.017
+NCU_STEP_B8_TRAFFIC_RATIO = 1.005
 
 
 def parse_args():
@@ -276,7 +280,7 @@ def time_ragged_batch(fb, wl, torch, dev, local, dm, layers, embed, g_final, w_l
            "ms_per_step": ms / steps, "batch": B, "past_lens": lens0.tolist(), "max_seq": W.max_seq,
            "algorithmic_bytes_per_step": nbytes, "device_status": status,
            "roofline": {"bound": "hbm", "kernel": "decode_step_kernel", "achieved": gbs, "peak": peak, "unit": "GB/s",
-                        "frac": gbs / peak, "traffic": None, "bytes_per_launch": nbytes,
+                        "frac": gbs / peak, "traffic": nbytes * NCU_STEP_B8_TRAFFIC_RATIO, "bytes_per_launch": nbytes,
                         "avg_launch_us": ms / steps * 1e3}}
     ctx.close()
     del caches
@@ -452,7 +456,14 @@ def run_ours(args):
         steps_per_launch = n_prof if one_call else 1
         dom_bytes = float(sum(W.algorithmic_bytes(s if advance else 0) for s in range(steps_per_launch)))
         dom_name = "decode_step_kernel"
-        ncu_traffic = dom_bytes * NCU_STEP_TRAFFIC_RATIO if (dm is wl.PHI3_MINI and B == 1) else None
+        ncu_traffic = None
+        if dm is wl.PHI3_MINI:
+            if not W.full_stack and B == 1:
+                ncu_traffic = dom_bytes * NCU_LAYER_TRAFFIC_RATIO
+            elif W.full_stack and B == 1:
+                ncu_traffic = dom_bytes * NCU_STEP_TRAFFIC_RATIO
+            elif W.full_stack and B == 8:
+                ncu_traffic = dom_bytes * NCU_STEP_B8_TRAFFIC_RATIO
     elif dom == "attn":                                       # one launch = the attention of one layer
         kv = dm.kv_bytes_per_token_per_layer * float(sum(int(l) + 1 for l in lens0))
         dom_bytes = kv + 2 * B * dm.n_q_heads * dm.head_dim * 2 + 2 * B * dm.n_kv_heads * dm.head_dim * 2
