@@ -7,7 +7,7 @@ import torch
 
 from oracle import oracle as orc
 from paper_2607_11211_b200 import workload as wl
-from tests.helpers import assert_close_bits
+from tests.helpers import assert_close_bits, ulp_distance, from_bf16_bits as F32
 
 pytestmark = pytest.mark.gpu
 
@@ -68,6 +68,35 @@ def test_attn_decode_fp8_saturates_and_reports_a_full_cache(fb):
     new = kg[1, :, 10] & 0x7f
     assert (new == 0x7e).mean() > 0.9                           # scales far too small: nearly every new code is +-448
     assert_close_bits(got[1:], want[1:], what="attention over a saturated E4M3 cache")
+
+
+def test_attn_decode_fp8_keeps_subnormal_codes(fb):
+    # a cache made of the SUBNORMAL codes of the format (magnitudes 2^-9 .. 7 * 2^-9) and of zeros only: widened to
+    # fp16 they are normal numbers, and the products must see them (an implementation that flushed them would
+    # return zeros)
+    dims, max_seq, lens = wl.SMALL_GQA, 128, np.array([100, 37], np.int32)
+    B, d, Hq, Hkv = 2, dims.head_dim, dims.n_q_heads, dims.n_kv_heads
+    rng = np.random.default_rng(3)
+    sub = lambda *s: (rng.integers(0, 8, size=s) | (rng.integers(0, 2, size=s) << 7)).astype(np.uint8)
+    k0, v0 = sub(B, Hkv, max_seq, d), sub(B, Hkv, max_seq, d)
+    q = orc.f32_to_bf16((rng.standard_normal((B, Hq, d)) * 8).astype(np.float32))
+    tiny = orc.f32_to_bf16((rng.standard_normal((B, Hkv, d)) * 2.0 ** -8).astype(np.float32))
+    ctx = fb.Context.from_dims(dims, B, max_seq)
+    kc, vc = torch.from_numpy(k0.copy()).cuda(), torch.from_numpy(v0.copy()).cuda()
+    out = torch.zeros(B, Hq, d, dtype=torch.bfloat16, device="cuda")
+    k_scale, v_scale = 64.0, 2.0
+    ctx.attn_decode_fp8(wl.from_bits(q, "cuda"), wl.from_bits(tiny, "cuda"), wl.from_bits(tiny, "cuda"), kc, vc, k_scale, v_scale,
+                        i32(lens), i32(lens), out)
+    torch.cuda.synchronize()
+    assert ctx.get_status() == 0
+    ko, vo = k0.copy(), v0.copy()
+    want = orc.attn_decode_fp8(q, tiny, tiny, ko, vo, k_scale, v_scale, lens, lens, dims.rope_theta)
+    got = wl.bits(out)
+    assert (kc.cpu().numpy() == ko).all() and (vc.cpu().numpy() == vo).all()
+    w = F32(want).astype(np.float64)
+    assert np.abs(w).max() > 1e-3                                        # the expected outputs are far from zero
+    assert ulp_distance(got, want).max() <= 2                            # outputs of about 0.01: two bf16 units are 2e-4
+    ctx.close()
 
 
 def test_attn_decode_fp8_rejects_bad_scales_and_groups(fb):
