@@ -489,10 +489,10 @@ void orc_mlp_decode(const uint16_t *x, const uint16_t *w_gu, const uint16_t *w_d
 static void layer_decode_n(const uint16_t *g_attn, const uint16_t *w_qkv, const uint16_t *w_o,
                            const uint16_t *g_mlp, const uint16_t *w_gu, const uint16_t *w_down,
                            const uint16_t *x_in, uint16_t *x_out,
-                           uint16_t *k_cache, uint16_t *v_cache,
+                           void *k_cache, void *v_cache,
                            const int32_t *pos, const int32_t *seq_lens,
                            int n_seq, int n_new, int D, int Hq, int Hkv, int d, int K, int max_seq,
-                           double eps, double theta)
+                           double eps, double theta, int fp8, float k_scale, float v_scale)
 {
     /* B: token rows of the step = sequences x new tokens per sequence; only the attention tells them apart */
     int B = n_seq * n_new;
@@ -517,8 +517,9 @@ static void layer_decode_n(const uint16_t *g_attn, const uint16_t *w_qkv, const 
     }
     /* a skipped sequence (bad length) leaves its attention output at zero */
     memset(ab, 0, 2 * (size_t)B * nq);
-    if (n_new == 1) orc_attn_decode(qb, kb, vb, k_cache, v_cache, pos, seq_lens, ab, B, Hq, Hkv, d, max_seq, theta);
-    else orc_attn_decode_multi(qb, kb, vb, k_cache, v_cache, pos, seq_lens, ab, n_seq, n_new, Hq, Hkv, d, max_seq, theta);
+    if (fp8) orc_attn_decode_fp8(qb, kb, vb, (uint8_t *)k_cache, (uint8_t *)v_cache, k_scale, v_scale, pos, seq_lens, ab, B, Hq, Hkv, d, max_seq, theta);
+    else if (n_new == 1) orc_attn_decode(qb, kb, vb, (uint16_t *)k_cache, (uint16_t *)v_cache, pos, seq_lens, ab, B, Hq, Hkv, d, max_seq, theta);
+    else orc_attn_decode_multi(qb, kb, vb, (uint16_t *)k_cache, (uint16_t *)v_cache, pos, seq_lens, ab, n_seq, n_new, Hq, Hkv, d, max_seq, theta);
     orc_gemv(ab, w_o, proj, B, nq, D);
     for (size_t i = 0; i < (size_t)B * D; ++i)
         h[i] = orc_f64_to_bf16((double)orc_bf16_to_f32(x_in[i]) + proj[i]);
@@ -539,7 +540,21 @@ void orc_layer_decode(const uint16_t *g_attn, const uint16_t *w_qkv, const uint1
                       double eps, double theta)
 {
     layer_decode_n(g_attn, w_qkv, w_o, g_mlp, w_gu, w_down, x_in, x_out, k_cache, v_cache, pos, seq_lens,
-                   B, 1, D, Hq, Hkv, d, K, max_seq, eps, theta);
+                   B, 1, D, Hq, Hkv, d, K, max_seq, eps, theta, 0, 1.f, 1.f);
+}
+
+/* The same layer over caches of E4M3 codes (orc_attn_decode_fp8 in place of orc_attn_decode; everything else,
+ * including the bf16 q | k | v handed to the attention, unchanged). */
+void orc_layer_decode_fp8(const uint16_t *g_attn, const uint16_t *w_qkv, const uint16_t *w_o,
+                          const uint16_t *g_mlp, const uint16_t *w_gu, const uint16_t *w_down,
+                          const uint16_t *x_in, uint16_t *x_out,
+                          uint8_t *k_cache, uint8_t *v_cache, float k_scale, float v_scale,
+                          const int32_t *pos, const int32_t *seq_lens,
+                          int B, int D, int Hq, int Hkv, int d, int K, int max_seq,
+                          double eps, double theta)
+{
+    layer_decode_n(g_attn, w_qkv, w_o, g_mlp, w_gu, w_down, x_in, x_out, k_cache, v_cache, pos, seq_lens,
+                   B, 1, D, Hq, Hkv, d, K, max_seq, eps, theta, 1, k_scale, v_scale);
 }
 
 /* The same layer for N new tokens per sequence: x_in, x_out [B*N, D] (token j of sequence b in row b*N + j);
@@ -553,7 +568,7 @@ void orc_layer_decode_multi(const uint16_t *g_attn, const uint16_t *w_qkv, const
                             double eps, double theta)
 {
     layer_decode_n(g_attn, w_qkv, w_o, g_mlp, w_gu, w_down, x_in, x_out, k_cache, v_cache, pos, seq_lens,
-                   B, N, D, Hq, Hkv, d, K, max_seq, eps, theta);
+                   B, N, D, Hq, Hkv, d, K, max_seq, eps, theta, 0, 1.f, 1.f);
 }
 
 /* ------------------------------------------------------------ model decode */

@@ -279,6 +279,26 @@ def layer_decode_multi(w: dict, x_in, n_new, k_cache, v_cache, pos, seq_lens, ep
     return x_out
 
 
+def layer_decode_fp8(w: dict, x_in, k_cache, v_cache, k_scale, v_scale, pos, seq_lens, eps=1e-5, theta=10000.0):
+    """layer_decode over caches of E4M3 codes (uint8 [B,Hkv,max_seq,d], appended in place); returns x_out [B, D]."""
+    x_in = _u16(x_in)
+    B, D = x_in.shape
+    assert k_cache.dtype == np.uint8 and v_cache.dtype == np.uint8 and k_cache.flags.c_contiguous and v_cache.flags.c_contiguous
+    _, Hkv, max_seq, d = k_cache.shape
+    Hq = w["w_o"].shape[0] // d
+    K = w["w_down"].shape[0]
+    pos, seq_lens = _i32(pos), _i32(seq_lens)
+    x_out = np.empty_like(x_in)
+    u8p = C.POINTER(C.c_uint8)
+    lib().orc_layer_decode_fp8(_p(_u16(w["g_attn"]), _u16p), _p(_u16(w["w_qkv"]), _u16p), _p(_u16(w["w_o"]), _u16p),
+                               _p(_u16(w["g_mlp"]), _u16p), _p(_u16(w["w_gu"]), _u16p), _p(_u16(w["w_down"]), _u16p),
+                               _p(x_in, _u16p), _p(x_out, _u16p), _p(k_cache, u8p), _p(v_cache, u8p),
+                               C.c_float(k_scale), C.c_float(v_scale), _p(pos, _i32p), _p(seq_lens, _i32p), C.c_int(B),
+                               C.c_int(D), C.c_int(Hq), C.c_int(Hkv), C.c_int(d), C.c_int(K), C.c_int(max_seq),
+                               C.c_double(eps), C.c_double(theta))
+    return x_out
+
+
 def model_decode(embed, layers, g_final, w_lm, k_caches, v_caches, token_ids, pos, seq_lens,
                  eps=1e-5, theta=10000.0, want_hidden=False):
     """layers: list of dicts as in layer_decode.  Returns (logits f32 [B,V], next_ids i32 [B]

@@ -739,3 +739,25 @@ def test_fp8_attention_skips_a_full_cache_and_saturates_large_rows():
     vbig = B16(np.full(vn.shape, 3.0, np.float32))
     orc.attn_decode_fp8(q, kn, vbig, kc, vc, 1.0, 1e-3, lens, lens)
     assert (vc[1, :, 2] == 0x7e).all()
+
+
+def test_fp8_layer_equals_the_blocks_chained_by_hand():
+    # the layer over an E4M3 cache: norm -> QKV -> attention over the codes -> output projection + residual -> norm -> MLP
+    D, H, d, K, Bn, max_seq = 8, 2, 4, 16, 2, 10
+    w = _tiny_layer(D, H, d, K)
+    x = rnd(Bn, D)
+    _, _, _, kc, vc, _ = _fp8_case(Bn=Bn, Hq=H, Hkv=H, d=d, max_seq=max_seq)
+    lens, pos = np.array([3, 0], np.int32), np.array([3, 1], np.int32)
+    ks, vs = 0.3, 0.7
+    k1, v1 = kc.copy(), vc.copy()
+    got = orc.layer_decode_fp8(w, x, k1, v1, ks, vs, pos, lens)
+    qkv = orc.f64_to_bf16(orc.gemv(orc.rmsnorm(x, w["g_attn"], 1e-5), w["w_qkv"]))
+    nq = H * d
+    sp = lambda t: t.reshape(Bn, H, d)
+    k2, v2 = kc.copy(), vc.copy()
+    a = orc.attn_decode_fp8(sp(qkv[:, :nq]), sp(qkv[:, nq:2 * nq]), sp(qkv[:, 2 * nq:]), k2, v2, ks, vs, pos, lens)
+    h = orc.f64_to_bf16(F32(x).astype(np.float64) + orc.gemv(a.reshape(Bn, nq), w["w_o"]))
+    want = orc.f64_to_bf16(F32(h).astype(np.float64) + orc.mlp_f64(orc.rmsnorm(h, w["g_mlp"], 1e-5), w["w_gu"], w["w_down"]))
+    assert (got == want).all() and (k1 == k2).all() and (v1 == v2).all()
+    # and the bf16 layer is untouched by the new path: same inputs, bf16 caches of the dequantised codes, position 0
+    # rotation-free, is covered by test_fp8_attention_on_exactly_representable_data_is_the_bf16_attention
