@@ -214,6 +214,13 @@ int fasttps_layer_decode(fasttps_ctx *ctx, const fasttps_layer_weights *w, const
                          void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens,
                          int batch, void *stream);
 
+/* The same layer over caches of E4M3 codes (fasttps_attn_decode_fp8 in place of fasttps_attn_decode; Section 6.2):
+ * k_cache, v_cache uint8 [B,H_kv,max_seq,d], one scale per tensor; batch <= 32.  Runs one kernel per product (the
+ * persistent layer kernel reads bf16 caches).  1 to 16 query heads per kv head, else FASTTPS_INVALID_ARG. */
+int fasttps_layer_decode_fp8(fasttps_ctx *ctx, const fasttps_layer_weights *w, const void *x_in, void *x_out,
+                             void *k_cache, void *v_cache, float k_scale, float v_scale, const int32_t *pos,
+                             const int32_t *seq_lens, int batch, void *stream);
+
 /* The same layer for n_new tokens per sequence (Algorithm 3 and Algorithm 4 for general N): x_in, x_out
  * [B * n_new, D], token j of sequence b in row b * n_new + j; pos, seq_lens [B]; 1 <= n_new <= 8 and
  * batch * n_new <= max_batch.  The projections and the MLP treat the token rows alike; the attention is

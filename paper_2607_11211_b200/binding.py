@@ -69,6 +69,7 @@ def load_library() -> C.CDLL:
     lib.fasttps_attn_decode.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, vp, i, vp]
     lib.fasttps_attn_decode_multi.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, vp, i, i, vp]
     lib.fasttps_attn_decode_fp8.argtypes = [vp, vp, vp, vp, vp, vp, C.c_float, C.c_float, ip, ip, vp, i, vp]
+    lib.fasttps_layer_decode_fp8.argtypes = [vp, C.POINTER(LayerWeights), vp, vp, vp, vp, C.c_float, C.c_float, ip, ip, i, vp]
     lib.fasttps_layer_decode_multi.argtypes = [vp, C.POINTER(LayerWeights), vp, vp, vp, vp, ip, ip, i, i, vp]
     lib.fasttps_mlp_decode.argtypes = [vp, vp, vp, vp, vp, i, vp]
     lib.fasttps_mlp_decode_static.argtypes = [vp, vp, vp, vp, vp, i, vp]
@@ -235,6 +236,13 @@ class Context:
                                                   _ptr(v_cache), _ptr(pos), _ptr(seq_lens), _ptr(out), batch, n_new,
                                                   _stream(stream)), "fasttps_attn_decode_multi")
         return out
+
+    def layer_decode_fp8(self, lw: LayerWeights, x_in, x_out, k_cache, v_cache, k_scale, v_scale, pos, seq_lens, stream=None):
+        """The layer over uint8 caches of E4M3 codes."""
+        _check(self.lib.fasttps_layer_decode_fp8(self.handle, C.byref(lw), _ptr(x_in), _ptr(x_out), _ptr(k_cache),
+                                                 _ptr(v_cache), float(k_scale), float(v_scale), _ptr(pos), _ptr(seq_lens),
+                                                 x_in.shape[0], _stream(stream)), "fasttps_layer_decode_fp8")
+        return x_out
 
     def layer_decode_multi(self, lw: LayerWeights, x_in, x_out, n_new, k_cache, v_cache, pos, seq_lens, stream=None):
         """x_in [B * n_new, D]: token j of sequence b in row b * n_new + j."""

@@ -423,7 +423,8 @@ int fasttps_linear_decode(fasttps_ctx *ctx, int kind, const void *x, const void 
 // prep folds them in (the input of the next layer, or the layer output).
 static int layer_body_wide(Ctx *c, const fasttps_layer_weights &w, const __nv_bfloat16 *x_res, float *pend,
                            __nv_bfloat16 *x_store, void *k_cache, void *v_cache, const int32_t *pos,
-                           const int32_t *seq_lens, int batch, int n_new, cudaStream_t st)
+                           const int32_t *seq_lens, int batch, int n_new, cudaStream_t st, bool fp8 = false,
+                           float k_scale = 1.f, float v_scale = 1.f)
 {
     const fasttps_config &f = c->cfg;
     const int D = f.hidden, nq = f.n_q_heads * f.head_dim, nkv = f.n_kv_heads * f.head_dim, nqkv = nq + 2 * nkv;
@@ -437,7 +438,7 @@ static int layer_body_wide(Ctx *c, const fasttps_layer_weights &w, const __nv_bf
     if (rc) return rc;
     // the attention writes its output straight into the chunked activations of the output projection
     rc = attn_impl(c, c->qkv, c->qkv + nq, c->qkv + nq + nkv, nqkv, nqkv, k_cache, v_cache, pos, seq_lens, c->wide_n, nq,
-                   batch, st, n_new, /*out_chunked=*/1);
+                   batch, st, n_new, /*out_chunked=*/1, fp8, k_scale, v_scale);
     if (rc) return rc;
     a = wide_args(c, c->wide_n, w.w_o, nq, D, batch);            // h = x + attn . W_o
     a.res = resid; a.res_stride = D; a.out_bf16 = c->h; a.out_stride = D; a.pair_rows = 1;
@@ -449,10 +450,11 @@ static int layer_body_wide(Ctx *c, const fasttps_layer_weights &w, const __nv_bf
 // batch: token rows (sequences x n_new)
 static int layer_impl(Ctx *c, const fasttps_layer_weights &w, const __nv_bfloat16 *x_in, __nv_bfloat16 *x_out,
                       void *k_cache, void *v_cache, const int32_t *pos, const int32_t *seq_lens, int batch,
-                      cudaStream_t st, int n_new = 1)
+                      cudaStream_t st, int n_new = 1, bool fp8 = false, float k_scale = 1.f, float v_scale = 1.f)
 {
     if (wide_batch(c, batch) && batch <= kWideMaxB) {
-        int rc = layer_body_wide(c, w, x_in, nullptr, nullptr, k_cache, v_cache, pos, seq_lens, batch, n_new, st);
+        int rc = layer_body_wide(c, w, x_in, nullptr, nullptr, k_cache, v_cache, pos, seq_lens, batch, n_new, st, fp8,
+                                 k_scale, v_scale);
         if (rc) return rc;
         // x' = h + MLP sums
         return wide_prep(c, c->h, c->cfg.hidden, c->mlp_acc, nullptr, x_out, nullptr, c->cfg.hidden, batch, kProfMlp, st);
@@ -465,7 +467,7 @@ static int layer_impl(Ctx *c, const fasttps_layer_weights &w, const __nv_bfloat1
                      c->qkv, nullptr, nqkv, batch, nullptr, nullptr, nullptr, kProfQkv, st);
     if (rc) return rc;
     rc = attn_impl(c, c->qkv, c->qkv + nq, c->qkv + nq + nkv, nqkv, nqkv, k_cache, v_cache, pos, seq_lens,
-                   c->attn_out, nq, batch, st, n_new);
+                   c->attn_out, nq, batch, st, n_new, 0, fp8, k_scale, v_scale);
     if (rc) return rc;
     // h = x + attn . W_o
     rc = linear_impl(c, nq, D, c->attn_out, nq, nullptr, w.w_o, x_in, D, c->h, nullptr, D, batch, nullptr, nullptr,
@@ -516,6 +518,21 @@ int fasttps_layer_decode_multi(fasttps_ctx *ctx, const fasttps_layer_weights *w,
     // the projections and the MLP see batch * n_new token rows; only the attention tells the tokens of a sequence apart
     return layer_impl(c, *w, static_cast<const __nv_bfloat16 *>(x_in), static_cast<__nv_bfloat16 *>(x_out), k_cache,
                       v_cache, pos, seq_lens, batch * n_new, static_cast<cudaStream_t>(stream), n_new);
+}
+
+int fasttps_layer_decode_fp8(fasttps_ctx *ctx, const fasttps_layer_weights *w, const void *x_in, void *x_out,
+                             void *k_cache, void *v_cache, float k_scale, float v_scale, const int32_t *pos,
+                             const int32_t *seq_lens, int batch, void *stream)
+{
+    if (!ctx) return FASTTPS_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (batch < 1 || batch > c->cfg.max_batch || batch > kWideMaxB || !layer_ok(w)) return FASTTPS_INVALID_ARG;
+    if (!aligned16(x_in) || !aligned16(x_out) || !aligned16(k_cache) || !aligned16(v_cache) || !pos || !seq_lens)
+        return FASTTPS_INVALID_ARG;
+    if (!(k_scale > 0.f) || !(v_scale > 0.f) || std::isinf(k_scale) || std::isinf(v_scale)) return FASTTPS_INVALID_ARG;
+    // one kernel per product (the persistent layer kernel reads bf16 caches)
+    return layer_impl(c, *w, static_cast<const __nv_bfloat16 *>(x_in), static_cast<__nv_bfloat16 *>(x_out), k_cache,
+                      v_cache, pos, seq_lens, batch, static_cast<cudaStream_t>(stream), 1, /*fp8=*/true, k_scale, v_scale);
 }
 
 static bool use_step_kernel(const Ctx *c, int batch)

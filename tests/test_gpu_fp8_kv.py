@@ -109,3 +109,52 @@ def test_attn_decode_fp8_rejects_bad_scales_and_groups(fb):
         with pytest.raises(fb.FasttpsError):
             ctx.attn_decode_fp8(act["q"], act["k_new"], act["v_new"], kc, vc, ks, vs, i32([0]), i32([0]), out)
     ctx.close()
+
+
+def _e4m3_order(c):
+    """Order-preserving integer image of E4M3 codes (+0 and -0 coincide)."""
+    c = np.asarray(c, np.uint8).astype(np.int32)
+    return np.where(c & 0x80, -(c & 0x7F), c)
+
+
+@pytest.mark.parametrize("dims,lens", [(wl.TINY, [5, 30]), (wl.SMALL_GQA, [100, 3, 250]), (wl.PHI3_MINI, [700, 64, 5]),
+                                       (wl.SMALL, [17] * 12)])
+def test_layer_decode_fp8_matches_oracle(fb, dims, lens):
+    from tests.helpers import layer_output_ok
+    B, max_seq = len(lens), 1024
+    lens = np.asarray(lens, np.int32)
+    k_scale, v_scale = 0.0625 * 1.3, 0.05
+    ctx = fb.Context.from_dims(dims, B, max_seq)
+    w = wl.layer_weights(dims, 0, device="cuda")
+    pw = ctx.pack_layer(w)
+    wb = {k: wl.bits(v) for k, v in w.items()}
+    x = wl.normal_bf16(5, 77, (B, dims.hidden), device="cuda")
+    kc, vc = wl.kv_cache_e4m3(dims, 0, B, max_seq, k_scale, v_scale, device="cuda")
+    k0, v0 = kc.cpu().numpy().copy(), vc.cpu().numpy().copy()
+    xo = torch.zeros_like(x)
+    ctx.layer_decode_fp8(pw["struct"], x, xo, kc, vc, k_scale, v_scale, i32(lens), i32(lens))
+    torch.cuda.synchronize()
+    assert ctx.get_status() == 0
+    ko, vo = k0.copy(), v0.copy()
+    want = orc.layer_decode_fp8(wb, wl.bits(x), ko, vo, k_scale, v_scale, lens, lens, dims.rms_eps, dims.rope_theta)
+    # the residual stream before its rounding, from the oracle's primitives (see tests/helpers.py: layer_output_ok)
+    nq, nkv, d = dims.n_q_heads * dims.head_dim, dims.n_kv_heads * dims.head_dim, dims.head_dim
+    qkv = orc.f64_to_bf16(orc.gemv(orc.rmsnorm(wl.bits(x), wb["g_attn"], dims.rms_eps), wb["w_qkv"]))
+    sp = lambda t, h: t.reshape(B, h, d)
+    a = orc.attn_decode_fp8(sp(qkv[:, :nq], dims.n_q_heads), sp(qkv[:, nq:nq + nkv], dims.n_kv_heads),
+                            sp(qkv[:, nq + nkv:], dims.n_kv_heads), k0.copy(), v0.copy(), k_scale, v_scale, lens, lens,
+                            dims.rope_theta)
+    h_exact = F32(wl.bits(x)).astype(np.float64) + orc.gemv(a.reshape(B, nq), wb["w_o"])
+    ok = layer_output_ok(wl.bits(xo), want, h_exact)
+    assert ok.all(), int((~ok).sum())
+    kg, vg = kc.cpu().numpy(), vc.cpu().numpy()
+    mask = np.ones(kg.shape, bool)
+    for b in range(B):
+        mask[b, :, lens[b]] = False
+    assert (kg[mask] == k0[mask]).all() and (vg[mask] == v0[mask]).all()       # nothing but the new rows changed
+    # k and v are outputs of the QKV block here: where the two sides round them to neighbouring bf16 values next to a
+    # boundary between two codes, the stored codes are neighbours too; that must stay rare and never exceed one unit
+    for got, ref in ((kg, ko), (vg, vo)):
+        diff = np.abs(_e4m3_order(got[~mask]) - _e4m3_order(ref[~mask]))
+        assert diff.max() <= 1 and (diff != 0).mean() < 0.01
+    ctx.close()
