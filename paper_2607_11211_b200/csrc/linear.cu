@@ -127,6 +127,7 @@ int configure_linear_kernels()
     FT_CUDA(allow_big_smem(linear_kernel<4, 416>));
     FT_CUDA(allow_big_smem(linear_kernel<4, 800>));
     FT_CUDA(allow_big_smem(linear_kernel<8, 416>));
+    FT_CUDA(allow_big_smem(linear_kernel<8, 544>));
     FT_CUDA(allow_big_smem(linear_kernel<8, 800>));
     return FASTTPS_OK;
 }
@@ -143,8 +144,11 @@ static int launch_linear_tile(Ctx *c, const LinearArgs &a, cudaStream_t st)
     // the register budget follows the block size: one instantiation per size class
     int rc;
     if (lay.ipw == 8)
-        rc = threads <= 416 ? launch_stream_kernel(linear_kernel<8, 416>, grid, threads, lay.total, st, &a)
-                            : launch_stream_kernel(linear_kernel<8, 800>, grid, threads, lay.total, st, &a);
+        // 17 warps (hidden 4096: 16 consumer warps) get a register budget of their own: under the 800-thread bound a
+        // thread has 72 registers and the tile loops spill
+        rc = threads <= 416   ? launch_stream_kernel(linear_kernel<8, 416>, grid, threads, lay.total, st, &a)
+             : threads <= 544 ? launch_stream_kernel(linear_kernel<8, 544>, grid, threads, lay.total, st, &a)
+                              : launch_stream_kernel(linear_kernel<8, 800>, grid, threads, lay.total, st, &a);
     else
         rc = threads <= 416 ? launch_stream_kernel(linear_kernel<4, 416>, grid, threads, lay.total, st, &a)
                             : launch_stream_kernel(linear_kernel<4, 800>, grid, threads, lay.total, st, &a);
