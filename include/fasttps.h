@@ -287,6 +287,10 @@ int fasttps_set_option(fasttps_ctx *ctx, const char *name, int value);
  * that ran out, the workspace's accumulators, tickets and barrier words are cleared as well: the kernels of the
  * abandoned call left them in an unknown state, and the next call must find them at zero. */
 int fasttps_get_status(fasttps_ctx *ctx, uint32_t *host_status);
+/* Test hook: puts the workspace into the state an abandoned call leaves behind -- garbage in the accumulators,
+ * tickets and barrier words, the FASTTPS_DEV_WAIT_TIMEOUT bit set -- with host-side memsets only (no kernel runs,
+ * nothing waits).  The next fasttps_get_status() must report the bit and make the context usable again. */
+int fasttps_debug_leave_workspace_dirty(fasttps_ctx *ctx);
 /* Optional per-launch timing for benchmarks: while enabled, every kernel launch of this
  * context is bracketed by CUDA events on its stream (up to 8192 launches; not usable during
  * stream capture).  fasttps_profile_read() synchronises and sums the elapsed time and the

@@ -82,6 +82,7 @@ def load_library() -> C.CDLL:
     lib.fasttps_model_generate.argtypes = [vp, vp, C.POINTER(LayerWeights), vp, vp, C.POINTER(vp), C.POINTER(vp),
                                            ip, ip, ip, ip, i, i, vp]
     lib.fasttps_get_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+    lib.fasttps_debug_leave_workspace_dirty.argtypes = [vp]
     lib.fasttps_profile.argtypes = [vp, i]
     lib.fasttps_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
     lib.fasttps_launch_count.argtypes = [vp]
@@ -220,6 +221,10 @@ class Context:
                                             _ptr(v_cache), _ptr(pos), _ptr(seq_lens), _ptr(out), batch,
                                             _stream(stream)), "fasttps_attn_decode")
         return out
+
+    def debug_leave_workspace_dirty(self):
+        """Test hook: the aftermath of an abandoned call, made with host-side memsets."""
+        _check(self.lib.fasttps_debug_leave_workspace_dirty(self.handle), "fasttps_debug_leave_workspace_dirty")
 
     def attn_decode_fp8(self, q, k_new, v_new, k_cache, v_cache, k_scale, v_scale, pos, seq_lens, out, stream=None):
         """k_cache / v_cache: uint8 tensors of E4M3 codes [B,Hkv,max_seq,d]; a code c stands for c * scale."""

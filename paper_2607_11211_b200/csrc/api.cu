@@ -743,6 +743,26 @@ int fasttps_get_status(fasttps_ctx *ctx, uint32_t *host_status)
     return FASTTPS_OK;
 }
 
+// Test hook: the state an abandoned call leaves behind, made on the host (no kernel is involved, nothing waits or
+// faults): partial sums in the accumulators, tickets taken, barrier words counted up, and the time-out bit set.
+int fasttps_debug_leave_workspace_dirty(fasttps_ctx *ctx)
+{
+    if (!ctx) return FASTTPS_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    const fasttps_config &f = c->cfg;
+    const size_t B = f.max_batch, D = f.hidden;
+    FT_CUDA(cudaDeviceSynchronize());
+    FT_CUDA(cudaMemset(c->mlp_acc, 0x3f, 2 * B * D * sizeof(float)));          // 0x3f3f3f3f = 0.747 in every sum
+    FT_CUDA(cudaMemset(c->hacc, 0x3f, 2 * B * D * sizeof(float)));
+    FT_CUDA(cudaMemset(c->mlp_ticket, 0x01, sizeof(int)));
+    FT_CUDA(cudaMemset(c->amax_ticket, 0x01, sizeof(int)));
+    FT_CUDA(cudaMemset(c->attn_ticket, 0x01, B * f.n_q_heads * sizeof(int)));
+    FT_CUDA(cudaMemset(c->grid_bar, 0x01, kGridBarWords * sizeof(unsigned)));
+    const uint32_t bit = FASTTPS_DEV_WAIT_TIMEOUT;
+    FT_CUDA(cudaMemcpy(c->status, &bit, sizeof(bit), cudaMemcpyHostToDevice));
+    return FASTTPS_OK;
+}
+
 int fasttps_profile(fasttps_ctx *ctx, int enable)
 {
     if (!ctx) return FASTTPS_INVALID_ARG;

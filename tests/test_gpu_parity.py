@@ -393,6 +393,42 @@ def test_mlp_decode_right_after_a_persistent_kernel_launch_many_times(fb):
     ctx.close()
 
 
+@pytest.mark.parametrize("batch", [2, 12])
+def test_context_is_usable_again_after_a_reported_timeout(fb, batch):
+    # A call that gave up on a bounded wait leaves partial sums, taken tickets and counted-up barrier words behind.
+    # That state is made on the host here (memsets through a test hook: no kernel waits, nothing faults);
+    # get_status must report the time-out bit, clear the workspace, and every path must then match the oracle again:
+    # fused MLP, the layer (persistent kernel or thin-GEMM chain) and a model step.
+    dims, max_seq = wl.SMALL, 128
+    lens = np.arange(batch, dtype=np.int32) * 7 + 3
+    ctx = make_ctx(fb, dims, batch, max_seq)
+    w = wl.layer_weights(dims, 0, device="cuda")
+    pw = ctx.pack_layer(w)
+    wb = {k: wl.bits(v) for k, v in w.items()}
+    x = wl.activations(dims, batch, device="cuda")["x"]
+    ctx.debug_leave_workspace_dirty()
+    assert ctx.get_status() & fb.DEV_WAIT_TIMEOUT
+    assert ctx.get_status() == 0
+    out = torch.empty_like(x)
+    ctx.mlp_decode(x, pw["w_gu"], pw["w_down"], out)
+    assert_close_bits(wl.bits(out), orc.mlp_decode(wl.bits(x), wb["w_gu"], wb["w_down"]), what="MLP after the reset")
+    kc, vc = wl.kv_cache(dims, 0, batch, max_seq, device="cuda")
+    ko, vo = wl.bits(kc), wl.bits(vc)
+    xo = torch.empty_like(x)
+    ctx.layer_decode(pw["struct"], x, xo, kc, vc, i32(lens), i32(lens))
+    torch.cuda.synchronize()
+    want = orc.layer_decode(wb, wl.bits(x), ko, vo, lens, lens, dims.rms_eps, dims.rope_theta)
+    assert_close_bits(wl.bits(xo), want, what="layer after the reset")
+    assert ctx.get_status() == 0
+    # and once more with the garbage left in place: the status word says so, whatever the outputs are
+    ctx.debug_leave_workspace_dirty()
+    ctx.mlp_decode(x, pw["w_gu"], pw["w_down"], out)
+    assert ctx.get_status() & fb.DEV_WAIT_TIMEOUT
+    ctx.mlp_decode(x, pw["w_gu"], pw["w_down"], out)
+    assert_close_bits(wl.bits(out), orc.mlp_decode(wl.bits(x), wb["w_gu"], wb["w_down"]), what="MLP after the second reset")
+    ctx.close()
+
+
 # -------------------------------------------------------------------- layer
 
 def rotate_rows(bits, pos, theta):
